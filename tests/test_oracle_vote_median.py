@@ -1,0 +1,201 @@
+"""Pins for the oracle's majority vote (Eq. 3) and coordinate-wise median.  CPU only."""
+import struct
+from collections import Counter
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2010_04902_b200 import inputs
+
+
+def _f(bits):
+    return struct.unpack("<f", struct.pack("<I", bits))[0]
+
+
+def _bits(a):
+    return np.ascontiguousarray(a, np.float32).view(np.uint32)
+
+
+def _cluster(l, r, q, d, attack, seed=0, **kw):
+    wf, fw, _ = oracle.assign(l, r)
+    _, byz, _ = oracle.worst_case(wf, l * l, r, q)
+    g = inputs.true_gradients(l * l, d, seed=seed)
+    rep = inputs.build_replicas(g, fw, byz, attack, **kw)
+    return g.numpy(), rep.numpy(), fw, byz
+
+
+# ------------------------------------------------------------------ vote
+
+def test_vote_hand_cases():
+    # one file, one coordinate each; columns are the r copies in order k = 0..r-1
+    a, b, c = 1.5, -2.25, 7.0
+    cases = [
+        ([a, a, a], a), ([a, b, a], a), ([b, a, a], a), ([a, a, b], a),
+        ([a, b, c], a),                       # three-way tie: first occurrence
+        ([a, b, b, a, c], a),                 # 2-2 tie: value first seen at k = 0
+        ([b, a, a, b, b], b), ([c, a, b, a, a], a),
+        ([a, b, c, c, b, a, a], a), ([a, b, b, c, c, c, b], b),  # 3-3 tie at r = 7
+    ]
+    for copies, want in cases:
+        rep = np.array(copies, np.float32).reshape(len(copies), 1, 1)
+        assert oracle.vote(rep)[0, 0] == np.float32(want), copies
+
+
+def test_vote_is_bitwise():
+    pz, nz = _f(0x00000000), _f(0x80000000)
+    n1, n2 = _f(0x7FC00001), _f(0x7FC00002)  # two NaNs with different payloads
+    cases = [([pz, nz, nz], 0x80000000), ([nz, pz, pz], 0x00000000), ([pz, nz, 1.0], 0x00000000),
+             ([n1, n2, n2], 0x7FC00002), ([n1, n1, n2], 0x7FC00001), ([1.0, n1, n1], 0x7FC00001)]
+    for copies, want_bits in cases:
+        rep = np.array([_bits(np.float32(x)) for x in copies], np.uint32).view(np.float32).reshape(3, 1, 1)
+        assert int(_bits(oracle.vote(rep))[0, 0]) == want_bits
+
+
+def test_vote_against_counter_brute_force():
+    rng = np.random.default_rng(5)
+    for r in (1, 3, 5, 7):
+        # few distinct values so that ties and pluralities of every shape occur
+        rep = rng.integers(0, 3, size=(r, 4, 200)).astype(np.float32)
+        got = oracle.vote(rep)
+        for i in range(4):
+            for j in range(200):
+                col = [float(x) for x in rep[:, i, j]]
+                cnt = Counter(col)
+                top = max(cnt.values())
+                want = next(x for x in col if cnt[x] == top)
+                assert got[i, j] == want
+
+
+def test_vote_r1_is_identity():
+    rep = np.random.default_rng(0).standard_normal((1, 9, 33)).astype(np.float32)
+    assert np.array_equal(_bits(oracle.vote(rep)), _bits(rep[0]))
+
+
+@pytest.mark.parametrize("l,r,q,attack,want_distorted", [
+    (5, 3, 2, "alie", 1),       # table (15,25,5,3), q = 2
+    (5, 3, 3, "reversed", 3),   # q = 3
+    (7, 3, 5, "alie", 8),       # table (21,49,7,3), q = 5
+    (5, 5, 6, "constant", 4),   # table (25,25,5,5), q = 6
+])
+def test_vote_count_identity_at_worst_case_placement(l, r, q, attack, want_distorted):
+    # Sec. 2: a file's gradient is distorted only if at least r' of its copies are Byzantine; at
+    # the worst-case placement the number of such files is the printed c_max.
+    g, rep, fw, byz = _cluster(l, r, q, 257, attack)
+    voted = oracle.vote(rep)
+    distorted = [i for i in range(l * l) if not np.array_equal(_bits(voted[i]), _bits(g[i]))]
+    assert len(distorted) == want_distorted
+    rp = (r + 1) // 2
+    for i in range(l * l):
+        n_byz = sum(1 for u in fw[i] if u in set(byz.tolist()))
+        assert (i in distorted) == (n_byz >= rp)
+    # colluding attackers: the element-wise vote equals the whole-vector vote of the paper
+    win = oracle.vote_vectorwise(rep)
+    for i in range(l * l):
+        assert np.array_equal(_bits(voted[i]), _bits(rep[win[i], i]))
+
+
+def test_vote_minority_corruption_is_harmless():
+    # q < r' Byzantine workers cannot change any winner (Sec. 2).
+    wf, fw, _ = oracle.assign(5, 3)
+    g = inputs.true_gradients(25, 101, seed=3)
+    for byz in ([4], [7], [13]):
+        for attack in ("alie", "reversed", "constant", "independent"):
+            rep = inputs.build_replicas(g, fw, byz, attack).numpy()
+            assert np.array_equal(_bits(oracle.vote(rep)), _bits(g.numpy()))
+
+
+def test_vote_independent_attackers_plurality():
+    # Honest copies in the minority and Byzantine copies all different: the honest value wins a
+    # file only where it is the earliest of the equally frequent patterns.
+    wf, fw, _ = oracle.assign(5, 5)
+    g = inputs.true_gradients(25, 64, seed=1)
+    byz = [0, 5, 10, 15]           # four of the five holders of file 0 (one per class)
+    assert all(0 in wf[u] for u in byz)
+    rep = inputs.build_replicas(g, fw, byz, "independent").numpy()
+    voted = oracle.vote(rep)
+    # file 0: copies k = 0..3 are distinct random vectors, k = 4 is honest -> all counts are 1,
+    # the copy of class 0 wins
+    assert np.array_equal(_bits(voted[0]), _bits(rep[0, 0]))
+    for i in range(1, 25):
+        n_byz = sum(1 for u in fw[i] if u in byz)
+        assert n_byz <= 1
+        assert np.array_equal(_bits(voted[i]), _bits(g.numpy()[i]))
+
+
+# ------------------------------------------------------------------ median
+
+def test_median_hand_cases():
+    cases = [([3, 1, 2], 2.0), ([5, 5, 5], 5.0), ([1, 9, 2, 8, 3], 3.0), ([-1, -7, 4, 0, 2, 2, -3], 0.0),
+             ([1, 2, 3, 4], 2.5), ([4, 1], 2.5), ([6], 6.0)]
+    for vals, want in cases:
+        v = np.array(vals, np.float32).reshape(len(vals), 1)
+        assert oracle.median(v)[0] == np.float32(want), vals
+
+
+def test_median_total_order_on_zeros_and_nans():
+    pz, nz = 0x00000000, 0x80000000
+    pnan, nnan = 0x7FC00000, 0xFFC00000
+    one, two = 0x3F800000, 0x40000000
+    cases = [([nz, pz, pz], pz), ([nz, nz, pz], nz), ([pz, nz, one], pz), ([pnan, one, two], two),
+             ([nnan, one, two], one), ([pnan, pnan, one], pnan), ([nnan, nnan, pnan], nnan)]
+    for bits, want in cases:
+        v = np.array(bits, np.uint32).view(np.float32).reshape(3, 1)
+        assert int(_bits(oracle.median(v))[0]) == want, [hex(b) for b in bits]
+
+
+@pytest.mark.parametrize("f", [1, 3, 5, 9, 25, 49, 63])
+def test_median_matches_numpy(f):
+    v = np.random.default_rng(f).standard_normal((f, 1000)).astype(np.float32)
+    v[:, :50] = np.round(v[:, :50]) + np.float32(0.0)  # many duplicates; "+ 0" turns -0.0 into +0.0
+    want = np.median(v, axis=0)      # odd count: numpy returns the middle element itself
+    assert np.array_equal(_bits(oracle.median(v)), _bits(want))
+    want2 = np.sort(v, axis=0)[(f - 1) // 2]
+    assert np.array_equal(_bits(oracle.median(v)), _bits(want2))
+
+
+@pytest.mark.parametrize("f", [2, 4, 16, 64])
+def test_median_even_count(f):
+    v = np.random.default_rng(f).standard_normal((f, 500)).astype(np.float32)
+    s = np.sort(v, axis=0)
+    want = np.float32(0.5) * s[f // 2 - 1] + np.float32(0.5) * s[f // 2]
+    assert np.array_equal(_bits(oracle.median(v)), _bits(want))
+
+
+def test_median_permutation_invariant_and_constant():
+    rng = np.random.default_rng(2)
+    v = rng.standard_normal((25, 300)).astype(np.float32)
+    base = oracle.median(v)
+    for _ in range(3):
+        assert np.array_equal(_bits(oracle.median(v[rng.permutation(25)])), _bits(base))
+    c = np.full((25, 17), -3.75, np.float32)
+    assert (oracle.median(c) == np.float32(-3.75)).all()
+
+
+@pytest.mark.parametrize("l,r,q,attack", [(5, 3, 2, "alie"), (5, 3, 3, "reversed"), (5, 3, 5, "constant"),
+                                          (7, 3, 5, "alie"), (5, 5, 6, "constant")])
+def test_median_stays_in_honest_range(l, r, q, attack):
+    # With fewer than f/2 distorted files the median lies between the smallest and the largest
+    # honest value of every coordinate - the property the defence relies on (Sec. 6.1).
+    g, rep, fw, byz = _cluster(l, r, q, 513, attack)
+    voted = oracle.vote(rep)
+    honest = [i for i in range(l * l) if np.array_equal(_bits(voted[i]), _bits(g[i]))]
+    assert len(honest) > (l * l) / 2
+    out = oracle.median(voted)
+    assert (out >= g[honest].min(0)).all() and (out <= g[honest].max(0)).all()
+    assert np.array_equal(_bits(oracle.vote_median(rep)), _bits(out))
+
+
+def test_inputs_are_seeded():
+    a = inputs.true_gradients(25, 1000, seed=0)
+    b = inputs.true_gradients(25, 1000, seed=0)
+    c = inputs.true_gradients(25, 1000, seed=1)
+    assert torch.equal(a, b) and not torch.equal(a, c)
+    # per-coordinate spread sigma = 0.1 around a shared N(0,1) mean
+    assert abs(float(a.std(dim=0, unbiased=True).mean()) - 0.1) < 0.01
+    assert abs(float(a.mean(dim=0).std()) - 1.0) < 0.1
+    h = inputs.true_gradients(25, 200000, seed=0, heavy_tail_frac=0.01)
+    dev = (h - h.median(dim=0).values).abs().max(dim=0).values
+    frac_wide = float((dev > 0.6).float().mean())   # 6 sigma: only heavy-tailed coordinates get there
+    assert 0.002 < frac_wide < 0.012
