@@ -1,0 +1,196 @@
+/*
+ * libbz - parameter-server aggregation of ByzShield (Konstantinidis & Ramamoorthy, MLSys 2021)
+ * on one NVIDIA B200 (sm_100a).  C ABI: plain pointers and sizes, no framework types.
+ *
+ * The library covers the per-round work of the parameter server once the K = r*l workers have
+ * reported one gradient for each of their l files: the majority vote over the r copies of every
+ * file gradient (Eq. 3, Algorithm 1), the robust aggregation of the f winners (coordinate-wise
+ * median in ByzShield, Sec. 2 and Sec. 6.1; Multi-Krum and Bulyan as the alternatives named in
+ * Sec. 6.1 and Sec. 7), the task assignment that decides which r workers hold a file
+ * (Algorithm 2, Sec. 4.2.1) and the exhaustive worst-case count c_max^(q) (Sec. 5.3.2).
+ *
+ * Conventions
+ *   - "device" pointers are CUDA global-memory addresses of the current device; "host" pointers
+ *     are ordinary process memory.  The caller owns every buffer.  The library never allocates
+ *     or frees device memory and keeps no device state between calls; scratch space is a
+ *     caller-provided device workspace whose size bz_workspace_bytes() reports.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls with
+ *     device outputs only enqueue work on that stream and return; outputs are valid once the
+ *     caller has synchronised it.  Calls with host outputs synchronise the stream themselves.
+ *   - Leading dimensions (ld_*) are in elements.  Gradients are IEEE binary32.  Row layout:
+ *     replicas[k][i][j] sits at replicas + k*ld_replica + i*ld_file + j, with k the parallel
+ *     class (Latin square) of the worker that sent the copy, i the file, j the coordinate.
+ *     The vectorised kernels need 16-byte aligned bases and leading dimensions that are
+ *     multiples of 4; anything else takes a slower scalar path, never an error.
+ *   - Every function returns BZ_OK or a negative status.  Arguments are validated on the host
+ *     before anything is launched; on a non-zero status no output has been written and nothing
+ *     has been enqueued (BZ_ERR_CUDA excepted: the runtime's message is kept for
+ *     bz_last_cuda_error()).  Nothing aborts or throws.
+ *   - Limits: r odd, 1 <= r <= BZ_MAX_R; 1 <= f <= BZ_MAX_F; d >= 0 (d == 0 is a successful no-op).
+ */
+#ifndef BZ_H_
+#define BZ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BZ_OK 0
+#define BZ_ERR_INVALID_ARG (-1)  /* null pointer, size out of range, r even, l not prime, r > l ... */
+#define BZ_ERR_UNSUPPORTED (-2)  /* a shape outside the compiled limits                              */
+#define BZ_ERR_PRECONDITION (-3) /* f < 2c+3 (Multi-Krum) or f < 4c+3 (Bulyan), m outside [1, f]     */
+#define BZ_ERR_WORKSPACE (-4)    /* workspace missing, misaligned (256 B) or too small               */
+#define BZ_ERR_BUDGET (-5)       /* C(K, q) exceeds max_subsets                                      */
+#define BZ_ERR_CUDA (-6)         /* a CUDA runtime call or launch failed                             */
+
+#define BZ_MAX_R 15
+#define BZ_MAX_F 128
+
+/* operations known to bz_workspace_bytes() */
+#define BZ_OP_PAIRDIST 1
+#define BZ_OP_MULTIKRUM 2
+#define BZ_OP_BULYAN 3
+#define BZ_OP_WORST_CASE 4
+#define BZ_OP_VOTE_MEDIAN_HOST 5
+
+/*
+ * Task assignment (Algorithm 2; Sec. 4.1.1 for the squares L_alpha(i,j) = alpha*i + j over F_l).
+ * Square k = 0..r-1 uses alpha = k+1 when r < l.  When r == l the l parallel classes are those of
+ * the Ramanujan Case 2 graph with m = s = l (Sec. 4.2.1), i.e. alpha = k.  File i*l + j is given
+ * to worker k*l + L(i, j).  Host only, synchronous.
+ *   l              prime; r in [1, l]
+ *   worker_files   host, int32 [r*l][l]: files of each worker, ascending        (may be NULL)
+ *   file_workers   host, int32 [l*l][r]: holder of each file in class k         (may be NULL)
+ *   worker_mask    host, uint64 [r*l]: bit x set iff the worker holds file x; requires l*l <= 64
+ *                  (may be NULL; BZ_ERR_INVALID_ARG if non-NULL and l*l > 64)
+ */
+int bz_assign_mols(int l, int r, int32_t* worker_files, int32_t* file_workers, uint64_t* worker_mask);
+
+/*
+ * Majority vote (Eq. 3; Algorithm 1, the loop over files), element by element: voted[i][j] is
+ * the 32-bit pattern that occurs most often among replicas[0..r-1][i][j]; among equally frequent
+ * patterns the one first seen at the lowest k wins.  Equality is bitwise (+0 != -0, NaNs are
+ * equal only with equal payloads).  For colluding attackers this equals the whole-vector vote
+ * the paper describes; r odd rules out two-way ties (Sec. 2).
+ *   replicas  device, [r][f][d] with ld_file, ld_replica;  voted  device, [f][d] with ld_voted.
+ *   voted must not overlap replicas.
+ */
+int bz_vote(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica, float* voted,
+            int64_t ld_voted, void* stream);
+
+/*
+ * Coordinate-wise median of the f voted gradients (Sec. 2, Sec. 6.1): out[j] is the element of
+ * rank (f-1)/2 of voted[0..f-1][j] under the IEEE total order (-NaN < -inf < ... < -0 < +0 < ...
+ * < +inf < +NaN).  For even f the two middle values lo <= hi give 0.5f*lo + 0.5f*hi.
+ *   voted device [f][d] with ld;  out device [d].
+ */
+int bz_median(const float* voted, int f, int64_t d, int64_t ld, float* out, void* stream);
+
+/*
+ * ByzShield's aggregation in one pass: bz_median(bz_vote(replicas)) without materialising the
+ * voted gradients.  Reads 4*r*f bytes and writes 4 bytes per coordinate.
+ */
+int bz_vote_median(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica,
+                   float* out, void* stream);
+
+/*
+ * The same aggregation for a caller whose gradients sit in HOST memory (ideally page-locked):
+ * coordinate slabs are copied to the device workspace, aggregated there and the result is copied
+ * back; the call returns after out_host is complete.  replicas_host is contiguous [r][f][d],
+ * out_host is [d].  workspace: device, at least bz_workspace_bytes(BZ_OP_VOTE_MEDIAN_HOST, ...)
+ * (more lets it use larger slabs, up to the whole array).
+ */
+int bz_vote_median_host(const float* replicas_host, int r, int f, int64_t d, float* out_host, void* workspace,
+                        size_t workspace_bytes, void* stream);
+
+/*
+ * Squared Euclidean distances between all pairs of voted gradients, the O(f^2 d) part of the
+ * Krum family (Sec. 1.2; cost in Appendix A.1): dist[a][b] = sum_j (v_a[j] - v_b[j])^2.
+ * Differences and squares are formed in binary32, added in binary32 over runs of at most 256
+ * coordinates and in binary64 across runs, in a fixed order (results are reproducible).
+ *   dist  device, double [f][f], symmetric with a zero diagonal.
+ *   workspace  device, bz_workspace_bytes(BZ_OP_PAIRDIST, 0, f, d, 0, 0) bytes, 256-byte aligned.
+ */
+int bz_pairdist(const float* voted, int f, int64_t d, int64_t ld, double* dist, void* workspace,
+                size_t workspace_bytes, void* stream);
+
+/*
+ * Multi-Krum selection on a distance matrix (Sec. 1.2: the gradient closest to its nearest
+ * neighbours; Sec. 6.1 for the operand requirement f >= 2c+3).  score[a] = sum of the f-c-2
+ * smallest dist[a][b], b != a, added in ascending order; rows are ranked by (score, index) and
+ * the first m are written to selected (m = 1 is Krum).  c counts corrupted OPERANDS (files).
+ *   dist device double [f][f];  selected device int32 [m].
+ */
+int bz_krum_select(const double* dist, int f, int c, int m, int32_t* selected, void* stream);
+
+/*
+ * Coordinate-wise mean of m selected rows: binary64 sum in the order of `selected`, divided by m,
+ * rounded once to binary32.   selected device int32 [m], values in [0, f).
+ */
+int bz_mean_rows(const float* voted, int f, int64_t d, int64_t ld, const int32_t* selected, int m, float* out,
+                 void* stream);
+
+/*
+ * Multi-Krum end to end: bz_pairdist, bz_krum_select, bz_mean_rows.
+ *   out device [d];  selected device int32 [m];  dist device double [f][f] or NULL (then the
+ *   matrix lives in the workspace);  workspace >= bz_workspace_bytes(BZ_OP_MULTIKRUM, 0, f, d, c, m).
+ */
+int bz_multikrum(const float* voted, int f, int64_t d, int64_t ld, int c, int m, float* out, int32_t* selected,
+                 double* dist, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Bulyan, first stage (Sec. 1.2; requirement f >= 4c+3 from Sec. 6.1): theta = f - 2c rows are
+ * picked one at a time.  With R the rows not yet picked, a pick takes the (score, index)-smallest
+ * row of R, scores being Krum scores inside R with clamp(|R|-c-2, 1, |R|-1) neighbours.
+ *   selected device int32 [f - 2c], in pick order.
+ */
+int bz_bulyan_select(const double* dist, int f, int c, int32_t* selected, void* stream);
+
+/*
+ * Bulyan, second stage - the trimmed mean around the median described in Sec. 1.2: per
+ * coordinate, of the theta selected values the beta closest to their median (rank (theta-1)/2 in
+ * total order) are averaged.  Closeness is |v - median| in binary32; the window grows from the
+ * median outward, ties go to the lower side; the mean is a binary64 sum in ascending order
+ * divided by beta, rounded once.   1 <= beta <= theta <= f.
+ */
+int bz_trimmed_mean(const float* voted, int f, int64_t d, int64_t ld, const int32_t* selected, int theta,
+                    int beta, float* out, void* stream);
+
+/*
+ * Bulyan end to end with theta = f - 2c, beta = theta - 2c.
+ *   selected device int32 [f - 2c];  workspace >= bz_workspace_bytes(BZ_OP_BULYAN, 0, f, d, c, 0).
+ */
+int bz_bulyan(const float* voted, int f, int64_t d, int64_t ld, int c, float* out, int32_t* selected,
+              void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Worst-case number of distorted files (Sec. 5.3.2 "exhaustive simulations"; Sec. 6.1: the
+ * attacked set is the maximiser): over all q-subsets S of the K workers, the largest number of
+ * files with at least r' = (r+1)/2 holders in S, and the lexicographically first S attaining it.
+ *   worker_mask host uint64 [K] (bit x = holds file x), f <= 64, r <= 7, 0 <= q <= K <= 64.
+ *   max_subsets: BZ_ERR_BUDGET if C(K, q) is larger (0 = no limit).
+ *   c_max host int32 [1];  argmax host int32 [q] ascending (may be NULL);  n_subsets host (may be NULL).
+ *   workspace device, bz_workspace_bytes(BZ_OP_WORST_CASE, ...) bytes.  Synchronises `stream`.
+ */
+int bz_worst_case(const uint64_t* worker_mask, int K, int f, int r, int q, uint64_t max_subsets, int32_t* c_max,
+                  int32_t* argmax, uint64_t* n_subsets, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of device workspace `op` needs for the given shape (arguments an op ignores may be 0). */
+size_t bz_workspace_bytes(int op, int r, int f, int64_t d, int c, int m);
+
+/* Static description of a status code; never NULL. */
+const char* bz_status_string(int status);
+
+/* Message of the last CUDA runtime error seen by the calling thread ("" if none). */
+const char* bz_last_cuda_error(void);
+
+/* Number of kernels this library has launched from the calling process since it was loaded. */
+uint64_t bz_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BZ_H_ */

@@ -1,0 +1,280 @@
+"""Thin ctypes binding over libbz.so: one Python function per C entry point, same names minus the
+``bz_`` prefix.  It only marshals arguments (pointers, sizes, the current CUDA stream) - every step
+of the aggregation runs in the library's kernels.  There is no fallback: a missing library or a
+non-zero status raises.
+
+Device arrays are torch CUDA tensors (torch is used for allocation and streams only).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libbz.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_PRECONDITION, ERR_WORKSPACE, ERR_BUDGET, ERR_CUDA = -1, -2, -3, -4, -5, -6
+OP_PAIRDIST, OP_MULTIKRUM, OP_BULYAN, OP_WORST_CASE, OP_VOTE_MEDIAN_HOST = 1, 2, 3, 4, 5
+MAX_R, MAX_F = 15, 128
+
+
+class BzError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        msg = "%s failed: %s (%d)" % (what, status_string(status), status)
+        if status == ERR_CUDA:
+            msg += " - " + last_cuda_error()
+        super().__init__(msg)
+
+
+_lib = None
+
+_c_int, _c_i64, _c_sz, _c_vp, _c_u64 = ctypes.c_int, ctypes.c_int64, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_uint64
+
+_SIGNATURES = {
+    "bz_assign_mols": (_c_int, [_c_int, _c_int, _c_vp, _c_vp, _c_vp]),
+    "bz_vote": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_i64, _c_vp]),
+    "bz_median": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_vp]),
+    "bz_vote_median": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_vp]),
+    "bz_vote_median_host": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_vp, _c_vp, _c_sz, _c_vp]),
+    "bz_pairdist": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_vp, _c_sz, _c_vp]),
+    "bz_krum_select": (_c_int, [_c_vp, _c_int, _c_int, _c_int, _c_vp, _c_vp]),
+    "bz_mean_rows": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_int, _c_vp, _c_vp]),
+    "bz_multikrum": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_int, _c_int, _c_vp, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp]),
+    "bz_bulyan_select": (_c_int, [_c_vp, _c_int, _c_int, _c_vp, _c_vp]),
+    "bz_trimmed_mean": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_int, _c_int, _c_vp, _c_vp]),
+    "bz_bulyan": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_int, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp]),
+    "bz_worst_case": (_c_int, [_c_vp, _c_int, _c_int, _c_int, _c_int, _c_u64, _c_vp, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp]),
+    "bz_workspace_bytes": (_c_sz, [_c_int, _c_int, _c_int, _c_i64, _c_int, _c_int]),
+    "bz_status_string": (ctypes.c_char_p, [_c_int]),
+    "bz_last_cuda_error": (ctypes.c_char_p, []),
+    "bz_kernel_launch_count": (_c_u64, []),
+}
+
+EXPORTS = sorted(_SIGNATURES)
+
+
+def lib() -> ctypes.CDLL:
+    """Load libbz.so (built in-tree by ``python -m paper_2010_04902_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("libbz.so is missing at %s: run `python -m paper_2010_04902_b200.build` "
+                              "(there is no CPU fallback)" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().bz_status_string(status).decode()
+
+
+def last_cuda_error() -> str:
+    return lib().bz_last_cuda_error().decode()
+
+
+def kernel_launch_count() -> int:
+    return int(lib().bz_kernel_launch_count())
+
+
+def _check(status: int, what: str):
+    if status != OK:
+        raise BzError(status, what)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> int:
+    if not t.is_cuda or t.dtype != dtype:
+        raise TypeError("%s must be a CUDA tensor of dtype %s" % (name, dtype))
+    return t.data_ptr()
+
+
+def _rows(t: torch.Tensor, name: str):
+    """(f, d, ld) of a [f][d] tensor whose last dimension is contiguous."""
+    if t.dim() != 2 or (t.shape[1] > 1 and t.stride(1) != 1):
+        raise ValueError("%s must be [f][d] with unit stride along d" % name)
+    f, d = t.shape
+    return f, d, (max(d, t.stride(0)) if f > 1 else d)
+
+
+def _replicas(t: torch.Tensor):
+    """(r, f, d, ld_file, ld_replica) of a [r][f][d] tensor whose last dimension is contiguous."""
+    if t.dim() != 3 or (t.shape[2] > 1 and t.stride(2) != 1):
+        raise ValueError("replicas must be [r][f][d] with unit stride along d")
+    r, f, d = t.shape
+    ld_file = max(d, t.stride(1)) if f > 1 else d
+    ld_rep = max(d, t.stride(0)) if r > 1 else f * ld_file
+    return r, f, d, ld_file, ld_rep
+
+
+def workspace_bytes(op: int, r: int = 0, f: int = 0, d: int = 0, c: int = 0, m: int = 0) -> int:
+    return int(lib().bz_workspace_bytes(op, r, f, d, c, m))
+
+
+def alloc_workspace(op: int, r: int = 0, f: int = 0, d: int = 0, c: int = 0, m: int = 0, device="cuda") -> torch.Tensor:
+    n = workspace_bytes(op, r, f, d, c, m)
+    return torch.empty(max(n, 256), dtype=torch.uint8, device=device)
+
+
+# --------------------------------------------------------------------------------------------- host
+
+def assign_mols(l: int, r: int):
+    """Algorithm 2.  Returns numpy (worker_files[K][l], file_workers[f][r], worker_mask[K] or None)."""
+    K, f = max(r * l, 1), max(l * l, 1)
+    wf = np.zeros((K, max(l, 1)), np.int32)
+    fw = np.zeros((f, max(r, 1)), np.int32)
+    mask = np.zeros(K, np.uint64) if l * l <= 64 else None
+    st = lib().bz_assign_mols(l, r, wf.ctypes.data, fw.ctypes.data, mask.ctypes.data if mask is not None else None)
+    _check(st, "bz_assign_mols(l=%d, r=%d)" % (l, r))
+    return wf, fw, mask
+
+
+def worst_case(worker_mask, f: int, r: int, q: int, max_subsets: int = 0, workspace: torch.Tensor | None = None):
+    """Exhaustive c_max^(q).  Returns (c_max, argmax[q] numpy, n_subsets)."""
+    mask = np.ascontiguousarray(worker_mask, np.uint64)
+    K = int(mask.shape[0])
+    ws = workspace if workspace is not None else alloc_workspace(OP_WORST_CASE, r, f)
+    cmax = ctypes.c_int32(0)
+    n = ctypes.c_uint64(0)
+    arg = np.zeros(max(q, 1), np.int32)
+    st = lib().bz_worst_case(mask.ctypes.data, K, f, r, q, max_subsets, ctypes.addressof(cmax), arg.ctypes.data,
+                             ctypes.addressof(n), ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "bz_worst_case(K=%d, q=%d)" % (K, q))
+    return int(cmax.value), arg[:q].copy(), int(n.value)
+
+
+# --------------------------------------------------------------------------------------------- device
+
+def vote(replicas: torch.Tensor, voted: torch.Tensor | None = None) -> torch.Tensor:
+    r, f, d, ld_file, ld_rep = _replicas(replicas)
+    if voted is None:
+        voted = torch.empty((f, d), dtype=torch.float32, device=replicas.device)
+    vf, vd, ld_v = _rows(voted, "voted")
+    if (vf, vd) != (f, d):
+        raise ValueError("voted must be [%d][%d]" % (f, d))
+    st = lib().bz_vote(_dev(replicas, torch.float32, "replicas"), r, f, d, ld_file, ld_rep,
+                       _dev(voted, torch.float32, "voted"), ld_v, _stream())
+    _check(st, "bz_vote")
+    return voted
+
+
+def median(voted: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    f, d, ld = _rows(voted, "voted")
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=voted.device)
+    st = lib().bz_median(_dev(voted, torch.float32, "voted"), f, d, ld, _dev(out, torch.float32, "out"), _stream())
+    _check(st, "bz_median")
+    return out
+
+
+def vote_median(replicas: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    r, f, d, ld_file, ld_rep = _replicas(replicas)
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=replicas.device)
+    st = lib().bz_vote_median(_dev(replicas, torch.float32, "replicas"), r, f, d, ld_file, ld_rep,
+                              _dev(out, torch.float32, "out"), _stream())
+    _check(st, "bz_vote_median")
+    return out
+
+
+def vote_median_host(replicas_host: torch.Tensor, out_host: torch.Tensor, workspace: torch.Tensor) -> torch.Tensor:
+    """replicas_host: contiguous CPU [r][f][d] (pin it for full copy speed); out_host: CPU [d]."""
+    if replicas_host.is_cuda or out_host.is_cuda or not replicas_host.is_contiguous() or not out_host.is_contiguous():
+        raise TypeError("replicas_host / out_host must be contiguous CPU tensors")
+    if replicas_host.dtype != torch.float32 or out_host.dtype != torch.float32:
+        raise TypeError("float32 expected")
+    r, f, d = replicas_host.shape
+    st = lib().bz_vote_median_host(replicas_host.data_ptr(), r, f, d, out_host.data_ptr(), workspace.data_ptr(),
+                                   workspace.numel(), _stream())
+    _check(st, "bz_vote_median_host")
+    return out_host
+
+
+def pairdist(voted: torch.Tensor, workspace: torch.Tensor | None = None, dist: torch.Tensor | None = None) -> torch.Tensor:
+    f, d, ld = _rows(voted, "voted")
+    ws = workspace if workspace is not None else alloc_workspace(OP_PAIRDIST, 0, f, d, device=voted.device)
+    if dist is None:
+        dist = torch.empty((f, f), dtype=torch.float64, device=voted.device)
+    st = lib().bz_pairdist(_dev(voted, torch.float32, "voted"), f, d, ld, _dev(dist, torch.float64, "dist"),
+                           ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "bz_pairdist")
+    return dist
+
+
+def krum_select(dist: torch.Tensor, c: int, m: int) -> torch.Tensor:
+    f = dist.shape[0]
+    sel = torch.empty(max(m, 1), dtype=torch.int32, device=dist.device)
+    st = lib().bz_krum_select(_dev(dist, torch.float64, "dist"), f, c, m, sel.data_ptr(), _stream())
+    _check(st, "bz_krum_select")
+    return sel[:m]
+
+
+def mean_rows(voted: torch.Tensor, selected: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    f, d, ld = _rows(voted, "voted")
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=voted.device)
+    st = lib().bz_mean_rows(_dev(voted, torch.float32, "voted"), f, d, ld, _dev(selected, torch.int32, "selected"),
+                            selected.numel(), _dev(out, torch.float32, "out"), _stream())
+    _check(st, "bz_mean_rows")
+    return out
+
+
+def multikrum(voted: torch.Tensor, c: int, m: int, workspace: torch.Tensor | None = None,
+              out: torch.Tensor | None = None, want_dist: bool = False):
+    """Returns (out[d], selected[m]) or (out, selected, dist) with want_dist."""
+    f, d, ld = _rows(voted, "voted")
+    ws = workspace if workspace is not None else alloc_workspace(OP_MULTIKRUM, 0, f, d, c, m, device=voted.device)
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=voted.device)
+    sel = torch.empty(max(m, 1), dtype=torch.int32, device=voted.device)
+    dist = torch.empty((f, f), dtype=torch.float64, device=voted.device) if want_dist else None
+    st = lib().bz_multikrum(_dev(voted, torch.float32, "voted"), f, d, ld, c, m, _dev(out, torch.float32, "out"),
+                            sel.data_ptr(), dist.data_ptr() if dist is not None else None, ws.data_ptr(), ws.numel(),
+                            _stream())
+    _check(st, "bz_multikrum")
+    return (out, sel[:m], dist) if want_dist else (out, sel[:m])
+
+
+def bulyan_select(dist: torch.Tensor, c: int) -> torch.Tensor:
+    f = dist.shape[0]
+    theta = f - 2 * c
+    sel = torch.empty(max(theta, 1), dtype=torch.int32, device=dist.device)
+    st = lib().bz_bulyan_select(_dev(dist, torch.float64, "dist"), f, c, sel.data_ptr(), _stream())
+    _check(st, "bz_bulyan_select")
+    return sel[:theta]
+
+
+def trimmed_mean(voted: torch.Tensor, selected: torch.Tensor, beta: int, out: torch.Tensor | None = None) -> torch.Tensor:
+    f, d, ld = _rows(voted, "voted")
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=voted.device)
+    st = lib().bz_trimmed_mean(_dev(voted, torch.float32, "voted"), f, d, ld, _dev(selected, torch.int32, "selected"),
+                               selected.numel(), beta, _dev(out, torch.float32, "out"), _stream())
+    _check(st, "bz_trimmed_mean")
+    return out
+
+
+def bulyan(voted: torch.Tensor, c: int, workspace: torch.Tensor | None = None, out: torch.Tensor | None = None):
+    """Returns (out[d], selected[f - 2c])."""
+    f, d, ld = _rows(voted, "voted")
+    ws = workspace if workspace is not None else alloc_workspace(OP_BULYAN, 0, f, d, c, device=voted.device)
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=voted.device)
+    theta = f - 2 * c
+    sel = torch.empty(max(theta, 1), dtype=torch.int32, device=voted.device)
+    st = lib().bz_bulyan(_dev(voted, torch.float32, "voted"), f, d, ld, c, _dev(out, torch.float32, "out"),
+                         sel.data_ptr(), ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "bz_bulyan")
+    return out, sel[:max(theta, 0)]

@@ -1,0 +1,297 @@
+// Majority vote (Eq. 3), coordinate-wise median, and the two fused in one pass over the replicas.
+//
+// Register path: every thread owns VEC consecutive coordinates (VEC = 4 with 128-bit loads, 1 on the
+// scalar path), streams the r copies of each of the f files once, votes them on their bit
+// patterns, keeps the f winners as order keys in registers and selects the median with a
+// comparator network.  HBM traffic is the algorithmic minimum: 4*r*f bytes in, 4 bytes out per
+// coordinate.
+#include "bz_common.cuh"
+
+namespace bz {
+
+namespace {
+
+constexpr int kBlock = 128;
+
+template <typename V> struct Lanes;
+template <> struct Lanes<uint4> {
+    static constexpr int n = 4;
+    __device__ __forceinline__ static uint32_t get(const uint4& v, int c) {
+        return c == 0 ? v.x : (c == 1 ? v.y : (c == 2 ? v.z : v.w));
+    }
+    __device__ __forceinline__ static uint4 make(const uint32_t (&a)[4]) { return make_uint4(a[0], a[1], a[2], a[3]); }
+};
+template <> struct Lanes<uint32_t> {
+    static constexpr int n = 1;
+    __device__ __forceinline__ static uint32_t get(const uint32_t& v, int) { return v; }
+    __device__ __forceinline__ static uint32_t make(const uint32_t (&a)[1]) { return a[0]; }
+};
+
+// files fetched together before their votes are taken: keeps about 12 wide loads in flight
+template <int R, int VEC> constexpr int files_per_batch() {
+    constexpr int target_regs = 48;
+    int b = target_regs / (R * VEC);
+    return b < 1 ? 1 : b;
+}
+
+// n = number of V-wide coordinate groups; ld_file / ld_rep in units of V.
+template <int R, int F, typename V>
+__global__ void __launch_bounds__(kBlock) vote_median_kernel(const V* __restrict__ rep, int64_t n, int64_t ld_file,
+                                                              int64_t ld_rep, V* __restrict__ out) {
+    constexpr int VEC = Lanes<V>::n;
+    constexpr int B = files_per_batch<R, VEC>();
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kBlock;
+    for (int64_t j = static_cast<int64_t>(blockIdx.x) * kBlock + threadIdx.x; j < n; j += stride) {
+        int key[VEC][F];
+        const V* p = rep + j;
+#pragma unroll
+        for (int i0 = 0; i0 < F; i0 += B) {
+            V x[B][R];
+#pragma unroll
+            for (int b = 0; b < B; ++b)
+#pragma unroll
+                for (int k = 0; k < R; ++k)
+                    if (i0 + b < F) x[b][k] = ld_stream(p + k * ld_rep + (i0 + b) * ld_file);
+#pragma unroll
+            for (int b = 0; b < B; ++b)
+                if (i0 + b < F) {
+#pragma unroll
+                    for (int c = 0; c < VEC; ++c) {
+                        uint32_t copies[R];
+#pragma unroll
+                        for (int k = 0; k < R; ++k) copies[k] = Lanes<V>::get(x[b][k], c);
+                        key[c][i0 + b] = order_key(vote_bits<R>(copies));
+                    }
+                }
+        }
+        uint32_t res[VEC];
+#pragma unroll
+        for (int c = 0; c < VEC; ++c) res[c] = key_bits(MedianNet<F>::run(key[c]));
+        out[j] = Lanes<V>::make(res);
+    }
+}
+
+// grid.y = file, grid.x strides over coordinate groups
+template <int R, typename V>
+__global__ void __launch_bounds__(256) vote_kernel(const V* __restrict__ rep, int64_t n, int64_t ld_file,
+                                                   int64_t ld_rep, V* __restrict__ voted, int64_t ld_voted) {
+    constexpr int VEC = Lanes<V>::n;
+    const int i = blockIdx.y;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < n; j += stride) {
+        V x[R];
+#pragma unroll
+        for (int k = 0; k < R; ++k) x[k] = ld_stream(rep + k * ld_rep + i * ld_file + j);
+        uint32_t res[VEC];
+#pragma unroll
+        for (int c = 0; c < VEC; ++c) {
+            uint32_t copies[R];
+#pragma unroll
+            for (int k = 0; k < R; ++k) copies[k] = Lanes<V>::get(x[k], c);
+            res[c] = vote_bits<R>(copies);
+        }
+        voted[i * ld_voted + j] = Lanes<V>::make(res);
+    }
+}
+
+// Any (r, f) within the limits, one coordinate per thread, arrays in local memory.  mode 0: vote
+// only (writes voted), mode 1: vote + median (writes out).
+__global__ void __launch_bounds__(128) generic_kernel(const uint32_t* __restrict__ rep, int r, int f, int64_t d,
+                                                      int64_t ld_file, int64_t ld_rep, uint32_t* __restrict__ voted,
+                                                      int64_t ld_voted, float* __restrict__ out, int mode) {
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < d; j += stride) {
+        int key[BZ_MAX_F];
+        for (int i = 0; i < f; ++i) {
+            uint32_t x[BZ_MAX_R];
+            for (int k = 0; k < r; ++k) x[k] = rep[k * ld_rep + i * ld_file + j];
+            const uint32_t w = vote_bits_dyn(x, r);
+            if (mode == 0)
+                voted[i * ld_voted + j] = w;
+            else
+                key[i] = order_key(w);
+        }
+        if (mode == 0) continue;
+        // element(s) of the wanted rank by counting, ties ordered by position
+        const int want_hi = f / 2, want_lo = (f - 1) / 2;
+        int k_lo = 0, k_hi = 0;
+        for (int i = 0; i < f; ++i) {
+            int rank = 0;
+            for (int t = 0; t < f; ++t) rank += (key[t] < key[i]) || (key[t] == key[i] && t < i);
+            if (rank == want_lo) k_lo = key[i];
+            if (rank == want_hi) k_hi = key[i];
+        }
+        if (f & 1)
+            out[j] = __uint_as_float(key_bits(k_lo));
+        else
+            out[j] = __fadd_rn(__fmul_rn(0.5f, __uint_as_float(key_bits(k_lo))),
+                               __fmul_rn(0.5f, __uint_as_float(key_bits(k_hi))));
+    }
+}
+
+int grid_for(int64_t work_items, int block, int ctas_per_sm) {
+    int64_t need = (work_items + block - 1) / block;
+    const int64_t cap = static_cast<int64_t>(kNumSMs) * ctas_per_sm;
+    if (need > cap) need = cap;
+    if (need < 1) need = 1;
+    return static_cast<int>(need);
+}
+
+template <int R, int F, typename V>
+int launch_vm(const float* rep, int64_t n, int64_t ld_file, int64_t ld_rep, float* out, cudaStream_t s) {
+    if (n <= 0) return BZ_OK;
+    constexpr int VEC = Lanes<V>::n;
+    vote_median_kernel<R, F, V><<<grid_for(n, kBlock, 16), kBlock, 0, s>>>(
+        reinterpret_cast<const V*>(rep), n, ld_file / VEC, ld_rep / VEC, reinterpret_cast<V*>(out));
+    note_launch();
+    return check_launch();
+}
+
+template <int R, int F>
+int vm_dispatch_vec(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, float* out, bool vec, cudaStream_t s) {
+    if (!vec) return launch_vm<R, F, uint32_t>(rep, d, ld_file, ld_rep, out, s);
+    const int64_t n4 = d / 4;
+    int st = launch_vm<R, F, uint4>(rep, n4, ld_file, ld_rep, out, s);
+    if (st != BZ_OK) return st;
+    return launch_vm<R, F, uint32_t>(rep + 4 * n4, d - 4 * n4, ld_file, ld_rep, out + 4 * n4, s);
+}
+
+template <int R>
+int vm_dispatch_f(const float* rep, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* out, bool vec,
+                  cudaStream_t s) {
+    switch (f) {
+        case 25: return vm_dispatch_vec<R, 25>(rep, d, ld_file, ld_rep, out, vec, s);
+        case 49: return vm_dispatch_vec<R, 49>(rep, d, ld_file, ld_rep, out, vec, s);
+        default: return 1;  // not specialised
+    }
+}
+
+int launch_generic(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted,
+                   int64_t ld_voted, float* out, int mode, cudaStream_t s) {
+    generic_kernel<<<grid_for(d, 128, 8), 128, 0, s>>>(reinterpret_cast<const uint32_t*>(rep), r, f, d, ld_file, ld_rep,
+                                                       reinterpret_cast<uint32_t*>(voted), ld_voted, out, mode);
+    note_launch();
+    return check_launch();
+}
+
+template <int R, typename V>
+int launch_vote(const float* rep, int f, int64_t n, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted,
+                cudaStream_t s) {
+    if (n <= 0) return BZ_OK;
+    constexpr int VEC = Lanes<V>::n;
+    // about 8 CTAs per SM over the whole (coordinate group, file) grid
+    int64_t gx = (n + 255) / 256;
+    const int64_t cap = (static_cast<int64_t>(kNumSMs) * 8 + f - 1) / f;
+    if (gx > cap) gx = cap;
+    if (gx < 1) gx = 1;
+    dim3 grid(static_cast<unsigned>(gx), f);
+    vote_kernel<R, V><<<grid, 256, 0, s>>>(reinterpret_cast<const V*>(rep), n, ld_file / VEC, ld_rep / VEC,
+                                           reinterpret_cast<V*>(voted), ld_voted / VEC);
+    note_launch();
+    return check_launch();
+}
+
+template <int R>
+int vote_dispatch(const float* rep, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted,
+                  bool vec, cudaStream_t s) {
+    if (!vec) return launch_vote<R, uint32_t>(rep, f, d, ld_file, ld_rep, voted, ld_voted, s);
+    const int64_t n4 = d / 4;
+    int st = launch_vote<R, uint4>(rep, f, n4, ld_file, ld_rep, voted, ld_voted, s);
+    if (st != BZ_OK) return st;
+    return launch_vote<R, uint32_t>(rep + 4 * n4, f, d - 4 * n4, ld_file, ld_rep, voted + 4 * n4, ld_voted, s);
+}
+
+int validate_replicas(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep) {
+    if (rep == nullptr || d < 0 || r < 1 || f < 1 || (r % 2) == 0) return BZ_ERR_INVALID_ARG;
+    if (r > BZ_MAX_R || f > BZ_MAX_F) return BZ_ERR_UNSUPPORTED;
+    if (ld_file < d) return BZ_ERR_INVALID_ARG;
+    if (r > 1 && ld_rep < d) return BZ_ERR_INVALID_ARG;
+    return BZ_OK;
+}
+
+}  // namespace
+
+int vote_median_on_device(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* out,
+                          cudaStream_t s) {
+    const bool vec = aligned16(rep) && aligned16(out) && (ld_file % 4 == 0) && (r == 1 || ld_rep % 4 == 0);
+    int st = 1;
+    switch (r) {
+        case 1: st = vm_dispatch_f<1>(rep, f, d, ld_file, ld_rep, out, vec, s); break;
+        case 3: st = vm_dispatch_f<3>(rep, f, d, ld_file, ld_rep, out, vec, s); break;
+        case 5: st = vm_dispatch_f<5>(rep, f, d, ld_file, ld_rep, out, vec, s); break;
+        case 7: st = vm_dispatch_f<7>(rep, f, d, ld_file, ld_rep, out, vec, s); break;
+        default: break;
+    }
+    if (st == 1) st = launch_generic(rep, r, f, d, ld_file, ld_rep, nullptr, 0, out, 1, s);
+    return st;
+}
+
+}  // namespace bz
+
+using namespace bz;
+
+extern "C" int bz_vote_median(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica,
+                              float* out, void* stream) {
+    int st = validate_replicas(replicas, r, f, d, ld_file, ld_replica);
+    if (st != BZ_OK) return st;
+    if (out == nullptr) return BZ_ERR_INVALID_ARG;
+    if (d == 0) return BZ_OK;
+    return vote_median_on_device(replicas, r, f, d, ld_file, ld_replica, out, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int bz_median(const float* voted, int f, int64_t d, int64_t ld, float* out, void* stream) {
+    int st = validate_replicas(voted, 1, f, d, ld, 0);
+    if (st != BZ_OK) return st;
+    if (out == nullptr) return BZ_ERR_INVALID_ARG;
+    if (d == 0) return BZ_OK;
+    return vote_median_on_device(voted, 1, f, d, ld, 0, out, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int bz_vote(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica,
+                       float* voted, int64_t ld_voted, void* stream) {
+    int st = validate_replicas(replicas, r, f, d, ld_file, ld_replica);
+    if (st != BZ_OK) return st;
+    if (voted == nullptr || ld_voted < d) return BZ_ERR_INVALID_ARG;
+    if (d == 0) return BZ_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool vec = aligned16(replicas) && aligned16(voted) && (ld_file % 4 == 0) && (ld_voted % 4 == 0) &&
+                     (r == 1 || ld_replica % 4 == 0);
+    switch (r) {
+        case 1: return vote_dispatch<1>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, vec, s);
+        case 3: return vote_dispatch<3>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, vec, s);
+        case 5: return vote_dispatch<5>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, vec, s);
+        case 7: return vote_dispatch<7>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, vec, s);
+        default: return launch_generic(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, nullptr, 0, s);
+    }
+}
+
+extern "C" int bz_vote_median_host(const float* replicas_host, int r, int f, int64_t d, float* out_host,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
+    int st = validate_replicas(replicas_host, r, f, d, d, static_cast<int64_t>(f) * d);
+    if (st != BZ_OK) return st;
+    if (out_host == nullptr) return BZ_ERR_INVALID_ARG;
+    if (d == 0) return BZ_OK;
+    if (workspace == nullptr || !aligned256(workspace)) return BZ_ERR_WORKSPACE;
+    if (workspace_bytes < bz_workspace_bytes(BZ_OP_VOTE_MEDIAN_HOST, r, f, d, 0, 0)) return BZ_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // slab of S coordinates: r*f input rows and one output row, each padded to a multiple of 64
+    const size_t rows = static_cast<size_t>(r) * f + 1;
+    int64_t S = static_cast<int64_t>(workspace_bytes / (rows * sizeof(float)));
+    S = S / 64 * 64;
+    if (S > (d + 63) / 64 * 64) S = (d + 63) / 64 * 64;
+    float* slab = static_cast<float*>(workspace);
+    float* out_dev = slab + static_cast<size_t>(r) * f * S;
+    for (int64_t j0 = 0; j0 < d; j0 += S) {
+        const int64_t n = (d - j0 < S) ? d - j0 : S;
+        cudaError_t e = cudaMemcpy2DAsync(slab, S * sizeof(float), replicas_host + j0, d * sizeof(float),
+                                          n * sizeof(float), static_cast<size_t>(r) * f, cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return cuda_failed(e);
+        st = vote_median_on_device(slab, r, f, n, S, static_cast<int64_t>(f) * S, out_dev, s);
+        if (st != BZ_OK) return st;
+        e = cudaMemcpyAsync(out_host + j0, out_dev, n * sizeof(float), cudaMemcpyDeviceToHost, s);
+        if (e != cudaSuccess) return cuda_failed(e);
+    }
+    cudaError_t e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_failed(e);
+    return BZ_OK;
+}
