@@ -1,0 +1,143 @@
+"""GPU parity of the Krum family against the CPU oracle: distances, selection indices (bit-exact),
+means (relative L2 <= 1e-5, the tolerance for averaged outputs in binary32)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2010_04902_b200 import binding as bz
+from paper_2010_04902_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda"
+MEAN_TOL = 1e-5      # relative L2 of averaged outputs
+DIST_TOL = 1e-7      # relative error of a squared distance (binary32 products, binary64 sums)
+
+
+def _rel_l2(got, want):
+    got = np.asarray(got, np.float64)
+    want = np.asarray(want, np.float64)
+    den = np.linalg.norm(want)
+    return np.linalg.norm(got - want) / (den if den > 0 else 1.0)
+
+
+def _voted(l, r, q, d, attack, seed=0, heavy=0.0):
+    wf, fw, _ = oracle.assign(l, r)
+    byz = oracle.worst_case(wf, l * l, r, q)[1]
+    g = inputs.true_gradients(l * l, d, seed=seed, heavy_tail_frac=heavy)
+    rep = inputs.build_replicas(g, fw, byz, attack)
+    return torch.from_numpy(oracle.vote(rep.numpy()))
+
+
+@pytest.mark.parametrize("f,d", [(25, 1), (25, 255), (25, 4097), (49, 3), (49, 1000), (49, 70001), (9, 513), (121, 300)])
+def test_pairdist_exact_on_integer_rows(f, d):
+    v = inputs.integer_gradients(f, d, seed=f + d)
+    want = oracle.pairdist(v.numpy())
+    got = bz.pairdist(v.to(DEV)).cpu().numpy()
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("l,r,q,attack,d", [(5, 3, 3, "reversed", 50001), (7, 3, 5, "alie", 50001),
+                                            (5, 5, 6, "constant", 20000), (3, 3, 2, "alie", 999)])
+def test_pairdist_close_on_gradients(l, r, q, attack, d):
+    v = _voted(l, r, q, d, attack)
+    want = oracle.pairdist(v.numpy())
+    got = bz.pairdist(v.to(DEV)).cpu().numpy()
+    assert np.array_equal(got, got.T) and (np.diag(got) == 0).all()
+    off = ~np.eye(v.shape[0], dtype=bool)
+    nz = off & (want > 0)
+    assert (np.abs(got[nz] - want[nz]) <= DIST_TOL * want[nz]).all()
+    assert (got[off & (want == 0)] == 0).all()     # identical (colluding) rows
+    # twice the same call: fixed summation order
+    assert np.array_equal(bz.pairdist(v.to(DEV)).cpu().numpy(), got)
+
+
+def test_pairdist_unaligned_rows():
+    v = inputs.integer_gradients(25, 1003, seed=2)
+    buf = torch.zeros((25, 1100), dtype=torch.float32, device=DEV)
+    buf[:, 1:1004] = v.to(DEV)
+    assert np.array_equal(bz.pairdist(buf[:, 1:1004]).cpu().numpy(), oracle.pairdist(v.numpy()))
+    buf[:, 4:1007] = v.to(DEV)
+    assert np.array_equal(bz.pairdist(buf[:, 4:1007]).cpu().numpy(), oracle.pairdist(v.numpy()))
+
+
+def test_krum_hand_cases_on_device():
+    v = torch.tensor([[0.0], [1.0], [2.0], [3.0], [10.0]])
+    D = bz.pairdist(v.to(DEV))
+    assert bz.krum_select(D, 1, 1).cpu().tolist() == [1]
+    assert bz.krum_select(D, 1, 3).cpu().tolist() == [1, 2, 0]
+    out, sel = bz.multikrum(v.to(DEV), 1, 4)
+    assert sel.cpu().tolist() == [1, 2, 0, 3] and float(out[0]) == 1.5
+    v7 = torch.tensor([[0.0], [1.0], [2.0], [3.0], [4.0], [5.0], [100.0]])
+    assert bz.bulyan_select(bz.pairdist(v7.to(DEV)), 1).cpu().tolist() == [2, 3, 1, 4, 0]
+    out, sel = bz.bulyan(v7.to(DEV), 1)
+    assert float(out[0]) == 2.0
+
+
+@pytest.mark.parametrize("l,r,q,attack,d,c,m", [
+    (7, 3, 5, "alie", 30011, 5, 44),        # benchmark parameters of the multi-Krum configuration
+    (7, 3, 5, "alie", 30011, 8, 41),        # the paper's reading: c = c_max = 8 distorted files
+    (5, 3, 3, "reversed", 12345, 3, 22),
+    (5, 5, 6, "constant", 8000, 4, 1),      # Krum
+    (3, 3, 2, "reversed", 777, 1, 5),       # generic (f = 9) path
+])
+def test_multikrum_parity(l, r, q, attack, d, c, m):
+    v = _voted(l, r, q, d, attack)
+    want_out, want_sel, want_D = oracle.multikrum(v.numpy(), c, m)
+    out, sel, D = bz.multikrum(v.to(DEV), c, m, want_dist=True)
+    assert sel.cpu().tolist() == want_sel.tolist()
+    assert _rel_l2(out.cpu().numpy(), want_out) <= MEAN_TOL
+    # stage by stage through the separate entry points
+    sel2 = bz.krum_select(torch.from_numpy(want_D).to(DEV), c, m)
+    assert sel2.cpu().tolist() == want_sel.tolist()
+    out2 = bz.mean_rows(v.to(DEV), sel2)
+    assert np.array_equal(out2.cpu().numpy(), want_out)        # same binary64 sums, same order
+
+
+def test_multikrum_c0_is_plain_mean():
+    v = inputs.true_gradients(25, 5001, seed=6)
+    out, sel = bz.multikrum(v.to(DEV), 0, 25)
+    assert sorted(sel.cpu().tolist()) == list(range(25))
+    assert _rel_l2(out.cpu().numpy(), v.double().mean(0).numpy()) <= MEAN_TOL
+
+
+@pytest.mark.parametrize("l,r,q,attack,d,c,heavy", [
+    (5, 5, 6, "constant", 30011, 4, 0.01),   # benchmark parameters of the Bulyan configuration
+    (7, 3, 5, "alie", 9001, 8, 0.0),
+    (7, 3, 3, "reversed", 4000, 11, 0.0),    # largest c for f = 49: theta = 27, beta = 5
+    (5, 3, 2, "alie", 4000, 0, 0.0),         # c = 0: theta = beta = f
+    (3, 3, 2, "reversed", 600, 1, 0.0),      # generic (f = 9) path, theta = 7
+])
+def test_bulyan_parity(l, r, q, attack, d, c, heavy):
+    v = _voted(l, r, q, d, attack, heavy=heavy)
+    want_out, want_sel, want_D = oracle.bulyan(v.numpy(), c)
+    out, sel = bz.bulyan(v.to(DEV), c)
+    assert sel.cpu().tolist() == want_sel.tolist()
+    assert _rel_l2(out.cpu().numpy(), want_out) <= MEAN_TOL
+    sel2 = bz.bulyan_select(torch.from_numpy(want_D).to(DEV), c)
+    assert sel2.cpu().tolist() == want_sel.tolist()
+
+
+@pytest.mark.parametrize("theta,beta", [(5, 3), (7, 1), (9, 9), (17, 9), (25, 17), (27, 5), (49, 49), (49, 1),
+                                        (8, 3), (12, 12), (11, 5), (13, 7)])
+def test_trimmed_mean_parity(theta, beta):
+    # specialised (odd theta with a network) and generic thetas; many duplicates and ties
+    rng = np.random.default_rng(theta * 64 + beta)
+    f = max(theta, 25)
+    v = rng.standard_normal((f, 2049)).astype(np.float32)
+    v[:, :512] = np.round(v[:, :512] * 2) / 2
+    sel = rng.permutation(f)[:theta].astype(np.int32)
+    want = oracle.trimmed_mean(v, sel, beta)
+    got = bz.trimmed_mean(torch.from_numpy(v).to(DEV), torch.from_numpy(sel).to(DEV), beta)
+    assert np.array_equal(got.cpu().numpy(), want)
+
+
+def test_preconditions_reported():
+    v = torch.zeros((25, 16), dtype=torch.float32, device=DEV)
+    with pytest.raises(bz.BzError) as e:
+        bz.bulyan(v, 6)          # 4*6+3 > 25: the case the paper calls inapplicable
+    assert e.value.status == bz.ERR_PRECONDITION
+    with pytest.raises(bz.BzError) as e:
+        bz.multikrum(v, 12, 1)   # 2*12+3 > 25
+    assert e.value.status == bz.ERR_PRECONDITION
