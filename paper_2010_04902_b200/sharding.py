@@ -1,0 +1,70 @@
+"""Coordinate sharding of the aggregation path over several GPUs (one process per GPU).
+
+The vote, the median, the means and the trimmed means are independent per coordinate: each rank
+aggregates its own contiguous slab of coordinates and nothing is exchanged.  The Krum family needs
+one exchange: squared distances are sums over coordinates, so the ranks' partial f x f matrices are
+added with a single all-reduce (at most 128 x 128 doubles) before the - replicated - selection.
+
+``ops`` is the module that supplies the per-rank operations; it defaults to the CUDA binding.  The
+functions here contain only the partitioning and the exchange.
+"""
+from __future__ import annotations
+
+import torch
+import torch.distributed as dist
+
+
+def coordinate_slab(d: int, rank: int, world: int, align: int = 4):
+    """[begin, end) of the coordinates rank `rank` of `world` owns.  Slab boundaries are multiples of
+    `align` (so every slab starts on a 16-byte boundary for fp32), slabs are contiguous, disjoint and
+    cover [0, d), and sizes differ by less than 2 * `align`."""
+    if world < 1 or not (0 <= rank < world) or d < 0 or align < 1:
+        raise ValueError("bad slab request d=%d rank=%d world=%d" % (d, rank, world))
+    units = (d + align - 1) // align
+    base, extra = divmod(units, world)
+    first = rank * base + min(rank, extra)
+    last = first + base + (1 if rank < extra else 0)
+    return min(first * align, d), min(last * align, d)
+
+
+def _world(group=None):
+    if dist.is_available() and dist.is_initialized():
+        return dist.get_world_size(group)
+    return 1
+
+
+def allreduce_sum_(t: torch.Tensor, group=None) -> torch.Tensor:
+    """In-place sum over ranks; identity for a single process."""
+    if _world(group) > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.SUM, group=group)
+    return t
+
+
+def _ops(ops):
+    if ops is None:
+        from . import binding as ops  # the CUDA path; raises if the library is missing
+    return ops
+
+
+def vote_median(replicas_slab: torch.Tensor, ops=None) -> torch.Tensor:
+    """Fused vote + median on this rank's slab [r][f][d_local]; no exchange."""
+    return _ops(ops).vote_median(replicas_slab)
+
+
+def multikrum(voted_slab: torch.Tensor, c: int, m: int, ops=None, group=None):
+    """Multi-Krum over coordinate slabs.  Returns (out_slab[d_local], selected[m], dist[f][f])."""
+    ops = _ops(ops)
+    D = ops.pairdist(voted_slab)
+    allreduce_sum_(D, group)
+    sel = ops.krum_select(D, c, m)
+    return ops.mean_rows(voted_slab, sel), sel, D
+
+
+def bulyan(voted_slab: torch.Tensor, c: int, ops=None, group=None):
+    """Bulyan over coordinate slabs.  Returns (out_slab[d_local], selected[f-2c], dist[f][f])."""
+    ops = _ops(ops)
+    D = ops.pairdist(voted_slab)
+    allreduce_sum_(D, group)
+    sel = ops.bulyan_select(D, c)
+    theta = voted_slab.shape[0] - 2 * c
+    return ops.trimmed_mean(voted_slab, sel, theta - 2 * c), sel, D

@@ -1,0 +1,103 @@
+"""The multi-rank path on CPU: two gloo ranks, each aggregating its coordinate slab with the CPU
+checker standing in for the per-rank kernels, must reproduce the single-rank result - no exchange
+for vote/median, one all-reduce of the distance matrix for the Krum family."""
+import os
+import socket
+import types
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import oracle
+from paper_2010_04902_b200 import inputs, sharding
+
+
+def test_coordinate_slabs_partition_the_range():
+    for d in [0, 1, 3, 4, 5, 1000, 1001, 11_200_000, 11_173_962]:
+        for world in [1, 2, 3, 4, 8]:
+            ends = [sharding.coordinate_slab(d, rk, world) for rk in range(world)]
+            assert ends[0][0] == 0 and ends[-1][1] == d
+            for (a0, a1), (b0, b1) in zip(ends, ends[1:]):
+                assert a1 == b0 and a0 <= a1
+            for a0, a1 in ends:
+                assert a0 % 4 == 0 or a0 == d
+            sizes = [b - a for a, b in ends]
+            assert max(sizes) - min(sizes) < 8
+    with pytest.raises(ValueError):
+        sharding.coordinate_slab(10, 2, 2)
+
+
+def _oracle_ops():
+    """Per-rank operations backed by the CPU checker, with the binding's signatures."""
+    t = torch.from_numpy
+    return types.SimpleNamespace(
+        vote_median=lambda rep: t(oracle.vote_median(rep.numpy())),
+        pairdist=lambda v: t(oracle.pairdist(v.numpy())),
+        krum_select=lambda D, c, m: t(oracle.multikrum_select(D.numpy(), c, m)),
+        mean_rows=lambda v, sel: t(oracle.mean_rows(v.numpy(), sel.numpy())),
+        bulyan_select=lambda D, c: t(oracle.bulyan_select(D.numpy(), c)),
+        trimmed_mean=lambda v, sel, beta: t(oracle.trimmed_mean(v.numpy(), sel.numpy(), beta)),
+    )
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def _worker(rank, world, port, d, ret):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        ops = _oracle_ops()
+        wf, fw, _ = oracle.assign(5, 3)
+        _, byz, _ = oracle.worst_case(wf, 25, 3, 3)
+        g = inputs.true_gradients(25, d, seed=0)
+        rep = inputs.build_replicas(g, fw, byz, "reversed")
+        j0, j1 = sharding.coordinate_slab(d, rank, world)
+        rep_slab = rep[:, :, j0:j1].contiguous()
+        med = sharding.vote_median(rep_slab, ops=ops)
+        voted_slab = torch.from_numpy(oracle.vote(rep_slab.numpy()))
+        mk_out, mk_sel, D = sharding.multikrum(voted_slab, 3, 22, ops=ops)
+        bu_out, bu_sel, _ = sharding.bulyan(voted_slab, 3, ops=ops)
+        ret[rank] = dict(j=(j0, j1), med=med.numpy(), mk_out=mk_out.numpy(), mk_sel=mk_sel.numpy(), D=D.numpy(),
+                         bu_out=bu_out.numpy(), bu_sel=bu_sel.numpy())
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("d", [4001, 1026])
+def test_two_ranks_reproduce_the_single_rank_result(d):
+    world = 2
+    ctx = mp.get_context("spawn")
+    mgr = ctx.Manager()
+    ret = mgr.dict()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(rk, world, port, d, ret)) for rk in range(world)]
+    for p in procs:
+        p.start()
+    for p in procs:
+        p.join(180)
+        assert p.exitcode == 0
+    wf, fw, _ = oracle.assign(5, 3)
+    _, byz, _ = oracle.worst_case(wf, 25, 3, 3)
+    g = inputs.true_gradients(25, d, seed=0)
+    rep = inputs.build_replicas(g, fw, byz, "reversed").numpy()
+    voted = oracle.vote(rep)
+    want_med = oracle.median(voted)
+    want_mk, want_mk_sel, want_D = oracle.multikrum(voted, 3, 22)
+    want_bu, want_bu_sel, _ = oracle.bulyan(voted, 3)
+    parts = [ret[rk] for rk in range(world)]
+    assert parts[0]["j"][1] == parts[1]["j"][0] and parts[1]["j"][1] == d
+    assert np.array_equal(np.concatenate([p["med"] for p in parts]).view(np.uint32), want_med.view(np.uint32))
+    for p in parts:
+        assert np.allclose(p["D"], want_D, rtol=1e-12, atol=0)           # summed in two pieces
+        assert p["mk_sel"].tolist() == want_mk_sel.tolist() and p["bu_sel"].tolist() == want_bu_sel.tolist()
+    assert np.array_equal(np.concatenate([p["mk_out"] for p in parts]), want_mk)
+    assert np.array_equal(np.concatenate([p["bu_out"] for p in parts]), want_bu)
