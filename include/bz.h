@@ -187,6 +187,13 @@ const char* bz_status_string(int status);
 /* Message of the last CUDA runtime error seen by the calling thread ("" if none). */
 const char* bz_last_cuda_error(void);
 
+/*
+ * The TMA-staged kernels bound every wait on a shared-memory barrier; a wait that runs out makes
+ * the kernel stop early and bump a device-side counter instead of hanging.  This reads that
+ * counter (synchronously; 0 after any number of healthy launches) into *count (host).
+ */
+int bz_pipeline_timeouts(unsigned int* count);
+
 /* Number of kernels this library has launched from the calling process since it was loaded. */
 uint64_t bz_kernel_launch_count(void);
 

@@ -53,6 +53,7 @@ _SIGNATURES = {
     "bz_status_string": (ctypes.c_char_p, [_c_int]),
     "bz_last_cuda_error": (ctypes.c_char_p, []),
     "bz_kernel_launch_count": (_c_u64, []),
+    "bz_pipeline_timeouts": (_c_int, [_c_vp]),
 }
 
 EXPORTS = sorted(_SIGNATURES)
@@ -84,6 +85,13 @@ def last_cuda_error() -> str:
 
 def kernel_launch_count() -> int:
     return int(lib().bz_kernel_launch_count())
+
+
+def pipeline_timeouts() -> int:
+    """Barrier waits that ran out inside the TMA-staged kernels since the library was loaded (0 when healthy)."""
+    n = ctypes.c_uint(0)
+    _check(lib().bz_pipeline_timeouts(ctypes.addressof(n)), "bz_pipeline_timeouts")
+    return int(n.value)
 
 
 def _check(status: int, what: str):

@@ -10,6 +10,7 @@ namespace bz {
 
 size_t krum_workspace_bytes(int op, int f);   // krum.cu
 size_t worst_case_workspace_bytes();          // worst_case.cu
+int pipeline_timeouts(unsigned int* count);   // vote_median_tma.cu
 
 namespace {
 std::atomic<uint64_t> g_launches{0};
@@ -96,6 +97,11 @@ extern "C" const char* bz_status_string(int status) {
         case BZ_ERR_CUDA: return "CUDA runtime error";
         default: return "unknown status";
     }
+}
+
+extern "C" int bz_pipeline_timeouts(unsigned int* count) {
+    if (count == nullptr) return BZ_ERR_INVALID_ARG;
+    return pipeline_timeouts(count);
 }
 
 extern "C" const char* bz_last_cuda_error(void) { return g_cuda_msg; }

@@ -499,7 +499,7 @@ int trimmed_mean_on_device(const float* v, int64_t d, int64_t ld, const int32_t*
 }
 
 int validate_rows(const float* v, int f, int64_t d, int64_t ld) {
-    if (v == nullptr || d < 0 || f < 1) return BZ_ERR_INVALID_ARG;
+    if (d < 0 || f < 1 || (v == nullptr && d > 0)) return BZ_ERR_INVALID_ARG;  // an empty array may have no address
     if (f > BZ_MAX_F) return BZ_ERR_UNSUPPORTED;
     if (ld < d) return BZ_ERR_INVALID_ARG;
     return BZ_OK;
@@ -546,7 +546,7 @@ extern "C" int bz_mean_rows(const float* voted, int f, int64_t d, int64_t ld, co
                             float* out, void* stream) {
     int st = validate_rows(voted, f, d, ld);
     if (st != BZ_OK) return st;
-    if (selected == nullptr || out == nullptr) return BZ_ERR_INVALID_ARG;
+    if (selected == nullptr || (out == nullptr && d > 0)) return BZ_ERR_INVALID_ARG;
     if (m < 1 || m > f) return BZ_ERR_PRECONDITION;
     if (d == 0) return BZ_OK;
     return mean_rows_on_device(voted, d, ld, selected, m, out, static_cast<cudaStream_t>(stream));
@@ -556,7 +556,7 @@ extern "C" int bz_multikrum(const float* voted, int f, int64_t d, int64_t ld, in
                             int32_t* selected, double* dist, void* workspace, size_t workspace_bytes, void* stream) {
     int st = validate_rows(voted, f, d, ld);
     if (st != BZ_OK) return st;
-    if (out == nullptr || selected == nullptr) return BZ_ERR_INVALID_ARG;
+    if ((out == nullptr && d > 0) || selected == nullptr) return BZ_ERR_INVALID_ARG;
     if (c < 0 || f < 2 * c + 3 || m < 1 || m > f) return BZ_ERR_PRECONDITION;
     st = check_workspace(workspace, workspace_bytes, krum_workspace_bytes(BZ_OP_MULTIKRUM, f));
     if (st != BZ_OK) return st;
@@ -583,7 +583,7 @@ extern "C" int bz_trimmed_mean(const float* voted, int f, int64_t d, int64_t ld,
                                int beta, float* out, void* stream) {
     int st = validate_rows(voted, f, d, ld);
     if (st != BZ_OK) return st;
-    if (selected == nullptr || out == nullptr) return BZ_ERR_INVALID_ARG;
+    if (selected == nullptr || (out == nullptr && d > 0)) return BZ_ERR_INVALID_ARG;
     if (theta < 1 || theta > f || beta < 1 || beta > theta) return BZ_ERR_PRECONDITION;
     if (d == 0) return BZ_OK;
     return trimmed_mean_on_device(voted, d, ld, selected, theta, beta, out, static_cast<cudaStream_t>(stream));
@@ -593,7 +593,7 @@ extern "C" int bz_bulyan(const float* voted, int f, int64_t d, int64_t ld, int c
                          void* workspace, size_t workspace_bytes, void* stream) {
     int st = validate_rows(voted, f, d, ld);
     if (st != BZ_OK) return st;
-    if (out == nullptr || selected == nullptr) return BZ_ERR_INVALID_ARG;
+    if ((out == nullptr && d > 0) || selected == nullptr) return BZ_ERR_INVALID_ARG;
     if (c < 0 || f < 4 * c + 3) return BZ_ERR_PRECONDITION;
     st = check_workspace(workspace, workspace_bytes, krum_workspace_bytes(BZ_OP_BULYAN, f));
     if (st != BZ_OK) return st;

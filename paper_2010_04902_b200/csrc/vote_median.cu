@@ -5,13 +5,30 @@
 // patterns, keeps the f winners as order keys in registers and selects the median with a
 // comparator network.  HBM traffic is the algorithmic minimum: 4*r*f bytes in, 4 bytes out per
 // coordinate.
+#include <cstdlib>
+#include <cstring>
+
 #include "bz_common.cuh"
 
 namespace bz {
 
+// vote_median_tma.cu: BZ_OK / error, or 1 when the staged path does not apply
+int vote_median_tma(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* out,
+                    cudaStream_t s);
+
 namespace {
 
 constexpr int kBlock = 128;
+
+// BZ_VOTE_MEDIAN_PATH=registers keeps the fused pass on the register path (for profiling the two
+// against each other); anything else lets the TMA-staged path run where it applies.
+bool staged_path_enabled() {
+    static const bool on = [] {
+        const char* v = std::getenv("BZ_VOTE_MEDIAN_PATH");
+        return !(v != nullptr && std::strcmp(v, "registers") == 0);
+    }();
+    return on;
+}
 
 template <typename V> struct Lanes;
 template <> struct Lanes<uint4> {
@@ -202,7 +219,8 @@ int vote_dispatch(const float* rep, int f, int64_t d, int64_t ld_file, int64_t l
 }
 
 int validate_replicas(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep) {
-    if (rep == nullptr || d < 0 || r < 1 || f < 1 || (r % 2) == 0) return BZ_ERR_INVALID_ARG;
+    if (d < 0 || r < 1 || f < 1 || (r % 2) == 0) return BZ_ERR_INVALID_ARG;
+    if (rep == nullptr && d > 0) return BZ_ERR_INVALID_ARG;  // an empty array may have no address
     if (r > BZ_MAX_R || f > BZ_MAX_F) return BZ_ERR_UNSUPPORTED;
     if (ld_file < d) return BZ_ERR_INVALID_ARG;
     if (r > 1 && ld_rep < d) return BZ_ERR_INVALID_ARG;
@@ -215,6 +233,10 @@ int vote_median_on_device(const float* rep, int r, int f, int64_t d, int64_t ld_
                           cudaStream_t s) {
     const bool vec = aligned16(rep) && aligned16(out) && (ld_file % 4 == 0) && (r == 1 || ld_rep % 4 == 0);
     int st = 1;
+    if (staged_path_enabled()) {
+        st = vote_median_tma(rep, r, f, d, ld_file, ld_rep, out, s);
+        if (st != 1) return st;
+    }
     switch (r) {
         case 1: st = vm_dispatch_f<1>(rep, f, d, ld_file, ld_rep, out, vec, s); break;
         case 3: st = vm_dispatch_f<3>(rep, f, d, ld_file, ld_rep, out, vec, s); break;
@@ -234,7 +256,7 @@ extern "C" int bz_vote_median(const float* replicas, int r, int f, int64_t d, in
                               float* out, void* stream) {
     int st = validate_replicas(replicas, r, f, d, ld_file, ld_replica);
     if (st != BZ_OK) return st;
-    if (out == nullptr) return BZ_ERR_INVALID_ARG;
+    if (out == nullptr && d > 0) return BZ_ERR_INVALID_ARG;
     if (d == 0) return BZ_OK;
     return vote_median_on_device(replicas, r, f, d, ld_file, ld_replica, out, static_cast<cudaStream_t>(stream));
 }
@@ -242,7 +264,7 @@ extern "C" int bz_vote_median(const float* replicas, int r, int f, int64_t d, in
 extern "C" int bz_median(const float* voted, int f, int64_t d, int64_t ld, float* out, void* stream) {
     int st = validate_replicas(voted, 1, f, d, ld, 0);
     if (st != BZ_OK) return st;
-    if (out == nullptr) return BZ_ERR_INVALID_ARG;
+    if (out == nullptr && d > 0) return BZ_ERR_INVALID_ARG;
     if (d == 0) return BZ_OK;
     return vote_median_on_device(voted, 1, f, d, ld, 0, out, static_cast<cudaStream_t>(stream));
 }
@@ -251,7 +273,7 @@ extern "C" int bz_vote(const float* replicas, int r, int f, int64_t d, int64_t l
                        float* voted, int64_t ld_voted, void* stream) {
     int st = validate_replicas(replicas, r, f, d, ld_file, ld_replica);
     if (st != BZ_OK) return st;
-    if (voted == nullptr || ld_voted < d) return BZ_ERR_INVALID_ARG;
+    if ((voted == nullptr && d > 0) || ld_voted < d) return BZ_ERR_INVALID_ARG;
     if (d == 0) return BZ_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool vec = aligned16(replicas) && aligned16(voted) && (ld_file % 4 == 0) && (ld_voted % 4 == 0) &&
@@ -269,7 +291,7 @@ extern "C" int bz_vote_median_host(const float* replicas_host, int r, int f, int
                                    void* workspace, size_t workspace_bytes, void* stream) {
     int st = validate_replicas(replicas_host, r, f, d, d, static_cast<int64_t>(f) * d);
     if (st != BZ_OK) return st;
-    if (out_host == nullptr) return BZ_ERR_INVALID_ARG;
+    if (out_host == nullptr && d > 0) return BZ_ERR_INVALID_ARG;
     if (d == 0) return BZ_OK;
     if (workspace == nullptr || !aligned256(workspace)) return BZ_ERR_WORKSPACE;
     if (workspace_bytes < bz_workspace_bytes(BZ_OP_VOTE_MEDIAN_HOST, r, f, d, 0, 0)) return BZ_ERR_WORKSPACE;

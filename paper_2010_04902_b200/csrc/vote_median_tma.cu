@@ -1,0 +1,229 @@
+// Fused vote + median, staged through shared memory by the TMA unit.
+//
+// One producer thread per CTA issues cp.async.bulk.tensor loads of boxes
+// [R copies][FC files][kTileD coordinates] from a rank-3 tensor map over replicas[r][f][d] into a
+// ring of shared-memory stages; four consumer warps take one coordinate per thread, vote the FC
+// files of a stage straight out of shared memory and keep the winners' order keys in registers.
+// After the last file chunk of a coordinate tile the median network runs and one float is stored.
+// The bytes in flight are set by the ring (stages x ~37 KB per CTA), not by registers, and every
+// replica byte is read from HBM exactly once.  No cluster multicast is used anywhere.
+//
+// Every mbarrier wait is bounded: on expiry the kernel raises g_pipeline_timeouts, stops taking
+// new tiles, drains the loads it has already issued (bounded as well) and returns.
+#include <cuda.h>
+
+#include "bz_common.cuh"
+
+namespace bz {
+
+namespace {
+
+constexpr int kTileD = 128;            // coordinates per tile = consumer threads per CTA
+constexpr int kConsumers = kTileD;
+constexpr int kThreads = kConsumers + 32;
+constexpr uint32_t kSpinLimit = 1u << 20;  // try_wait attempts before a wait is declared dead
+
+__device__ unsigned int g_pipeline_timeouts = 0;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait for the phase with the given parity.  Returns false if the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    const uint32_t addr = smem_u32(bar);
+    for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+        uint32_t done;
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            "selp.u32 %0, 1, 0, p;\n"
+            "}\n"
+            : "=r"(done)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int x, int y, int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
+
+template <int R, int F, int FC> struct Shape {
+    static constexpr int kChunks = (F + FC - 1) / FC;
+    static constexpr int kStageFloats = R * FC * kTileD;
+    static constexpr int kStageBytes = kStageFloats * 4;
+};
+
+// Dynamic shared memory: [STAGES][R][FC][kTileD] floats (each stage 128-byte aligned), then the
+// full/empty barriers.
+template <int R, int F, int FC, int STAGES>
+__global__ void __launch_bounds__(kThreads)
+    vote_median_tma_kernel(const __grid_constant__ CUtensorMap map, int64_t d, float* __restrict__ out) {
+    using S = Shape<R, F, FC>;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    float* stages = reinterpret_cast<float*>(smem_raw);
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + static_cast<size_t>(STAGES) * S::kStageBytes);
+    uint64_t* empty = full + STAGES;
+
+    const int tid = threadIdx.x;
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], kConsumers / 32);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    const int64_t n_tiles = (d + kTileD - 1) / kTileD;
+    const int64_t my_tiles = blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const int64_t n_items = my_tiles * S::kChunks;  // (tile, file chunk) pairs this CTA streams
+
+    if (tid >= kConsumers) {
+        // ---------------------------------------------------------------- producer warp
+        if (tid == kConsumers) {
+            int64_t issued = 0;
+            bool alive = true;
+            for (; issued < n_items && alive; ++issued) {
+                const int s = static_cast<int>(issued % STAGES);
+                const uint32_t round = static_cast<uint32_t>(issued / STAGES);
+                if (round > 0 && !mbar_wait(&empty[s], (round - 1) & 1)) {
+                    alive = false;
+                    break;
+                }
+                const int64_t tile = blockIdx.x + (issued / S::kChunks) * gridDim.x;
+                const int chunk = static_cast<int>(issued % S::kChunks);
+                mbar_expect_tx(&full[s], S::kStageBytes);
+                tma_load_3d(stages + static_cast<size_t>(s) * S::kStageFloats, &map, &full[s],
+                            static_cast<int>(tile * kTileD), chunk * FC, 0);
+            }
+            if (!alive) {
+                atomicAdd(&g_pipeline_timeouts, 1u);
+                // shared memory must outlive the loads already issued: wait for each stage's last load
+                for (int64_t it = issued > STAGES ? issued - STAGES : 0; it < issued; ++it)
+                    mbar_wait(&full[it % STAGES], static_cast<uint32_t>(it / STAGES) & 1);
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- consumers: one coordinate each
+        int key[F];
+        int64_t item = 0;
+        bool alive = true;
+        for (int64_t t = 0; t < my_tiles && alive; ++t) {
+            const int64_t j = (blockIdx.x + t * gridDim.x) * kTileD + tid;
+#pragma unroll
+            for (int chunk = 0; chunk < S::kChunks; ++chunk, ++item) {
+                const int s = static_cast<int>(item % STAGES);
+                if (!mbar_wait(&full[s], static_cast<uint32_t>(item / STAGES) & 1)) {
+                    alive = false;
+                    break;
+                }
+                const uint32_t* base = reinterpret_cast<const uint32_t*>(stages + static_cast<size_t>(s) * S::kStageFloats) + tid;
+#pragma unroll
+                for (int fi = 0; fi < FC; ++fi) {
+                    if (chunk * FC + fi < F) {
+                        uint32_t copies[R];
+#pragma unroll
+                        for (int k = 0; k < R; ++k) copies[k] = base[(k * FC + fi) * kTileD];
+                        key[chunk * FC + fi] = order_key(vote_bits<R>(copies));
+                    }
+                }
+                __syncwarp();
+                if ((tid & 31) == 0) mbar_arrive(&empty[s]);  // this warp is done reading the stage
+            }
+            if (alive && j < d) out[j] = __uint_as_float(key_bits(MedianNet<F>::run(key)));
+        }
+        if (!alive && (tid & 31) == 0) atomicAdd(&g_pipeline_timeouts, 1u);
+    }
+}
+
+// ---- host side ----------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            (void)cudaGetLastError();
+    }
+    return fn;
+}
+
+template <int R, int F, int FC, int STAGES>
+int launch_tma(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, float* out, cudaStream_t s) {
+    using S = Shape<R, F, FC>;
+    EncodeTiledFn enc = encode_tiled();
+    if (enc == nullptr) return 1;
+    CUtensorMap map;
+    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(F), static_cast<cuuint64_t>(R)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(ld_file) * 4, static_cast<cuuint64_t>(R > 1 ? ld_rep : ld_file * F) * 4};
+    const cuuint32_t box[3] = {kTileD, FC, R};
+    const cuuint32_t elem[3] = {1, 1, 1};
+    const CUresult cr = enc(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(rep), dims, strides, box, elem,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return 1;  // shape the descriptor cannot express: use the register path
+    constexpr int smem = STAGES * S::kStageBytes + 2 * STAGES * 8;
+    auto kern = vote_median_tma_kernel<R, F, FC, STAGES>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return cuda_failed(e);
+    constexpr int ctas_per_sm = (227 * 1024) / (smem + 1024) >= 2 ? 2 : 1;
+    int64_t grid = (d + kTileD - 1) / kTileD;
+    if (grid > kNumSMs * ctas_per_sm) grid = kNumSMs * ctas_per_sm;
+    kern<<<static_cast<int>(grid), kThreads, smem, s>>>(map, d, out);
+    note_launch();
+    return check_launch();
+}
+
+}  // namespace
+
+// Returns BZ_OK / an error, or 1 when this path does not apply and the caller should use the
+// register path.  Requirements: 16-byte aligned base, leading dimensions multiples of 4 floats,
+// d below 2^31, a specialised (r, f).
+int vote_median_tma(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* out,
+                    cudaStream_t s) {
+    if (!aligned16(rep) || (ld_file % 4) != 0 || (r > 1 && (ld_rep % 4) != 0) || d >= (int64_t(1) << 31)) return 1;
+    if (d < 4 * kTileD) return 1;  // tiny inputs: not worth a descriptor
+#define BZ_TMA_CASE(R_, F_, FC_, ST_) \
+    if (r == R_ && f == F_) return launch_tma<R_, F_, FC_, ST_>(rep, d, ld_file, ld_rep, out, s);
+    BZ_TMA_CASE(3, 25, 25, 2)
+    BZ_TMA_CASE(3, 49, 25, 2)
+    BZ_TMA_CASE(5, 25, 13, 2)
+    BZ_TMA_CASE(5, 49, 13, 2)
+    BZ_TMA_CASE(7, 49, 10, 2)
+    BZ_TMA_CASE(1, 25, 25, 4)
+    BZ_TMA_CASE(1, 49, 49, 3)
+#undef BZ_TMA_CASE
+    return 1;
+}
+
+int pipeline_timeouts(unsigned int* count) {
+    const cudaError_t e = cudaMemcpyFromSymbol(count, g_pipeline_timeouts, sizeof(unsigned int));
+    return e == cudaSuccess ? BZ_OK : cuda_failed(e);
+}
+
+}  // namespace bz

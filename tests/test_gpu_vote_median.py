@@ -121,6 +121,38 @@ def test_host_entry_point():
     assert np.array_equal(_bits(out2), _bits(want))
 
 
+_REGISTER_PATH_SCRIPT = r"""
+import numpy as np, torch, oracle
+from paper_2010_04902_b200 import binding as bz, inputs
+n0 = bz.kernel_launch_count()
+for (l, r, q, attack, d) in [(5, 3, 3, "reversed", 70001), (7, 3, 5, "alie", 33333), (5, 5, 6, "constant", 20480),
+                             (7, 7, 9, "reversed", 9999)]:
+    wf, fw, _ = oracle.assign(l, r)
+    byz = oracle.worst_case(wf, l * l, r, q)[1]
+    rep = inputs.build_replicas(inputs.true_gradients(l * l, d, seed=2), fw, byz, attack)
+    got = bz.vote_median(rep.cuda()).cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), oracle.vote_median(rep.numpy()).view(np.uint32)), (l, r)
+assert bz.pipeline_timeouts() == 0
+print("register path ok", bz.kernel_launch_count() - n0)
+"""
+
+
+def test_register_path_at_sizes_the_staged_path_normally_takes():
+    # the fused pass has two implementations; the environment switch pins the register one
+    import os
+    import subprocess
+    import sys
+    from conftest import ROOT
+    env = dict(os.environ, BZ_VOTE_MEDIAN_PATH="registers", PYTHONPATH=ROOT)
+    res = subprocess.run([sys.executable, "-c", _REGISTER_PATH_SCRIPT], env=env, cwd=ROOT, capture_output=True, text=True)
+    assert res.returncode == 0 and "register path ok" in res.stdout, res.stdout + res.stderr
+
+
+def test_no_barrier_wait_ran_out():
+    # after everything above: the staged kernels' bounded waits never expired
+    assert bz.pipeline_timeouts() == 0
+
+
 def _sampled_columns(d, n, rng):
     return np.unique(np.concatenate([np.arange(0, 600), np.arange(d - 600, d), rng.integers(0, d, size=n)]))
 
