@@ -145,6 +145,8 @@ def run_ours(args):
     bz.lib()
 
     cfg = dict(WORKLOAD)
+    if args.coords > 0:
+        cfg["d"] = args.coords
     l, r, d = cfg["l"], cfg["r"], cfg["d"]
     f = l * l
     rep, fw, byz, cmax = make_inputs(bz, inputs, torch, cfg, device, seed_offset=rank)
@@ -369,6 +371,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the multi-Krum / Bulyan / worst-case extras")
+    ap.add_argument("--coords", type=int, default=0,
+                    help="profiling only: override the number of coordinates d (the JSON line then names the smaller workload)")
+    ap.add_argument("--no-e2e", action="store_true", help="profiling only: skip the host-buffer leg")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

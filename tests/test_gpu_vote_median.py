@@ -39,7 +39,7 @@ def _check_all(rep_cpu, rep_dev=None):
 # sizes: below one vector, ragged tails, several CTAs' worth with a ragged tail
 @pytest.mark.parametrize("d", [1, 3, 4, 5, 127, 1025, 70001])
 @pytest.mark.parametrize("l,r,q,attack", [(5, 3, 3, "reversed"), (5, 5, 6, "constant"), (7, 3, 5, "alie"),
-                                          (7, 5, 6, "alie"), (7, 7, 9, "reversed"), (3, 3, 2, "constant")])
+                                          (7, 5, 6, "alie"), (7, 7, 5, "reversed"), (3, 3, 2, "constant")])
 def test_parity_specialised_and_generic_shapes(l, r, q, attack, d):
     _check_all(_cluster(l, r, q, d, attack))
 
@@ -126,7 +126,7 @@ import numpy as np, torch, oracle
 from paper_2010_04902_b200 import binding as bz, inputs
 n0 = bz.kernel_launch_count()
 for (l, r, q, attack, d) in [(5, 3, 3, "reversed", 70001), (7, 3, 5, "alie", 33333), (5, 5, 6, "constant", 20480),
-                             (7, 7, 9, "reversed", 9999)]:
+                             (7, 7, 5, "reversed", 9999)]:
     wf, fw, _ = oracle.assign(l, r)
     byz = oracle.worst_case(wf, l * l, r, q)[1]
     rep = inputs.build_replicas(inputs.true_gradients(l * l, d, seed=2), fw, byz, attack)
