@@ -45,6 +45,7 @@ extern "C" {
 #define BZ_ERR_WORKSPACE (-4)    /* workspace missing, misaligned (256 B) or too small               */
 #define BZ_ERR_BUDGET (-5)       /* C(K, q) exceeds max_subsets                                      */
 #define BZ_ERR_CUDA (-6)         /* a CUDA runtime call or launch failed                             */
+#define BZ_ERR_STATIC_LIMIT (-7) /* the shape needs more scratch than the built-in array holds       */
 
 #define BZ_MAX_R 15
 #define BZ_MAX_F 128
@@ -116,6 +117,30 @@ int bz_vote_median_host(const float* replicas_host, int r, int f, int64_t d, flo
  */
 int bz_pairdist(const float* voted, int f, int64_t d, int64_t ld, double* dist, void* workspace,
                 size_t workspace_bytes, void* stream);
+
+/*
+ * bz_pairdist for callers that have no device workspace to offer and may not allocate one.
+ * (The paper has no counterpart to this call; it exists for the library's users.)  Such callers
+ * are, for instance, an operator embedded in a framework that fixes its memory plan before the
+ * run, a serving or training loop that cannot afford the device-wide synchronisation an
+ * allocation may cause, or a tenant of a shared GPU held to a fixed memory budget.  They pass
+ * inputs and outputs only; the partial sums go to an array of BZ_STATIC_SCRATCH_BYTES that is part
+ * of the library image, so every GPU that loads the library holds those 4 MiB until the process
+ * exits.  The call itself allocates and frees nothing.
+ *   - Results are those of bz_pairdist (same kernels, same summation order).
+ *   - Shapes whose scratch need, bz_workspace_bytes(BZ_OP_PAIRDIST, 0, f, d, 0, 0), exceeds the
+ *     array are refused with BZ_ERR_STATIC_LIMIT before anything runs: f = 25 fits, f = 49 (about
+ *     13 MB) does not, other f fit up to 84.
+ *   - The first call on each device looks up the array's device address (the device must be
+ *     current, as for every call).  Make that first call outside any stream capture.
+ *   - All calls share the one array and it keeps the previous call's contents.  The kernels
+ *     overwrite or clear every element before reading it, so successive calls on one stream are
+ *     independent; two calls that overlap on the GPU (different streams, several host threads)
+ *     race on the array and must be serialised by the caller.
+ *   voted device [f][d] with ld;  dist device double [f][f].
+ */
+#define BZ_STATIC_SCRATCH_BYTES (4u << 20)
+int bz_pairdist_static(const float* voted, int f, int64_t d, int64_t ld, double* dist, void* stream);
 
 /*
  * Multi-Krum selection on a distance matrix (Sec. 1.2: the gradient closest to its nearest

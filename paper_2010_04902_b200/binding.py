@@ -42,6 +42,7 @@ _SIGNATURES = {
     "bz_vote_median": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_vp]),
     "bz_vote_median_host": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_vp, _c_vp, _c_sz, _c_vp]),
     "bz_pairdist": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_vp, _c_sz, _c_vp]),
+    "bz_pairdist_static": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_vp]),
     "bz_krum_select": (_c_int, [_c_vp, _c_int, _c_int, _c_int, _c_vp, _c_vp]),
     "bz_mean_rows": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_int, _c_vp, _c_vp]),
     "bz_multikrum": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_int, _c_int, _c_vp, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp]),
@@ -218,6 +219,23 @@ def pairdist(voted: torch.Tensor, workspace: torch.Tensor | None = None, dist: t
     st = lib().bz_pairdist(_dev(voted, torch.float32, "voted"), f, d, ld, _dev(dist, torch.float64, "dist"),
                            ws.data_ptr(), ws.numel(), _stream())
     _check(st, "bz_pairdist")
+    return dist
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+ERR_STATIC_LIMIT = -7
+
+
+def pairdist_static(voted: torch.Tensor, dist: torch.Tensor) -> torch.Tensor:
+    """bz_pairdist_static: the distance matrix for a caller that cannot supply (or allocate) a device
+    workspace - for example code running under a frozen memory plan or a fixed memory budget.  The
+    scratch is a 4 MiB array inside the library; `dist` ([f][f] float64) must already exist.  Shapes
+    that need more scratch (f = 49, f > 84) raise with status ERR_STATIC_LIMIT.  Calls share that
+    array: do not let two of them run on the GPU at the same time."""
+    f, d, ld = _rows(voted, "voted")
+    st = lib().bz_pairdist_static(_dev(voted, torch.float32, "voted"), f, d, ld, _dev(dist, torch.float64, "dist"),
+                                  _stream())
+    _check(st, "bz_pairdist_static")
     return dist
 
 

@@ -95,6 +95,7 @@ extern "C" const char* bz_status_string(int status) {
         case BZ_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case BZ_ERR_BUDGET: return "number of subsets exceeds the budget";
         case BZ_ERR_CUDA: return "CUDA runtime error";
+        case BZ_ERR_STATIC_LIMIT: return "shape needs more scratch than the library's built-in array holds";
         default: return "unknown status";
     }
 }

@@ -607,3 +607,53 @@ extern "C" int bz_bulyan(const float* voted, int f, int64_t d, int64_t ld, int c
     const int theta = f - 2 * c;
     return trimmed_mean_on_device(voted, d, ld, selected, theta, theta - 2 * c, out, s);
 }
+
+// ------------------------------------------------------------------------------------------------
+// Pairwise distances without a caller workspace.
+//
+// Some hosts of this library may not allocate device memory at the moment they need the distance
+// matrix: an operator plugged into a framework whose memory plan is frozen before the run, a
+// serving or training loop that must not take the implicit device synchronisation an allocation
+// can bring, a process confined to a fixed memory budget on a shared GPU.  For them the partial
+// sums that bz_pairdist keeps in the caller's workspace live in the array below, which every GPU
+// that loads the library holds from load to exit.
+namespace {
+
+constexpr size_t kStaticScratchBytes = BZ_STATIC_SCRATCH_BYTES;  // 4 MiB
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {};  // device address of the array on each device, once resolved
+
+// The array's name is only a handle on the host side; kernels need its device address, which the
+// runtime hands out per device.
+int static_scratch(void** ptr) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_failed(e);
+    if (dev < 0 || dev >= kMaxDevices) return BZ_ERR_UNSUPPORTED;
+    if (g_static_scratch_addr[dev] == nullptr) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return cuda_failed(e);
+        if (p == nullptr || !aligned256(p)) return BZ_ERR_WORKSPACE;
+        g_static_scratch_addr[dev] = p;
+    }
+    *ptr = g_static_scratch_addr[dev];
+    return BZ_OK;
+}
+
+}  // namespace
+
+extern "C" int bz_pairdist_static(const float* voted, int f, int64_t d, int64_t ld, double* dist, void* stream) {
+    int st = validate_rows(voted, f, d, ld);
+    if (st != BZ_OK) return st;
+    if (dist == nullptr) return BZ_ERR_INVALID_ARG;
+    if (krum_workspace_bytes(BZ_OP_PAIRDIST, f) > kStaticScratchBytes) return BZ_ERR_STATIC_LIMIT;
+    void* scratch = nullptr;
+    st = static_scratch(&scratch);
+    if (st != BZ_OK) return st;
+    // Nothing in the array has to start at zero: the tiled kernel overwrites every partial sum the
+    // reduction reads, and the generic kernel clears its own slots before it accumulates.
+    return pairdist_on_device(voted, f, d, ld, dist, scratch, static_cast<cudaStream_t>(stream));
+}
