@@ -7,6 +7,8 @@ replicated file gradients: K = 15 workers, r = 3, l = 5, f = 25 files, d = 11.2 
 q = 3 Byzantine workers at the worst-case placement sending -100 x the true gradient.
 With N > 1 (torchrun) every rank aggregates its own coordinate slab of the same size; the path needs
 no collective.  Rank 0 prints ONE JSON line.  `--impl reference` times the CPU checker instead.
+`--coords`, `--no-e2e`, `--no-cpu` shrink the run for profiler captures; their JSON line names the
+smaller workload and is not a benchmark value.
 """
 from __future__ import annotations
 
@@ -25,8 +27,16 @@ if ROOT not in sys.path:
 METRIC = "aggregated gradient coordinates/sec (fused vote+median)"
 UNIT = "coordinates/s"
 WORKLOAD = dict(l=5, r=3, q=3, d=11_200_000, attack="reversed", seed=0)
-WORKLOAD_NAME = ("K=15 r=3 l=5 f=25 d=11.2M fp32, q=3 Byzantine (worst-case placement) sending -100 x gradient; "
-                 "fused vote + coordinate-wise median")
+
+# DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum, scaled to a full launch), or None when no capture of the current kernel exists.
+TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def workload_name(cfg):
+    return ("K=%d r=%d l=%d f=%d d=%s fp32, q=%d Byzantine (worst-case placement) sending -100 x gradient; "
+            "fused vote + coordinate-wise median" % (cfg["r"] * cfg["l"], cfg["r"], cfg["l"], cfg["l"] ** 2,
+                                                     ("%.1fM" % (cfg["d"] / 1e6)), cfg["q"]))
 
 
 def log(*a):
@@ -37,7 +47,7 @@ def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(path) as fh:
-            return float(json.load(fh)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+            return float(json.load(fh)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy read+write)"
     except Exception:
         return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
@@ -95,7 +105,7 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def make_inputs(bz, inputs, torch, cfg, device, seed_offset=0, heavy=0.0):
+def make_inputs(bz, inputs, cfg, device, seed_offset=0, heavy=0.0):
     """Assignment and Byzantine set through the library, synthetic replicas on the device."""
     l, r, q, d = cfg["l"], cfg["r"], cfg["q"], cfg["d"]
     _, fw, mask = bz.assign_mols(l, r)
@@ -118,6 +128,31 @@ def timed(torch, fn, steps, warmup):
     e1.record()
     torch.cuda.synchronize()
     return e0.elapsed_time(e1) / steps
+
+
+def e2e_leg(bz, torch, dist, world, rep, out, device, steps):
+    """The same aggregation through the host entry point: pinned host buffers, copies inside the timing."""
+    r, f, d = rep.shape
+    rep_host = torch.empty((r, f, d), dtype=torch.float32, pin_memory=True)
+    rep_host.copy_(rep)
+    out_host = torch.empty(d, dtype=torch.float32, pin_memory=True)
+    ws = torch.empty((r * f + 1) * ((d + 63) // 64 * 64) * 4 + 256, dtype=torch.uint8, device=device)
+    step = lambda: bz.vote_median_host(rep_host, out_host, ws)
+    step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    n = max(2, min(5, steps))
+    t0 = time.perf_counter()
+    for _ in range(n):
+        step()
+    torch.cuda.synchronize()
+    secs = torch.tensor([(time.perf_counter() - t0) / n], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(secs, op=dist.ReduceOp.MAX)
+    matches = bool(torch.equal(out_host.to(device), out))
+    return {"value": world * d / float(secs.item()), "unit": UNIT, "h2d_bytes_per_step": r * f * d * 4,
+            "d2h_bytes_per_step": d * 4, "steps": n, "matches_device_result": matches}, rep_host
 
 
 def run_ours(args):
@@ -149,7 +184,7 @@ def run_ours(args):
         cfg["d"] = args.coords
     l, r, d = cfg["l"], cfg["r"], cfg["d"]
     f = l * l
-    rep, fw, byz, cmax = make_inputs(bz, inputs, torch, cfg, device, seed_offset=rank)
+    rep, fw, byz, cmax = make_inputs(bz, inputs, cfg, device, seed_offset=rank)
     out = torch.empty(d, dtype=torch.float32, device=device)
     step = lambda: bz.vote_median(rep, out)
 
@@ -178,74 +213,55 @@ def run_ours(args):
     ms_step = float(ms_total.item()) / args.steps
     value = world * d / (ms_step * 1e-3)
 
-    # ---- end to end through the host entry point: pinned host buffers, copies inside the timing -------
-    h2d = r * f * d * 4
-    d2h = d * 4
-    rep_host = torch.empty((r, f, d), dtype=torch.float32, pin_memory=True)
-    rep_host.copy_(rep)
-    out_host = torch.empty(d, dtype=torch.float32, pin_memory=True)
-    ws = torch.empty((r * f + 1) * ((d + 63) // 64 * 64) * 4 + 256, dtype=torch.uint8, device=device)
-    e2e_step = lambda: bz.vote_median_host(rep_host, out_host, ws)
-    e2e_step()
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    e2e_steps = max(2, min(5, args.steps))
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        e2e_step()
-    torch.cuda.synchronize()
-    e2e_s = torch.tensor([(time.perf_counter() - t0) / e2e_steps], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(e2e_s, op=dist.ReduceOp.MAX)
-    e2e_value = world * d / float(e2e_s.item())
-    e2e_matches = bool(torch.equal(out_host.to(device), out))
-    del ws
+    e2e, rep_host = (None, None)
+    if not args.no_e2e:
+        e2e, rep_host = e2e_leg(bz, torch, dist, world, rep, out, device, args.steps)
 
     result = None
     if rank == 0:
         peak, peak_src = measured_peaks()
         alg_bytes = (4 * r * f + 4) * d
         achieved = alg_bytes / (ms_step * 1e-3) / 1e9
+        traffic = TRAFFIC_BYTES_PER_LAUNCH if args.coords == 0 else None
         result = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32",
             "data": "synthetic",
-            "config": {"workload": WORKLOAD_NAME, "coordinates_per_gpu": d, "c_max": cmax,
+            "config": {"workload": workload_name(cfg), "coordinates_per_gpu": d, "c_max": cmax,
                        "byzantine_workers": [int(u) for u in byz],
-                       "l2": "inputs are 3.36 GB per step, far larger than the 126 MB L2; no flush needed",
+                       "l2": "inputs are %.2f GB per step, far larger than the 126 MB L2; no flush needed" % (4 * r * f * d / 1e9),
                        "parallelism": "coordinate slabs, no collective" if world > 1 else "single GPU"},
             "clocks": sampler.summary(),
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "steps": e2e_steps, "matches_device_result": e2e_matches},
+            "e2e": e2e,
             "gpu_launches": int(launches),
+            "pipeline_timeouts": bz.pipeline_timeouts(),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": TRAFFIC_BYTES_PER_LAUNCH, "peak_source": peak_src,
-                         "frac_of_nominal_8TBs": achieved / 8000.0, "algorithmic_bytes_per_launch": alg_bytes,
-                         "kernel": "vote_median_kernel<3,25>"},
+                         "traffic": traffic, "peak_source": peak_src, "frac_of_nominal_8TBs": achieved / 8000.0,
+                         "algorithmic_bytes_per_launch": alg_bytes,
+                         "kernel": "vote_median_tma_kernel<3,25,25,2> (one launch per step)"},
         }
 
     # ---- CPU baseline and parity of the timed output (single-GPU run only) ----------------------------
-    if rank == 0 and world == 1:
+    if rank == 0 and world == 1 and not args.no_cpu:
         import oracle
         cores = oracle.num_threads()
-        probe = rep[:, :, :200_000].cpu().numpy()
+        probe = rep[:, :, :min(d, 200_000)].cpu().numpy()
         t0 = time.perf_counter()
         oracle.vote_median(probe)
-        rate = 200_000 / (time.perf_counter() - t0)
+        rate = probe.shape[2] / (time.perf_counter() - t0)
         n_sample = int(min(d, max(200_000, rate * 15.0)))
-        sample = rep_host[:, :, :n_sample].contiguous().numpy()
+        sample = (rep_host[:, :, :n_sample] if rep_host is not None else rep[:, :, :n_sample].cpu()).contiguous().numpy()
         t0 = time.perf_counter()
         want = oracle.vote_median(sample)
         dt = time.perf_counter() - t0
         got = out[:n_sample].cpu().numpy()
         parity = bool(np.array_equal(got.view(np.uint32), want.view(np.uint32)))
         result["cpu_baseline"] = {"value": n_sample / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                  "sample": "first %d of %d coordinates of the same replicas (all 75 rows)" % (n_sample, d)}
+                                  "sample": "first %d of %d coordinates of the same replicas (all %d rows)" % (n_sample, d, r * f)}
         result["parity"] = {"bit_exact_vs_oracle_on_sample": parity, "sample_coordinates": n_sample}
         if not parity:
             raise RuntimeError("bench output differs from the CPU checker")
-    del rep_host, out_host, rep, out
+    del rep_host, rep, out
     torch.cuda.empty_cache()
 
     if rank == 0 and world == 1 and not args.no_extra:
@@ -258,63 +274,68 @@ def run_ours(args):
         print(json.dumps(result), flush=True)
 
 
-# DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum), or None when no capture of the current kernel exists.
-TRAFFIC_BYTES_PER_LAUNCH = None
-
-
 def extra_paths(bz, inputs, torch, device):
     """The other aggregators at their own configurations (not part of the headline value)."""
     res = {}
     peak, _ = measured_peaks()
+
+    def hbm(nbytes, ms):
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        return {"achieved_GBs": gbs, "frac_of_measured_hbm": gbs / peak}
+
     # vote -> multi-Krum: K=21, r=3, l=7, f=49, d=11.2M, q=5 ALIE, c=5, m=44
     cfg = dict(l=7, r=3, q=5, d=11_200_000, attack="alie", seed=0)
-    rep, fw, byz, cmax = make_inputs(bz, inputs, torch, cfg, device)
+    rep, fw, byz, cmax = make_inputs(bz, inputs, cfg, device)
     f, d, r = 49, cfg["d"], 3
     voted = torch.empty((f, d), dtype=torch.float32, device=device)
     out = torch.empty(d, dtype=torch.float32, device=device)
     ws = bz.alloc_workspace(bz.OP_MULTIKRUM, 0, f, d, 5, 44, device=device)
+    sel44 = torch.arange(44, dtype=torch.int32, device=device)
     t_vote = timed(torch, lambda: bz.vote(rep, voted), 5, 2)
     t_pd = timed(torch, lambda: bz.pairdist(voted, ws), 5, 2)
+    t_mean = timed(torch, lambda: bz.mean_rows(voted, sel44, out), 5, 2)
     t_mk = timed(torch, lambda: bz.multikrum(voted, 5, 44, workspace=ws, out=out), 5, 2)
     t_vm = timed(torch, lambda: bz.vote_median(rep, out), 5, 2)
+    t_med = timed(torch, lambda: bz.median(voted, out), 5, 2)
     bytes_pipeline = (4 * r * f + 4 * f + 4 * f + 4 * 44 + 4) * d
-    res["vote+multikrum"] = {
-        "workload": "K=21 r=3 l=7 f=49 d=11.2M, q=5 ALIE, c=5 m=44", "c_max": cmax,
-        "coordinates_per_s": d / ((t_vote + t_mk) * 1e-3), "ms_vote": t_vote, "ms_multikrum": t_mk, "ms_pairdist": t_pd,
-        "pairdist_fma_lane_ops_per_s": 2 * (f * (f - 1) // 2) * d / (t_pd * 1e-3),
-        "achieved_GBs": bytes_pipeline / ((t_vote + t_mk) * 1e-3) / 1e9, "frac_of_measured_hbm": bytes_pipeline / ((t_vote + t_mk) * 1e-3) / 1e9 / peak,
-    }
-    res["vote+median f=49"] = {"workload": "same replicas, fused vote+median", "ms": t_vm,
-                               "coordinates_per_s": d / (t_vm * 1e-3),
-                               "achieved_GBs": (4 * r * f + 4) * d / (t_vm * 1e-3) / 1e9,
-                               "frac_of_measured_hbm": (4 * r * f + 4) * d / (t_vm * 1e-3) / 1e9 / peak}
+    res["vote+multikrum"] = dict(
+        workload="K=21 r=3 l=7 f=49 d=11.2M, q=5 ALIE, c=5 m=44", c_max=cmax,
+        coordinates_per_s=d / ((t_vote + t_mk) * 1e-3), ms_vote=t_vote, ms_multikrum=t_mk, ms_pairdist=t_pd,
+        ms_mean_rows=t_mean, pairdist_fma_lane_ops_per_s=2 * (f * (f - 1) // 2) * d / (t_pd * 1e-3),
+        vote=hbm((4 * r * f + 4 * f) * d, t_vote), mean_rows=hbm((4 * 44 + 4) * d, t_mean),
+        pipeline=hbm(bytes_pipeline, t_vote + t_mk))
+    res["vote+median f=49"] = dict(workload="same replicas, fused vote+median", ms=t_vm, coordinates_per_s=d / (t_vm * 1e-3),
+                                   **hbm((4 * r * f + 4) * d, t_vm))
+    res["median f=49"] = dict(workload="median of the 49 voted rows", ms=t_med, coordinates_per_s=d / (t_med * 1e-3),
+                              **hbm((4 * f + 4) * d, t_med))
     del rep, voted, out, ws
     torch.cuda.empty_cache()
+
     # vote -> Bulyan: K=25, r=5, l=5, f=25, d=25M heavy-tailed, q=6 constant, c=4
     cfg = dict(l=5, r=5, q=6, d=25_000_000, attack="constant", seed=0)
-    rep, fw, byz, cmax = make_inputs(bz, inputs, torch, cfg, device, heavy=0.01)
+    rep, fw, byz, cmax = make_inputs(bz, inputs, cfg, device, heavy=0.01)
     f, d, r = 25, cfg["d"], 5
     voted = torch.empty((f, d), dtype=torch.float32, device=device)
     out = torch.empty(d, dtype=torch.float32, device=device)
     ws = bz.alloc_workspace(bz.OP_BULYAN, 0, f, d, 4, device=device)
+    sel17 = torch.arange(17, dtype=torch.int32, device=device)
     t_vote = timed(torch, lambda: bz.vote(rep, voted), 5, 2)
+    t_pd = timed(torch, lambda: bz.pairdist(voted, ws), 5, 2)
+    t_tm = timed(torch, lambda: bz.trimmed_mean(voted, sel17, 9, out), 5, 2)
     t_bu = timed(torch, lambda: bz.bulyan(voted, 4, workspace=ws, out=out), 5, 2)
     t_vm = timed(torch, lambda: bz.vote_median(rep, out), 5, 2)
     theta = f - 8
     bytes_pipeline = (4 * r * f + 4 * f + 4 * f + 4 * theta + 4) * d
-    res["vote+bulyan"] = {
-        "workload": "K=25 r=5 l=5 f=25 d=25M (1% Student-t coordinates), q=6 constant, c=4 (theta=17, beta=9)",
-        "c_max": cmax, "coordinates_per_s": d / ((t_vote + t_bu) * 1e-3), "ms_vote": t_vote, "ms_bulyan": t_bu,
-        "achieved_GBs": bytes_pipeline / ((t_vote + t_bu) * 1e-3) / 1e9,
-        "frac_of_measured_hbm": bytes_pipeline / ((t_vote + t_bu) * 1e-3) / 1e9 / peak,
-    }
-    res["vote+median r=5"] = {"workload": "same replicas, fused vote+median", "ms": t_vm,
-                              "coordinates_per_s": d / (t_vm * 1e-3),
-                              "achieved_GBs": (4 * r * f + 4) * d / (t_vm * 1e-3) / 1e9,
-                              "frac_of_measured_hbm": (4 * r * f + 4) * d / (t_vm * 1e-3) / 1e9 / peak}
+    res["vote+bulyan"] = dict(
+        workload="K=25 r=5 l=5 f=25 d=25M (1% Student-t coordinates), q=6 constant, c=4 (theta=17, beta=9)",
+        c_max=cmax, coordinates_per_s=d / ((t_vote + t_bu) * 1e-3), ms_vote=t_vote, ms_bulyan=t_bu, ms_pairdist=t_pd,
+        ms_trimmed_mean=t_tm, vote=hbm((4 * r * f + 4 * f) * d, t_vote), pairdist=hbm(4 * f * d, t_pd),
+        trimmed_mean=hbm((4 * theta + 4) * d, t_tm), pipeline=hbm(bytes_pipeline, t_vote + t_bu))
+    res["vote+median r=5"] = dict(workload="same replicas, fused vote+median", ms=t_vm, coordinates_per_s=d / (t_vm * 1e-3),
+                                  **hbm((4 * r * f + 4) * d, t_vm))
     del rep, voted, out, ws
     torch.cuda.empty_cache()
+
     # exhaustive worst case: (K, f, l, r) = (35, 49, 7, 5), q = 13 - the largest row the paper printed
     _, _, mask = bz.assign_mols(7, 5)
     ws = bz.alloc_workspace(bz.OP_WORST_CASE, 5, 49)
@@ -323,8 +344,8 @@ def extra_paths(bz, inputs, torch, device):
     t0 = time.perf_counter()
     cmax, arg, n = bz.worst_case(mask, 49, 5, 13, workspace=ws)
     dt = time.perf_counter() - t0
-    res["worst_case"] = {"workload": "(K,f,l,r)=(35,49,7,5), q=13, all C(35,13) subsets", "c_max": cmax,
-                         "subsets": n, "seconds": dt, "subsets_per_s": n / dt, "argmax": [int(u) for u in arg]}
+    res["worst_case"] = dict(workload="(K,f,l,r)=(35,49,7,5), q=13, all C(35,13) subsets", c_max=cmax, subsets=n,
+                             seconds=dt, subsets_per_s=n / dt, argmax=[int(u) for u in arg])
     return res
 
 
@@ -333,8 +354,6 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    import torch
-
     import oracle
     from paper_2010_04902_b200 import inputs
     cfg = dict(WORKLOAD)
@@ -358,7 +377,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u32", "data": "synthetic",
-        "config": {"workload": WORKLOAD_NAME, "sample": sample},
+        "config": {"workload": workload_name(cfg), "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }), flush=True)
@@ -371,9 +390,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the multi-Krum / Bulyan / worst-case extras")
-    ap.add_argument("--coords", type=int, default=0,
-                    help="profiling only: override the number of coordinates d (the JSON line then names the smaller workload)")
+    ap.add_argument("--coords", type=int, default=0, help="profiling only: override the number of coordinates d")
     ap.add_argument("--no-e2e", action="store_true", help="profiling only: skip the host-buffer leg")
+    ap.add_argument("--no-cpu", action="store_true", help="profiling only: skip the CPU baseline / parity leg")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
