@@ -129,8 +129,8 @@ int bz_pairdist(const float* voted, int f, int64_t d, int64_t ld, double* dist, 
  * exits.  The call itself allocates and frees nothing.
  *   - Results are those of bz_pairdist (same kernels, same summation order).
  *   - Shapes whose scratch need, bz_workspace_bytes(BZ_OP_PAIRDIST, 0, f, d, 0, 0), exceeds the
- *     array are refused with BZ_ERR_STATIC_LIMIT before anything runs: f = 25 fits, f = 49 (about
- *     13 MB) does not, other f fit up to 84.
+ *     array are refused with BZ_ERR_STATIC_LIMIT before anything runs: f = 25 (0.9 MB) and f = 49
+ *     (1.6 MB) fit, any other f fits up to 84; f from 85 to BZ_MAX_F is refused.
  *   - The first call on each device looks up the array's device address (the device must be
  *     current, as for every call).  Make that first call outside any stream capture.
  *   - All calls share the one array and it keeps the previous call's contents.  The kernels

@@ -230,7 +230,7 @@ def pairdist_static(voted: torch.Tensor, dist: torch.Tensor) -> torch.Tensor:
     """bz_pairdist_static: the distance matrix for a caller that cannot supply (or allocate) a device
     workspace - for example code running under a frozen memory plan or a fixed memory budget.  The
     scratch is a 4 MiB array inside the library; `dist` ([f][f] float64) must already exist.  Shapes
-    that need more scratch (f = 49, f > 84) raise with status ERR_STATIC_LIMIT.  Calls share that
+    that need more scratch (f > 84) raise with status ERR_STATIC_LIMIT.  Calls share that
     array: do not let two of them run on the GPU at the same time."""
     f, d, ld = _rows(voted, "voted")
     st = lib().bz_pairdist_static(_dev(voted, torch.float32, "voted"), f, d, ld, _dev(dist, torch.float64, "dist"),

@@ -1,204 +1,18 @@
-// The Krum family on the f voted gradients: pairwise squared distances, Multi-Krum selection and
-// mean, Bulyan's iterated selection and its trimmed mean around the median (Sec. 1.2, Sec. 6.1).
+// The Krum family on the f voted gradients (Sec. 1.2, Sec. 6.1): Multi-Krum selection and mean,
+// Bulyan's iterated selection and its trimmed mean around the median, and the end-to-end calls.
+// The pairwise distances they start from are in pairdist.cu.
 #include "bz_common.cuh"
 
 namespace bz {
 
+// pairdist.cu
+size_t pairdist_workspace(int f);
+size_t krum_workspace_bytes(int op, int f);
+int pairdist_on_device(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, cudaStream_t s);
+int validate_rows(const float* v, int f, int64_t d, int64_t ld);
+int check_workspace(void* ws, size_t have, size_t need);
+
 namespace {
-
-// ------------------------------------------------------------------------------------------------
-// Pairwise distances, register-tiled.  The f rows are split into NB = F/T residue classes; a thread
-// owns one unordered pair of classes (bi <= bj), i.e. the T x T row pairs (bi + NB*t, bj + NB*t'),
-// and one of G interleaved coordinate groups of every tile.  A CTA streams tiles of TD coordinates
-// of all F rows through a double-buffered shared-memory stage (cp.async, 16 bytes per request).
-// Sums: binary32 inside one tile (TD / G coordinates per thread), binary64 across tiles, then one
-// fixed-order reduction over CTAs and groups - bit-reproducible from run to run.
-template <int F, int T> struct PairTile {
-    static constexpr int NB = F / T;
-    static constexpr int NPB = NB * (NB + 1) / 2;
-    static_assert(NB * T == F, "T must divide F");
-};
-
-constexpr int kTD = 256;        // coordinates per tile
-constexpr int kRowPad = 4;      // floats; keeps the row stride an odd number of 16-byte units
-constexpr int kRowStride = kTD + kRowPad;
-
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src, int src_bytes) {
-    const unsigned dst = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(gmem_src), "r"(src_bytes));
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
-
-template <int F, int T, int G>
-__global__ void __launch_bounds__(PairTile<F, T>::NPB* G)
-    pairdist_tiled_kernel(const float* __restrict__ v, int64_t d, int64_t ld, double* __restrict__ partial) {
-    using PT = PairTile<F, T>;
-    constexpr int NB = PT::NB, NPB = PT::NPB, NT = NPB * G;
-    extern __shared__ __align__(16) float smem[];
-    float* stage[2] = {smem, smem + F * kRowStride};
-
-    const int tid = threadIdx.x;
-    const int pb = tid % NPB, g = tid / NPB;
-    int bi = 0, bj = 0;
-    {
-        int rest = pb;
-        while (rest >= NB - bi) {
-            rest -= NB - bi;
-            ++bi;
-        }
-        bj = bi + rest;
-    }
-
-    const int64_t n_tiles = (d + kTD - 1) / kTD;
-    auto load_tile = [&](int buf, int64_t tile) {
-        const int64_t j0 = tile * kTD;
-        constexpr int per_row = kTD / 4;
-        for (int idx = tid; idx < F * per_row; idx += NT) {
-            const int row = idx / per_row, c4 = idx - row * per_row;
-            const int64_t j = j0 + 4 * c4;
-            const int64_t left = d - j;
-            const int bytes = left >= 4 ? 16 : (left > 0 ? static_cast<int>(left) * 4 : 0);
-            const float* src = bytes ? v + row * ld + j : v;  // zero-byte requests still name a valid address
-            cp_async16(stage[buf] + row * kRowStride + 4 * c4, src, bytes);
-        }
-        cp_async_commit();
-    };
-
-    double dacc[T * T];
-#pragma unroll
-    for (int e = 0; e < T * T; ++e) dacc[e] = 0.0;
-
-    int64_t tile = blockIdx.x;
-    int buf = 0;
-    if (tile < n_tiles) load_tile(0, tile);
-    for (; tile < n_tiles; tile += gridDim.x) {
-        const int64_t next = tile + gridDim.x;
-        if (next < n_tiles) {
-            load_tile(buf ^ 1, next);
-            cp_async_wait<1>();
-        } else {
-            cp_async_wait<0>();
-        }
-        __syncthreads();
-
-        float acc[T * T];
-#pragma unroll
-        for (int e = 0; e < T * T; ++e) acc[e] = 0.f;
-        const float* base = stage[buf];
-#pragma unroll 1
-        for (int c4 = g; c4 < kTD / 4; c4 += G) {
-            float4 a[T], b[T];
-#pragma unroll
-            for (int t = 0; t < T; ++t) {
-                a[t] = *reinterpret_cast<const float4*>(base + (bi + NB * t) * kRowStride + 4 * c4);
-                b[t] = *reinterpret_cast<const float4*>(base + (bj + NB * t) * kRowStride + 4 * c4);
-            }
-#pragma unroll
-            for (int t = 0; t < T; ++t)
-#pragma unroll
-                for (int u = 0; u < T; ++u) {
-                    float s = acc[t * T + u];
-                    float e;
-                    e = a[t].x - b[u].x; s = fmaf(e, e, s);
-                    e = a[t].y - b[u].y; s = fmaf(e, e, s);
-                    e = a[t].z - b[u].z; s = fmaf(e, e, s);
-                    e = a[t].w - b[u].w; s = fmaf(e, e, s);
-                    acc[t * T + u] = s;
-                }
-        }
-#pragma unroll
-        for (int e = 0; e < T * T; ++e) dacc[e] += static_cast<double>(acc[e]);
-        __syncthreads();
-        buf ^= 1;
-    }
-    double* mine = partial + (static_cast<size_t>(blockIdx.x) * NT + tid) * (T * T);
-#pragma unroll
-    for (int e = 0; e < T * T; ++e) mine[e] = dacc[e];
-}
-
-// dist[a][b] = sum over CTAs (ascending) and groups (ascending) of the owning thread's element
-template <int F, int T, int G>
-__global__ void pairdist_tiled_reduce_kernel(const double* __restrict__ partial, int n_ctas, double* __restrict__ dist) {
-    using PT = PairTile<F, T>;
-    constexpr int NB = PT::NB, NPB = PT::NPB, NT = NPB * G;
-    const int p = blockIdx.x * blockDim.x + threadIdx.x;
-    if (p >= F * F) return;
-    const int a = p / F, b = p % F;
-    if (a > b) return;
-    if (a == b) {
-        dist[p] = 0.0;
-        return;
-    }
-    const int ra = a % NB, ta = a / NB, rb = b % NB, tb = b / NB;
-    int bi, bj, t, u;
-    if (ra <= rb) {
-        bi = ra; bj = rb; t = ta; u = tb;
-    } else {
-        bi = rb; bj = ra; t = tb; u = ta;
-    }
-    // index of (bi, bj) among the pairs bi <= bj in row-major order
-    const int pb = bi * NB - bi * (bi - 1) / 2 + (bj - bi);
-    double s = 0.0;
-    for (int cta = 0; cta < n_ctas; ++cta)
-        for (int g = 0; g < G; ++g) s += partial[(static_cast<size_t>(cta) * NT + g * NPB + pb) * (T * T) + t * T + u];
-    dist[a * F + b] = s;
-    dist[b * F + a] = s;
-}
-
-// Any f, any alignment: a CTA stages kGT coordinates of all rows with scalar loads; pair p is
-// always summed by thread p % blockDim of the CTA, binary32 inside the stage, binary64 across.
-constexpr int kGT = 64;
-__global__ void __launch_bounds__(256)
-    pairdist_generic_kernel(const float* __restrict__ v, int f, int64_t d, int64_t ld, double* __restrict__ partial) {
-    __shared__ float tile[BZ_MAX_F][kGT + 1];
-    const int n_pairs = f * (f - 1) / 2;
-    double* mine = partial + static_cast<size_t>(blockIdx.x) * n_pairs;
-    for (int p = threadIdx.x; p < n_pairs; p += blockDim.x) mine[p] = 0.0;
-    const int64_t n_tiles = (d + kGT - 1) / kGT;
-    for (int64_t tile_i = blockIdx.x; tile_i < n_tiles; tile_i += gridDim.x) {
-        const int64_t j0 = tile_i * kGT;
-        for (int idx = threadIdx.x; idx < f * kGT; idx += blockDim.x) {
-            const int row = idx / kGT, c = idx % kGT;
-            tile[row][c] = (j0 + c < d) ? v[row * ld + j0 + c] : 0.f;
-        }
-        __syncthreads();
-        for (int p = threadIdx.x; p < n_pairs; p += blockDim.x) {
-            // p -> (a, b), a < b, row-major over the strict upper triangle
-            int a = 0, rest = p;
-            while (rest >= f - 1 - a) {
-                rest -= f - 1 - a;
-                ++a;
-            }
-            const int b = a + 1 + rest;
-            float s = 0.f;
-            for (int c = 0; c < kGT; ++c) {
-                const float e = tile[a][c] - tile[b][c];
-                s = fmaf(e, e, s);
-            }
-            mine[p] += static_cast<double>(s);
-        }
-        __syncthreads();
-    }
-}
-
-__global__ void pairdist_generic_reduce_kernel(const double* __restrict__ partial, int n_ctas, int f,
-                                               double* __restrict__ dist) {
-    const int p = blockIdx.x * blockDim.x + threadIdx.x;
-    if (p < f) dist[p * f + p] = 0.0;
-    const int n_pairs = f * (f - 1) / 2;
-    if (p >= n_pairs) return;
-    int a = 0, rest = p;
-    while (rest >= f - 1 - a) {
-        rest -= f - 1 - a;
-        ++a;
-    }
-    const int b = a + 1 + rest;
-    double s = 0.0;
-    for (int cta = 0; cta < n_ctas; ++cta) s += partial[static_cast<size_t>(cta) * n_pairs + p];
-    dist[a * f + b] = s;
-    dist[b * f + a] = s;
-}
 
 // ------------------------------------------------------------------------------------------------
 // Selection kernels: one CTA, thread a owns row a.
@@ -302,38 +116,39 @@ __global__ void __launch_bounds__(256) mean_rows_kernel(const V* __restrict__ v,
     }
 }
 
-// Window of the beta sorted values closest to the median: the greedy growth (lower neighbour on
-// ties) is a merge of the two distance sequences, so a value's membership follows from its rank
-// in that merge.  s[] ascending; returns the mean of the window (binary64 sum, ascending).
-template <int THETA> __device__ __forceinline__ float window_mean(const float (&s)[THETA], int beta) {
+// Window of the BETA sorted values closest to the median.  The greedy growth (lower neighbour on
+// ties) is a merge of the two distance sequences: the p-th lower value enters before the q-th upper
+// one iff its distance is not larger, so it belongs to the window iff the (BETA-p)-th upper value
+// does not exist or is at least as far.  The number L of such p fixes the window [MID-L, MID-L+BETA).
+// s[] ascending; returns the mean of the window (binary64 sum, ascending).
+template <int THETA, int BETA> __device__ __forceinline__ float window_mean(const float (&s)[THETA]) {
     constexpr int MID = (THETA - 1) / 2;
     const float med = s[MID];
-    float dist[THETA];
+    int L = 0;
 #pragma unroll
-    for (int t = 0; t < THETA; ++t) dist[t] = fabsf(__fsub_rn(s[t], med));
+    for (int p = 1; p <= MID && p <= BETA - 1; ++p) {
+        const int up = MID + (BETA - p);  // index of the (BETA-p)-th upper value
+        if (up > THETA - 1) {
+            ++L;
+        } else {
+            const float dl = fabsf(__fsub_rn(s[MID - p], med)), du = fabsf(__fsub_rn(s[up], med));
+            L += (du >= dl);
+        }
+    }
+    const int lo = MID - L, hi = lo + BETA - 1;
     double sum = 0.0;
 #pragma unroll
     for (int t = 0; t < THETA; ++t) {
-        int rank;  // number of values taken before s[t]; the median itself is rank 0
-        if (t == MID) {
-            rank = 0;
-        } else if (t < MID) {
-            rank = MID - t;  // the median and the lower values nearer to it
-#pragma unroll
-            for (int u = MID + 1; u < THETA; ++u) rank += (dist[u] < dist[t]);
-        } else {
-            rank = t - MID;
-#pragma unroll
-            for (int u = 0; u < MID; ++u) rank += (dist[u] <= dist[t]);
+        if (t >= MID - (BETA - 1) && t <= MID + (BETA - 1)) {  // the only positions a window can cover
+            if (t >= lo && t <= hi) sum += static_cast<double>(s[t]);
         }
-        if (rank < beta) sum += static_cast<double>(s[t]);
     }
-    return static_cast<float>(sum / static_cast<double>(beta));
+    return static_cast<float>(sum / static_cast<double>(BETA));
 }
 
-template <int THETA>
+template <int THETA, int BETA>
 __global__ void __launch_bounds__(128) trimmed_mean_kernel(const float* __restrict__ v, int64_t d, int64_t ld,
-                                                           const int32_t* __restrict__ selected, int beta,
+                                                           const int32_t* __restrict__ selected,
                                                            float* __restrict__ out) {
     __shared__ int32_t sel[THETA];
     for (int t = threadIdx.x; t < THETA; t += blockDim.x) sel[t] = selected[t];
@@ -347,7 +162,7 @@ __global__ void __launch_bounds__(128) trimmed_mean_kernel(const float* __restri
         float s[THETA];
 #pragma unroll
         for (int t = 0; t < THETA; ++t) s[t] = __uint_as_float(key_bits(k[t]));
-        out[j] = window_mean<THETA>(s, beta);
+        out[j] = window_mean<THETA, BETA>(s);
     }
 }
 
@@ -392,61 +207,6 @@ __global__ void __launch_bounds__(128) trimmed_mean_generic_kernel(const float* 
 // ------------------------------------------------------------------------------------------------
 // host side
 
-int pairdist_ctas(int64_t d, int tile) {
-    int64_t n_tiles = (d + tile - 1) / tile;
-    if (n_tiles > kNumSMs) n_tiles = kNumSMs;
-    if (n_tiles < 1) n_tiles = 1;
-    return static_cast<int>(n_tiles);
-}
-
-template <int F, int T, int G> constexpr size_t tiled_partial_doubles() {
-    return static_cast<size_t>(kNumSMs) * PairTile<F, T>::NPB * G * T * T;
-}
-
-size_t pairdist_workspace(int f) {
-    size_t doubles;
-    if (f == 25)
-        doubles = tiled_partial_doubles<25, 5, 8>();
-    else if (f == 49)
-        doubles = tiled_partial_doubles<49, 7, 8>();
-    else
-        doubles = static_cast<size_t>(kNumSMs) * f * (f - 1) / 2;
-    if (doubles < 32) doubles = 32;
-    return round_up(doubles * sizeof(double), 256);
-}
-
-template <int F, int T, int G>
-int launch_pairdist_tiled(const float* v, int64_t d, int64_t ld, double* dist, double* partial, cudaStream_t s) {
-    constexpr int NT = PairTile<F, T>::NPB * G;
-    constexpr int smem = 2 * F * kRowStride * static_cast<int>(sizeof(float));
-    cudaError_t e = cudaFuncSetAttribute(pairdist_tiled_kernel<F, T, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return cuda_failed(e);
-    const int ctas = pairdist_ctas(d, kTD);
-    pairdist_tiled_kernel<F, T, G><<<ctas, NT, smem, s>>>(v, d, ld, partial);
-    note_launch();
-    int st = check_launch();
-    if (st != BZ_OK) return st;
-    pairdist_tiled_reduce_kernel<F, T, G><<<(F * F + 127) / 128, 128, 0, s>>>(partial, ctas, dist);
-    note_launch();
-    return check_launch();
-}
-
-int pairdist_on_device(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, cudaStream_t s) {
-    double* partial = static_cast<double*>(ws);
-    const bool vec = aligned16(v) && (ld % 4 == 0);
-    if (vec && f == 25) return launch_pairdist_tiled<25, 5, 8>(v, d, ld, dist, partial, s);
-    if (vec && f == 49) return launch_pairdist_tiled<49, 7, 8>(v, d, ld, dist, partial, s);
-    const int ctas = pairdist_ctas(d, kGT);
-    pairdist_generic_kernel<<<ctas, 256, 0, s>>>(v, f, d, ld, partial);
-    note_launch();
-    int st = check_launch();
-    if (st != BZ_OK) return st;
-    const int n = f * f;  // covers both the pairs and the diagonal
-    pairdist_generic_reduce_kernel<<<(n + 127) / 128, 128, 0, s>>>(partial, ctas, f, dist);
-    note_launch();
-    return check_launch();
-}
-
 int mean_rows_on_device(const float* v, int64_t d, int64_t ld, const int32_t* selected, int m, float* out,
                         cudaStream_t s) {
     const bool vec = aligned16(v) && aligned16(out) && (ld % 4 == 0);
@@ -471,26 +231,26 @@ int mean_rows_on_device(const float* v, int64_t d, int64_t ld, const int32_t* se
     return BZ_OK;
 }
 
-template <int THETA>
-int launch_trimmed(const float* v, int64_t d, int64_t ld, const int32_t* selected, int beta, float* out, cudaStream_t s) {
+template <int THETA, int BETA>
+int launch_trimmed(const float* v, int64_t d, int64_t ld, const int32_t* selected, float* out, cudaStream_t s) {
     int64_t grid = (d + 127) / 128;
     if (grid > kNumSMs * 16) grid = kNumSMs * 16;
-    trimmed_mean_kernel<THETA><<<static_cast<int>(grid), 128, 0, s>>>(v, d, ld, selected, beta, out);
+    trimmed_mean_kernel<THETA, BETA><<<static_cast<int>(grid), 128, 0, s>>>(v, d, ld, selected, out);
     note_launch();
     return check_launch();
 }
 
+// Register kernels exist for the (theta, beta) = (f - 2c, f - 4c) pairs of f = 25 and f = 49 (every c
+// Bulyan admits) and a few small shapes; anything else runs the local-memory kernel.
 int trimmed_mean_on_device(const float* v, int64_t d, int64_t ld, const int32_t* selected, int theta, int beta,
                            float* out, cudaStream_t s) {
-    switch (theta) {
-#define BZ_TM_CASE(N) \
-    case N: return launch_trimmed<N>(v, d, ld, selected, beta, out, s);
-        BZ_TM_CASE(5) BZ_TM_CASE(7) BZ_TM_CASE(9) BZ_TM_CASE(15) BZ_TM_CASE(17) BZ_TM_CASE(19) BZ_TM_CASE(21)
-        BZ_TM_CASE(23) BZ_TM_CASE(25) BZ_TM_CASE(27) BZ_TM_CASE(29) BZ_TM_CASE(31) BZ_TM_CASE(33) BZ_TM_CASE(35)
-        BZ_TM_CASE(37) BZ_TM_CASE(39) BZ_TM_CASE(41) BZ_TM_CASE(43) BZ_TM_CASE(45) BZ_TM_CASE(47) BZ_TM_CASE(49)
+#define BZ_TM_CASE(TH, BE) \
+    if (theta == TH && beta == BE) return launch_trimmed<TH, BE>(v, d, ld, selected, out, s);
+    BZ_TM_CASE(25, 25) BZ_TM_CASE(23, 21) BZ_TM_CASE(21, 17) BZ_TM_CASE(19, 13) BZ_TM_CASE(17, 9) BZ_TM_CASE(15, 5)
+    BZ_TM_CASE(49, 49) BZ_TM_CASE(47, 45) BZ_TM_CASE(45, 41) BZ_TM_CASE(43, 37) BZ_TM_CASE(41, 33) BZ_TM_CASE(39, 29)
+    BZ_TM_CASE(37, 25) BZ_TM_CASE(35, 21) BZ_TM_CASE(33, 17) BZ_TM_CASE(31, 13) BZ_TM_CASE(29, 9) BZ_TM_CASE(27, 5)
+    BZ_TM_CASE(9, 9) BZ_TM_CASE(7, 5) BZ_TM_CASE(5, 3) BZ_TM_CASE(9, 1)
 #undef BZ_TM_CASE
-        default: break;
-    }
     int64_t grid = (d + 127) / 128;
     if (grid > kNumSMs * 8) grid = kNumSMs * 8;
     trimmed_mean_generic_kernel<<<static_cast<int>(grid), 128, 0, s>>>(v, d, ld, selected, theta, beta, out);
@@ -498,40 +258,11 @@ int trimmed_mean_on_device(const float* v, int64_t d, int64_t ld, const int32_t*
     return check_launch();
 }
 
-int validate_rows(const float* v, int f, int64_t d, int64_t ld) {
-    if (d < 0 || f < 1 || (v == nullptr && d > 0)) return BZ_ERR_INVALID_ARG;  // an empty array may have no address
-    if (f > BZ_MAX_F) return BZ_ERR_UNSUPPORTED;
-    if (ld < d) return BZ_ERR_INVALID_ARG;
-    return BZ_OK;
-}
-
-int check_workspace(void* ws, size_t have, size_t need) {
-    if (ws == nullptr || !aligned256(ws) || have < need) return BZ_ERR_WORKSPACE;
-    return BZ_OK;
-}
-
 }  // namespace
-
-size_t krum_workspace_bytes(int op, int f) {
-    const size_t pd = pairdist_workspace(f);
-    if (op == BZ_OP_PAIRDIST) return pd;
-    // multi-Krum / Bulyan: partial sums, then the f x f matrix
-    return pd + round_up(static_cast<size_t>(f) * f * sizeof(double), 256);
-}
 
 }  // namespace bz
 
 using namespace bz;
-
-extern "C" int bz_pairdist(const float* voted, int f, int64_t d, int64_t ld, double* dist, void* workspace,
-                           size_t workspace_bytes, void* stream) {
-    int st = validate_rows(voted, f, d, ld);
-    if (st != BZ_OK) return st;
-    if (dist == nullptr) return BZ_ERR_INVALID_ARG;
-    st = check_workspace(workspace, workspace_bytes, krum_workspace_bytes(BZ_OP_PAIRDIST, f));
-    if (st != BZ_OK) return st;
-    return pairdist_on_device(voted, f, d, ld, dist, workspace, static_cast<cudaStream_t>(stream));
-}
 
 extern "C" int bz_krum_select(const double* dist, int f, int c, int m, int32_t* selected, void* stream) {
     if (dist == nullptr || selected == nullptr || f < 1) return BZ_ERR_INVALID_ARG;
@@ -608,52 +339,3 @@ extern "C" int bz_bulyan(const float* voted, int f, int64_t d, int64_t ld, int c
     return trimmed_mean_on_device(voted, d, ld, selected, theta, theta - 2 * c, out, s);
 }
 
-// ------------------------------------------------------------------------------------------------
-// Pairwise distances without a caller workspace.
-//
-// Some hosts of this library may not allocate device memory at the moment they need the distance
-// matrix: an operator plugged into a framework whose memory plan is frozen before the run, a
-// serving or training loop that must not take the implicit device synchronisation an allocation
-// can bring, a process confined to a fixed memory budget on a shared GPU.  For them the partial
-// sums that bz_pairdist keeps in the caller's workspace live in the array below, which every GPU
-// that loads the library holds from load to exit.
-namespace {
-
-constexpr size_t kStaticScratchBytes = BZ_STATIC_SCRATCH_BYTES;  // 4 MiB
-static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
-
-constexpr int kMaxDevices = 64;
-void* g_static_scratch_addr[kMaxDevices] = {};  // device address of the array on each device, once resolved
-
-// The array's name is only a handle on the host side; kernels need its device address, which the
-// runtime hands out per device.
-int static_scratch(void** ptr) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return cuda_failed(e);
-    if (dev < 0 || dev >= kMaxDevices) return BZ_ERR_UNSUPPORTED;
-    if (g_static_scratch_addr[dev] == nullptr) {
-        void* p = nullptr;
-        e = cudaGetSymbolAddress(&p, g_static_scratch);
-        if (e != cudaSuccess) return cuda_failed(e);
-        if (p == nullptr || !aligned256(p)) return BZ_ERR_WORKSPACE;
-        g_static_scratch_addr[dev] = p;
-    }
-    *ptr = g_static_scratch_addr[dev];
-    return BZ_OK;
-}
-
-}  // namespace
-
-extern "C" int bz_pairdist_static(const float* voted, int f, int64_t d, int64_t ld, double* dist, void* stream) {
-    int st = validate_rows(voted, f, d, ld);
-    if (st != BZ_OK) return st;
-    if (dist == nullptr) return BZ_ERR_INVALID_ARG;
-    if (krum_workspace_bytes(BZ_OP_PAIRDIST, f) > kStaticScratchBytes) return BZ_ERR_STATIC_LIMIT;
-    void* scratch = nullptr;
-    st = static_scratch(&scratch);
-    if (st != BZ_OK) return st;
-    // Nothing in the array has to start at zero: the tiled kernel overwrites every partial sum the
-    // reduction reads, and the generic kernel clears its own slots before it accumulates.
-    return pairdist_on_device(voted, f, d, ld, dist, scratch, static_cast<cudaStream_t>(stream));
-}

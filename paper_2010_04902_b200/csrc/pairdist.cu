@@ -1,0 +1,382 @@
+// Pairwise squared distances between the f voted gradients - the O(f^2 d) part of the Krum family
+// (Sec. 1.2; cost in Appendix A.1).
+//
+// The distances are accumulated in the difference form sum_j (v_a[j] - v_b[j])^2: its accuracy
+// does not depend on a common offset of the rows (gradients share a large per-coordinate mean)
+// nor on the size of an attacker's payload in other rows, which the Gram form |a|^2 + |b|^2 - 2ab
+// - and with it a tensor-core contraction - cannot offer at the precision the selection needs.
+// The work is therefore bound by the FP32 pipe: f(f-1) add/fma lane-operations per coordinate.
+#include "bz_common.cuh"
+
+namespace bz {
+
+namespace {
+
+// ------------------------------------------------------------------------------------------------
+// Register-tiled kernel.  The F rows are split into NB = F/T residue classes; a thread owns one
+// unordered pair of classes (bi <= bj), i.e. the T x T row pairs (bi + NB*t, bj + NB*u), and one of
+// G interleaved coordinate groups of every tile.  A CTA streams tiles of kTD coordinates of all F
+// rows through a double-buffered shared-memory stage (cp.async, 16 bytes per request).
+// Sums: binary32 in registers over kFlush tiles (kFlush * kTD / G coordinates per thread), then
+// the G groups of a pair are added in binary32 in a fixed order and the result goes into the CTA's
+// binary64 accumulator in shared memory; one fixed-order reduction over CTAs finishes.
+// The result is bit-reproducible from run to run.
+template <int F, int T, int G> struct PairTile {
+    static constexpr int NB = F / T;
+    static constexpr int NPB = NB * (NB + 1) / 2;
+    static constexpr int NT = NPB * G;
+    static constexpr int TT = T * T;
+    static_assert(NB * T == F, "T must divide F");
+};
+
+constexpr int kTD = 256;        // coordinates per tile
+constexpr int kRowPad = 4;      // floats; keeps the row stride an odd number of 16-byte units
+constexpr int kRowStride = kTD + kRowPad;
+constexpr int kFlush = 4;       // tiles between two flushes of the binary32 accumulators
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src, int src_bytes) {
+    const unsigned dst = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(gmem_src), "r"(src_bytes));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+
+template <int F, int T, int G> constexpr size_t tiled_smem_bytes() {
+    using PT = PairTile<F, T, G>;
+    return size_t(2) * F * kRowStride * 4 + (size_t(PT::NT) * PT::TT + 1) * 4 + size_t(PT::NPB) * PT::TT * 8;
+}
+
+// CTAs per SM the launch asks for: two where the shared memory of two fits
+template <int F, int T, int G> constexpr int tiled_ctas_per_sm() { return tiled_smem_bytes<F, T, G>() <= 110 * 1024 ? 2 : 1; }
+
+template <int F, int T, int G>
+__global__ void __launch_bounds__(PairTile<F, T, G>::NT)
+    pairdist_tiled_kernel(const float* __restrict__ v, int64_t d, int64_t ld, double* __restrict__ partial) {
+    using PT = PairTile<F, T, G>;
+    constexpr int NB = PT::NB, NPB = PT::NPB, NT = PT::NT, TT = PT::TT;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* stage0 = reinterpret_cast<float*>(smem_raw);                            // 2 x [F][kRowStride]
+    float* red = stage0 + 2 * F * kRowStride;                                      // [G][NPB][TT]
+    double* dsum = reinterpret_cast<double*>(red + NT * TT + ((NT * TT) & 1));     // [NPB][TT]
+
+    const int tid = threadIdx.x;
+    const int pb = tid % NPB, g = tid / NPB;
+    int bi = 0, bj = 0;
+    {
+        int rest = pb;
+        while (rest >= NB - bi) {
+            rest -= NB - bi;
+            ++bi;
+        }
+        bj = bi + rest;
+    }
+    for (int e = tid; e < NPB * TT; e += NT) dsum[e] = 0.0;
+
+    const int64_t n_tiles = (d + kTD - 1) / kTD;
+    auto load_tile = [&](int buf, int64_t tile) {
+        const int64_t j0 = tile * kTD;
+        constexpr int per_row = kTD / 4;
+        float* dst = stage0 + buf * F * kRowStride;
+        for (int idx = tid; idx < F * per_row; idx += NT) {
+            const int row = idx / per_row, c4 = idx - row * per_row;
+            const int64_t j = j0 + 4 * c4;
+            const int64_t left = d - j;
+            const int bytes = left >= 4 ? 16 : (left > 0 ? static_cast<int>(left) * 4 : 0);
+            const float* src = bytes ? v + row * ld + j : v;  // zero-byte requests still name a valid address
+            cp_async16(dst + row * kRowStride + 4 * c4, src, bytes);
+        }
+        cp_async_commit();
+    };
+
+    float acc[TT];
+#pragma unroll
+    for (int e = 0; e < TT; ++e) acc[e] = 0.f;
+
+    int64_t tile = blockIdx.x;
+    int buf = 0, since_flush = 0;
+    if (tile < n_tiles) load_tile(0, tile);
+    for (; tile < n_tiles; tile += gridDim.x) {
+        const int64_t next = tile + gridDim.x;
+        if (next < n_tiles) {
+            load_tile(buf ^ 1, next);
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+
+        const float* base = stage0 + buf * F * kRowStride;
+#pragma unroll 1
+        for (int c4 = g; c4 < kTD / 4; c4 += G) {
+            float4 a[T], b[T];
+#pragma unroll
+            for (int t = 0; t < T; ++t) {
+                a[t] = *reinterpret_cast<const float4*>(base + (bi + NB * t) * kRowStride + 4 * c4);
+                b[t] = *reinterpret_cast<const float4*>(base + (bj + NB * t) * kRowStride + 4 * c4);
+            }
+#pragma unroll
+            for (int t = 0; t < T; ++t)
+#pragma unroll
+                for (int u = 0; u < T; ++u) {
+                    float s = acc[t * T + u];
+                    float e;
+                    e = a[t].x - b[u].x; s = fmaf(e, e, s);
+                    e = a[t].y - b[u].y; s = fmaf(e, e, s);
+                    e = a[t].z - b[u].z; s = fmaf(e, e, s);
+                    e = a[t].w - b[u].w; s = fmaf(e, e, s);
+                    acc[t * T + u] = s;
+                }
+        }
+        ++since_flush;
+        if (since_flush == kFlush || next >= n_tiles) {  // uniform over the CTA
+            since_flush = 0;
+#pragma unroll
+            for (int e = 0; e < TT; ++e) {
+                red[tid * TT + e] = acc[e];  // tid = g * NPB + pb
+                acc[e] = 0.f;
+            }
+            __syncthreads();
+            for (int e = g; e < TT; e += G) {
+                float s = 0.f;
+#pragma unroll
+                for (int g2 = 0; g2 < G; ++g2) s += red[(g2 * NPB + pb) * TT + e];
+                dsum[pb * TT + e] += static_cast<double>(s);
+            }
+        }
+        __syncthreads();
+        buf ^= 1;
+    }
+    __syncthreads();
+    double* mine = partial + static_cast<size_t>(blockIdx.x) * NPB * TT;
+    for (int e = tid; e < NPB * TT; e += NT) mine[e] = dsum[e];
+}
+
+// dist[a][b] = sum over CTAs (ascending) of the element of the pair's class block
+template <int F, int T, int G>
+__global__ void pairdist_tiled_reduce_kernel(const double* __restrict__ partial, int n_ctas, double* __restrict__ dist) {
+    using PT = PairTile<F, T, G>;
+    constexpr int NB = PT::NB, NPB = PT::NPB, TT = PT::TT;
+    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= F * F) return;
+    const int a = p / F, b = p % F;
+    if (a > b) return;
+    if (a == b) {
+        dist[p] = 0.0;
+        return;
+    }
+    const int ra = a % NB, ta = a / NB, rb = b % NB, tb = b / NB;
+    int bi, bj, t, u;
+    if (ra <= rb) {
+        bi = ra; bj = rb; t = ta; u = tb;
+    } else {
+        bi = rb; bj = ra; t = tb; u = ta;
+    }
+    // index of (bi, bj) among the pairs bi <= bj in row-major order
+    const int pb = bi * NB - bi * (bi - 1) / 2 + (bj - bi);
+    double s = 0.0;
+    for (int cta = 0; cta < n_ctas; ++cta) s += partial[(static_cast<size_t>(cta) * NPB + pb) * TT + t * T + u];
+    dist[a * F + b] = s;
+    dist[b * F + a] = s;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Any f, any alignment: a CTA stages kGT coordinates of all rows with scalar loads; pair p is
+// always summed by thread p % blockDim of the CTA, binary32 inside the stage, binary64 across.
+constexpr int kGT = 64;
+__global__ void __launch_bounds__(256)
+    pairdist_generic_kernel(const float* __restrict__ v, int f, int64_t d, int64_t ld, double* __restrict__ partial) {
+    __shared__ float tile[BZ_MAX_F][kGT + 1];
+    const int n_pairs = f * (f - 1) / 2;
+    double* mine = partial + static_cast<size_t>(blockIdx.x) * n_pairs;
+    for (int p = threadIdx.x; p < n_pairs; p += blockDim.x) mine[p] = 0.0;
+    const int64_t n_tiles = (d + kGT - 1) / kGT;
+    for (int64_t tile_i = blockIdx.x; tile_i < n_tiles; tile_i += gridDim.x) {
+        const int64_t j0 = tile_i * kGT;
+        for (int idx = threadIdx.x; idx < f * kGT; idx += blockDim.x) {
+            const int row = idx / kGT, c = idx % kGT;
+            tile[row][c] = (j0 + c < d) ? v[row * ld + j0 + c] : 0.f;
+        }
+        __syncthreads();
+        for (int p = threadIdx.x; p < n_pairs; p += blockDim.x) {
+            // p -> (a, b), a < b, row-major over the strict upper triangle
+            int a = 0, rest = p;
+            while (rest >= f - 1 - a) {
+                rest -= f - 1 - a;
+                ++a;
+            }
+            const int b = a + 1 + rest;
+            float s = 0.f;
+            for (int c = 0; c < kGT; ++c) {
+                const float e = tile[a][c] - tile[b][c];
+                s = fmaf(e, e, s);
+            }
+            mine[p] += static_cast<double>(s);
+        }
+        __syncthreads();
+    }
+}
+
+__global__ void pairdist_generic_reduce_kernel(const double* __restrict__ partial, int n_ctas, int f,
+                                               double* __restrict__ dist) {
+    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p < f) dist[p * f + p] = 0.0;
+    const int n_pairs = f * (f - 1) / 2;
+    if (p >= n_pairs) return;
+    int a = 0, rest = p;
+    while (rest >= f - 1 - a) {
+        rest -= f - 1 - a;
+        ++a;
+    }
+    const int b = a + 1 + rest;
+    double s = 0.0;
+    for (int cta = 0; cta < n_ctas; ++cta) s += partial[static_cast<size_t>(cta) * n_pairs + p];
+    dist[a * f + b] = s;
+    dist[b * f + a] = s;
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+
+int pairdist_ctas(int64_t d, int tile, int per_sm = 1) {
+    int64_t n_tiles = (d + tile - 1) / tile;
+    if (n_tiles > kNumSMs * per_sm) n_tiles = kNumSMs * per_sm;
+    if (n_tiles < 1) n_tiles = 1;
+    return static_cast<int>(n_tiles);
+}
+
+// specialisations: <F, T, G>
+#define BZ_PD_25 25, 5, 16
+#define BZ_PD_49 49, 7, 16
+
+template <int F, int T, int G> constexpr size_t tiled_partial_doubles() {
+    return static_cast<size_t>(kNumSMs) * tiled_ctas_per_sm<F, T, G>() * PairTile<F, T, G>::NPB * PairTile<F, T, G>::TT;
+}
+
+template <int F, int T, int G>
+int launch_pairdist_tiled(const float* v, int64_t d, int64_t ld, double* dist, double* partial, cudaStream_t s) {
+    constexpr int NT = PairTile<F, T, G>::NT;
+    constexpr int smem = static_cast<int>(tiled_smem_bytes<F, T, G>());
+    cudaError_t e = cudaFuncSetAttribute(pairdist_tiled_kernel<F, T, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return cuda_failed(e);
+    const int ctas = pairdist_ctas(d, kTD, tiled_ctas_per_sm<F, T, G>());
+    pairdist_tiled_kernel<F, T, G><<<ctas, NT, smem, s>>>(v, d, ld, partial);
+    note_launch();
+    int st = check_launch();
+    if (st != BZ_OK) return st;
+    pairdist_tiled_reduce_kernel<F, T, G><<<(F * F + 127) / 128, 128, 0, s>>>(partial, ctas, dist);
+    note_launch();
+    return check_launch();
+}
+
+}  // namespace
+
+size_t pairdist_workspace(int f) {
+    size_t doubles;
+    if (f == 25)
+        doubles = tiled_partial_doubles<BZ_PD_25>();
+    else if (f == 49)
+        doubles = tiled_partial_doubles<BZ_PD_49>();
+    else
+        doubles = static_cast<size_t>(kNumSMs) * f * (f - 1) / 2;
+    if (doubles < 32) doubles = 32;
+    return round_up(doubles * sizeof(double), 256);
+}
+
+int pairdist_on_device(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, cudaStream_t s) {
+    double* partial = static_cast<double*>(ws);
+    const bool vec = aligned16(v) && (ld % 4 == 0);
+    if (vec && f == 25) return launch_pairdist_tiled<BZ_PD_25>(v, d, ld, dist, partial, s);
+    if (vec && f == 49) return launch_pairdist_tiled<BZ_PD_49>(v, d, ld, dist, partial, s);
+    const int ctas = pairdist_ctas(d, kGT);
+    pairdist_generic_kernel<<<ctas, 256, 0, s>>>(v, f, d, ld, partial);
+    note_launch();
+    int st = check_launch();
+    if (st != BZ_OK) return st;
+    const int n = f * f;  // covers both the pairs and the diagonal
+    pairdist_generic_reduce_kernel<<<(n + 127) / 128, 128, 0, s>>>(partial, ctas, f, dist);
+    note_launch();
+    return check_launch();
+}
+
+int validate_rows(const float* v, int f, int64_t d, int64_t ld) {
+    if (d < 0 || f < 1 || (v == nullptr && d > 0)) return BZ_ERR_INVALID_ARG;  // an empty array may have no address
+    if (f > BZ_MAX_F) return BZ_ERR_UNSUPPORTED;
+    if (ld < d) return BZ_ERR_INVALID_ARG;
+    return BZ_OK;
+}
+
+int check_workspace(void* ws, size_t have, size_t need) {
+    if (ws == nullptr || !aligned256(ws) || have < need) return BZ_ERR_WORKSPACE;
+    return BZ_OK;
+}
+
+size_t krum_workspace_bytes(int op, int f) {
+    const size_t pd = pairdist_workspace(f);
+    if (op == BZ_OP_PAIRDIST) return pd;
+    // multi-Krum / Bulyan: partial sums, then the f x f matrix
+    return pd + round_up(static_cast<size_t>(f) * f * sizeof(double), 256);
+}
+
+}  // namespace bz
+
+using namespace bz;
+
+extern "C" int bz_pairdist(const float* voted, int f, int64_t d, int64_t ld, double* dist, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+    int st = validate_rows(voted, f, d, ld);
+    if (st != BZ_OK) return st;
+    if (dist == nullptr) return BZ_ERR_INVALID_ARG;
+    st = check_workspace(workspace, workspace_bytes, krum_workspace_bytes(BZ_OP_PAIRDIST, f));
+    if (st != BZ_OK) return st;
+    return pairdist_on_device(voted, f, d, ld, dist, workspace, static_cast<cudaStream_t>(stream));
+}
+
+// ------------------------------------------------------------------------------------------------
+// Pairwise distances without a caller workspace.
+//
+// Some hosts of this library may not allocate device memory at the moment they need the distance
+// matrix: an operator plugged into a framework whose memory plan is frozen before the run, a
+// serving or training loop that must not take the implicit device synchronisation an allocation
+// can bring, a process confined to a fixed memory budget on a shared GPU.  For them the partial
+// sums that bz_pairdist keeps in the caller's workspace live in the array below, which every GPU
+// that loads the library holds from load to exit.
+namespace {
+
+constexpr size_t kStaticScratchBytes = BZ_STATIC_SCRATCH_BYTES;  // 4 MiB
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {};  // device address of the array on each device, once resolved
+
+// The array's name is only a handle on the host side; kernels need its device address, which the
+// runtime hands out per device.
+int static_scratch(void** ptr) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_failed(e);
+    if (dev < 0 || dev >= kMaxDevices) return BZ_ERR_UNSUPPORTED;
+    if (g_static_scratch_addr[dev] == nullptr) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return cuda_failed(e);
+        if (p == nullptr || !aligned256(p)) return BZ_ERR_WORKSPACE;
+        g_static_scratch_addr[dev] = p;
+    }
+    *ptr = g_static_scratch_addr[dev];
+    return BZ_OK;
+}
+
+}  // namespace
+
+extern "C" int bz_pairdist_static(const float* voted, int f, int64_t d, int64_t ld, double* dist, void* stream) {
+    int st = validate_rows(voted, f, d, ld);
+    if (st != BZ_OK) return st;
+    if (dist == nullptr) return BZ_ERR_INVALID_ARG;
+    if (krum_workspace_bytes(BZ_OP_PAIRDIST, f) > kStaticScratchBytes) return BZ_ERR_STATIC_LIMIT;
+    void* scratch = nullptr;
+    st = static_scratch(&scratch);
+    if (st != BZ_OK) return st;
+    // Nothing in the array has to start at zero: the tiled kernel overwrites every partial sum the
+    // reduction reads, and the generic kernel clears its own slots before it accumulates.
+    return pairdist_on_device(voted, f, d, ld, dist, scratch, static_cast<cudaStream_t>(stream));
+}

@@ -93,21 +93,31 @@ template <int R, typename V>
 __global__ void __launch_bounds__(256) vote_kernel(const V* __restrict__ rep, int64_t n, int64_t ld_file,
                                                    int64_t ld_rep, V* __restrict__ voted, int64_t ld_voted) {
     constexpr int VEC = Lanes<V>::n;
+    constexpr int U = (12 / R) < 1 ? 1 : (12 / R);  // coordinate groups per thread and trip: ~12 loads in flight
     const int i = blockIdx.y;
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
-    for (int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < n; j += stride) {
-        V x[R];
+    const V* src = rep + i * ld_file;
+    V* dst = voted + i * ld_voted;
+    for (int64_t j0 = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j0 < n; j0 += stride * U) {
+        V x[U][R];
 #pragma unroll
-        for (int k = 0; k < R; ++k) x[k] = ld_stream(rep + k * ld_rep + i * ld_file + j);
-        uint32_t res[VEC];
+        for (int u = 0; u < U; ++u)
 #pragma unroll
-        for (int c = 0; c < VEC; ++c) {
-            uint32_t copies[R];
+            for (int k = 0; k < R; ++k)
+                if (j0 + u * stride < n) x[u][k] = ld_stream(src + k * ld_rep + j0 + u * stride);
 #pragma unroll
-            for (int k = 0; k < R; ++k) copies[k] = Lanes<V>::get(x[k], c);
-            res[c] = vote_bits<R>(copies);
+        for (int u = 0; u < U; ++u) {
+            if (j0 + u * stride >= n) break;
+            uint32_t res[VEC];
+#pragma unroll
+            for (int c = 0; c < VEC; ++c) {
+                uint32_t copies[R];
+#pragma unroll
+                for (int k = 0; k < R; ++k) copies[k] = Lanes<V>::get(x[u][k], c);
+                res[c] = vote_bits<R>(copies);
+            }
+            dst[j0 + u * stride] = Lanes<V>::make(res);
         }
-        voted[i * ld_voted + j] = Lanes<V>::make(res);
     }
 }
 

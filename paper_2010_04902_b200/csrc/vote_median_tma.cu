@@ -191,7 +191,8 @@ int launch_tma(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, flo
     auto kern = vote_median_tma_kernel<R, F, FC, STAGES>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return cuda_failed(e);
-    constexpr int ctas_per_sm = (227 * 1024) / (smem + 1024) >= 2 ? 2 : 1;
+    constexpr int fit = (227 * 1024) / (smem + 1024);  // CTAs whose rings fit in one SM (1 KB reserved each)
+    constexpr int ctas_per_sm = fit >= 4 ? 4 : (fit >= 1 ? fit : 1);
     int64_t grid = (d + kTileD - 1) / kTileD;
     if (grid > kNumSMs * ctas_per_sm) grid = kNumSMs * ctas_per_sm;
     kern<<<static_cast<int>(grid), kThreads, smem, s>>>(map, d, out);
@@ -216,7 +217,7 @@ int vote_median_tma(const float* rep, int r, int f, int64_t d, int64_t ld_file, 
     BZ_TMA_CASE(5, 49, 13, 2)
     BZ_TMA_CASE(7, 49, 10, 2)
     BZ_TMA_CASE(1, 25, 25, 4)
-    BZ_TMA_CASE(1, 49, 49, 3)
+    BZ_TMA_CASE(1, 49, 49, 2)
 #undef BZ_TMA_CASE
     return 1;
 }

@@ -4,9 +4,18 @@
 // Every worker is a 64-bit mask of the files it holds.  The number of holders of each file inside
 // S is kept bit-sliced in three 64-bit planes (counts 0..7, enough for r <= 7): adding a worker is
 // a ripple-carry add of its mask, the threshold ">= r'" is a Boolean function of the planes and the
-// answer is one popcount.  Threads take fixed-size runs of consecutive lexicographic ranks, unrank
-// the first subset of a run with the combinatorial number system and then walk successors,
-// keeping the plane state of every prefix so that a successor only redoes the changed suffix.
+// answer is one popcount.
+//
+// Enumeration: a subset is a prefix of p = q - T workers followed by a tail of T <= 5 workers.  The
+// tail is T nested loops with all state in registers - about twenty integer instructions per
+// subset.  Prefixes are grouped by their largest worker l: inside a group every prefix has the same
+// tail range (l, K), so the threads of a warp run the nested loops with identical trip counts.  A
+// group's prefixes are l plus the (p-1)-subsets of {0..l-1}; threads take chunks of consecutive
+// ones, unrank the first with the combinatorial number system and walk lexicographic successors,
+// keeping the plane state of every prefix length so that a successor redoes only the changed suffix.
+// The answer is the largest (count, membership mask with worker u at bit 63-u): the larger mask is
+// the lexicographically earlier subset, so ties resolve to the first maximiser whatever the order
+// of enumeration.
 #include "bz_common.cuh"
 
 namespace bz {
@@ -15,8 +24,9 @@ namespace {
 
 constexpr int kMaxK = 64;
 constexpr int kMaxQ = 64;
+constexpr int kMaxTail = 5;
 constexpr int kWcBlock = 128;
-constexpr uint64_t kRun = 2048;  // subsets per run
+constexpr uint64_t kSubsetsPerChunk = 16384;  // target work per chunk
 
 struct Planes {
     uint64_t c0, c1, c2;
@@ -32,71 +42,122 @@ __device__ __forceinline__ Planes add_mask(const Planes& s, uint64_t m) {
     return o;
 }
 
-// files with at least rp holders (rp in 1..4)
-__device__ __forceinline__ int count_at_least(const Planes& s, int rp) {
+// files with at least RP holders
+template <int RP> __device__ __forceinline__ int count_at_least(const Planes& s) {
     uint64_t hit;
-    if (rp == 1)
+    if constexpr (RP == 1)
         hit = s.c0 | s.c1 | s.c2;
-    else if (rp == 2)
+    else if constexpr (RP == 2)
         hit = s.c1 | s.c2;
-    else if (rp == 3)
+    else if constexpr (RP == 3)
         hit = s.c2 | (s.c1 & s.c0);
     else
         hit = s.c2;
     return __popcll(hit);
 }
 
+struct Best {
+    int cnt;
+    uint64_t mem;
+};
+
+__device__ __forceinline__ void offer(Best& b, int cnt, uint64_t mem) {
+    if (cnt > b.cnt || (cnt == b.cnt && mem > b.mem)) {
+        b.cnt = cnt;
+        b.mem = mem;
+    }
+}
+
+// LEVEL nested loops over the tail workers start <= w_1 < ... < w_LEVEL < K
+template <int RP, int LEVEL>
+__device__ __forceinline__ void tail_loops(const uint64_t* __restrict__ s_mask, const Planes& s, int start, int K,
+                                           uint64_t mem, Best& best) {
+    if constexpr (LEVEL == 1) {
+        for (int x = start; x < K; ++x) {
+            const int cnt = count_at_least<RP>(add_mask(s, s_mask[x]));
+            if (cnt >= best.cnt) offer(best, cnt, mem | (1ull << (63 - x)));
+        }
+    } else {
+        for (int y = start; y <= K - LEVEL; ++y)
+            tail_loops<RP, LEVEL - 1>(s_mask, add_mask(s, s_mask[y]), y + 1, K, mem | (1ull << (63 - y)), best);
+    }
+}
+
+// the outermost tail loop restricted to [y_lo, y_hi)
+template <int RP, int LEVEL>
+__device__ __forceinline__ void tail_top(const uint64_t* __restrict__ s_mask, const Planes& s, int y_lo, int y_hi, int K,
+                                         uint64_t mem, Best& best) {
+    if constexpr (LEVEL == 1) {
+        for (int x = y_lo; x < y_hi; ++x) {
+            const int cnt = count_at_least<RP>(add_mask(s, s_mask[x]));
+            if (cnt >= best.cnt) offer(best, cnt, mem | (1ull << (63 - x)));
+        }
+    } else {
+        for (int y = y_lo; y < y_hi; ++y)
+            tail_loops<RP, LEVEL - 1>(s_mask, add_mask(s, s_mask[y]), y + 1, K, mem | (1ull << (63 - y)), best);
+    }
+}
+
+// A group (all prefixes with the same largest worker) is cut into chunks along two axes: runs of
+// chunk_len consecutive prefixes, and - where one prefix alone has too many tails - pieces of y_width
+// values of the first tail worker.  Chunk index = piece * prefix_chunks + run, so neighbouring
+// threads hold neighbouring prefix runs of the same piece and loop in step.
 struct WcParams {
     uint64_t mask[kMaxK];
-    uint64_t total;  // C(K, q)
-    int K, q, rp;
+    uint64_t chunk_begin[kMaxK + 1];   // first chunk of each group; chunk_begin[n_groups] = number of chunks
+    uint64_t prefix_chunks[kMaxK];     // runs of prefixes in each group
+    uint32_t chunk_len[kMaxK];         // prefixes per run
+    uint32_t y_width[kMaxK];           // first-tail-worker values per piece
+    int K, q, p, n_groups, first_l;   // group g holds the prefixes whose largest worker is first_l + g
 };
 
 struct WcResult {
-    // a larger (count, members) pair is a better answer: count first, then the lexicographically
-    // earlier subset (worker u is bit 63-u of `members`, so an earlier subset is a larger integer)
-    uint32_t count;
+    int32_t count;
     uint32_t pad;
     uint64_t members;
 };
 
-__device__ __forceinline__ bool better(uint32_t c1, uint64_t m1, uint32_t c2, uint64_t m2) {
-    return c1 > c2 || (c1 == c2 && m1 > m2);
-}
-
 // binom[n][k] for n, k <= 64 (saturating), filled by the host into constant memory
 __constant__ uint64_t c_binom[kMaxK + 1][kMaxK + 1];
 
+template <int RP, int T>
 __global__ void __launch_bounds__(kWcBlock)
     worst_case_kernel(const __grid_constant__ WcParams prm, WcResult* __restrict__ results) {
     __shared__ uint64_t s_mask[kMaxK];
-    __shared__ uint32_t s_cnt[kWcBlock];
+    __shared__ uint64_t s_begin[kMaxK + 1];
+    __shared__ int32_t s_cnt[kWcBlock];
     __shared__ uint64_t s_mem[kWcBlock];
     for (int u = threadIdx.x; u < prm.K; u += blockDim.x) s_mask[u] = prm.mask[u];
+    for (int u = threadIdx.x; u <= prm.n_groups; u += blockDim.x) s_begin[u] = prm.chunk_begin[u];
     __syncthreads();
 
-    const int K = prm.K, q = prm.q, rp = prm.rp;
-    uint32_t best_cnt = 0;
-    uint64_t best_mem = 0;
-    bool have = false;
-
+    const int K = prm.K, p = prm.p;
+    Best best{-1, 0};
     int comb[kMaxQ];
-    Planes prefix[kMaxQ];  // prefix[i] = planes of comb[0..i-1]
+    Planes state[kMaxQ + 1];  // state[i] = planes of comb[0..i-1]
 
-    const uint64_t n_runs = (prm.total + kRun - 1) / kRun;
-    const uint64_t first_run = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    const uint64_t run_stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
-    for (uint64_t run = first_run; run < n_runs; run += run_stride) {
-        const uint64_t rank = run * kRun;
-        uint64_t left = prm.total - rank < kRun ? prm.total - rank : kRun;
-        // unrank: the rank-th q-subset in lexicographic order
+    const uint64_t n_chunks = s_begin[prm.n_groups];
+    const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
+    int g = 0;
+    for (uint64_t chunk = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; chunk < n_chunks; chunk += stride) {
+        while (chunk >= s_begin[g + 1]) ++g;  // chunks only move forward
+        const int l = prm.first_l + g;        // largest worker of the prefix (p >= 1), or -1 when p == 0
+        const int m = p - 1;                  // free prefix elements, from {0..l-1}
+        const uint64_t in_group = m > 0 ? c_binom[l][m] : 1;
+        const uint64_t in_g = chunk - s_begin[g];
+        const uint64_t piece = in_g / prm.prefix_chunks[g];
+        const uint64_t rank = (in_g - piece * prm.prefix_chunks[g]) * prm.chunk_len[g];
+        const int y_lo = l + 1 + static_cast<int>(piece) * static_cast<int>(prm.y_width[g]);
+        const int y_end = K - T + 1;  // the first tail worker leaves room for the other T-1
+        const int y_hi = y_lo + static_cast<int>(prm.y_width[g]) < y_end ? y_lo + static_cast<int>(prm.y_width[g]) : y_end;
+        uint64_t left = in_group - rank < prm.chunk_len[g] ? in_group - rank : prm.chunk_len[g];
+        // unrank: the rank-th m-subset of {0..l-1} in lexicographic order
         {
             int x = 0;
             uint64_t rest = rank;
-            for (int i = 0; i < q; ++i) {
-                // subsets whose element i is x (earlier elements fixed): C(K-1-x, q-1-i)
+            for (int i = 0; i < m; ++i) {
                 while (true) {
-                    const uint64_t cnt = c_binom[K - 1 - x][q - 1 - i];
+                    const uint64_t cnt = c_binom[l - 1 - x][m - 1 - i];  // subsets whose element i is x
                     if (rest < cnt) break;
                     rest -= cnt;
                     ++x;
@@ -104,43 +165,36 @@ __global__ void __launch_bounds__(kWcBlock)
                 comb[i] = x++;
             }
         }
-        prefix[0] = Planes{0, 0, 0};
-        for (int i = 0; i + 1 < q; ++i) prefix[i + 1] = add_mask(prefix[i], s_mask[comb[i]]);
+        if (p > 0) comb[p - 1] = l;
+        state[0] = Planes{0, 0, 0};
+        for (int i = 0; i < p; ++i) state[i + 1] = add_mask(state[i], s_mask[comb[i]]);
 
         while (true) {
-            // last position: sweep its remaining values with the prefix state fixed
-            const Planes base = prefix[q - 1];
-            for (int x = comb[q - 1]; x < K && left > 0; ++x, --left) {
-                const uint32_t cnt = static_cast<uint32_t>(count_at_least(add_mask(base, s_mask[x]), rp));
-                // a thread meets subsets in lexicographic order: only a larger count replaces
-                if (!have || cnt > best_cnt) {
-                    uint64_t mem = 1ull << (63 - x);
-                    for (int i = 0; i + 1 < q; ++i) mem |= 1ull << (63 - comb[i]);
-                    best_cnt = cnt;
-                    best_mem = mem;
-                    have = true;
-                }
-            }
-            if (left == 0) break;
-            // successor of the prefix comb[0..q-2]
-            int i = q - 2;
-            while (i >= 0 && comb[i] == K - q + i) --i;
-            if (i < 0) break;  // the last subset was reached; cannot happen while left > 0
+            uint64_t mem = 0;
+            for (int i = 0; i < p; ++i) mem |= 1ull << (63 - comb[i]);
+            tail_top<RP, T>(s_mask, state[p], y_lo, y_hi, K, mem, best);
+            if (--left == 0) break;
+            // successor of the free elements inside {0..l-1}
+            int i = m - 1;
+            while (i >= 0 && comb[i] == l - m + i) --i;
+            if (i < 0) break;  // the group's last prefix; cannot happen while left > 0
             ++comb[i];
-            for (int t = i + 1; t < q; ++t) comb[t] = comb[t - 1] + 1;
-            for (int t = i; t + 1 < q; ++t) prefix[t + 1] = add_mask(prefix[t], s_mask[comb[t]]);
+            for (int t = i + 1; t < m; ++t) comb[t] = comb[t - 1] + 1;
+            for (int t = i; t < p; ++t) state[t + 1] = add_mask(state[t], s_mask[comb[t]]);
         }
     }
 
-    // threads interleave their runs: reduce with the full (count, members) order
-    s_cnt[threadIdx.x] = have ? best_cnt : 0;
-    s_mem[threadIdx.x] = have ? best_mem : 0;
+    s_cnt[threadIdx.x] = best.cnt;
+    s_mem[threadIdx.x] = best.mem;
     __syncthreads();
     for (int off = kWcBlock / 2; off > 0; off >>= 1) {
-        if (threadIdx.x < off &&
-            better(s_cnt[threadIdx.x + off], s_mem[threadIdx.x + off], s_cnt[threadIdx.x], s_mem[threadIdx.x])) {
-            s_cnt[threadIdx.x] = s_cnt[threadIdx.x + off];
-            s_mem[threadIdx.x] = s_mem[threadIdx.x + off];
+        if (threadIdx.x < off) {
+            const int c2 = s_cnt[threadIdx.x + off];
+            const uint64_t m2 = s_mem[threadIdx.x + off];
+            if (c2 > s_cnt[threadIdx.x] || (c2 == s_cnt[threadIdx.x] && m2 > s_mem[threadIdx.x])) {
+                s_cnt[threadIdx.x] = c2;
+                s_mem[threadIdx.x] = m2;
+            }
         }
         __syncthreads();
     }
@@ -176,6 +230,17 @@ int upload_binom() {
     return BZ_OK;
 }
 
+template <int RP>
+void launch_tail(int tail, int grid, cudaStream_t s, const WcParams& prm, WcResult* dev) {
+    switch (tail) {
+        case 1: worst_case_kernel<RP, 1><<<grid, kWcBlock, 0, s>>>(prm, dev); break;
+        case 2: worst_case_kernel<RP, 2><<<grid, kWcBlock, 0, s>>>(prm, dev); break;
+        case 3: worst_case_kernel<RP, 3><<<grid, kWcBlock, 0, s>>>(prm, dev); break;
+        case 4: worst_case_kernel<RP, 4><<<grid, kWcBlock, 0, s>>>(prm, dev); break;
+        default: worst_case_kernel<RP, 5><<<grid, kWcBlock, 0, s>>>(prm, dev); break;
+    }
+}
+
 }  // namespace
 
 size_t worst_case_workspace_bytes() { return round_up(sizeof(WcResult) * kWcMaxBlocks, 256); }
@@ -207,16 +272,54 @@ extern "C" int bz_worst_case(const uint64_t* worker_mask, int K, int f, int r, i
     }
     WcParams prm;
     for (int u = 0; u < kMaxK; ++u) prm.mask[u] = u < K ? worker_mask[u] : 0;
-    prm.total = total;
+    const int tail = q < kMaxTail ? q : kMaxTail;
+    const int p = q - tail;
     prm.K = K;
     prm.q = q;
-    prm.rp = (r + 1) / 2;
-    const uint64_t n_runs = (total + kRun - 1) / kRun;
-    uint64_t blocks = (n_runs + kWcBlock - 1) / kWcBlock;
+    prm.p = p;
+    // chunk size: about kSubsetsPerChunk subsets, fewer when the whole search is small
+    uint64_t per_chunk = total / (static_cast<uint64_t>(kWcMaxBlocks) * kWcBlock * 4);
+    if (per_chunk > kSubsetsPerChunk) per_chunk = kSubsetsPerChunk;
+    if (per_chunk < 512) per_chunk = 512;
+    uint64_t n_chunks = 0;
+    // group g: prefixes whose largest worker is l = first_l + g (p == 0: the empty prefix, l = -1)
+    prm.first_l = p - 1;
+    prm.n_groups = p == 0 ? 1 : (K - tail - 1) - (p - 1) + 1;
+    for (int g = 0; g < prm.n_groups; ++g) {
+        const int l = prm.first_l + g;
+        const uint64_t prefixes = p == 0 ? 1 : h_binom[l][p - 1];
+        const uint64_t tails = h_binom[K - 1 - l][tail];
+        const int n_y = K - tail - l;  // values of the first tail worker
+        uint64_t len = 1, width = static_cast<uint64_t>(n_y);
+        if (tails <= per_chunk) {
+            len = per_chunk / tails;
+        } else {
+            // tails under the first value of the first tail worker (the largest share)
+            const uint64_t under_first = h_binom[K - 2 - l][tail - 1];
+            width = per_chunk / under_first;
+            if (width < 1) width = 1;
+            if (width > static_cast<uint64_t>(n_y)) width = static_cast<uint64_t>(n_y);
+        }
+        if (len > 0xffffffffull) len = 0xffffffffull;
+        const uint64_t pieces = (static_cast<uint64_t>(n_y) + width - 1) / width;
+        prm.chunk_begin[g] = n_chunks;
+        prm.chunk_len[g] = static_cast<uint32_t>(len);
+        prm.prefix_chunks[g] = (prefixes + len - 1) / len;
+        prm.y_width[g] = static_cast<uint32_t>(width);
+        n_chunks += pieces * prm.prefix_chunks[g];
+    }
+    prm.chunk_begin[prm.n_groups] = n_chunks;
+    uint64_t blocks = (n_chunks + kWcBlock - 1) / kWcBlock;
     if (blocks > static_cast<uint64_t>(kWcMaxBlocks)) blocks = kWcMaxBlocks;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     WcResult* dev = static_cast<WcResult*>(workspace);
-    worst_case_kernel<<<static_cast<int>(blocks), kWcBlock, 0, s>>>(prm, dev);
+    const int grid = static_cast<int>(blocks);
+    switch ((r + 1) / 2) {
+        case 1: launch_tail<1>(tail, grid, s, prm, dev); break;
+        case 2: launch_tail<2>(tail, grid, s, prm, dev); break;
+        case 3: launch_tail<3>(tail, grid, s, prm, dev); break;
+        default: launch_tail<4>(tail, grid, s, prm, dev); break;
+    }
     note_launch();
     st = check_launch();
     if (st != BZ_OK) return st;
@@ -225,14 +328,15 @@ extern "C" int bz_worst_case(const uint64_t* worker_mask, int K, int f, int r, i
     if (e != cudaSuccess) return cuda_failed(e);
     e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_failed(e);
-    uint32_t best_cnt = host[0].count;
+    int32_t best_cnt = host[0].count;
     uint64_t best_mem = host[0].members;
     for (uint64_t b = 1; b < blocks; ++b)
         if (host[b].count > best_cnt || (host[b].count == best_cnt && host[b].members > best_mem)) {
             best_cnt = host[b].count;
             best_mem = host[b].members;
         }
-    *c_max = static_cast<int32_t>(best_cnt);
+    if (best_cnt < 0) return BZ_ERR_CUDA;  // no thread saw a subset: cannot happen for a valid launch
+    *c_max = best_cnt;
     if (argmax) {
         int t = 0;
         for (int u = 0; u < K && t < q; ++u)

@@ -119,10 +119,11 @@ def test_bulyan_parity(l, r, q, attack, d, c, heavy):
     assert sel2.cpu().tolist() == want_sel.tolist()
 
 
-@pytest.mark.parametrize("theta,beta", [(5, 3), (7, 1), (9, 9), (17, 9), (25, 17), (27, 5), (49, 49), (49, 1),
-                                        (8, 3), (12, 12), (11, 5), (13, 7)])
+@pytest.mark.parametrize("theta,beta", [(5, 3), (7, 5), (9, 9), (9, 1), (15, 5), (17, 9), (19, 13), (23, 21), (25, 25),
+                                        (27, 5), (29, 9), (37, 25), (47, 45), (49, 49),          # register kernels
+                                        (7, 1), (25, 17), (49, 1), (8, 3), (12, 12), (11, 5), (13, 7)])  # generic
 def test_trimmed_mean_parity(theta, beta):
-    # specialised (odd theta with a network) and generic thetas; many duplicates and ties
+    # (theta, beta) pairs with a register kernel and pairs that take the generic one; many duplicates and ties
     rng = np.random.default_rng(theta * 64 + beta)
     f = max(theta, 25)
     v = rng.standard_normal((f, 2049)).astype(np.float32)

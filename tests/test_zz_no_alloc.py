@@ -51,7 +51,7 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
 
 def test_other_shapes_and_a_third_call():
     # generic kernel (f = 9 and the largest f that fits), unaligned rows, then f = 25 again
-    for f, d in [(9, 4001), (84, 700)]:
+    for f, d in [(9, 4001), (84, 700), (49, 30_001)]:
         v = inputs.true_gradients(f, d, seed=f).to(DEV)
         got = torch.empty((f, f), dtype=torch.float64, device=DEV)
         bz.pairdist_static(v, got)
@@ -67,7 +67,7 @@ def test_other_shapes_and_a_third_call():
 
 
 def test_shapes_beyond_the_built_in_scratch_are_refused():
-    for f in (49, 85, 121):
+    for f in (85, 100, 121):
         v = torch.zeros((f, 64), dtype=torch.float32, device=DEV)
         out = torch.full((f, f), -1.0, dtype=torch.float64, device=DEV)
         assert bz.workspace_bytes(bz.OP_PAIRDIST, 0, f, 64) > bz.STATIC_SCRATCH_BYTES
