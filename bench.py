@@ -349,6 +349,56 @@ def extra_paths(bz, inputs, torch, device):
     return res
 
 
+def profile_op(args):
+    """Profiling only: run ONE entry point `--steps` times on a synthetic case of `--coords` coordinates
+    (shape `--shape l,r,q`), so that a profiler capture sees just that kernel.  Prints its timing."""
+    import torch
+
+    from paper_2010_04902_b200 import binding as bz
+    from paper_2010_04902_b200 import build as bz_build
+    from paper_2010_04902_b200 import inputs
+    bz_build.build()
+    torch.cuda.set_device(0)
+    device = torch.device("cuda", 0)
+    l, r, q = (int(x) for x in args.shape.split(","))
+    f = l * l
+    d = args.coords if args.coords > 0 else 2_000_000
+    op = args.op
+    if op == "worst_case":
+        _, _, mask = bz.assign_mols(l, r)
+        ws = bz.alloc_workspace(bz.OP_WORST_CASE, r, f)
+        fn = lambda: bz.worst_case(mask, f, r, q, workspace=ws)
+    else:
+        cfg = dict(l=l, r=r, q=q, d=d, attack="reversed", seed=0)
+        rep, fw, byz, cmax = make_inputs(bz, inputs, cfg, device)
+        voted = bz.vote(rep)
+        out = torch.empty(d, dtype=torch.float32, device=device)
+        c = max(0, min(cmax, (f - 3) // 4))
+        ws = bz.alloc_workspace(bz.OP_MULTIKRUM, 0, f, d, c, f - c, device=device)
+        theta = f - 2 * c
+        sel = torch.arange(theta, dtype=torch.int32, device=device)
+        fn = {
+            "vote_median": lambda: bz.vote_median(rep, out),
+            "vote": lambda: bz.vote(rep, voted),
+            "median": lambda: bz.median(voted, out),
+            "pairdist": lambda: bz.pairdist(voted, ws),
+            "multikrum": lambda: bz.multikrum(voted, c, f - c, workspace=ws, out=out),
+            "bulyan": lambda: bz.bulyan(voted, c, workspace=ws, out=out),
+            "mean_rows": lambda: bz.mean_rows(voted, sel, out),
+            "trimmed_mean": lambda: bz.trimmed_mean(voted, sel, theta - 2 * c, out),
+        }[op]
+    t0 = time.perf_counter()
+    ms = timed(torch, fn, args.steps, args.warmup) if op != "worst_case" else None
+    if op == "worst_case":
+        for _ in range(args.warmup):
+            fn()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            fn()
+        ms = (time.perf_counter() - t0) / args.steps * 1e3
+    print(json.dumps({"profile_op": op, "shape": [l, r, q], "coordinates": d, "ms_per_call": ms}), flush=True)
+
+
 def run_reference(args):
     """The CPU checker, as it stands, on the host cores: each step is a bounded sample of the workload."""
     rank = int(os.environ.get("RANK", "0"))
@@ -393,10 +443,15 @@ def main():
     ap.add_argument("--coords", type=int, default=0, help="profiling only: override the number of coordinates d")
     ap.add_argument("--no-e2e", action="store_true", help="profiling only: skip the host-buffer leg")
     ap.add_argument("--no-cpu", action="store_true", help="profiling only: skip the CPU baseline / parity leg")
+    ap.add_argument("--op", default="", help="profiling only: run a single entry point (vote_median, vote, median, "
+                    "pairdist, multikrum, bulyan, mean_rows, trimmed_mean, worst_case) instead of the benchmark")
+    ap.add_argument("--shape", default="5,3,3", help="profiling only: l,r,q of the cluster for --op")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.impl == "reference":
+    if args.op:
+        profile_op(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

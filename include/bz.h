@@ -110,8 +110,9 @@ int bz_vote_median_host(const float* replicas_host, int r, int f, int64_t d, flo
 /*
  * Squared Euclidean distances between all pairs of voted gradients, the O(f^2 d) part of the
  * Krum family (Sec. 1.2; cost in Appendix A.1): dist[a][b] = sum_j (v_a[j] - v_b[j])^2.
- * Differences and squares are formed in binary32, added in binary32 over runs of at most 256
- * coordinates and in binary64 across runs, in a fixed order (results are reproducible).
+ * Differences and squares are formed in binary32, added in binary32 inside blocks of at most 1024
+ * coordinates (as interleaved partial sums of at most 128 terms) and in binary64 across blocks, in
+ * a fixed order (results are reproducible from run to run).
  *   dist  device, double [f][f], symmetric with a zero diagonal.
  *   workspace  device, bz_workspace_bytes(BZ_OP_PAIRDIST, 0, f, d, 0, 0) bytes, 256-byte aligned.
  */

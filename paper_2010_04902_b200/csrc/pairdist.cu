@@ -29,10 +29,10 @@ template <int F, int T, int G> struct PairTile {
     static_assert(NB * T == F, "T must divide F");
 };
 
-constexpr int kTD = 256;        // coordinates per tile
+constexpr int kTD = 128;        // coordinates per tile
 constexpr int kRowPad = 4;      // floats; keeps the row stride an odd number of 16-byte units
 constexpr int kRowStride = kTD + kRowPad;
-constexpr int kFlush = 4;       // tiles between two flushes of the binary32 accumulators
+constexpr int kFlush = 8;       // tiles between two flushes of the binary32 accumulators
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src, int src_bytes) {
     const unsigned dst = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
@@ -46,11 +46,15 @@ template <int F, int T, int G> constexpr size_t tiled_smem_bytes() {
     return size_t(2) * F * kRowStride * 4 + (size_t(PT::NT) * PT::TT + 1) * 4 + size_t(PT::NPB) * PT::TT * 8;
 }
 
-// CTAs per SM the launch asks for: two where the shared memory of two fits
-template <int F, int T, int G> constexpr int tiled_ctas_per_sm() { return tiled_smem_bytes<F, T, G>() <= 110 * 1024 ? 2 : 1; }
+// CTAs per SM the launch asks for: as many as the shared memory holds (1 KB reserved each), at most 3.
+// Two or more let one CTA's barrier waits overlap another CTA's arithmetic.
+template <int F, int T, int G> constexpr int tiled_ctas_per_sm() {
+    const int fit = static_cast<int>((227 * 1024) / (tiled_smem_bytes<F, T, G>() + 1024));
+    return fit >= 3 ? 3 : (fit >= 1 ? fit : 1);
+}
 
 template <int F, int T, int G>
-__global__ void __launch_bounds__(PairTile<F, T, G>::NT)
+__global__ void __launch_bounds__(PairTile<F, T, G>::NT, tiled_ctas_per_sm<F, T, G>())
     pairdist_tiled_kernel(const float* __restrict__ v, int64_t d, int64_t ld, double* __restrict__ partial) {
     using PT = PairTile<F, T, G>;
     constexpr int NB = PT::NB, NPB = PT::NPB, NT = PT::NT, TT = PT::TT;
@@ -108,24 +112,23 @@ __global__ void __launch_bounds__(PairTile<F, T, G>::NT)
         const float* base = stage0 + buf * F * kRowStride;
 #pragma unroll 1
         for (int c4 = g; c4 < kTD / 4; c4 += G) {
-            float4 a[T], b[T];
+            float4 b[T];
+#pragma unroll
+            for (int u = 0; u < T; ++u) b[u] = *reinterpret_cast<const float4*>(base + (bj + NB * u) * kRowStride + 4 * c4);
 #pragma unroll
             for (int t = 0; t < T; ++t) {
-                a[t] = *reinterpret_cast<const float4*>(base + (bi + NB * t) * kRowStride + 4 * c4);
-                b[t] = *reinterpret_cast<const float4*>(base + (bj + NB * t) * kRowStride + 4 * c4);
-            }
-#pragma unroll
-            for (int t = 0; t < T; ++t)
+                const float4 a = *reinterpret_cast<const float4*>(base + (bi + NB * t) * kRowStride + 4 * c4);
 #pragma unroll
                 for (int u = 0; u < T; ++u) {
                     float s = acc[t * T + u];
                     float e;
-                    e = a[t].x - b[u].x; s = fmaf(e, e, s);
-                    e = a[t].y - b[u].y; s = fmaf(e, e, s);
-                    e = a[t].z - b[u].z; s = fmaf(e, e, s);
-                    e = a[t].w - b[u].w; s = fmaf(e, e, s);
+                    e = a.x - b[u].x; s = fmaf(e, e, s);
+                    e = a.y - b[u].y; s = fmaf(e, e, s);
+                    e = a.z - b[u].z; s = fmaf(e, e, s);
+                    e = a.w - b[u].w; s = fmaf(e, e, s);
                     acc[t * T + u] = s;
                 }
+            }
         }
         ++since_flush;
         if (since_flush == kFlush || next >= n_tiles) {  // uniform over the CTA
@@ -246,7 +249,7 @@ int pairdist_ctas(int64_t d, int tile, int per_sm = 1) {
 
 // specialisations: <F, T, G>
 #define BZ_PD_25 25, 5, 16
-#define BZ_PD_49 49, 7, 16
+#define BZ_PD_49 49, 7, 8
 
 template <int F, int T, int G> constexpr size_t tiled_partial_doubles() {
     return static_cast<size_t>(kNumSMs) * tiled_ctas_per_sm<F, T, G>() * PairTile<F, T, G>::NPB * PairTile<F, T, G>::TT;

@@ -7,8 +7,8 @@
 // answer is one popcount.
 //
 // Enumeration: a subset is a prefix of p = q - T workers followed by a tail of T <= 5 workers.  The
-// tail is T nested loops with all state in registers - about twenty integer instructions per
-// subset.  Prefixes are grouped by their largest worker l: inside a group every prefix has the same
+// tail is T nested loops with all state in registers; in the innermost one a subset costs a
+// load, an AND and a popcount.  Prefixes are grouped by their largest worker l: inside a group every prefix has the same
 // tail range (l, K), so the threads of a warp run the nested loops with identical trip counts.  A
 // group's prefixes are l plus the (p-1)-subsets of {0..l-1}; threads take chunks of consecutive
 // ones, unrank the first with the combinatorial number system and walk lexicographic successors,
@@ -56,10 +56,39 @@ template <int RP> __device__ __forceinline__ int count_at_least(const Planes& s)
     return __popcll(hit);
 }
 
+// files with exactly RP-1 holders: those one more holder would tip over the threshold
+template <int RP> __device__ __forceinline__ uint64_t one_short(const Planes& s) {
+    if constexpr (RP == 1)
+        return ~(s.c0 | s.c1 | s.c2);  // bits above the last file never meet a worker mask
+    else if constexpr (RP == 2)
+        return s.c0 & ~s.c1 & ~s.c2;
+    else if constexpr (RP == 3)
+        return s.c1 & ~s.c0 & ~s.c2;
+    else
+        return s.c0 & s.c1 & ~s.c2;
+}
+
 struct Best {
     int cnt;
     uint64_t mem;
 };
+
+// tail workers chosen by the enclosing loops (outermost first); only read when a candidate is offered
+struct TailIds {
+    int w[4];
+};
+
+__device__ __forceinline__ uint64_t member_bits(uint64_t prefix_mem, const TailIds& ids, int n_ids, int x) {
+    uint64_t mem = prefix_mem | (1ull << (63 - x));
+    for (int i = 0; i < n_ids; ++i) mem |= 1ull << (63 - ids.w[i]);
+    return mem;
+}
+
+// innermost loop: adding worker x distorts exactly the files that were one holder short, so the
+// count under each x is the count of the enclosing subset plus one popcount
+template <int RP, int DEPTH>
+__device__ __forceinline__ void leaf_loop(const uint64_t* __restrict__ s_mask, const Planes& s, int x_lo, int x_hi,
+                                          uint64_t prefix_mem, const TailIds& ids, Best& best);
 
 __device__ __forceinline__ void offer(Best& b, int cnt, uint64_t mem) {
     if (cnt > b.cnt || (cnt == b.cnt && mem > b.mem)) {
@@ -68,18 +97,28 @@ __device__ __forceinline__ void offer(Best& b, int cnt, uint64_t mem) {
     }
 }
 
+template <int RP, int DEPTH>
+__device__ __forceinline__ void leaf_loop(const uint64_t* __restrict__ s_mask, const Planes& s, int x_lo, int x_hi,
+                                          uint64_t prefix_mem, const TailIds& ids, Best& best) {
+    const int base = count_at_least<RP>(s);
+    const uint64_t tip = one_short<RP>(s);
+    for (int x = x_lo; x < x_hi; ++x) {
+        const int cnt = base + __popcll(s_mask[x] & tip);
+        if (cnt >= best.cnt) offer(best, cnt, member_bits(prefix_mem, ids, DEPTH, x));
+    }
+}
+
 // LEVEL nested loops over the tail workers start <= w_1 < ... < w_LEVEL < K
-template <int RP, int LEVEL>
+template <int RP, int LEVEL, int DEPTH>
 __device__ __forceinline__ void tail_loops(const uint64_t* __restrict__ s_mask, const Planes& s, int start, int K,
-                                           uint64_t mem, Best& best) {
+                                           uint64_t prefix_mem, TailIds& ids, Best& best) {
     if constexpr (LEVEL == 1) {
-        for (int x = start; x < K; ++x) {
-            const int cnt = count_at_least<RP>(add_mask(s, s_mask[x]));
-            if (cnt >= best.cnt) offer(best, cnt, mem | (1ull << (63 - x)));
-        }
+        leaf_loop<RP, DEPTH>(s_mask, s, start, K, prefix_mem, ids, best);
     } else {
-        for (int y = start; y <= K - LEVEL; ++y)
-            tail_loops<RP, LEVEL - 1>(s_mask, add_mask(s, s_mask[y]), y + 1, K, mem | (1ull << (63 - y)), best);
+        for (int y = start; y <= K - LEVEL; ++y) {
+            ids.w[DEPTH] = y;
+            tail_loops<RP, LEVEL - 1, DEPTH + 1>(s_mask, add_mask(s, s_mask[y]), y + 1, K, prefix_mem, ids, best);
+        }
     }
 }
 
@@ -87,14 +126,14 @@ __device__ __forceinline__ void tail_loops(const uint64_t* __restrict__ s_mask, 
 template <int RP, int LEVEL>
 __device__ __forceinline__ void tail_top(const uint64_t* __restrict__ s_mask, const Planes& s, int y_lo, int y_hi, int K,
                                          uint64_t mem, Best& best) {
+    TailIds ids;
     if constexpr (LEVEL == 1) {
-        for (int x = y_lo; x < y_hi; ++x) {
-            const int cnt = count_at_least<RP>(add_mask(s, s_mask[x]));
-            if (cnt >= best.cnt) offer(best, cnt, mem | (1ull << (63 - x)));
-        }
+        leaf_loop<RP, 0>(s_mask, s, y_lo, y_hi, mem, ids, best);
     } else {
-        for (int y = y_lo; y < y_hi; ++y)
-            tail_loops<RP, LEVEL - 1>(s_mask, add_mask(s, s_mask[y]), y + 1, K, mem | (1ull << (63 - y)), best);
+        for (int y = y_lo; y < y_hi; ++y) {
+            ids.w[0] = y;
+            tail_loops<RP, LEVEL - 1, 1>(s_mask, add_mask(s, s_mask[y]), y + 1, K, mem, ids, best);
+        }
     }
 }
 
