@@ -30,7 +30,7 @@ WORKLOAD = dict(l=5, r=3, q=3, d=11_200_000, attack="reversed", seed=0)
 
 # DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum, scaled to a full launch), or None when no capture of the current kernel exists.
-TRAFFIC_BYTES_PER_LAUNCH = None
+TRAFFIC_BYTES_PER_LAUNCH = 3_426_670_000  # (600.03 + 11.87) MB at d = 2 M, scaled by 5.6 to d = 11.2 M
 
 
 def workload_name(cfg):
