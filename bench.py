@@ -30,7 +30,7 @@ WORKLOAD = dict(l=5, r=3, q=3, d=11_200_000, attack="reversed", seed=0)
 
 # DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum, scaled to a full launch), or None when no capture of the current kernel exists.
-TRAFFIC_BYTES_PER_LAUNCH = 3_426_670_000  # (600.03 + 11.87) MB at d = 2 M, scaled by 5.6 to d = 11.2 M
+TRAFFIC_BYTES_PER_LAUNCH = 3_429_614_000  # (600.03 + 12.40) MB at d = 2 M, scaled by 5.6 to d = 11.2 M
 
 
 def workload_name(cfg):
@@ -238,7 +238,7 @@ def run_ours(args):
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "peak_source": peak_src, "frac_of_nominal_8TBs": achieved / 8000.0,
                          "algorithmic_bytes_per_launch": alg_bytes,
-                         "kernel": "vote_median_tma_kernel<3,25,25,2> (one launch per step)"},
+                         "kernel": "vote_median_tma_kernel<3,25,25,3> (one launch per step)"},
         }
 
     # ---- CPU baseline and parity of the timed output (single-GPU run only) ----------------------------

@@ -211,8 +211,8 @@ int vote_median_tma(const float* rep, int r, int f, int64_t d, int64_t ld_file, 
     if (d < 4 * kTileD) return 1;  // tiny inputs: not worth a descriptor
 #define BZ_TMA_CASE(R_, F_, FC_, ST_) \
     if (r == R_ && f == F_) return launch_tma<R_, F_, FC_, ST_>(rep, d, ld_file, ld_rep, out, s);
-    BZ_TMA_CASE(3, 25, 25, 2)
-    BZ_TMA_CASE(3, 49, 25, 2)
+    BZ_TMA_CASE(3, 25, 25, 3)
+    BZ_TMA_CASE(3, 49, 25, 3)
     BZ_TMA_CASE(5, 25, 13, 2)
     BZ_TMA_CASE(5, 49, 13, 2)
     BZ_TMA_CASE(7, 49, 10, 2)
