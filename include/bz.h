@@ -71,6 +71,18 @@ extern "C" {
 int bz_assign_mols(int l, int r, int32_t* worker_files, int32_t* file_workers, uint64_t* worker_mask);
 
 /*
+ * Task assignment from the Ramanujan bigraph of Sec. 4.2.1 (array-code matrix B whose block (a, b)
+ * is the a*b-th power of the s x s cyclic shift; H = B for m >= s, H = B^T for m < s).  Cluster
+ * shape per Eq. (7): (K, f, l, r) = (m*s, s*s, s, m) if m < s ("Case 1"), (s*s, m*s, m, s) otherwise
+ * ("Case 2"); m = s gives the same tables as bz_assign_mols(s, s).  Host only, synchronous.
+ *   m >= 2; s prime
+ *   worker_files   host, int32 [K][l] ascending            (may be NULL)
+ *   file_workers   host, int32 [f][r] ascending            (may be NULL)
+ *   worker_mask    host, uint64 [K]; requires f <= 64      (may be NULL)
+ */
+int bz_assign_ramanujan(int m, int s, int32_t* worker_files, int32_t* file_workers, uint64_t* worker_mask);
+
+/*
  * Majority vote (Eq. 3; Algorithm 1, the loop over files), element by element: voted[i][j] is
  * the 32-bit pattern that occurs most often among replicas[0..r-1][i][j]; among equally frequent
  * patterns the one first seen at the lowest k wins.  Equality is bitwise (+0 != -0, NaNs are

@@ -56,6 +56,26 @@ def assign(l: int, r: int):
     return wf, fw, (mask if f <= 64 else None)
 
 
+def ramanujan_dims(m: int, s: int):
+    """(K, f, l, r) of Eq. (7)."""
+    return (m * s, s * s, s, m) if m < s else (s * s, m * s, m, s)
+
+
+def assign_ramanujan(m: int, s: int):
+    """Sec. 4.2.1 array-code bigraph.  Returns (worker_files[K][l], file_workers[f][r], worker_mask or None)."""
+    lib = _load()
+    if m < 2 or s < 2:
+        raise ValueError("orc_assign_ramanujan(m=%d, s=%d) rejected" % (m, s))
+    K, f, l, r = ramanujan_dims(m, s)
+    wf = np.zeros((K, l), np.int32)
+    fw = np.zeros((f, r), np.int32)
+    mask = np.zeros(K, np.uint64)
+    rc = lib.orc_assign_ramanujan(ctypes.c_int(m), ctypes.c_int(s), _p(wf, _i32p), _p(fw, _i32p), _p(mask, _u64p))
+    if rc != 0:
+        raise ValueError("orc_assign_ramanujan(m=%d, s=%d) rejected: %d" % (m, s, rc))
+    return wf, fw, (mask if f <= 64 else None)
+
+
 def vote(replicas):
     """replicas [r][f][d] float32 -> voted [f][d] (Eq. 3, element by element)."""
     lib = _load()

@@ -15,6 +15,7 @@
 // where a header comment says "parity unpinned".
 //
 //   orc_assign            Algorithm 2 (MOLS placement) + Sec. 4.2.1 (Ramanujan Case 2, m = s = l)
+//   orc_assign_ramanujan  Sec. 4.2.1 Steps 1-3 and Eq. (7): the array-code matrix B, H = B or B^T
 //   orc_vote              Eq. (3): per-file majority over the r returned copies
 //   orc_vote_vectorwise   Eq. (3) read on whole vectors (Sec. 2, "Training Protocol")
 //   orc_median            coordinate-wise median of the f winners (Sec. 2 / Sec. 6.1)
@@ -122,6 +123,62 @@ int orc_assign(int l, int r, int32_t* worker_files, int32_t* file_workers, uint6
             worker_mask[u] = m;
         }
     }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Sec. 4.2.1, written out: P is the s x s cyclic shift with P[i][j] = 1 iff j = i - 1 (mod s); B is
+// the s x m block matrix whose block (a, b) is P^(a*b) (matrix powers by repeated multiplication);
+// H = B when m >= s (Case 2: K = s*s workers, f = m*s files) and H = B^T when m < s (Case 1:
+// K = m*s workers, f = s*s files), Eq. (7).  Rows of H are workers, columns are files.
+// worker_files[K][l] ascending, file_workers[f][r] ascending, worker_mask as in orc_assign.
+int orc_assign_ramanujan(int m, int s, int32_t* worker_files, int32_t* file_workers, uint64_t* worker_mask) {
+    if (m < 2 || !is_prime(s)) return -1;
+    typedef std::vector<std::vector<int>> Mat;
+    auto matmul = [&](const Mat& X, const Mat& Y) {
+        Mat Z(s, std::vector<int>(s, 0));
+        for (int i = 0; i < s; ++i)
+            for (int k = 0; k < s; ++k)
+                if (X[i][k])
+                    for (int j = 0; j < s; ++j) Z[i][j] += X[i][k] * Y[k][j];
+        return Z;
+    };
+    Mat I(s, std::vector<int>(s, 0)), P(s, std::vector<int>(s, 0));
+    for (int i = 0; i < s; ++i) {
+        I[i][i] = 1;
+        P[i][((i - 1) % s + s) % s] = 1;
+    }
+    const int rows = s * s, cols = m * s;
+    std::vector<std::vector<int>> B(rows, std::vector<int>(cols, 0));
+    for (int a = 0; a < s; ++a)
+        for (int b = 0; b < m; ++b) {
+            Mat blk = I;
+            for (int t = 0; t < a * b; ++t) blk = matmul(blk, P);
+            for (int x = 0; x < s; ++x)
+                for (int y = 0; y < s; ++y) B[a * s + x][b * s + y] = blk[x][y];
+        }
+    const bool case2 = m >= s;
+    const int K = case2 ? rows : cols, f = case2 ? cols : rows;
+    const int l = case2 ? m : s, r = case2 ? s : m;
+    std::vector<int> n_workers(f, 0);
+    for (int u = 0; u < K; ++u) {
+        int n = 0;
+        uint64_t mask = 0;
+        for (int x = 0; x < f; ++x) {
+            const int h = case2 ? B[u][x] : B[x][u];
+            if (h != 0 && h != 1) return -2;
+            if (h) {
+                if (n >= l || n_workers[x] >= r) return -2;
+                worker_files[u * l + n++] = x;
+                file_workers[x * r + n_workers[x]++] = u;
+                if (f <= 64) mask |= (uint64_t)1 << x;
+            }
+        }
+        if (n != l) return -2;
+        if (worker_mask && f <= 64) worker_mask[u] = mask;
+    }
+    for (int x = 0; x < f; ++x)
+        if (n_workers[x] != r) return -2;
     return 0;
 }
 

@@ -37,6 +37,7 @@ _c_int, _c_i64, _c_sz, _c_vp, _c_u64 = ctypes.c_int, ctypes.c_int64, ctypes.c_si
 
 _SIGNATURES = {
     "bz_assign_mols": (_c_int, [_c_int, _c_int, _c_vp, _c_vp, _c_vp]),
+    "bz_assign_ramanujan": (_c_int, [_c_int, _c_int, _c_vp, _c_vp, _c_vp]),
     "bz_vote": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_i64, _c_vp]),
     "bz_median": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_vp]),
     "bz_vote_median": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_vp]),
@@ -147,6 +148,22 @@ def assign_mols(l: int, r: int):
     mask = np.zeros(K, np.uint64) if l * l <= 64 else None
     st = lib().bz_assign_mols(l, r, wf.ctypes.data, fw.ctypes.data, mask.ctypes.data if mask is not None else None)
     _check(st, "bz_assign_mols(l=%d, r=%d)" % (l, r))
+    return wf, fw, mask
+
+
+def ramanujan_dims(m: int, s: int):
+    """(K, f, l, r) of Eq. (7) for the Ramanujan construction with parameters (m, s)."""
+    return (m * s, s * s, s, m) if m < s else (s * s, m * s, m, s)
+
+
+def assign_ramanujan(m: int, s: int):
+    """Sec. 4.2.1.  Returns numpy (worker_files[K][l], file_workers[f][r], worker_mask[K] or None)."""
+    K, f, l, r = ramanujan_dims(max(m, 1), max(s, 1))
+    wf = np.zeros((K, l), np.int32)
+    fw = np.zeros((f, r), np.int32)
+    mask = np.zeros(K, np.uint64) if f <= 64 else None
+    st = lib().bz_assign_ramanujan(m, s, wf.ctypes.data, fw.ctypes.data, mask.ctypes.data if mask is not None else None)
+    _check(st, "bz_assign_ramanujan(m=%d, s=%d)" % (m, s))
     return wf, fw, mask
 
 

@@ -66,6 +66,35 @@ extern "C" int bz_assign_mols(int l, int r, int32_t* worker_files, int32_t* file
     return BZ_OK;
 }
 
+extern "C" int bz_assign_ramanujan(int m, int s, int32_t* worker_files, int32_t* file_workers, uint64_t* worker_mask) {
+    if (m < 2 || s < 2 || s > 46340 || m > 46340 || !is_prime(s)) return BZ_ERR_INVALID_ARG;
+    // Block (a, b) of the array-code matrix is the a*b-th power of the cyclic shift: its entry (x, y)
+    // is 1 iff y = x - a*b (mod s).  m >= s: H = B, worker a*s + x holds file b*s + y.
+    // m < s: H = B^T, worker b*s + y holds file a*s + x.
+    const bool case2 = m >= s;
+    const int64_t K = case2 ? static_cast<int64_t>(s) * s : static_cast<int64_t>(m) * s;
+    const int64_t f = case2 ? static_cast<int64_t>(m) * s : static_cast<int64_t>(s) * s;
+    const int l = case2 ? m : s, r = case2 ? s : m;
+    if (worker_mask != nullptr && f > 64) return BZ_ERR_INVALID_ARG;
+    if (worker_mask)
+        for (int64_t u = 0; u < K; ++u) worker_mask[u] = 0;
+    for (int a = 0; a < s; ++a)
+        for (int b = 0; b < m; ++b) {
+            const int shift = static_cast<int>((static_cast<int64_t>(a) * b) % s);
+            for (int x = 0; x < s; ++x) {
+                const int y = (x - shift + s) % s;
+                const int64_t row = static_cast<int64_t>(a) * s + x, col = static_cast<int64_t>(b) * s + y;
+                const int64_t worker = case2 ? row : col, file = case2 ? col : row;
+                // the class of a worker (a resp. b) and the block index on the file side (b resp. a) order both lists
+                const int in_worker = case2 ? b : a, in_file = case2 ? a : b;
+                if (worker_files) worker_files[worker * l + in_worker] = static_cast<int32_t>(file);
+                if (file_workers) file_workers[file * r + in_file] = static_cast<int32_t>(worker);
+                if (worker_mask) worker_mask[worker] |= 1ull << file;
+            }
+        }
+    return BZ_OK;
+}
+
 extern "C" size_t bz_workspace_bytes(int op, int r, int f, int64_t d, int c, int m) {
     (void)c;
     (void)m;

@@ -65,6 +65,32 @@ def test_vote_median_and_multikrum_at_1m(l, r, qsel):
         assert e.value.status == bz.ERR_PRECONDITION
 
 
+def test_ramanujan_clusters():
+    from conftest import read_golden_rows
+    # Case 1, (m, s) = (3, 5): the printed (15,25,5,3) table holds for this graph too (Sec. 5.3.2)
+    wf, fw, mask = bz.assign_ramanujan(3, 5)
+    for K, f, l, r, q, cmax, _ in read_golden_rows("cmax_tables.txt"):
+        if (K, f, l, r) == ("15", "25", "5", "3"):
+            got, arg, _ = bz.worst_case(mask, 25, 3, int(q))
+            assert got == int(cmax) and oracle.count_distorted(fw, arg) == int(cmax)
+            want, warg, _ = oracle.worst_case(oracle.assign_ramanujan(3, 5)[0], 25, 3, int(q))
+            assert arg.tolist() == warg.tolist()
+    # Case 2 with m > s, (m, s) = (10, 5): K = 25 workers, f = 50 files (even: two middle values), r = 5
+    wf, fw, mask = bz.assign_ramanujan(10, 5)
+    cmax, byz, _ = bz.worst_case(mask, 50, 5, 6)
+    ocmax, obyz, _ = oracle.worst_case(oracle.assign_ramanujan(10, 5)[0], 50, 5, 6)
+    assert (cmax, byz.tolist()) == (ocmax, obyz.tolist())
+    g = inputs.true_gradients(50, 30_001, seed=3)
+    rep = inputs.build_replicas(g, fw, byz, "constant")
+    want_voted = oracle.vote(rep.numpy())
+    assert np.array_equal(_bits(bz.vote(rep.to(DEV))), _bits(want_voted))
+    assert np.array_equal(_bits(bz.vote_median(rep.to(DEV))), _bits(oracle.median(want_voted)))
+    out, sel = bz.multikrum(torch.from_numpy(want_voted).to(DEV), cmax, 50 - cmax)
+    want_out, want_sel, _ = oracle.multikrum(want_voted, cmax, 50 - cmax)
+    assert sel.cpu().tolist() == want_sel.tolist()
+    assert np.linalg.norm(out.cpu().numpy().astype(np.float64) - want_out) <= 1e-5 * np.linalg.norm(want_out)
+
+
 def test_hundred_million_coordinates():
     # (l, r) = (5, 3), d = 1e8: 30 GB of replicas, 7.5e9 elements - offsets need 64 bits
     l, r, q, d = 5, 3, 3, 100_000_000
