@@ -211,3 +211,14 @@ def count_distorted(file_workers, byz) -> int:
     b = np.ascontiguousarray(byz, np.int32)
     return int(lib.orc_count_distorted(_p(fw, _i32p), ctypes.c_int(f), ctypes.c_int(r), _p(b, _i32p),
                                        ctypes.c_int(len(b))))
+
+
+def model_update(w, g, eta: float, velocity=None, mu: float = 0.0):
+    """Eq. (1) step on copies of the state: returns (w_new, velocity_new or None)."""
+    lib = _load()
+    w = _f32(w).copy()
+    g = _f32(g)
+    v = None if velocity is None else _f32(velocity).copy()
+    lib.orc_model_update(_p(w, _f32p), None if v is None else _p(v, _f32p), _p(g, _f32p), ctypes.c_int64(w.shape[0]),
+                         ctypes.c_float(eta), ctypes.c_float(mu))
+    return w, v

@@ -22,6 +22,7 @@
 //   orc_pairdist ... orc_mean_rows      Krum / Multi-Krum (Sec. 1.2, Sec. 6.1)
 //   orc_bulyan_select, orc_trimmed_mean Bulyan (Sec. 1.2 trimmed mean, Sec. 6.1)
 //   orc_worst_case        c_max^(q) by exhaustive search (Sec. 5.3.2, Sec. 6.1)
+//   orc_model_update      Eq. (1) step on the aggregate, optional momentum (Sec. 6.1)
 
 #include <algorithm>
 #include <cmath>
@@ -436,6 +437,23 @@ int orc_count_distorted(const int32_t* file_workers, int f, int r, const int32_t
         if (holders >= rp) ++cnt;
     }
     return cnt;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Eq. (1) / Algorithm 1, the parameter server's last step: w <- w - eta * g with g the aggregate.
+// With a momentum coefficient mu (Sec. 6.1 trains with 0.9; the paper gives no formula, so the
+// heavy-ball form of the framework it trained with is taken): v <- mu * v + g, w <- w - eta * v.
+// v == null is the plain step of Eq. (1).  w and v are single-precision state; each new value is
+// formed in double from the stored singles and rounded once.
+void orc_model_update(float* w, float* v, const float* g, int64_t d, float eta, float mu) {
+    for (int64_t j = 0; j < d; ++j) {
+        double step = static_cast<double>(g[j]);
+        if (v != nullptr) {
+            v[j] = static_cast<float>(static_cast<double>(mu) * static_cast<double>(v[j]) + static_cast<double>(g[j]));
+            step = static_cast<double>(v[j]);
+        }
+        w[j] = static_cast<float>(static_cast<double>(w[j]) - static_cast<double>(eta) * step);
+    }
 }
 
 }  // extern "C"
