@@ -336,6 +336,22 @@ def extra_paths(bz, inputs, torch, device):
     del rep, voted, out, ws
     torch.cuda.empty_cache()
 
+    # vote + median + model update (Eq. 1 with momentum) in one pass, headline shape
+    cfg = dict(l=5, r=3, q=3, d=11_200_000, attack="reversed", seed=0)
+    rep, fw, byz, cmax = make_inputs(bz, inputs, cfg, device)
+    f, d, r = 25, cfg["d"], 3
+    w = torch.zeros(d, dtype=torch.float32, device=device)
+    vel = torch.zeros(d, dtype=torch.float32, device=device)
+    out = torch.empty(d, dtype=torch.float32, device=device)
+    t_fused = timed(torch, lambda: bz.vote_median_update(rep, w, 0.01, vel, 0.9), 20, 3)
+    t_vm = timed(torch, lambda: bz.vote_median(rep, out), 20, 3)
+    t_upd = timed(torch, lambda: bz.model_update(out, w, 0.01, vel, 0.9), 20, 3)
+    res["vote+median+update"] = dict(
+        workload="K=15 r=3 l=5 f=25 d=11.2M, aggregate applied to w with momentum in the same kernel",
+        ms=t_fused, ms_unfused=t_vm + t_upd, coordinates_per_s=d / (t_fused * 1e-3), **hbm((4 * r * f + 16) * d, t_fused))
+    del rep, w, vel, out
+    torch.cuda.empty_cache()
+
     # exhaustive worst case: (K, f, l, r) = (35, 49, 7, 5), q = 13 - the largest row the paper printed
     _, _, mask = bz.assign_mols(7, 5)
     ws = bz.alloc_workspace(bz.OP_WORST_CASE, 5, 49)

@@ -110,6 +110,28 @@ int bz_vote_median(const float* replicas, int r, int f, int64_t d, int64_t ld_fi
                    float* out, void* stream);
 
 /*
+ * bz_vote_median followed by the parameter server's model update (Eq. 1, last step of Algorithm 1)
+ * in the same pass, so the aggregate never makes a round trip through memory:
+ *     velocity == NULL:  w[j] <- w[j] - eta * g[j]
+ *     otherwise:         velocity[j] <- mu * velocity[j] + g[j];  w[j] <- w[j] - eta * velocity[j]
+ * with g the coordinate-wise median of the voted gradients (bit-identical to bz_vote_median's out).
+ * The momentum form is the heavy-ball one (Sec. 6.1 trains with mu = 0.9 and gives no formula).
+ * Each assignment is one fused multiply-add in binary32.
+ *   w, velocity  device [d], read and written in place; velocity may be NULL.  Neither may
+ *                overlap replicas or out.
+ *   out          device [d] or NULL: where non-NULL the aggregate is written as well.
+ * Errors as bz_vote_median; BZ_ERR_INVALID_ARG when w is NULL and d > 0.
+ */
+int bz_vote_median_update(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica,
+                          float* w, float* velocity, float eta, float mu, float* out, void* stream);
+
+/*
+ * The same update from an aggregate g[d] already in device memory (for the Multi-Krum and Bulyan
+ * outputs).  g must not overlap w or velocity.
+ */
+int bz_model_update(const float* g, int64_t d, float* w, float* velocity, float eta, float mu, void* stream);
+
+/*
  * The same aggregation for a caller whose gradients sit in HOST memory (ideally page-locked):
  * coordinate slabs are copied to the device workspace, aggregated there and the result is copied
  * back; the call returns after out_host is complete.  replicas_host is contiguous [r][f][d],

@@ -42,6 +42,9 @@ _SIGNATURES = {
     "bz_median": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_vp]),
     "bz_vote_median": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_vp]),
     "bz_vote_median_host": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_vp, _c_vp, _c_sz, _c_vp]),
+    "bz_vote_median_update": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_vp, ctypes.c_float,
+                                       ctypes.c_float, _c_vp, _c_vp]),
+    "bz_model_update": (_c_int, [_c_vp, _c_i64, _c_vp, _c_vp, ctypes.c_float, ctypes.c_float, _c_vp]),
     "bz_pairdist": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_vp, _c_sz, _c_vp]),
     "bz_pairdist_static": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_vp]),
     "bz_krum_select": (_c_int, [_c_vp, _c_int, _c_int, _c_int, _c_vp, _c_vp]),
@@ -213,6 +216,33 @@ def vote_median(replicas: torch.Tensor, out: torch.Tensor | None = None) -> torc
                               _dev(out, torch.float32, "out"), _stream())
     _check(st, "bz_vote_median")
     return out
+
+
+def _state(t, d: int, name: str):
+    if t is None:
+        return None
+    if t.dim() != 1 or t.numel() != d or not t.is_contiguous():
+        raise TypeError("%s must be a contiguous [d] tensor" % name)
+    return _dev(t, torch.float32, name)
+
+
+def vote_median_update(replicas: torch.Tensor, w: torch.Tensor, eta: float, velocity: torch.Tensor | None = None,
+                       mu: float = 0.0, out: torch.Tensor | None = None) -> None:
+    """bz_vote_median_update: aggregate and apply Eq. (1) to w (and velocity) in place; `out`, when given,
+    also receives the aggregate."""
+    r, f, d, ld_file, ld_rep = _replicas(replicas)
+    st = lib().bz_vote_median_update(_dev(replicas, torch.float32, "replicas"), r, f, d, ld_file, ld_rep,
+                                     _state(w, d, "w"), _state(velocity, d, "velocity"), eta, mu,
+                                     _state(out, d, "out"), _stream())
+    _check(st, "bz_vote_median_update")
+
+
+def model_update(g: torch.Tensor, w: torch.Tensor, eta: float, velocity: torch.Tensor | None = None,
+                 mu: float = 0.0) -> None:
+    d = g.numel()
+    st = lib().bz_model_update(_state(g, d, "g"), d, _state(w, d, "w"), _state(velocity, d, "velocity"), eta, mu,
+                               _stream())
+    _check(st, "bz_model_update")
 
 
 def vote_median_host(replicas_host: torch.Tensor, out_host: torch.Tensor, workspace: torch.Tensor) -> torch.Tensor:

@@ -87,6 +87,43 @@ __device__ __forceinline__ uint32_t vote_bits_dyn(const uint32_t* x, int r) {
     return best;
 }
 
+// ---- Eq. (1): the model update, applied where an aggregate is produced -------------------------
+// w == nullptr means "no update".  With a velocity buffer: v <- mu*v + g, w <- w - eta*v (one
+// fused multiply-add each); without: w <- w - eta*g.
+struct ModelUpdate {
+    float* w;
+    float* v;
+    float eta, mu;
+};
+__device__ __forceinline__ float update_lane(float w, float& v, float g, float eta, float mu, bool has_v) {
+    float step = g;
+    if (has_v) {
+        v = __fmaf_rn(mu, v, g);
+        step = v;
+    }
+    return __fmaf_rn(-eta, step, w);
+}
+__device__ __forceinline__ void apply_update(const ModelUpdate& u, int64_t j, float g) {
+    float v = 0.f;
+    const bool has_v = u.v != nullptr;
+    if (has_v) v = u.v[j];
+    u.w[j] = update_lane(u.w[j], v, g, u.eta, u.mu, has_v);
+    if (has_v) u.v[j] = v;
+}
+// four consecutive coordinates starting at 4*j4 (w and v 16-byte aligned)
+__device__ __forceinline__ void apply_update4(const ModelUpdate& u, int64_t j4, const uint4& gbits) {
+    const bool has_v = u.v != nullptr;
+    float4 w = reinterpret_cast<float4*>(u.w)[j4];
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (has_v) v = reinterpret_cast<float4*>(u.v)[j4];
+    w.x = update_lane(w.x, v.x, __uint_as_float(gbits.x), u.eta, u.mu, has_v);
+    w.y = update_lane(w.y, v.y, __uint_as_float(gbits.y), u.eta, u.mu, has_v);
+    w.z = update_lane(w.z, v.z, __uint_as_float(gbits.z), u.eta, u.mu, has_v);
+    w.w = update_lane(w.w, v.w, __uint_as_float(gbits.w), u.eta, u.mu, has_v);
+    reinterpret_cast<float4*>(u.w)[j4] = w;
+    if (has_v) reinterpret_cast<float4*>(u.v)[j4] = v;
+}
+
 // ---- streaming loads (read-once data: evict-first) -------------------------------------------
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }
 __device__ __forceinline__ uint32_t ld_stream(const uint32_t* p) { return __ldcs(p); }

@@ -14,11 +14,12 @@ namespace bz {
 
 // vote_median_tma.cu: BZ_OK / error, or 1 when the staged path does not apply
 int vote_median_tma(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* out,
-                    cudaStream_t s);
+                    const ModelUpdate& upd, cudaStream_t s);
 
 namespace {
 
 constexpr int kBlock = 128;
+constexpr ModelUpdate kNoUpdate = {nullptr, nullptr, 0.f, 0.f};
 
 // BZ_VOTE_MEDIAN_PATH=registers keeps the fused pass on the register path (for profiling the two
 // against each other); anything else lets the TMA-staged path run where it applies.
@@ -37,12 +38,24 @@ template <> struct Lanes<uint4> {
         return c == 0 ? v.x : (c == 1 ? v.y : (c == 2 ? v.z : v.w));
     }
     __device__ __forceinline__ static uint4 make(const uint32_t (&a)[4]) { return make_uint4(a[0], a[1], a[2], a[3]); }
+    __device__ __forceinline__ static void update(const ModelUpdate& u, int64_t j, const uint4& g) { apply_update4(u, j, g); }
 };
 template <> struct Lanes<uint32_t> {
     static constexpr int n = 1;
     __device__ __forceinline__ static uint32_t get(const uint32_t& v, int) { return v; }
     __device__ __forceinline__ static uint32_t make(const uint32_t (&a)[1]) { return a[0]; }
+    __device__ __forceinline__ static void update(const ModelUpdate& u, int64_t j, uint32_t g) {
+        apply_update(u, j, __uint_as_float(g));
+    }
 };
+
+// the same update for coordinates n and up
+ModelUpdate shifted(const ModelUpdate& u, int64_t n) {
+    ModelUpdate t = u;
+    if (t.w != nullptr) t.w += n;
+    if (t.v != nullptr) t.v += n;
+    return t;
+}
 
 // files fetched together before their votes are taken: keeps about 12 wide loads in flight
 template <int R, int VEC> constexpr int files_per_batch() {
@@ -51,10 +64,11 @@ template <int R, int VEC> constexpr int files_per_batch() {
     return b < 1 ? 1 : b;
 }
 
-// n = number of V-wide coordinate groups; ld_file / ld_rep in units of V.
+// n = number of V-wide coordinate groups; ld_file / ld_rep in units of V.  out may be null when
+// only the model update is wanted.
 template <int R, int F, typename V>
 __global__ void __launch_bounds__(kBlock) vote_median_kernel(const V* __restrict__ rep, int64_t n, int64_t ld_file,
-                                                              int64_t ld_rep, V* __restrict__ out) {
+                                                              int64_t ld_rep, V* __restrict__ out, const ModelUpdate upd) {
     constexpr int VEC = Lanes<V>::n;
     constexpr int B = files_per_batch<R, VEC>();
     const int64_t stride = static_cast<int64_t>(gridDim.x) * kBlock;
@@ -84,7 +98,9 @@ __global__ void __launch_bounds__(kBlock) vote_median_kernel(const V* __restrict
         uint32_t res[VEC];
 #pragma unroll
         for (int c = 0; c < VEC; ++c) res[c] = key_bits(MedianNet<F>::run(key[c]));
-        out[j] = Lanes<V>::make(res);
+        const V packed = Lanes<V>::make(res);
+        if (out != nullptr) out[j] = packed;
+        if (upd.w != nullptr) Lanes<V>::update(upd, j, packed);
     }
 }
 
@@ -125,7 +141,8 @@ __global__ void __launch_bounds__(256) vote_kernel(const V* __restrict__ rep, in
 // only (writes voted), mode 1: vote + median (writes out).
 __global__ void __launch_bounds__(128) generic_kernel(const uint32_t* __restrict__ rep, int r, int f, int64_t d,
                                                       int64_t ld_file, int64_t ld_rep, uint32_t* __restrict__ voted,
-                                                      int64_t ld_voted, float* __restrict__ out, int mode) {
+                                                      int64_t ld_voted, float* __restrict__ out, int mode,
+                                                      const ModelUpdate upd) {
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
     for (int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < d; j += stride) {
         int key[BZ_MAX_F];
@@ -148,11 +165,11 @@ __global__ void __launch_bounds__(128) generic_kernel(const uint32_t* __restrict
             if (rank == want_lo) k_lo = key[i];
             if (rank == want_hi) k_hi = key[i];
         }
-        if (f & 1)
-            out[j] = __uint_as_float(key_bits(k_lo));
-        else
-            out[j] = __fadd_rn(__fmul_rn(0.5f, __uint_as_float(key_bits(k_lo))),
-                               __fmul_rn(0.5f, __uint_as_float(key_bits(k_hi))));
+        const float med = (f & 1) ? __uint_as_float(key_bits(k_lo))
+                                  : __fadd_rn(__fmul_rn(0.5f, __uint_as_float(key_bits(k_lo))),
+                                              __fmul_rn(0.5f, __uint_as_float(key_bits(k_hi))));
+        if (out != nullptr) out[j] = med;
+        if (upd.w != nullptr) apply_update(upd, j, med);
     }
 }
 
@@ -165,38 +182,41 @@ int grid_for(int64_t work_items, int block, int ctas_per_sm) {
 }
 
 template <int R, int F, typename V>
-int launch_vm(const float* rep, int64_t n, int64_t ld_file, int64_t ld_rep, float* out, cudaStream_t s) {
+int launch_vm(const float* rep, int64_t n, int64_t ld_file, int64_t ld_rep, float* out, const ModelUpdate& upd,
+              cudaStream_t s) {
     if (n <= 0) return BZ_OK;
     constexpr int VEC = Lanes<V>::n;
     vote_median_kernel<R, F, V><<<grid_for(n, kBlock, 16), kBlock, 0, s>>>(
-        reinterpret_cast<const V*>(rep), n, ld_file / VEC, ld_rep / VEC, reinterpret_cast<V*>(out));
+        reinterpret_cast<const V*>(rep), n, ld_file / VEC, ld_rep / VEC, reinterpret_cast<V*>(out), upd);
     note_launch();
     return check_launch();
 }
 
 template <int R, int F>
-int vm_dispatch_vec(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, float* out, bool vec, cudaStream_t s) {
-    if (!vec) return launch_vm<R, F, uint32_t>(rep, d, ld_file, ld_rep, out, s);
+int vm_dispatch_vec(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, float* out, const ModelUpdate& upd,
+                    bool vec, cudaStream_t s) {
+    if (!vec) return launch_vm<R, F, uint32_t>(rep, d, ld_file, ld_rep, out, upd, s);
     const int64_t n4 = d / 4;
-    int st = launch_vm<R, F, uint4>(rep, n4, ld_file, ld_rep, out, s);
+    int st = launch_vm<R, F, uint4>(rep, n4, ld_file, ld_rep, out, upd, s);
     if (st != BZ_OK) return st;
-    return launch_vm<R, F, uint32_t>(rep + 4 * n4, d - 4 * n4, ld_file, ld_rep, out + 4 * n4, s);
+    return launch_vm<R, F, uint32_t>(rep + 4 * n4, d - 4 * n4, ld_file, ld_rep, out != nullptr ? out + 4 * n4 : nullptr,
+                                     shifted(upd, 4 * n4), s);
 }
 
 template <int R>
-int vm_dispatch_f(const float* rep, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* out, bool vec,
-                  cudaStream_t s) {
+int vm_dispatch_f(const float* rep, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* out,
+                  const ModelUpdate& upd, bool vec, cudaStream_t s) {
     switch (f) {
-        case 25: return vm_dispatch_vec<R, 25>(rep, d, ld_file, ld_rep, out, vec, s);
-        case 49: return vm_dispatch_vec<R, 49>(rep, d, ld_file, ld_rep, out, vec, s);
+        case 25: return vm_dispatch_vec<R, 25>(rep, d, ld_file, ld_rep, out, upd, vec, s);
+        case 49: return vm_dispatch_vec<R, 49>(rep, d, ld_file, ld_rep, out, upd, vec, s);
         default: return 1;  // not specialised
     }
 }
 
 int launch_generic(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted,
-                   int64_t ld_voted, float* out, int mode, cudaStream_t s) {
+                   int64_t ld_voted, float* out, int mode, const ModelUpdate& upd, cudaStream_t s) {
     generic_kernel<<<grid_for(d, 128, 8), 128, 0, s>>>(reinterpret_cast<const uint32_t*>(rep), r, f, d, ld_file, ld_rep,
-                                                       reinterpret_cast<uint32_t*>(voted), ld_voted, out, mode);
+                                                       reinterpret_cast<uint32_t*>(voted), ld_voted, out, mode, upd);
     note_launch();
     return check_launch();
 }
@@ -239,22 +259,24 @@ int validate_replicas(const float* rep, int r, int f, int64_t d, int64_t ld_file
 
 }  // namespace
 
+// out may be null when upd.w is not: then only the updated state is written.
 int vote_median_on_device(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* out,
-                          cudaStream_t s) {
-    const bool vec = aligned16(rep) && aligned16(out) && (ld_file % 4 == 0) && (r == 1 || ld_rep % 4 == 0);
+                          const ModelUpdate& upd, cudaStream_t s) {
+    const bool vec = aligned16(rep) && aligned16(out) && aligned16(upd.w) && aligned16(upd.v) && (ld_file % 4 == 0) &&
+                     (r == 1 || ld_rep % 4 == 0);
     int st = 1;
     if (staged_path_enabled()) {
-        st = vote_median_tma(rep, r, f, d, ld_file, ld_rep, out, s);
+        st = vote_median_tma(rep, r, f, d, ld_file, ld_rep, out, upd, s);
         if (st != 1) return st;
     }
     switch (r) {
-        case 1: st = vm_dispatch_f<1>(rep, f, d, ld_file, ld_rep, out, vec, s); break;
-        case 3: st = vm_dispatch_f<3>(rep, f, d, ld_file, ld_rep, out, vec, s); break;
-        case 5: st = vm_dispatch_f<5>(rep, f, d, ld_file, ld_rep, out, vec, s); break;
-        case 7: st = vm_dispatch_f<7>(rep, f, d, ld_file, ld_rep, out, vec, s); break;
+        case 1: st = vm_dispatch_f<1>(rep, f, d, ld_file, ld_rep, out, upd, vec, s); break;
+        case 3: st = vm_dispatch_f<3>(rep, f, d, ld_file, ld_rep, out, upd, vec, s); break;
+        case 5: st = vm_dispatch_f<5>(rep, f, d, ld_file, ld_rep, out, upd, vec, s); break;
+        case 7: st = vm_dispatch_f<7>(rep, f, d, ld_file, ld_rep, out, upd, vec, s); break;
         default: break;
     }
-    if (st == 1) st = launch_generic(rep, r, f, d, ld_file, ld_rep, nullptr, 0, out, 1, s);
+    if (st == 1) st = launch_generic(rep, r, f, d, ld_file, ld_rep, nullptr, 0, out, 1, upd, s);
     return st;
 }
 
@@ -268,7 +290,7 @@ extern "C" int bz_vote_median(const float* replicas, int r, int f, int64_t d, in
     if (st != BZ_OK) return st;
     if (out == nullptr && d > 0) return BZ_ERR_INVALID_ARG;
     if (d == 0) return BZ_OK;
-    return vote_median_on_device(replicas, r, f, d, ld_file, ld_replica, out, static_cast<cudaStream_t>(stream));
+    return vote_median_on_device(replicas, r, f, d, ld_file, ld_replica, out, kNoUpdate, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int bz_median(const float* voted, int f, int64_t d, int64_t ld, float* out, void* stream) {
@@ -276,7 +298,7 @@ extern "C" int bz_median(const float* voted, int f, int64_t d, int64_t ld, float
     if (st != BZ_OK) return st;
     if (out == nullptr && d > 0) return BZ_ERR_INVALID_ARG;
     if (d == 0) return BZ_OK;
-    return vote_median_on_device(voted, 1, f, d, ld, 0, out, static_cast<cudaStream_t>(stream));
+    return vote_median_on_device(voted, 1, f, d, ld, 0, out, kNoUpdate, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int bz_vote(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica,
@@ -293,7 +315,7 @@ extern "C" int bz_vote(const float* replicas, int r, int f, int64_t d, int64_t l
         case 3: return vote_dispatch<3>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, vec, s);
         case 5: return vote_dispatch<5>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, vec, s);
         case 7: return vote_dispatch<7>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, vec, s);
-        default: return launch_generic(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, nullptr, 0, s);
+        default: return launch_generic(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, nullptr, 0, kNoUpdate, s);
     }
 }
 
@@ -318,7 +340,7 @@ extern "C" int bz_vote_median_host(const float* replicas_host, int r, int f, int
         cudaError_t e = cudaMemcpy2DAsync(slab, S * sizeof(float), replicas_host + j0, d * sizeof(float),
                                           n * sizeof(float), static_cast<size_t>(r) * f, cudaMemcpyHostToDevice, s);
         if (e != cudaSuccess) return cuda_failed(e);
-        st = vote_median_on_device(slab, r, f, n, S, static_cast<int64_t>(f) * S, out_dev, s);
+        st = vote_median_on_device(slab, r, f, n, S, static_cast<int64_t>(f) * S, out_dev, kNoUpdate, s);
         if (st != BZ_OK) return st;
         e = cudaMemcpyAsync(out_host + j0, out_dev, n * sizeof(float), cudaMemcpyDeviceToHost, s);
         if (e != cudaSuccess) return cuda_failed(e);
@@ -326,4 +348,36 @@ extern "C" int bz_vote_median_host(const float* replicas_host, int r, int f, int
     cudaError_t e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_failed(e);
     return BZ_OK;
+}
+
+namespace bz {
+namespace {
+
+__global__ void __launch_bounds__(256) model_update_kernel(const float* __restrict__ g, int64_t d, const ModelUpdate upd) {
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < d; j += stride)
+        apply_update(upd, j, g[j]);
+}
+
+}  // namespace
+}  // namespace bz
+
+extern "C" int bz_vote_median_update(const float* replicas, int r, int f, int64_t d, int64_t ld_file,
+                                     int64_t ld_replica, float* w, float* velocity, float eta, float mu, float* out,
+                                     void* stream) {
+    int st = validate_replicas(replicas, r, f, d, ld_file, ld_replica);
+    if (st != BZ_OK) return st;
+    if (w == nullptr && d > 0) return BZ_ERR_INVALID_ARG;
+    if (d == 0) return BZ_OK;
+    const ModelUpdate upd = {w, velocity, eta, mu};
+    return vote_median_on_device(replicas, r, f, d, ld_file, ld_replica, out, upd, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int bz_model_update(const float* g, int64_t d, float* w, float* velocity, float eta, float mu, void* stream) {
+    if (d < 0 || ((g == nullptr || w == nullptr) && d > 0)) return BZ_ERR_INVALID_ARG;
+    if (d == 0) return BZ_OK;
+    const ModelUpdate upd = {w, velocity, eta, mu};
+    model_update_kernel<<<grid_for(d, 256, 8), 256, 0, static_cast<cudaStream_t>(stream)>>>(g, d, upd);
+    note_launch();
+    return check_launch();
 }

@@ -72,7 +72,8 @@ template <int R, int F, int FC> struct Shape {
 // full/empty barriers.
 template <int R, int F, int FC, int STAGES>
 __global__ void __launch_bounds__(kThreads)
-    vote_median_tma_kernel(const __grid_constant__ CUtensorMap map, int64_t d, float* __restrict__ out) {
+    vote_median_tma_kernel(const __grid_constant__ CUtensorMap map, int64_t d, float* __restrict__ out,
+                           const ModelUpdate upd) {
     using S = Shape<R, F, FC>;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     float* stages = reinterpret_cast<float*>(smem_raw);
@@ -121,10 +122,18 @@ __global__ void __launch_bounds__(kThreads)
     } else {
         // ---------------------------------------------------------------- consumers: one coordinate each
         int key[F];
+        const bool has_w = upd.w != nullptr, has_v = upd.v != nullptr;
         int64_t item = 0;
         bool alive = true;
         for (int64_t t = 0; t < my_tiles && alive; ++t) {
             const int64_t j = (blockIdx.x + t * gridDim.x) * kTileD + tid;
+            // the state this coordinate's update needs is requested now, so that its latency is spent
+            // under the votes and the median network rather than after them
+            float w_old = 0.f, v_old = 0.f;
+            if (has_w && j < d) {
+                w_old = upd.w[j];
+                if (has_v) v_old = upd.v[j];
+            }
 #pragma unroll
             for (int chunk = 0; chunk < S::kChunks; ++chunk, ++item) {
                 const int s = static_cast<int>(item % STAGES);
@@ -145,7 +154,14 @@ __global__ void __launch_bounds__(kThreads)
                 __syncwarp();
                 if ((tid & 31) == 0) mbar_arrive(&empty[s]);  // this warp is done reading the stage
             }
-            if (alive && j < d) out[j] = __uint_as_float(key_bits(MedianNet<F>::run(key)));
+            if (alive && j < d) {
+                const float med = __uint_as_float(key_bits(MedianNet<F>::run(key)));
+                if (out != nullptr) out[j] = med;
+                if (has_w) {
+                    upd.w[j] = update_lane(w_old, v_old, med, upd.eta, upd.mu, has_v);
+                    if (has_v) upd.v[j] = v_old;
+                }
+            }
         }
         if (!alive && (tid & 31) == 0) atomicAdd(&g_pipeline_timeouts, 1u);
     }
@@ -174,7 +190,8 @@ EncodeTiledFn encode_tiled() {
 }
 
 template <int R, int F, int FC, int STAGES>
-int launch_tma(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, float* out, cudaStream_t s) {
+int launch_tma(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, float* out, const ModelUpdate& upd,
+               cudaStream_t s) {
     using S = Shape<R, F, FC>;
     EncodeTiledFn enc = encode_tiled();
     if (enc == nullptr) return 1;
@@ -195,7 +212,7 @@ int launch_tma(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, flo
     constexpr int ctas_per_sm = fit >= 4 ? 4 : (fit >= 1 ? fit : 1);
     int64_t grid = (d + kTileD - 1) / kTileD;
     if (grid > kNumSMs * ctas_per_sm) grid = kNumSMs * ctas_per_sm;
-    kern<<<static_cast<int>(grid), kThreads, smem, s>>>(map, d, out);
+    kern<<<static_cast<int>(grid), kThreads, smem, s>>>(map, d, out, upd);
     note_launch();
     return check_launch();
 }
@@ -206,11 +223,11 @@ int launch_tma(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, flo
 // register path.  Requirements: 16-byte aligned base, leading dimensions multiples of 4 floats,
 // d below 2^31, a specialised (r, f).
 int vote_median_tma(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* out,
-                    cudaStream_t s) {
+                    const ModelUpdate& upd, cudaStream_t s) {
     if (!aligned16(rep) || (ld_file % 4) != 0 || (r > 1 && (ld_rep % 4) != 0) || d >= (int64_t(1) << 31)) return 1;
     if (d < 4 * kTileD) return 1;  // tiny inputs: not worth a descriptor
 #define BZ_TMA_CASE(R_, F_, FC_, ST_) \
-    if (r == R_ && f == F_) return launch_tma<R_, F_, FC_, ST_>(rep, d, ld_file, ld_rep, out, s);
+    if (r == R_ && f == F_) return launch_tma<R_, F_, FC_, ST_>(rep, d, ld_file, ld_rep, out, upd, s);
     BZ_TMA_CASE(3, 25, 25, 3)
     BZ_TMA_CASE(3, 49, 25, 3)
     BZ_TMA_CASE(5, 25, 13, 2)
