@@ -56,6 +56,7 @@ extern "C" {
 #define BZ_OP_BULYAN 3
 #define BZ_OP_WORST_CASE 4
 #define BZ_OP_VOTE_MEDIAN_HOST 5
+#define BZ_OP_WORST_CASE_MOLS 6
 
 /*
  * Task assignment (Algorithm 2; Sec. 4.1.1 for the squares L_alpha(i,j) = alpha*i + j over F_l).
@@ -237,6 +238,27 @@ int bz_bulyan(const float* voted, int f, int64_t d, int64_t ld, int c, float* ou
  */
 int bz_worst_case(const uint64_t* worker_mask, int K, int f, int r, int q, uint64_t max_subsets, int32_t* c_max,
                   int32_t* argmax, uint64_t* n_subsets, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The same search for the placement bz_assign_mols(l, r) makes (Algorithm 2; Ramanujan Case 2 when
+ * r == l), shortened by the design's symmetry: shifting all files by (i, j) -> (i + a, j + b) maps
+ * worker (k, s) to (k, s + alpha_k*a + b), so the l*l translations permute the workers inside each
+ * parallel class and leave the number of distorted files unchanged.  One set of workers per orbit
+ * is evaluated - the smallest of the orbit in lexicographic order - which keeps both results of
+ * bz_worst_case: c_max, and the lexicographically first maximiser.  The work drops by nearly l*l,
+ * which moves the wall Sec. 6.1 reports for the exhaustive search (K = 49 and large q).
+ *   l prime, l <= 7;  r odd, 3 <= r <= l;  0 <= q <= r*l.
+ *   max_subsets: BZ_ERR_BUDGET if the number of orbits is larger (0 = no limit).
+ *   c_max host int32 [1];  argmax host int32 [q] ascending (may be NULL);
+ *   n_orbits host: sets evaluated = orbits of q-subsets under the translations (may be NULL).
+ *   workspace device, bz_workspace_bytes(BZ_OP_WORST_CASE_MOLS, r, l*l, 0, 0, 0) bytes.
+ * Synchronises `stream`.
+ */
+int bz_worst_case_mols(int l, int r, int q, uint64_t max_subsets, int32_t* c_max, int32_t* argmax,
+                       uint64_t* n_orbits, void* workspace, size_t workspace_bytes, void* stream);
+
+/* The number of sets bz_worst_case_mols(l, r, q) evaluates.  Host only; needs no GPU. */
+int bz_mols_orbit_count(int l, int r, int q, uint64_t* n_orbits);
 
 /* Bytes of device workspace `op` needs for the given shape (arguments an op ignores may be 0). */
 size_t bz_workspace_bytes(int op, int r, int f, int64_t d, int c, int m);

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libbz.so")
 
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_PRECONDITION, ERR_WORKSPACE, ERR_BUDGET, ERR_CUDA = -1, -2, -3, -4, -5, -6
-OP_PAIRDIST, OP_MULTIKRUM, OP_BULYAN, OP_WORST_CASE, OP_VOTE_MEDIAN_HOST = 1, 2, 3, 4, 5
+OP_PAIRDIST, OP_MULTIKRUM, OP_BULYAN, OP_WORST_CASE, OP_VOTE_MEDIAN_HOST, OP_WORST_CASE_MOLS = 1, 2, 3, 4, 5, 6
 MAX_R, MAX_F = 15, 128
 
 
@@ -54,6 +54,8 @@ _SIGNATURES = {
     "bz_trimmed_mean": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_int, _c_int, _c_vp, _c_vp]),
     "bz_bulyan": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_int, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp]),
     "bz_worst_case": (_c_int, [_c_vp, _c_int, _c_int, _c_int, _c_int, _c_u64, _c_vp, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp]),
+    "bz_worst_case_mols": (_c_int, [_c_int, _c_int, _c_int, _c_u64, _c_vp, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp]),
+    "bz_mols_orbit_count": (_c_int, [_c_int, _c_int, _c_int, _c_vp]),
     "bz_workspace_bytes": (_c_sz, [_c_int, _c_int, _c_int, _c_i64, _c_int, _c_int]),
     "bz_status_string": (ctypes.c_char_p, [_c_int]),
     "bz_last_cuda_error": (ctypes.c_char_p, []),
@@ -182,6 +184,25 @@ def worst_case(worker_mask, f: int, r: int, q: int, max_subsets: int = 0, worksp
                              ctypes.addressof(n), ws.data_ptr(), ws.numel(), _stream())
     _check(st, "bz_worst_case(K=%d, q=%d)" % (K, q))
     return int(cmax.value), arg[:q].copy(), int(n.value)
+
+
+def worst_case_mols(l: int, r: int, q: int, max_subsets: int = 0, workspace: torch.Tensor | None = None):
+    """bz_worst_case_mols: c_max^(q) of the placement assign_mols(l, r), one set per translation orbit.
+    Returns (c_max, argmax[q] numpy, n_orbits)."""
+    ws = workspace if workspace is not None else alloc_workspace(OP_WORST_CASE_MOLS, r, l * l)
+    cmax = ctypes.c_int32(0)
+    n = ctypes.c_uint64(0)
+    arg = np.zeros(max(q, 1), np.int32)
+    st = lib().bz_worst_case_mols(l, r, q, max_subsets, ctypes.addressof(cmax), arg.ctypes.data, ctypes.addressof(n),
+                                  ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "bz_worst_case_mols(l=%d, r=%d, q=%d)" % (l, r, q))
+    return int(cmax.value), arg[:q].copy(), int(n.value)
+
+
+def mols_orbit_count(l: int, r: int, q: int) -> int:
+    n = ctypes.c_uint64(0)
+    _check(lib().bz_mols_orbit_count(l, r, q, ctypes.addressof(n)), "bz_mols_orbit_count")
+    return int(n.value)
 
 
 # --------------------------------------------------------------------------------------------- device

@@ -15,8 +15,8 @@ CSRC = os.path.join(PKG, "csrc")
 OBJ_DIR = os.path.join(ROOT, "_build")
 LIB = os.path.join(PKG, "libbz.so")
 
-HEADERS = [os.path.join(CSRC, "bz_common.cuh"), os.path.join(CSRC, "sort_networks.inc"),
-           os.path.join(ROOT, "include", "bz.h")]
+HEADERS = [os.path.join(CSRC, "bz_common.cuh"), os.path.join(CSRC, "worst_case_common.cuh"),
+           os.path.join(CSRC, "sort_networks.inc"), os.path.join(ROOT, "include", "bz.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]

@@ -10,6 +10,7 @@ namespace bz {
 
 size_t krum_workspace_bytes(int op, int f);   // krum.cu
 size_t worst_case_workspace_bytes();          // worst_case.cu
+size_t worst_case_mols_workspace_bytes(int l, int r);  // worst_case_mols.cu
 int pipeline_timeouts(unsigned int* count);   // vote_median_tma.cu
 
 namespace {
@@ -104,6 +105,12 @@ extern "C" size_t bz_workspace_bytes(int op, int r, int f, int64_t d, int c, int
         case BZ_OP_MULTIKRUM:
         case BZ_OP_BULYAN: return krum_workspace_bytes(op, f);
         case BZ_OP_WORST_CASE: return worst_case_workspace_bytes();
+        case BZ_OP_WORST_CASE_MOLS: {
+            int l = 2;
+            while (l * l < f) ++l;
+            if (l * l != f || l > 7 || r < 1 || r > l) return 0;
+            return worst_case_mols_workspace_bytes(l, r);
+        }
         case BZ_OP_VOTE_MEDIAN_HOST: {
             if (r < 1 || d < 0) return 0;
             // smallest useful slab: 64K coordinates (or all of them) of r*f rows plus the output row

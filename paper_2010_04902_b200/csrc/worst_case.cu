@@ -16,7 +16,7 @@
 // The answer is the largest (count, membership mask with worker u at bit 63-u): the larger mask is
 // the lexicographically earlier subset, so ties resolve to the first maximiser whatever the order
 // of enumeration.
-#include "bz_common.cuh"
+#include "worst_case_common.cuh"
 
 namespace bz {
 
@@ -25,53 +25,7 @@ namespace {
 constexpr int kMaxK = 64;
 constexpr int kMaxQ = 64;
 constexpr int kMaxTail = 5;
-constexpr int kWcBlock = 128;
 constexpr uint64_t kSubsetsPerChunk = 16384;  // target work per chunk
-
-struct Planes {
-    uint64_t c0, c1, c2;
-};
-
-__device__ __forceinline__ Planes add_mask(const Planes& s, uint64_t m) {
-    Planes o;
-    o.c0 = s.c0 ^ m;
-    const uint64_t k0 = s.c0 & m;
-    o.c1 = s.c1 ^ k0;
-    const uint64_t k1 = s.c1 & k0;
-    o.c2 = s.c2 ^ k1;
-    return o;
-}
-
-// files with at least RP holders
-template <int RP> __device__ __forceinline__ int count_at_least(const Planes& s) {
-    uint64_t hit;
-    if constexpr (RP == 1)
-        hit = s.c0 | s.c1 | s.c2;
-    else if constexpr (RP == 2)
-        hit = s.c1 | s.c2;
-    else if constexpr (RP == 3)
-        hit = s.c2 | (s.c1 & s.c0);
-    else
-        hit = s.c2;
-    return __popcll(hit);
-}
-
-// files with exactly RP-1 holders: those one more holder would tip over the threshold
-template <int RP> __device__ __forceinline__ uint64_t one_short(const Planes& s) {
-    if constexpr (RP == 1)
-        return ~(s.c0 | s.c1 | s.c2);  // bits above the last file never meet a worker mask
-    else if constexpr (RP == 2)
-        return s.c0 & ~s.c1 & ~s.c2;
-    else if constexpr (RP == 3)
-        return s.c1 & ~s.c0 & ~s.c2;
-    else
-        return s.c0 & s.c1 & ~s.c2;
-}
-
-struct Best {
-    int cnt;
-    uint64_t mem;
-};
 
 // tail workers chosen by the enclosing loops (outermost first); only read when a candidate is offered
 struct TailIds {
@@ -89,13 +43,6 @@ __device__ __forceinline__ uint64_t member_bits(uint64_t prefix_mem, const TailI
 template <int RP, int DEPTH>
 __device__ __forceinline__ void leaf_loop(const uint64_t* __restrict__ s_mask, const Planes& s, int x_lo, int x_hi,
                                           uint64_t prefix_mem, const TailIds& ids, Best& best);
-
-__device__ __forceinline__ void offer(Best& b, int cnt, uint64_t mem) {
-    if (cnt > b.cnt || (cnt == b.cnt && mem > b.mem)) {
-        b.cnt = cnt;
-        b.mem = mem;
-    }
-}
 
 template <int RP, int DEPTH>
 __device__ __forceinline__ void leaf_loop(const uint64_t* __restrict__ s_mask, const Planes& s, int x_lo, int x_hi,
@@ -148,12 +95,6 @@ struct WcParams {
     uint32_t chunk_len[kMaxK];         // prefixes per run
     uint32_t y_width[kMaxK];           // first-tail-worker values per piece
     int K, q, p, n_groups, first_l;   // group g holds the prefixes whose largest worker is first_l + g
-};
-
-struct WcResult {
-    int32_t count;
-    uint32_t pad;
-    uint64_t members;
 };
 
 // binom[n][k] for n, k <= 64 (saturating), filled by the host into constant memory
@@ -223,28 +164,9 @@ __global__ void __launch_bounds__(kWcBlock)
         }
     }
 
-    s_cnt[threadIdx.x] = best.cnt;
-    s_mem[threadIdx.x] = best.mem;
-    __syncthreads();
-    for (int off = kWcBlock / 2; off > 0; off >>= 1) {
-        if (threadIdx.x < off) {
-            const int c2 = s_cnt[threadIdx.x + off];
-            const uint64_t m2 = s_mem[threadIdx.x + off];
-            if (c2 > s_cnt[threadIdx.x] || (c2 == s_cnt[threadIdx.x] && m2 > s_mem[threadIdx.x])) {
-                s_cnt[threadIdx.x] = c2;
-                s_mem[threadIdx.x] = m2;
-            }
-        }
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) {
-        results[blockIdx.x].count = s_cnt[0];
-        results[blockIdx.x].pad = 0;
-        results[blockIdx.x].members = s_mem[0];
-    }
+    block_best(best, s_cnt, s_mem, results);
 }
 
-constexpr int kWcMaxBlocks = kNumSMs * 8;
 
 uint64_t h_binom[kMaxK + 1][kMaxK + 1];
 bool binom_ready = false;
@@ -362,24 +284,5 @@ extern "C" int bz_worst_case(const uint64_t* worker_mask, int K, int f, int r, i
     note_launch();
     st = check_launch();
     if (st != BZ_OK) return st;
-    static thread_local WcResult host[kWcMaxBlocks];
-    cudaError_t e = cudaMemcpyAsync(host, dev, sizeof(WcResult) * blocks, cudaMemcpyDeviceToHost, s);
-    if (e != cudaSuccess) return cuda_failed(e);
-    e = cudaStreamSynchronize(s);
-    if (e != cudaSuccess) return cuda_failed(e);
-    int32_t best_cnt = host[0].count;
-    uint64_t best_mem = host[0].members;
-    for (uint64_t b = 1; b < blocks; ++b)
-        if (host[b].count > best_cnt || (host[b].count == best_cnt && host[b].members > best_mem)) {
-            best_cnt = host[b].count;
-            best_mem = host[b].members;
-        }
-    if (best_cnt < 0) return BZ_ERR_CUDA;  // no thread saw a subset: cannot happen for a valid launch
-    *c_max = best_cnt;
-    if (argmax) {
-        int t = 0;
-        for (int u = 0; u < K && t < q; ++u)
-            if (best_mem & (1ull << (63 - u))) argmax[t++] = u;
-    }
-    return BZ_OK;
+    return collect_best(dev, static_cast<int>(blocks), K, q, c_max, argmax, s);
 }

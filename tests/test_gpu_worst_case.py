@@ -48,3 +48,56 @@ def test_budget():
         bz.worst_case(mask, 49, 5, 17, max_subsets=10 ** 9)
     assert e.value.status == bz.ERR_BUDGET
     assert bz.worst_case(mask, 49, 5, 3, max_subsets=math.comb(35, 3))[0] == 1
+
+
+# ---- the same search, one worker set per translation orbit ------------------------------------------------
+
+@pytest.mark.parametrize("K,f,l,r,q,cmax", _rows())
+def test_symmetric_search_on_printed_tables(K, f, l, r, q, cmax):
+    _, fw, _ = bz.assign_mols(l, r)
+    got, arg, n = bz.worst_case_mols(l, r, q)
+    assert got == cmax and n == bz.mols_orbit_count(l, r, q)
+    assert len(arg) == q and list(arg) == sorted(set(arg.tolist()))
+    assert oracle.count_distorted(fw, arg) == cmax
+
+
+@pytest.mark.parametrize("l,r,qs", [(5, 3, range(0, 16)), (5, 5, range(0, 10)), (7, 3, range(0, 9)), (7, 5, [0, 1, 2, 3, 5, 6]),
+                                    (7, 7, [1, 2, 4, 5]), (3, 3, range(0, 10))])
+def test_symmetric_search_first_maximiser_matches_oracle(l, r, qs):
+    # the oracle knows nothing of the symmetry: it walks all C(K, q) sets
+    wf, _, _ = oracle.assign(l, r)
+    for q in qs:
+        want, warg, _ = oracle.worst_case(wf, l * l, r, q)
+        got, arg, _ = bz.worst_case_mols(l, r, q)
+        assert got == want and arg.tolist() == warg.tolist(), (l, r, q)
+
+
+def test_symmetric_search_beyond_the_oracle():
+    # (K, f, l, r) = (35, 49, 7, 5), every q up to the honest-majority limit; (49, 49, 7, 7) likewise (q = 24: 6.3e13 sets, 1.3e12 orbits).
+    # Checked by what holds at any size: the reported set really distorts c_max files (recounted by the
+    # oracle), c_max grows with q, and it never exceeds the full search on the same masks where that is
+    # affordable.
+    for l, r, q_top, q_full in [(7, 5, 17, 11), (7, 7, 24, 8)]:
+        _, fw, mask = bz.assign_mols(l, r)
+        ws = bz.alloc_workspace(bz.OP_WORST_CASE_MOLS, r, l * l)
+        prev = 0
+        for q in range(1, q_top + 1):
+            got, arg, n = bz.worst_case_mols(l, r, q, workspace=ws)
+            assert oracle.count_distorted(fw, arg) == got and got >= prev
+            assert n == bz.mols_orbit_count(l, r, q)
+            prev = got
+            if q <= q_full:
+                full, farg, _ = bz.worst_case(mask, l * l, r, q)
+                assert (full, farg.tolist()) == (got, arg.tolist()), (l, r, q)
+
+
+def test_symmetric_search_budget_and_arguments():
+    with pytest.raises(bz.BzError) as e:
+        bz.worst_case_mols(7, 7, 20, max_subsets=10 ** 6)
+    assert e.value.status == bz.ERR_BUDGET
+    with pytest.raises(bz.BzError) as e:
+        bz.worst_case_mols(7, 5, 3, workspace=bz.alloc_workspace(bz.OP_WORST_CASE, 5, 49))
+    assert e.value.status == bz.ERR_WORKSPACE
+    with pytest.raises(bz.BzError) as e:
+        bz.worst_case_mols(5, 1, 2)
+    assert e.value.status == bz.ERR_UNSUPPORTED
