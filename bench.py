@@ -362,6 +362,20 @@ def extra_paths(bz, inputs, torch, device):
     dt = time.perf_counter() - t0
     res["worst_case"] = dict(workload="(K,f,l,r)=(35,49,7,5), q=13, all C(35,13) subsets", c_max=cmax, subsets=n,
                              seconds=dt, subsets_per_s=n / dt, argmax=[int(u) for u in arg])
+    # the same maximum from one worker set per translation orbit, and the largest cluster of the sweep
+    # (K = 49) up to its honest-majority limit q = 24, which the plain search cannot reach
+    ws = bz.alloc_workspace(bz.OP_WORST_CASE_MOLS, 7, 49)
+    bz.worst_case_mols(7, 5, 8, workspace=ws)
+    sym = {}
+    for l_, r_, q_ in [(7, 5, 13), (7, 7, 16), (7, 7, 24)]:
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        c_, arg_, n_ = bz.worst_case_mols(l_, r_, q_, workspace=ws)
+        dt = time.perf_counter() - t0
+        sym["K=%d q=%d" % (l_ * r_, q_)] = dict(c_max=c_, orbits=n_, seconds=dt, orbits_per_s=n_ / dt,
+                                                argmax=[int(u) for u in arg_])
+    assert sym["K=35 q=13"]["c_max"] == cmax and sym["K=35 q=13"]["argmax"] == [int(u) for u in arg]
+    res["worst_case_orbits"] = sym
     return res
 
 

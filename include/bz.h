@@ -228,6 +228,31 @@ int bz_bulyan(const float* voted, int f, int64_t d, int64_t ld, int c, float* ou
               void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * bz_vote and bz_pairdist in one pass over the replicas: the winners of Eq. (3) are written to
+ * `voted` and enter the distance sums of Sec. 1.2 from on-chip memory, so the voted rows are not
+ * read back (4*f of the 4*(r*f + 2*f) bytes per coordinate the two calls move are saved).
+ * voted is bit-identical to bz_vote's; dist is summed as in bz_pairdist.  Shapes without a fused
+ * kernel (r*f outside {3,5}x{25,49} and 7x49, unaligned or short arrays) run the two calls.
+ *   replicas, ld_file, ld_replica as bz_vote;  voted device [f][d] with ld_voted (written);
+ *   dist device double [f][f];  workspace as bz_pairdist.
+ */
+int bz_vote_pairdist(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica, float* voted,
+                     int64_t ld_voted, double* dist, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Multi-Krum from the replicas: bz_vote_pairdist, bz_krum_select, bz_mean_rows.  Arguments as
+ * bz_multikrum, plus the replicas and the voted rows (written).
+ */
+int bz_vote_multikrum(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica, int c, int m,
+                      float* voted, int64_t ld_voted, float* out, int32_t* selected, double* dist, void* workspace,
+                      size_t workspace_bytes, void* stream);
+
+/* Bulyan from the replicas: bz_vote_pairdist, bz_bulyan_select, bz_trimmed_mean.  Arguments as bz_bulyan. */
+int bz_vote_bulyan(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica, int c,
+                   float* voted, int64_t ld_voted, float* out, int32_t* selected, void* workspace,
+                   size_t workspace_bytes, void* stream);
+
+/*
  * Worst-case number of distorted files (Sec. 5.3.2 "exhaustive simulations"; Sec. 6.1: the
  * attacked set is the maximiser): over all q-subsets S of the K workers, the largest number of
  * files with at least r' = (r+1)/2 holders in S, and the lexicographically first S attaining it.

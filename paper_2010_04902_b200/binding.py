@@ -54,6 +54,11 @@ _SIGNATURES = {
     "bz_trimmed_mean": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_int, _c_int, _c_vp, _c_vp]),
     "bz_bulyan": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_int, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp]),
     "bz_worst_case": (_c_int, [_c_vp, _c_int, _c_int, _c_int, _c_int, _c_u64, _c_vp, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp]),
+    "bz_vote_pairdist": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_i64, _c_vp, _c_vp, _c_sz, _c_vp]),
+    "bz_vote_multikrum": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_int, _c_int, _c_vp, _c_i64, _c_vp, _c_vp,
+                                   _c_vp, _c_vp, _c_sz, _c_vp]),
+    "bz_vote_bulyan": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_int, _c_vp, _c_i64, _c_vp, _c_vp, _c_vp,
+                                _c_sz, _c_vp]),
     "bz_worst_case_mols": (_c_int, [_c_int, _c_int, _c_int, _c_u64, _c_vp, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp]),
     "bz_mols_orbit_count": (_c_int, [_c_int, _c_int, _c_int, _c_vp]),
     "bz_workspace_bytes": (_c_sz, [_c_int, _c_int, _c_int, _c_i64, _c_int, _c_int]),
@@ -372,3 +377,60 @@ def bulyan(voted: torch.Tensor, c: int, workspace: torch.Tensor | None = None, o
                          sel.data_ptr(), ws.data_ptr(), ws.numel(), _stream())
     _check(st, "bz_bulyan")
     return out, sel[:max(theta, 0)]
+
+
+# ------------------------------------------------------------------------- from the replicas in one pass
+
+def _voted_for(replicas: torch.Tensor, voted: torch.Tensor | None):
+    r, f, d, ld_file, ld_rep = _replicas(replicas)
+    if voted is None:
+        voted = torch.empty((f, d), dtype=torch.float32, device=replicas.device)
+    vf, vd, ld_v = _rows(voted, "voted")
+    if (vf, vd) != (f, d):
+        raise ValueError("voted must be [%d][%d]" % (f, d))
+    return r, f, d, ld_file, ld_rep, voted, ld_v
+
+
+def vote_pairdist(replicas: torch.Tensor, voted: torch.Tensor | None = None, workspace: torch.Tensor | None = None,
+                  dist: torch.Tensor | None = None):
+    """bz_vote_pairdist: returns (voted[f][d], dist[f][f])."""
+    r, f, d, ld_file, ld_rep, voted, ld_v = _voted_for(replicas, voted)
+    ws = workspace if workspace is not None else alloc_workspace(OP_PAIRDIST, 0, f, d, device=replicas.device)
+    if dist is None:
+        dist = torch.empty((f, f), dtype=torch.float64, device=replicas.device)
+    st = lib().bz_vote_pairdist(_dev(replicas, torch.float32, "replicas"), r, f, d, ld_file, ld_rep,
+                                _dev(voted, torch.float32, "voted"), ld_v, _dev(dist, torch.float64, "dist"),
+                                ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "bz_vote_pairdist")
+    return voted, dist
+
+
+def vote_multikrum(replicas: torch.Tensor, c: int, m: int, voted: torch.Tensor | None = None,
+                   workspace: torch.Tensor | None = None, out: torch.Tensor | None = None):
+    """bz_vote_multikrum: returns (out[d], selected[m], voted[f][d])."""
+    r, f, d, ld_file, ld_rep, voted, ld_v = _voted_for(replicas, voted)
+    ws = workspace if workspace is not None else alloc_workspace(OP_MULTIKRUM, 0, f, d, c, m, device=replicas.device)
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=replicas.device)
+    sel = torch.empty(max(m, 1), dtype=torch.int32, device=replicas.device)
+    st = lib().bz_vote_multikrum(_dev(replicas, torch.float32, "replicas"), r, f, d, ld_file, ld_rep, c, m,
+                                 _dev(voted, torch.float32, "voted"), ld_v, _dev(out, torch.float32, "out"),
+                                 sel.data_ptr(), None, ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "bz_vote_multikrum")
+    return out, sel[:m], voted
+
+
+def vote_bulyan(replicas: torch.Tensor, c: int, voted: torch.Tensor | None = None,
+                workspace: torch.Tensor | None = None, out: torch.Tensor | None = None):
+    """bz_vote_bulyan: returns (out[d], selected[f - 2c], voted[f][d])."""
+    r, f, d, ld_file, ld_rep, voted, ld_v = _voted_for(replicas, voted)
+    ws = workspace if workspace is not None else alloc_workspace(OP_BULYAN, 0, f, d, c, device=replicas.device)
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=replicas.device)
+    theta = f - 2 * c
+    sel = torch.empty(max(theta, 1), dtype=torch.int32, device=replicas.device)
+    st = lib().bz_vote_bulyan(_dev(replicas, torch.float32, "replicas"), r, f, d, ld_file, ld_rep, c,
+                              _dev(voted, torch.float32, "voted"), ld_v, _dev(out, torch.float32, "out"),
+                              sel.data_ptr(), ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "bz_vote_bulyan")
+    return out, sel[:max(theta, 0)], voted

@@ -12,6 +12,7 @@ size_t krum_workspace_bytes(int op, int f);   // krum.cu
 size_t worst_case_workspace_bytes();          // worst_case.cu
 size_t worst_case_mols_workspace_bytes(int l, int r);  // worst_case_mols.cu
 int pipeline_timeouts(unsigned int* count);   // vote_median_tma.cu
+int vote_pairdist_timeouts(unsigned int* count);  // vote_pairdist.cu
 
 namespace {
 std::atomic<uint64_t> g_launches{0};
@@ -138,7 +139,11 @@ extern "C" const char* bz_status_string(int status) {
 
 extern "C" int bz_pipeline_timeouts(unsigned int* count) {
     if (count == nullptr) return BZ_ERR_INVALID_ARG;
-    return pipeline_timeouts(count);
+    unsigned int a = 0, b = 0;
+    int st = pipeline_timeouts(&a);
+    if (st == BZ_OK) st = vote_pairdist_timeouts(&b);
+    *count = a + b;
+    return st;
 }
 
 extern "C" const char* bz_last_cuda_error(void) { return g_cuda_msg; }

@@ -6,7 +6,7 @@
 // nor on the size of an attacker's payload in other rows, which the Gram form |a|^2 + |b|^2 - 2ab
 // - and with it a tensor-core contraction - cannot offer at the precision the selection needs.
 // The work is therefore bound by the FP32 pipe: f(f-1) add/fma lane-operations per coordinate.
-#include "bz_common.cuh"
+#include "pairdist_tile.cuh"
 
 namespace bz {
 
@@ -21,37 +21,12 @@ namespace {
 // the G groups of a pair are added in binary32 in a fixed order and the result goes into the CTA's
 // binary64 accumulator in shared memory; one fixed-order reduction over CTAs finishes.
 // The result is bit-reproducible from run to run.
-template <int F, int T, int G> struct PairTile {
-    static constexpr int NB = F / T;
-    static constexpr int NPB = NB * (NB + 1) / 2;
-    static constexpr int NT = NPB * G;
-    static constexpr int TT = T * T;
-    static_assert(NB * T == F, "T must divide F");
-};
-
-constexpr int kTD = 128;        // coordinates per tile
-constexpr int kRowPad = 4;      // floats; keeps the row stride an odd number of 16-byte units
-constexpr int kRowStride = kTD + kRowPad;
-constexpr int kFlush = 8;       // tiles between two flushes of the binary32 accumulators
-
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src, int src_bytes) {
     const unsigned dst = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(gmem_src), "r"(src_bytes));
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
-
-template <int F, int T, int G> constexpr size_t tiled_smem_bytes() {
-    using PT = PairTile<F, T, G>;
-    return size_t(2) * F * kRowStride * 4 + (size_t(PT::NT) * PT::TT + 1) * 4 + size_t(PT::NPB) * PT::TT * 8;
-}
-
-// CTAs per SM the launch asks for: as many as the shared memory holds (1 KB reserved each), at most 3.
-// Two or more let one CTA's barrier waits overlap another CTA's arithmetic.
-template <int F, int T, int G> constexpr int tiled_ctas_per_sm() {
-    const int fit = static_cast<int>((227 * 1024) / (tiled_smem_bytes<F, T, G>() + 1024));
-    return fit >= 3 ? 3 : (fit >= 1 ? fit : 1);
-}
 
 template <int F, int T, int G>
 __global__ void __launch_bounds__(PairTile<F, T, G>::NT, tiled_ctas_per_sm<F, T, G>())
@@ -109,27 +84,7 @@ __global__ void __launch_bounds__(PairTile<F, T, G>::NT, tiled_ctas_per_sm<F, T,
         }
         __syncthreads();
 
-        const float* base = stage0 + buf * F * kRowStride;
-#pragma unroll 1
-        for (int c4 = g; c4 < kTD / 4; c4 += G) {
-            float4 b[T];
-#pragma unroll
-            for (int u = 0; u < T; ++u) b[u] = *reinterpret_cast<const float4*>(base + (bj + NB * u) * kRowStride + 4 * c4);
-#pragma unroll
-            for (int t = 0; t < T; ++t) {
-                const float4 a = *reinterpret_cast<const float4*>(base + (bi + NB * t) * kRowStride + 4 * c4);
-#pragma unroll
-                for (int u = 0; u < T; ++u) {
-                    float s = acc[t * T + u];
-                    float e;
-                    e = a.x - b[u].x; s = fmaf(e, e, s);
-                    e = a.y - b[u].y; s = fmaf(e, e, s);
-                    e = a.z - b[u].z; s = fmaf(e, e, s);
-                    e = a.w - b[u].w; s = fmaf(e, e, s);
-                    acc[t * T + u] = s;
-                }
-            }
-        }
+        accumulate_tile<F, T, G>(stage0 + buf * F * kRowStride, bi, bj, g, acc);
         ++since_flush;
         if (since_flush == kFlush || next >= n_tiles) {  // uniform over the CTA
             since_flush = 0;
@@ -152,34 +107,6 @@ __global__ void __launch_bounds__(PairTile<F, T, G>::NT, tiled_ctas_per_sm<F, T,
     __syncthreads();
     double* mine = partial + static_cast<size_t>(blockIdx.x) * NPB * TT;
     for (int e = tid; e < NPB * TT; e += NT) mine[e] = dsum[e];
-}
-
-// dist[a][b] = sum over CTAs (ascending) of the element of the pair's class block
-template <int F, int T, int G>
-__global__ void pairdist_tiled_reduce_kernel(const double* __restrict__ partial, int n_ctas, double* __restrict__ dist) {
-    using PT = PairTile<F, T, G>;
-    constexpr int NB = PT::NB, NPB = PT::NPB, TT = PT::TT;
-    const int p = blockIdx.x * blockDim.x + threadIdx.x;
-    if (p >= F * F) return;
-    const int a = p / F, b = p % F;
-    if (a > b) return;
-    if (a == b) {
-        dist[p] = 0.0;
-        return;
-    }
-    const int ra = a % NB, ta = a / NB, rb = b % NB, tb = b / NB;
-    int bi, bj, t, u;
-    if (ra <= rb) {
-        bi = ra; bj = rb; t = ta; u = tb;
-    } else {
-        bi = rb; bj = ra; t = tb; u = ta;
-    }
-    // index of (bi, bj) among the pairs bi <= bj in row-major order
-    const int pb = bi * NB - bi * (bi - 1) / 2 + (bj - bi);
-    double s = 0.0;
-    for (int cta = 0; cta < n_ctas; ++cta) s += partial[(static_cast<size_t>(cta) * NPB + pb) * TT + t * T + u];
-    dist[a * F + b] = s;
-    dist[b * F + a] = s;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -246,10 +173,6 @@ int pairdist_ctas(int64_t d, int tile, int per_sm = 1) {
     if (n_tiles < 1) n_tiles = 1;
     return static_cast<int>(n_tiles);
 }
-
-// specialisations: <F, T, G>
-#define BZ_PD_25 25, 5, 16
-#define BZ_PD_49 49, 7, 8
 
 template <int F, int T, int G> constexpr size_t tiled_partial_doubles() {
     return static_cast<size_t>(kNumSMs) * tiled_ctas_per_sm<F, T, G>() * PairTile<F, T, G>::NPB * PairTile<F, T, G>::TT;
