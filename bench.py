@@ -297,13 +297,17 @@ def extra_paths(bz, inputs, torch, device):
     t_mk = timed(torch, lambda: bz.multikrum(voted, 5, 44, workspace=ws, out=out), 5, 2)
     t_vm = timed(torch, lambda: bz.vote_median(rep, out), 5, 2)
     t_med = timed(torch, lambda: bz.median(voted, out), 5, 2)
+    t_vpd = timed(torch, lambda: bz.vote_pairdist(rep, voted, ws), 5, 2)
+    t_vmk = timed(torch, lambda: bz.vote_multikrum(rep, 5, 44, voted=voted, workspace=ws, out=out), 5, 2)
     bytes_pipeline = (4 * r * f + 4 * f + 4 * f + 4 * 44 + 4) * d
     res["vote+multikrum"] = dict(
         workload="K=21 r=3 l=7 f=49 d=11.2M, q=5 ALIE, c=5 m=44", c_max=cmax,
         coordinates_per_s=d / ((t_vote + t_mk) * 1e-3), ms_vote=t_vote, ms_multikrum=t_mk, ms_pairdist=t_pd,
         ms_mean_rows=t_mean, pairdist_fma_lane_ops_per_s=2 * (f * (f - 1) // 2) * d / (t_pd * 1e-3),
         vote=hbm((4 * r * f + 4 * f) * d, t_vote), mean_rows=hbm((4 * 44 + 4) * d, t_mean),
-        pipeline=hbm(bytes_pipeline, t_vote + t_mk))
+        pipeline=hbm(bytes_pipeline, t_vote + t_mk),
+        single_pass=dict(ms_vote_pairdist=t_vpd, ms_vote_multikrum=t_vmk, coordinates_per_s=d / (t_vmk * 1e-3),
+                         **hbm((4 * r * f + 4 * f + 4 * 44 + 4) * d, t_vmk)))
     res["vote+median f=49"] = dict(workload="same replicas, fused vote+median", ms=t_vm, coordinates_per_s=d / (t_vm * 1e-3),
                                    **hbm((4 * r * f + 4) * d, t_vm))
     res["median f=49"] = dict(workload="median of the 49 voted rows", ms=t_med, coordinates_per_s=d / (t_med * 1e-3),
@@ -324,13 +328,16 @@ def extra_paths(bz, inputs, torch, device):
     t_tm = timed(torch, lambda: bz.trimmed_mean(voted, sel17, 9, out), 5, 2)
     t_bu = timed(torch, lambda: bz.bulyan(voted, 4, workspace=ws, out=out), 5, 2)
     t_vm = timed(torch, lambda: bz.vote_median(rep, out), 5, 2)
+    t_vbu = timed(torch, lambda: bz.vote_bulyan(rep, 4, voted=voted, workspace=ws, out=out), 5, 2)
     theta = f - 8
     bytes_pipeline = (4 * r * f + 4 * f + 4 * f + 4 * theta + 4) * d
     res["vote+bulyan"] = dict(
         workload="K=25 r=5 l=5 f=25 d=25M (1% Student-t coordinates), q=6 constant, c=4 (theta=17, beta=9)",
         c_max=cmax, coordinates_per_s=d / ((t_vote + t_bu) * 1e-3), ms_vote=t_vote, ms_bulyan=t_bu, ms_pairdist=t_pd,
         ms_trimmed_mean=t_tm, vote=hbm((4 * r * f + 4 * f) * d, t_vote), pairdist=hbm(4 * f * d, t_pd),
-        trimmed_mean=hbm((4 * theta + 4) * d, t_tm), pipeline=hbm(bytes_pipeline, t_vote + t_bu))
+        trimmed_mean=hbm((4 * theta + 4) * d, t_tm), pipeline=hbm(bytes_pipeline, t_vote + t_bu),
+        single_pass=dict(ms_vote_bulyan=t_vbu, coordinates_per_s=d / (t_vbu * 1e-3),
+                         **hbm((4 * r * f + 4 * f + 4 * theta + 4) * d, t_vbu)))
     res["vote+median r=5"] = dict(workload="same replicas, fused vote+median", ms=t_vm, coordinates_per_s=d / (t_vm * 1e-3),
                                   **hbm((4 * r * f + 4) * d, t_vm))
     del rep, voted, out, ws
@@ -398,6 +405,9 @@ def profile_op(args):
         _, _, mask = bz.assign_mols(l, r)
         ws = bz.alloc_workspace(bz.OP_WORST_CASE, r, f)
         fn = lambda: bz.worst_case(mask, f, r, q, workspace=ws)
+    elif op == "worst_case_mols":
+        ws = bz.alloc_workspace(bz.OP_WORST_CASE_MOLS, r, f)
+        fn = lambda: bz.worst_case_mols(l, r, q, workspace=ws)
     else:
         cfg = dict(l=l, r=r, q=q, d=d, attack="reversed", seed=0)
         rep, fw, byz, cmax = make_inputs(bz, inputs, cfg, device)
@@ -412,14 +422,16 @@ def profile_op(args):
             "vote": lambda: bz.vote(rep, voted),
             "median": lambda: bz.median(voted, out),
             "pairdist": lambda: bz.pairdist(voted, ws),
+            "vote_pairdist": lambda: bz.vote_pairdist(rep, voted, ws),
+            "vote_median_update": lambda: bz.vote_median_update(rep, out, 0.01, voted[0], 0.9),
             "multikrum": lambda: bz.multikrum(voted, c, f - c, workspace=ws, out=out),
             "bulyan": lambda: bz.bulyan(voted, c, workspace=ws, out=out),
             "mean_rows": lambda: bz.mean_rows(voted, sel, out),
             "trimmed_mean": lambda: bz.trimmed_mean(voted, sel, theta - 2 * c, out),
         }[op]
     t0 = time.perf_counter()
-    ms = timed(torch, fn, args.steps, args.warmup) if op != "worst_case" else None
-    if op == "worst_case":
+    ms = timed(torch, fn, args.steps, args.warmup) if not op.startswith("worst_case") else None
+    if op.startswith("worst_case"):
         for _ in range(args.warmup):
             fn()
         t0 = time.perf_counter()
@@ -474,7 +486,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="profiling only: skip the host-buffer leg")
     ap.add_argument("--no-cpu", action="store_true", help="profiling only: skip the CPU baseline / parity leg")
     ap.add_argument("--op", default="", help="profiling only: run a single entry point (vote_median, vote, median, "
-                    "pairdist, multikrum, bulyan, mean_rows, trimmed_mean, worst_case) instead of the benchmark")
+                    "pairdist, vote_pairdist, vote_median_update, multikrum, bulyan, mean_rows, trimmed_mean, worst_case, "
+                    "worst_case_mols) instead of the benchmark")
     ap.add_argument("--shape", default="5,3,3", help="profiling only: l,r,q of the cluster for --op")
     args = ap.parse_args()
     if args.warmup < 3:
