@@ -15,8 +15,12 @@ CSRC = os.path.join(PKG, "csrc")
 OBJ_DIR = os.path.join(ROOT, "_build")
 LIB = os.path.join(PKG, "libbz.so")
 
-HEADERS = [os.path.join(CSRC, "bz_common.cuh"), os.path.join(CSRC, "worst_case_common.cuh"),
-           os.path.join(CSRC, "sort_networks.inc"), os.path.join(ROOT, "include", "bz.h")]
+
+
+def _headers():
+    return (sorted(glob.glob(os.path.join(CSRC, "*.cuh"))) + sorted(glob.glob(os.path.join(CSRC, "*.inc")))
+            + [os.path.join(ROOT, "include", "bz.h")])
+
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
@@ -48,7 +52,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     for s in _sources():
         o = os.path.join(OBJ_DIR, os.path.basename(s).replace(".cu", ".o"))
         objs.append(o)
-        if force or _stale(o, [s] + HEADERS):
+        if force or _stale(o, [s] + _headers()):
             jobs.append([nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o])
 
     def run(cmd):
