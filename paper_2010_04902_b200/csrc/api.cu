@@ -13,6 +13,7 @@ size_t worst_case_workspace_bytes();          // worst_case.cu
 size_t worst_case_mols_workspace_bytes(int l, int r);  // worst_case_mols.cu
 int pipeline_timeouts(unsigned int* count);   // vote_median_tma.cu
 int vote_pairdist_timeouts(unsigned int* count);  // vote_pairdist.cu
+int pairdist_i8_timeouts(unsigned int* count);    // pairdist_i8.cu
 
 namespace {
 std::atomic<uint64_t> g_launches{0};
@@ -139,10 +140,11 @@ extern "C" const char* bz_status_string(int status) {
 
 extern "C" int bz_pipeline_timeouts(unsigned int* count) {
     if (count == nullptr) return BZ_ERR_INVALID_ARG;
-    unsigned int a = 0, b = 0;
+    unsigned int a = 0, b = 0, c = 0;
     int st = pipeline_timeouts(&a);
     if (st == BZ_OK) st = vote_pairdist_timeouts(&b);
-    *count = a + b;
+    if (st == BZ_OK) st = pairdist_i8_timeouts(&c);
+    *count = a + b + c;
     return st;
 }
 

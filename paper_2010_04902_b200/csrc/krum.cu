@@ -8,7 +8,7 @@ namespace bz {
 // pairdist.cu
 size_t pairdist_workspace(int f);
 size_t krum_workspace_bytes(int op, int f);
-int pairdist_on_device(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, cudaStream_t s);
+int pairdist_on_device(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, cudaStream_t s, bool tensor_cores);
 int validate_rows(const float* v, int f, int64_t d, int64_t ld);
 int check_workspace(void* ws, size_t have, size_t need);
 
@@ -293,7 +293,7 @@ extern "C" int bz_multikrum(const float* voted, int f, int64_t d, int64_t ld, in
     if (st != BZ_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     double* D = dist ? dist : reinterpret_cast<double*>(static_cast<char*>(workspace) + pairdist_workspace(f));
-    st = pairdist_on_device(voted, f, d, ld, D, workspace, s);
+    st = pairdist_on_device(voted, f, d, ld, D, workspace, s, true);
     if (st != BZ_OK) return st;
     st = bz_krum_select(D, f, c, m, selected, stream);
     if (st != BZ_OK) return st;
@@ -330,7 +330,7 @@ extern "C" int bz_bulyan(const float* voted, int f, int64_t d, int64_t ld, int c
     if (st != BZ_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     double* D = reinterpret_cast<double*>(static_cast<char*>(workspace) + pairdist_workspace(f));
-    st = pairdist_on_device(voted, f, d, ld, D, workspace, s);
+    st = pairdist_on_device(voted, f, d, ld, D, workspace, s, true);
     if (st != BZ_OK) return st;
     st = bz_bulyan_select(D, f, c, selected, stream);
     if (st != BZ_OK) return st;

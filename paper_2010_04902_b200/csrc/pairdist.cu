@@ -6,6 +6,9 @@
 // nor on the size of an attacker's payload in other rows, which the Gram form |a|^2 + |b|^2 - 2ab
 // - and with it a tensor-core contraction - cannot offer at the precision the selection needs.
 // The work is therefore bound by the FP32 pipe: f(f-1) add/fma lane-operations per coordinate.
+#include <cstdlib>
+#include <cstring>
+
 #include "pairdist_tile.cuh"
 
 namespace bz {
@@ -30,8 +33,10 @@ template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile(
 
 template <int F, int T, int G>
 __global__ void __launch_bounds__(PairTile<F, T, G>::NT, tiled_ctas_per_sm<F, T, G>())
-    pairdist_tiled_kernel(const float* __restrict__ v, int64_t d, int64_t ld, double* __restrict__ partial) {
+    pairdist_tiled_kernel(const float* __restrict__ v, int64_t d, int64_t ld, double* __restrict__ partial,
+                          const int* __restrict__ gate) {
     using PT = PairTile<F, T, G>;
+    if (gate != nullptr && *gate == 0) return;  // the integer kernel's distances stand
     constexpr int NB = PT::NB, NPB = PT::NPB, NT = PT::NT, TT = PT::TT;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float* stage0 = reinterpret_cast<float*>(smem_raw);                            // 2 x [F][kRowStride]
@@ -179,24 +184,43 @@ template <int F, int T, int G> constexpr size_t tiled_partial_doubles() {
 }
 
 template <int F, int T, int G>
-int launch_pairdist_tiled(const float* v, int64_t d, int64_t ld, double* dist, double* partial, cudaStream_t s) {
+int launch_pairdist_tiled(const float* v, int64_t d, int64_t ld, double* dist, double* partial, const int* gate, cudaStream_t s) {
     constexpr int NT = PairTile<F, T, G>::NT;
     constexpr int smem = static_cast<int>(tiled_smem_bytes<F, T, G>());
     cudaError_t e = cudaFuncSetAttribute(pairdist_tiled_kernel<F, T, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return cuda_failed(e);
     const int ctas = pairdist_ctas(d, kTD, tiled_ctas_per_sm<F, T, G>());
-    pairdist_tiled_kernel<F, T, G><<<ctas, NT, smem, s>>>(v, d, ld, partial);
+    pairdist_tiled_kernel<F, T, G><<<ctas, NT, smem, s>>>(v, d, ld, partial, gate);
     note_launch();
     int st = check_launch();
     if (st != BZ_OK) return st;
-    pairdist_tiled_reduce_kernel<F, T, G><<<(F * F + 127) / 128, 128, 0, s>>>(partial, ctas, dist);
+    pairdist_tiled_reduce_kernel<F, T, G><<<(F * F + 127) / 128, 128, 0, s>>>(partial, ctas, dist, gate);
     note_launch();
     return check_launch();
 }
 
+// BZ_PAIRDIST_PATH=fp32 keeps the distances off the tensor cores; =i8 takes the integer kernel's
+// result even where its error estimate asks for the binary32 kernel (for tests of that kernel).
+enum { kPathAuto = 0, kPathFp32 = 1, kPathI8 = 2 };
+int pairdist_path() {
+    const char* e = std::getenv("BZ_PAIRDIST_PATH");
+    if (e == nullptr) return kPathAuto;
+    if (std::strcmp(e, "fp32") == 0) return kPathFp32;
+    if (std::strcmp(e, "i8") == 0) return kPathI8;
+    return kPathAuto;
+}
+
 }  // namespace
 
-size_t pairdist_workspace(int f) {
+bool pairdist_i8_has(int f);                  // pairdist_i8.cu
+size_t pairdist_i8_workspace(int f);
+int pairdist_i8(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, int force, int** flag_out, cudaStream_t s);
+
+int pairdist_path_fp32_only() { return pairdist_path() == kPathFp32; }
+int pairdist_path_i8_forced() { return pairdist_path() == kPathI8; }
+
+// the partial sums of the binary32 kernels alone (what bz_pairdist_static keeps in its array)
+size_t pairdist_workspace_fp32(int f) {
     size_t doubles;
     if (f == 25)
         doubles = tiled_partial_doubles<BZ_PD_25>();
@@ -208,11 +232,35 @@ size_t pairdist_workspace(int f) {
     return round_up(doubles * sizeof(double), 256);
 }
 
-int pairdist_on_device(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, cudaStream_t s) {
+// binary32 partial sums, then the integer kernel's partial matrices
+size_t pairdist_workspace(int f) { return pairdist_workspace_fp32(f) + pairdist_i8_workspace(f); }
+
+// The binary32 difference-form kernels.  gate != nullptr (only after the integer kernel ran, so on a
+// shape with a tiled kernel): they run only if *gate (device) is not 0.
+int pairdist_fp32(const float* v, int f, int64_t d, int64_t ld, double* dist, double* partial, const int* gate, cudaStream_t s);
+
+// tensor_cores: the workspace has room for the integer kernel (pairdist_workspace, not _fp32)
+int pairdist_on_device(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, cudaStream_t s, bool tensor_cores) {
     double* partial = static_cast<double*>(ws);
+    const int* gate = nullptr;
+    const int path = pairdist_path();
+    if (tensor_cores && path != kPathFp32) {
+        int* flag = nullptr;
+        const int st = pairdist_i8(v, f, d, ld, dist, static_cast<char*>(ws) + pairdist_workspace_fp32(f), path == kPathI8, &flag, s);
+        if (st == BZ_OK) {
+            if (path == kPathI8) return BZ_OK;
+            gate = flag;  // the binary32 kernels below run only if the flag asks for them
+        } else if (st != 1) {
+            return st;
+        }
+    }
+    return pairdist_fp32(v, f, d, ld, dist, partial, gate, s);
+}
+
+int pairdist_fp32(const float* v, int f, int64_t d, int64_t ld, double* dist, double* partial, const int* gate, cudaStream_t s) {
     const bool vec = aligned16(v) && (ld % 4 == 0);
-    if (vec && f == 25) return launch_pairdist_tiled<BZ_PD_25>(v, d, ld, dist, partial, s);
-    if (vec && f == 49) return launch_pairdist_tiled<BZ_PD_49>(v, d, ld, dist, partial, s);
+    if (vec && f == 25) return launch_pairdist_tiled<BZ_PD_25>(v, d, ld, dist, partial, gate, s);
+    if (vec && f == 49) return launch_pairdist_tiled<BZ_PD_49>(v, d, ld, dist, partial, gate, s);
     const int ctas = pairdist_ctas(d, kGT);
     pairdist_generic_kernel<<<ctas, 256, 0, s>>>(v, f, d, ld, partial);
     note_launch();
@@ -254,7 +302,7 @@ extern "C" int bz_pairdist(const float* voted, int f, int64_t d, int64_t ld, dou
     if (dist == nullptr) return BZ_ERR_INVALID_ARG;
     st = check_workspace(workspace, workspace_bytes, krum_workspace_bytes(BZ_OP_PAIRDIST, f));
     if (st != BZ_OK) return st;
-    return pairdist_on_device(voted, f, d, ld, dist, workspace, static_cast<cudaStream_t>(stream));
+    return pairdist_on_device(voted, f, d, ld, dist, workspace, static_cast<cudaStream_t>(stream), true);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -298,11 +346,11 @@ extern "C" int bz_pairdist_static(const float* voted, int f, int64_t d, int64_t 
     int st = validate_rows(voted, f, d, ld);
     if (st != BZ_OK) return st;
     if (dist == nullptr) return BZ_ERR_INVALID_ARG;
-    if (krum_workspace_bytes(BZ_OP_PAIRDIST, f) > kStaticScratchBytes) return BZ_ERR_STATIC_LIMIT;
+    if (pairdist_workspace_fp32(f) > kStaticScratchBytes) return BZ_ERR_STATIC_LIMIT;
     void* scratch = nullptr;
     st = static_scratch(&scratch);
     if (st != BZ_OK) return st;
     // Nothing in the array has to start at zero: the tiled kernel overwrites every partial sum the
     // reduction reads, and the generic kernel clears its own slots before it accumulates.
-    return pairdist_on_device(voted, f, d, ld, dist, scratch, static_cast<cudaStream_t>(stream));
+    return pairdist_on_device(voted, f, d, ld, dist, scratch, static_cast<cudaStream_t>(stream), false);
 }

@@ -1,0 +1,159 @@
+// Pairwise squared distances of the Krum family (Sec. 1.2; cost in Appendix A.1) on the tensor cores,
+// in exact integer arithmetic.  Host side; the kernel is in pairdist_i8_kernel.cuh.
+#include "pairdist_i8_kernel.cuh"
+
+namespace bz {
+
+namespace {
+
+// D from the CTAs' partial matrices, then the error estimate of the conversion.
+// flag[0] = 1 asks for the binary32 kernel (estimate above the tolerance, or values the fixed-point
+// scale cannot hold); with force != 0 the flag stays 0 whatever the estimate says.
+// Estimate for a pair: each value is rounded to a multiple of its row's step, an unbiased error of
+// standard deviation 0.29 step; over d coordinates that moves D by about 2 sqrt(D var) + d var.
+constexpr double kRelTol = 5e-9;
+
+template <int F>
+__global__ void __launch_bounds__(1024)
+    pairdist_i8_reduce_kernel(const double* __restrict__ tpart, const int* __restrict__ info, int n_ctas, int64_t d, int force,
+                              double* __restrict__ dist, int* __restrict__ flag) {
+    __shared__ double D[F * F];
+    __shared__ int s_emax[F];
+    __shared__ int s_bad;
+    const int tid = threadIdx.x;
+    if (tid < F) s_emax[tid] = kELo;
+    if (tid == 0) s_bad = 0;
+    __syncthreads();
+    for (int e = tid; e < n_ctas * kInfoStride; e += blockDim.x) {
+        const int a = e % kInfoStride;
+        if (a < F) atomicMax(&s_emax[a], info[e]);
+        if (a == kInfoBad && info[e]) atomicOr(&s_bad, 1);
+    }
+    for (int p = tid; p < F * F; p += blockDim.x) {
+        const int a = p / F, b = p % F;
+        if (a > b) continue;
+        double s = 0.0;
+        if (a < b)
+            for (int c = 0; c < n_ctas; ++c) {
+                const double* T = tpart + static_cast<size_t>(c) * F * F;
+                s += (T[a * F + a] + T[b * F + b]) - (T[a * F + b] + T[b * F + a]);
+            }
+        D[a * F + b] = s;
+        D[b * F + a] = s;
+    }
+    __syncthreads();
+    if (tid < F) {
+        const int a = tid;
+        const double step_a = __longlong_as_double(static_cast<long long>(1023 + s_emax[a] - 30) << 52);
+        double min_nz = 1e300, zero_step = 0.0;
+        bool bad = false;
+        for (int b = 0; b < F; ++b) {
+            if (b == a) continue;
+            const double step_b = __longlong_as_double(static_cast<long long>(1023 + s_emax[b] - 30) << 52);
+            const double var = 0.0841 * (step_a * step_a + step_b * step_b);
+            const double v = D[a * F + b];
+            if (v > 0.0) {
+                if (2.0 * sqrt(var / v) + static_cast<double>(d) * var / v > kRelTol) bad = true;
+                min_nz = fmin(min_nz, v);
+            } else if (v == 0.0) {
+                zero_step = fmax(zero_step, fmax(step_a, step_b));
+            } else {
+                bad = true;
+            }
+        }
+        // rows that convert to the same integers may still differ by less than a step everywhere
+        if (zero_step > 0.0 && min_nz < 1e300 && static_cast<double>(d) * zero_step * zero_step > kRelTol * min_nz) bad = true;
+        if (bad) atomicOr(&s_bad, 1);
+    }
+    __syncthreads();
+    for (int p = tid; p < F * F; p += blockDim.x) dist[p] = D[p];
+    if (tid == 0) flag[0] = (s_bad && !force) ? 1 : 0;
+}
+
+template <int F, int W, int R, int DEPTH>
+int launch_i8(const Rows<R>& rows, double* dist, double* tpart, int* info, int* flag, int force, cudaStream_t s) {
+    using S = I8Shape<F, W>;
+    const int64_t d = rows.d;
+    auto kern = pairdist_i8_kernel<F, W, R, DEPTH>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kSmem);
+    if (e != cudaSuccess) return cuda_failed(e);
+    int64_t ctas = (d + kTK - 1) / kTK;
+    if (ctas > kNumSMs) ctas = kNumSMs;
+    kern<<<static_cast<int>(ctas), S::kThreads, S::kSmem, s>>>(rows, tpart, info);
+    note_launch();
+    int st = check_launch();
+    if (st != BZ_OK) return st;
+    pairdist_i8_reduce_kernel<F><<<1, 1024, 0, s>>>(tpart, info, static_cast<int>(ctas), d, force, dist, flag);
+    note_launch();
+    return check_launch();
+}
+
+size_t tpart_bytes(int f) { return round_up(static_cast<size_t>(kNumSMs) * f * f * sizeof(double), 256); }
+size_t info_bytes() { return round_up(static_cast<size_t>(kNumSMs) * kInfoStride * sizeof(int), 256); }
+
+struct Scratch {
+    double* tpart;
+    int* info;
+    int* flag;
+};
+Scratch carve(void* ws, int f) {
+    char* p = static_cast<char*>(ws);
+    Scratch s;
+    s.tpart = reinterpret_cast<double*>(p);
+    p += tpart_bytes(f);
+    s.info = reinterpret_cast<int*>(p);
+    p += info_bytes();
+    s.flag = reinterpret_cast<int*>(p);
+    return s;
+}
+
+}  // namespace
+
+bool pairdist_i8_has(int f) { return f == 25 || f == 49; }
+
+// bytes of the partial matrices, the per-CTA records and the flag
+size_t pairdist_i8_workspace(int f) {
+    if (!pairdist_i8_has(f)) return 0;
+    return tpart_bytes(f) + info_bytes() + 256;
+}
+
+// Returns BZ_OK / an error, or 1 when this path does not apply (shape, alignment, size).  On BZ_OK
+// dist holds the distances and *flag_out points at the device flag that is 1 if they must be
+// recomputed in binary32.
+int pairdist_i8(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, int force, int** flag_out, cudaStream_t s) {
+    if (!pairdist_i8_has(f) || !aligned16(v) || (ld % 4) != 0 || d < 64 * kTK) return 1;
+    const Scratch sc = carve(ws, f);
+    *flag_out = sc.flag;
+    const Rows<1> rows{v, ld, 0, d, nullptr, 0};
+    if (f == 25) return launch_i8<25, 13, 1, 3>(rows, dist, sc.tpart, sc.info, sc.flag, force, s);
+    return launch_i8<49, 13, 1, 3>(rows, dist, sc.tpart, sc.info, sc.flag, force, s);
+}
+
+// The same from the replicas: vote (Eq. 3) and distances in one pass; the winners go to `voted`.
+int vote_pairdist_i8(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted,
+                     double* dist, void* ws, int force, int** flag_out, cudaStream_t s) {
+    if (!pairdist_i8_has(f) || !aligned16(rep) || !aligned16(voted) || (ld_file % 4) != 0 || (ld_rep % 4) != 0 ||
+        (ld_voted % 4) != 0 || d < 64 * kTK)
+        return 1;
+    const Scratch sc = carve(ws, f);
+    *flag_out = sc.flag;
+#define BZ_I8_CASE(R_, F_, W_, DEPTH_)                                                          \
+    if (r == R_ && f == F_) {                                                                   \
+        const Rows<R_> rows{rep, ld_file, ld_rep, d, voted, ld_voted};                          \
+        return launch_i8<F_, W_, R_, DEPTH_>(rows, dist, sc.tpart, sc.info, sc.flag, force, s); \
+    }
+    BZ_I8_CASE(3, 25, 13, 1)
+    BZ_I8_CASE(3, 49, 13, 1)
+    BZ_I8_CASE(5, 25, 13, 1)
+    BZ_I8_CASE(5, 49, 13, 1)
+    BZ_I8_CASE(7, 49, 13, 1)
+#undef BZ_I8_CASE
+    return 1;
+}
+
+int pairdist_i8_timeouts(unsigned int* count) {
+    const cudaError_t e = cudaMemcpyFromSymbol(count, g_i8_timeouts, sizeof(unsigned int));
+    return e == cudaSuccess ? BZ_OK : cuda_failed(e);
+}
+
+}  // namespace bz

@@ -1,0 +1,483 @@
+// Pairwise squared distances of the Krum family (Sec. 1.2; cost in Appendix A.1) on the tensor cores,
+// in exact integer arithmetic.
+//
+// The f x f matrix of squared distances is a contraction over the d coordinates, but in floating
+// point only its difference form is accurate enough: gradients share a large per-coordinate mean, so
+// |a|^2 + |b|^2 - 2ab cancels most of its digits.  Integers do not round.  Every value of row a is
+// converted to 31-bit fixed point on the row's own power-of-two scale 2^(30 - E_a) (E_a grows when a
+// larger magnitude shows up, and only then), the fixed-point word is cut into four balanced signed
+// bytes
+//     q = s3*2^24 + s2*2^16 + s1*2^8 + s0,   -128 <= s_i <= 127,
+// and the Gram matrix of the q's is the sum over slice pairs (i, j) of 2^(8(i+j)) S_i S_j^T.  Each
+// S_i S_j^T is an 8-bit integer MMA (tcgen05, kind::i8) with 32-bit accumulators in tensor memory:
+// exact, and independent of the order of the coordinates.  The slices are stacked along M and N, so
+// one or two MMAs per 32 coordinates produce every block that is needed (a block whose transpose is
+// not produced is counted twice).  The accumulators stay in tensor memory over hundreds of tiles and
+// are read back ("drained") only when some row's scale changes or 512 tiles have gone by (32-bit
+// headroom); a drain combines the blocks in binary64 and adds
+//     T[a][b] += 2^(E_a + E_b - 60) * sum_blocks weight * S_i S_j^T [a][b]
+// to the CTA's partial matrix.  A last kernel forms, per CTA and then over CTAs in a fixed order,
+//     D[a][b] = (T[a][a] + T[b][b]) - (T[a][b] + T[b][a]).
+// Identical rows give identical integers and therefore exactly equal distances and D = 0.
+//
+// What is not exact is the conversion: a value of row a is rounded to a multiple of 2^(E_a - 30),
+// where 2^E_a bounds the row's magnitudes so far.  Values whose binary exponent lies within 6 of E_a
+// keep all 24 bits; smaller ones lose low bits.  The last kernel turns the steps into an error
+// estimate for every pair and raises a flag when it exceeds the library's distance tolerance; the
+// caller then runs the binary32 difference-form kernel, which starts by looking at that flag.
+//
+// Per 128-coordinate tile and SM: f*512 bytes from HBM, f*128 conversions, 4 or 8 MMA instructions;
+// shared memory carries the operand tile once in (ordinary stores) and the MMAs' reads of it.  The
+// rows go from global memory straight to registers: shared-memory bandwidth is what the MMAs need.
+//
+// Roles in a CTA (one CTA per SM, tiles dealt round-robin): W converter warps own fixed rows (row r
+// belongs to warp r % W), hold the tiles in flight in registers, track the rows' scales and write the
+// operand tiles (K-major, 128-byte swizzle) of a ring; one thread issues the MMAs; four warps drain.
+// Every mbarrier wait is bounded; on expiry the CTA stops and g_i8_timeouts is raised.  No cluster
+// multicast is used.
+#pragma once
+
+#include "umma.cuh"
+
+namespace bz {
+
+constexpr int kTK = 128;             // coordinates per tile = bytes per operand row
+constexpr int kDrainWarps = 4;       // warps 0-3: one per 32 lanes of tensor memory
+constexpr int kMmaWarp = 4;
+constexpr int kConvWarp0 = 5;
+constexpr int kFlushTiles = 512;     // 2^9 tiles * 2^7 coordinates * 2^14 per product < 2^31
+constexpr int kENone = -1000, kELo = -64, kEHi = 64;
+constexpr int kCtlBytes = 2048;
+constexpr int kInfoStride = 72;      // ints per CTA: the rows' largest exponents, then the "bad" mark
+constexpr int kInfoBad = 64;
+constexpr int kPrefetchTiles = 8;    // how far ahead of the register loads the L2 prefetch runs
+
+__device__ unsigned int g_i8_timeouts = 0;
+
+template <int F, int W> struct I8Shape {
+    static constexpr int RP = F <= 32 ? 32 : 64;          // rows of one slice in an operand tile (f padded)
+    static constexpr int SPM = 128 / RP;                   // slices stacked along M in one MMA
+    static constexpr int NMMA = 4 / SPM;                   // MMAs per 32 coordinates
+    static constexpr int kOpStageBytes = 4 * RP * kTK;     // slices 3, 2, 1, 0 one after the other
+    static constexpr int kOpStages = 4;
+    static constexpr int kTmemCols = RP == 64 ? 512 : 128;
+    static constexpr int RW = (F + W - 1) / W;             // rows per converter warp
+    static constexpr int kThreads = (kConvWarp0 + W) * 32;
+    static constexpr int kSmem = 1024 + kOpStages * kOpStageBytes + kCtlBytes;
+    static_assert(F <= 64, "at most 64 rows");
+    // MMA m covers slice indices m*SPM .. m*SPM+SPM-1 along M and m*SPM .. 3 along N
+    static constexpr int mma_n(int m) { return (4 - m * SPM) * RP; }
+    static constexpr int mma_col(int m) { return m == 0 ? 0 : 4 * RP; }
+};
+
+__device__ __forceinline__ int clamp_e(int e) { return e < kELo ? kELo : (e > kEHi ? kEHi : e); }
+
+// weight of block (si, sj) (slice indices: slice value 3 - index) in T: 2^(8(6-si-sj)), doubled when
+// the transposed block (sj, si) is not among the computed ones
+template <int SPM> __device__ __forceinline__ double block_weight(int si, int sj) {
+    const int twice = ((sj / SPM) * SPM <= si) ? 0 : 1;
+    return __longlong_as_double(static_cast<long long>(1023 + 8 * (6 - si - sj) + twice) << 52);
+}
+
+// Four scaled coordinates of one row -> one 32-bit word per slice (byte k = coordinate k).
+// q = round(t) (|q| <= 2^30); adding 128 to each of the three low bytes (carries ripple upward) and
+// flipping their top bits afterwards leaves the balanced signed bytes.
+__device__ __forceinline__ void slice4(const float4& t, uint32_t (&w)[4]) {
+    const uint32_t x0 = static_cast<uint32_t>(__float2int_rn(t.x) + 0x00808080);
+    const uint32_t x1 = static_cast<uint32_t>(__float2int_rn(t.y) + 0x00808080);
+    const uint32_t x2 = static_cast<uint32_t>(__float2int_rn(t.z) + 0x00808080);
+    const uint32_t x3 = static_cast<uint32_t>(__float2int_rn(t.w) + 0x00808080);
+    // 4 x 4 byte transpose
+    const uint32_t lo01 = __byte_perm(x0, x1, 0x5140), lo23 = __byte_perm(x2, x3, 0x5140);
+    const uint32_t hi01 = __byte_perm(x0, x1, 0x7362), hi23 = __byte_perm(x2, x3, 0x7362);
+    w[0] = __byte_perm(lo01, lo23, 0x5410) ^ 0x80808080u;
+    w[1] = __byte_perm(lo01, lo23, 0x7632) ^ 0x80808080u;
+    w[2] = __byte_perm(hi01, hi23, 0x5410) ^ 0x80808080u;
+    w[3] = __byte_perm(hi01, hi23, 0x7632);
+}
+
+// the larger magnitude of a and b (any sign); a NaN in either comes through
+__device__ __forceinline__ float max_abs_nan(float a, float b) {
+    float m;
+    asm("max.NaN.xorsign.abs.f32 %0, %1, %2;" : "=f"(m) : "f"(a), "f"(b));
+    return m;
+}
+
+// Asks the L2 cache to fetch `bytes` (a multiple of 16, 16-byte aligned) from global memory.
+__device__ __forceinline__ void prefetch_l2(const void* p, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+
+// Where the f rows come from.  R = 1: they are given (src[row*ld_file + j]).  R > 1: row `row` is the
+// vote (Eq. 3, element by element on bit patterns) over its R copies src[k*ld_rep + row*ld_file + j],
+// which is also written to voted[row*ld_voted + j].  All bases 16-byte aligned, all leading dimensions
+// multiples of 4.  interior: the whole tile lies below d (uniform over the warp); the ragged last
+// tile is handled element by element and coordinates past d count as zero.
+template <int R> struct Rows {
+    const float* src;
+    int64_t ld_file, ld_rep, d;
+    float* voted;
+    int64_t ld_voted;
+
+    // issued here and now (the values are used later): volatile, so that the compiler leaves them in place
+    __device__ __forceinline__ void load(int row, int64_t j, bool interior, uint4 (&x)[R]) const {
+#pragma unroll
+        for (int k = 0; k < R; ++k) {
+            const float* p = src + k * ld_rep + row * ld_file + j;
+            if (interior) {
+                asm volatile("ld.global.cs.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(x[k].x), "=r"(x[k].y), "=r"(x[k].z), "=r"(x[k].w) : "l"(p));
+            } else {
+                const uint32_t* q = reinterpret_cast<const uint32_t*>(p);
+                x[k] = make_uint4(0u, 0u, 0u, 0u);
+                if (j < d) x[k].x = q[0];
+                if (j + 1 < d) x[k].y = q[1];
+                if (j + 2 < d) x[k].z = q[2];
+                if (j + 3 < d) x[k].w = q[3];
+            }
+        }
+    }
+    __device__ __forceinline__ float4 finish(int row, int64_t j, bool interior, const uint4 (&x)[R]) const {
+        uint4 w;
+        if constexpr (R == 1) {
+            w = x[0];
+        } else {
+            uint32_t c[R];
+#pragma unroll
+            for (int k = 0; k < R; ++k) c[k] = x[k].x;
+            w.x = vote_bits<R>(c);
+#pragma unroll
+            for (int k = 0; k < R; ++k) c[k] = x[k].y;
+            w.y = vote_bits<R>(c);
+#pragma unroll
+            for (int k = 0; k < R; ++k) c[k] = x[k].z;
+            w.z = vote_bits<R>(c);
+#pragma unroll
+            for (int k = 0; k < R; ++k) c[k] = x[k].w;
+            w.w = vote_bits<R>(c);
+            uint32_t* q = reinterpret_cast<uint32_t*>(voted + row * ld_voted + j);
+            if (interior) {
+                __stcs(reinterpret_cast<uint4*>(q), w);
+            } else {
+                if (j < d) q[0] = w.x;
+                if (j + 1 < d) q[1] = w.y;
+                if (j + 2 < d) q[2] = w.z;
+                if (j + 3 < d) q[3] = w.w;
+            }
+        }
+        return make_float4(__uint_as_float(w.x), __uint_as_float(w.y), __uint_as_float(w.z), __uint_as_float(w.w));
+    }
+};
+
+// R = 1: distances of given rows.  R > 1: vote and distances in one pass over the replicas.
+// DEPTH: tiles a converter warp holds in registers (the one it works on and DEPTH - 1 in flight).
+template <int F, int W, int R, int DEPTH>
+__global__ void __launch_bounds__(I8Shape<F, W>::kThreads, 1)
+    pairdist_i8_kernel(const Rows<R> rows, double* __restrict__ tpart, int* __restrict__ info) {
+    using S = I8Shape<F, W>;
+    constexpr int RP = S::RP, SPM = S::SPM, NMMA = S::NMMA, NO = S::kOpStages, RW = S::RW;
+    const int64_t d = rows.d;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    unsigned char* op = base;
+    unsigned char* ctl = base + NO * S::kOpStageBytes;
+    uint64_t* op_full = reinterpret_cast<uint64_t*>(ctl);
+    uint64_t* op_empty = op_full + NO;
+    uint64_t* acc_ready = op_empty + NO;
+    uint64_t* drain_go = acc_ready + 1;
+    uint64_t* drained = drain_go + 1;
+    volatile int* e_stage = reinterpret_cast<volatile int*>(drained + 1);  // [NO][64]: the rows' exponents BEFORE a tile
+    int* op_flush = const_cast<int*>(e_stage) + NO * 64;                     // [NO]: some row's scale changes with this tile
+    volatile int* drain_stage = op_flush + NO;                               // which e_stage row a drain uses
+    volatile int* drain_final = drain_stage + 1;                             // is it the last drain
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(drain_final) + 1);
+    volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    static_assert((2 * NO + 3) * 8 + (NO * 64 + NO + 4) * 4 <= kCtlBytes, "control block");
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int64_t n_tiles = (d + kTK - 1) / kTK;
+    // tiles are dealt round-robin, so that at any moment the CTAs read neighbouring pieces of each row
+    const int64_t my_tiles = (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x;  // at least 1: the grid never exceeds n_tiles
+    double* tp = tpart + static_cast<size_t>(blockIdx.x) * F * F;
+
+    if (tid == 0) {
+        for (int o = 0; o < NO; ++o) {
+            mbar_init(&op_full[o], W);
+            mbar_init(&op_empty[o], 1);
+            op_flush[o] = 0;
+        }
+        mbar_init(acc_ready, 1);
+        mbar_init(drain_go, 1);
+        mbar_init(drained, kDrainWarps);
+        *dead = 0;
+        info[blockIdx.x * kInfoStride + kInfoBad] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // rows f .. RP-1 of every slice stay zero for the whole run
+    for (int e = tid; e < NO * S::kOpStageBytes / 16; e += S::kThreads) reinterpret_cast<uint4*>(op)[e] = make_uint4(0, 0, 0, 0);
+    for (int e = tid; e < F * F; e += S::kThreads) tp[e] = 0.0;
+    fence_async_smem();
+    if (warp == kMmaWarp) tmem_alloc(tmem_slot, S::kTmemCols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp < kDrainWarps) {
+        // ------------------------------------------------------------------ drain: tensor memory -> T
+        const int L = warp * 32 + lane, g = L / RP, a = L % RP;
+        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+        bool ok = true;
+        for (uint32_t k = 0; ok; ++k) {
+            // the first request may be a whole launch away: long naps, still bounded (about 10 s)
+            if (!mbar_wait_live(drain_go, k & 1, dead, 20000) || !mbar_wait_live(acc_ready, k & 1, dead)) {
+                ok = false;
+                break;
+            }
+            tc_fence_after_sync();
+            const volatile int* e_row = e_stage + *drain_stage * 64;
+            const bool last = *drain_final != 0;
+            const int e_a = a < F ? e_row[a] : 0;
+            for (int ph = 0; ph < SPM; ++ph) {
+                if (g == ph) {  // uniform over the warp
+                    for (int b0 = 0; b0 < F; b0 += 8) {
+                        double val[8];
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) val[c] = 0.0;
+#pragma unroll
+                        for (int m = 0; m < NMMA; ++m) {
+                            const int si = m * SPM + g;
+#pragma unroll
+                            for (int h = 0; h < 4 - m * SPM; ++h) {
+                                int32_t x[8];
+                                tmem_ld8(lane_base + S::mma_col(m) + h * RP + b0, x);
+                                tmem_ld_wait();
+                                const double w = block_weight<SPM>(si, m * SPM + h);
+#pragma unroll
+                                for (int c = 0; c < 8; ++c) val[c] += w * static_cast<double>(x[c]);
+                            }
+                        }
+                        if (a < F) {
+#pragma unroll
+                            for (int c = 0; c < 8; ++c)
+                                if (b0 + c < F) {
+                                    const double sc = __longlong_as_double(static_cast<long long>(1023 + e_a + e_row[b0 + c] - 60) << 52);
+                                    tp[a * F + b0 + c] += val[c] * sc;
+                                }
+                        }
+                    }
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(kDrainWarps * 32) : "memory");
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(drained);
+            if (last) break;
+        }
+        if (!ok && lane == 0) atomicAdd(&g_i8_timeouts, 1u);
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------------ MMA issue
+        if (lane == 0) {
+            uint32_t n_flush = 0, have_acc = 0;
+            int since = 0;
+            bool ok = true;
+            // tile my_tiles carries no data: it hands over the final exponents for the last drain
+            for (int64_t it = 0; it <= my_tiles && ok; ++it) {
+                const int o = static_cast<int>(it % NO);
+                if (!mbar_wait_live(&op_full[o], static_cast<uint32_t>(it / NO) & 1, dead)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after_sync();
+                const bool last = it == my_tiles;
+                const int wants = atomicExch(&op_flush[o], 0);
+                if (have_acc && (wants || since == kFlushTiles || last)) {
+                    *drain_stage = o;
+                    *drain_final = last ? 1 : 0;
+                    mma_commit(acc_ready);
+                    mbar_arrive(drain_go);
+                    if (!mbar_wait_live(drained, n_flush & 1, dead)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    ++n_flush;
+                    have_acc = 0;
+                    since = 0;
+                }
+                if (last) break;
+                const uint32_t op_addr = smem_u32(op + static_cast<size_t>(o) * S::kOpStageBytes);
+#pragma unroll
+                for (int ks = 0; ks < kTK / 32; ++ks) {
+#pragma unroll
+                    for (int m = 0; m < NMMA; ++m) {
+                        const uint64_t desc = smem_desc_k128(op_addr + m * SPM * RP * kTK + ks * 32);
+                        mma_s8(tmem_base + S::mma_col(m), desc, desc, idesc_s8(128, S::mma_n(m)), have_acc | (ks > 0));
+                    }
+                }
+                mma_commit(&op_empty[o]);
+                have_acc = 1;
+                ++since;
+            }
+            if (!ok) atomicAdd(&g_i8_timeouts, 1u);
+        }
+    } else {
+        // ------------------------------------------------------------------ converters: global -> registers -> operand tiles
+        const int cw = warp - kConvWarp0;
+        int E[RW], e_max[RW];
+#pragma unroll
+        for (int i = 0; i < RW; ++i) {
+            E[i] = kENone;
+            e_max[i] = kELo;
+        }
+        int unrepresentable = 0;
+        bool ok = true;
+        uint4 buf[DEPTH][RW][R];
+
+        // With few tiles in flight in registers the loads cover the latency of L2, not that of HBM:
+        // every copy of the rows of tile it + kPrefetchTiles is then requested into L2 now (one lane
+        // per row and copy).
+        auto prefetch_tile = [&](int64_t it) {
+            if constexpr (DEPTH >= 3) return;  // enough in flight without it
+            const int64_t tile = blockIdx.x + it * gridDim.x;
+            const int i = lane / R, k = lane % R;
+            if (it < my_tiles && i < RW && cw + W * i < F && (tile + 1) * kTK <= d)
+                prefetch_l2(rows.src + k * rows.ld_rep + (cw + W * i) * rows.ld_file + tile * kTK, kTK * 4);
+        };
+        auto load_tile = [&](uint4(&dst)[RW][R], int64_t it) {
+            prefetch_tile(it + kPrefetchTiles);
+            if (it < my_tiles) {
+                const int64_t tile = blockIdx.x + it * gridDim.x;
+                const int64_t j = tile * kTK + 4 * lane;
+                const bool interior = (tile + 1) * kTK <= d;
+#pragma unroll
+                for (int i = 0; i < RW; ++i) {
+                    const int r = cw + W * i;
+                    if (r < F) rows.load(r, j, interior, dst[i]);
+                }
+            }
+        };
+        // this lane's byte offset inside a slice, for each of the warp's rows:
+        // row r = 8-row group r/8, row r%8 in it, 16-byte chunk (lane/4) ^ (r%8)
+        uint32_t row_off[RW];
+#pragma unroll
+        for (int i = 0; i < RW; ++i) {
+            const int r = cw + W * i;
+            row_off[i] = (r >> 3) * 1024 + (r & 7) * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | ((lane & 3) << 2));
+        }
+        auto convert_tile = [&](const uint4(&raw)[RW][R], int64_t it) -> bool {
+            const int o = static_cast<int>(it % NO);
+            float4 val[RW];
+            {
+                const int64_t tile = blockIdx.x + it * gridDim.x;
+                const int64_t j = tile * kTK + 4 * lane;
+                const bool interior = (tile + 1) * kTK <= d;
+#pragma unroll
+                for (int i = 0; i < RW; ++i)
+                    if (cw + W * i < F) val[i] = rows.finish(cw + W * i, j, interior, raw[i]);
+            }
+            // Scale with the rows' current exponents and look at the largest result: below 2^30 (and no
+            // NaN) the tile converts as it is - nearly always.  Otherwise the rows' largest magnitudes are
+            // found exactly, exponents grow, and the tile is scaled again.
+            int old[RW];
+            float4 t[RW];
+            float m = (it == 0) ? __int_as_float(0x7f800000) : 0.f;  // no exponents yet on the first tile
+#pragma unroll
+            for (int i = 0; i < RW; ++i) {
+                old[i] = E[i];
+                if (cw + W * i < F) {
+                    const float scale = __int_as_float((30 - E[i] + 127) << 23);
+                    t[i] = make_float4(val[i].x * scale, val[i].y * scale, val[i].z * scale, val[i].w * scale);
+                    m = max_abs_nan(max_abs_nan(m, t[i].x), max_abs_nan(t[i].y, max_abs_nan(t[i].z, t[i].w)));
+                }
+            }
+            bool raise = false;
+            if (__any_sync(0xffffffffu, !(fabsf(m) < 1073741824.0f))) {
+#pragma unroll
+                for (int i = 0; i < RW; ++i) {
+                    if (cw + W * i < F) {
+                        const uint32_t m4 = max(max(__float_as_uint(val[i].x) & 0x7fffffffu, __float_as_uint(val[i].y) & 0x7fffffffu),
+                                                max(__float_as_uint(val[i].z) & 0x7fffffffu, __float_as_uint(val[i].w) & 0x7fffffffu));
+                        const int need = static_cast<int>(__reduce_max_sync(0xffffffffu, m4) >> 23) - 126;  // |v| < 2^need
+                        if (need > 60) unrepresentable = 1;  // infinities, NaNs, magnitudes beyond 2^60
+                        if (E[i] == kENone || need > E[i]) {   // |v| * 2^(30 - E) may reach 2^30
+                            raise = raise || E[i] != kENone;
+                            E[i] = clamp_e(need + 2);
+                            e_max[i] = max(e_max[i], E[i]);
+                        }
+                        const float scale = __int_as_float((30 - E[i] + 127) << 23);
+                        t[i] = make_float4(val[i].x * scale, val[i].y * scale, val[i].z * scale, val[i].w * scale);
+                    }
+                }
+            }
+            // The slot is free once the MMAs of tile it - NO are done.  A row whose scale changes hands
+            // its old exponent to the drain that comes before this tile.
+            {
+                if (it >= NO && !mbar_wait_live(&op_empty[o], (static_cast<uint32_t>(it / NO) - 1) & 1, dead)) return false;
+                int mine = 0;
+#pragma unroll
+                for (int i = 0; i < RW; ++i)
+                    if (lane == i) mine = old[i] == kENone ? E[i] : old[i];
+                if (lane < RW && cw + W * lane < F) e_stage[o * 64 + cw + W * lane] = mine;
+            }
+            unsigned char* tile = op + static_cast<size_t>(o) * S::kOpStageBytes;
+#pragma unroll
+            for (int i = 0; i < RW; ++i) {
+                if (cw + W * i < F) {
+                    uint32_t w[4];
+                    slice4(t[i], w);
+                    unsigned char* dst = tile + row_off[i];
+                    *reinterpret_cast<uint32_t*>(dst + 0 * RP * kTK) = w[3];
+                    *reinterpret_cast<uint32_t*>(dst + 1 * RP * kTK) = w[2];
+                    *reinterpret_cast<uint32_t*>(dst + 2 * RP * kTK) = w[1];
+                    *reinterpret_cast<uint32_t*>(dst + 3 * RP * kTK) = w[0];
+                }
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                if (raise) atomicOr(&op_flush[o], 1);
+                mbar_arrive_relaxed(&op_full[o]);
+            }
+            return true;
+        };
+
+        for (int64_t it = DEPTH - 1; it < kPrefetchTiles; ++it) prefetch_tile(it);
+#pragma unroll
+        for (int k = 0; k < DEPTH - 1; ++k) load_tile(buf[k], k);
+        for (int64_t it = 0; it < my_tiles && ok; it += DEPTH) {
+#pragma unroll
+            for (int k = 0; k < DEPTH; ++k) {
+                if (ok && it + k < my_tiles) {
+                    load_tile(buf[(k + DEPTH - 1) % DEPTH], it + k + DEPTH - 1);
+                    ok = convert_tile(buf[k], it + k);
+                }
+            }
+        }
+        if (ok) {
+            // the stage after the last tile: current exponents, nothing to multiply
+            const int o = static_cast<int>(my_tiles % NO);
+            if (my_tiles >= NO && !mbar_wait_live(&op_empty[o], (static_cast<uint32_t>(my_tiles / NO) - 1) & 1, dead)) ok = false;
+            if (ok) {
+                int mine = 0;
+#pragma unroll
+                for (int i = 0; i < RW; ++i)
+                    if (lane == i) mine = E[i];
+                if (lane < RW && cw + W * lane < F) e_stage[o * 64 + cw + W * lane] = mine;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&op_full[o]);
+            }
+        }
+        if (!ok && lane == 0) atomicAdd(&g_i8_timeouts, 1u);
+        int mine = kELo;
+#pragma unroll
+        for (int i = 0; i < RW; ++i)
+            if (lane == i) mine = e_max[i];
+        if (lane < RW && cw + W * lane < F) info[blockIdx.x * kInfoStride + cw + W * lane] = mine;
+        if (lane == 0 && (unrepresentable || !ok)) atomicOr(&info[blockIdx.x * kInfoStride + kInfoBad], 1);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == kMmaWarp) tmem_dealloc(tmem_base, S::kTmemCols);
+}
+
+}  // namespace bz

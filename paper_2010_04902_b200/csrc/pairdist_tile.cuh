@@ -78,8 +78,10 @@ __device__ __forceinline__ void accumulate_tile(const float* base, int bi, int b
 
 // dist[a][b] = sum over CTAs (ascending) of the element of the pair's class block
 template <int F, int T, int G>
-__global__ void pairdist_tiled_reduce_kernel(const double* __restrict__ partial, int n_ctas, double* __restrict__ dist) {
+__global__ void pairdist_tiled_reduce_kernel(const double* __restrict__ partial, int n_ctas, double* __restrict__ dist,
+                                             const int* __restrict__ gate = nullptr) {
     using PT = PairTile<F, T, G>;
+    if (gate != nullptr && *gate == 0) return;  // nothing was summed: the distances already there stand
     constexpr int NB = PT::NB, NPB = PT::NPB, TT = PT::TT;
     const int p = blockIdx.x * blockDim.x + threadIdx.x;
     if (p >= F * F) return;

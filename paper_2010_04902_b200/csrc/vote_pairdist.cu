@@ -9,8 +9,14 @@
 
 namespace bz {
 
-int pairdist_on_device(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, cudaStream_t s);  // pairdist.cu
+int pairdist_on_device(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, cudaStream_t s, bool tensor_cores);  // pairdist.cu
 size_t pairdist_workspace(int f);
+size_t pairdist_workspace_fp32(int f);
+int pairdist_fp32(const float* v, int f, int64_t d, int64_t ld, double* dist, double* partial, const int* gate, cudaStream_t s);
+int pairdist_path_fp32_only();
+int pairdist_path_i8_forced();
+int vote_pairdist_i8(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted,
+                     double* dist, void* ws, int force, int** flag_out, cudaStream_t s);  // pairdist_i8.cu
 size_t krum_workspace_bytes(int op, int f);
 int check_workspace(void* ws, size_t have, size_t need);
 
@@ -84,6 +90,14 @@ extern "C" int bz_vote_pairdist(const float* replicas, int r, int f, int64_t d, 
     if (ld_file < d || (r > 1 && ld_replica < d) || ld_voted < d) return BZ_ERR_INVALID_ARG;
     int st = check_workspace(workspace, workspace_bytes, krum_workspace_bytes(BZ_OP_PAIRDIST, f));
     if (st != BZ_OK) return st;
+    if (d > 0 && r > 1 && pairdist_path_i8_forced()) {
+        // vote + integer distances on the tensor cores (on request only: the binary32 single-pass
+        // kernel below is the faster of the two at present)
+        int* flag = nullptr;
+        st = vote_pairdist_i8(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, dist,
+                              static_cast<char*>(workspace) + pairdist_workspace_fp32(f), 1, &flag, static_cast<cudaStream_t>(stream));
+        if (st != 1) return st;
+    }
     if (d > 0 && r > 1) {
         st = vote_pairdist_fused(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, dist,
                                  static_cast<double*>(workspace), static_cast<cudaStream_t>(stream));

@@ -1,0 +1,125 @@
+"""GPU parity of the integer (tensor-core) distance kernel against the CPU oracle.
+
+BZ_PAIRDIST_PATH=i8 takes that kernel's result whatever its own error estimate says, =fp32 keeps the
+distances on the binary32 kernels; unset, the library decides.  Shapes here satisfy the kernel's
+conditions (f in {25, 49}, 16-byte aligned rows, d >= 8192), so "i8" really runs it."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2010_04902_b200 import binding as bz
+from paper_2010_04902_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda"
+DIST_TOL = 1e-7      # relative error of a squared distance, as for the binary32 kernels
+
+
+def _voted(l, r, q, d, attack, seed=0, heavy=0.0):
+    wf, fw, _ = oracle.assign(l, r)
+    byz = oracle.worst_case(wf, l * l, r, q)[1]
+    g = inputs.true_gradients(l * l, d, seed=seed, heavy_tail_frac=heavy)
+    rep = inputs.build_replicas(g, fw, byz, attack)
+    return rep, torch.from_numpy(oracle.vote(rep.numpy()))
+
+
+def _check_close(got, want):
+    assert np.array_equal(got, got.T) and (np.diag(got) == 0).all()
+    off = ~np.eye(want.shape[0], dtype=bool)
+    nz = off & (want > 0)
+    assert (np.abs(got[nz] - want[nz]) <= DIST_TOL * want[nz]).all()
+    assert (got[off & (want == 0)] == 0).all()     # identical (colluding) rows
+
+
+@pytest.mark.parametrize("f,d", [(25, 8192), (49, 8192), (25, 70004), (49, 100000), (49, 1_000_004)])
+def test_exact_on_integer_rows(f, d, monkeypatch):
+    monkeypatch.setenv("BZ_PAIRDIST_PATH", "i8")
+    v = inputs.integer_gradients(f, d, seed=f + d)
+    want = oracle.pairdist(v.numpy())
+    got = bz.pairdist(v.to(DEV)).cpu().numpy()
+    assert np.array_equal(got, want)
+    assert bz.pipeline_timeouts() == 0
+
+
+@pytest.mark.parametrize("l,r,q,attack,d,heavy", [(5, 3, 3, "reversed", 50004, 0.0), (7, 3, 5, "alie", 50004, 0.0),
+                                                  (5, 5, 6, "constant", 200000, 0.01), (7, 3, 5, "alie", 1_000_004, 0.0)])
+def test_close_on_gradients(l, r, q, attack, d, heavy, monkeypatch):
+    monkeypatch.setenv("BZ_PAIRDIST_PATH", "i8")
+    _, v = _voted(l, r, q, d, attack, heavy=heavy)
+    want = oracle.pairdist(v.numpy())
+    got = bz.pairdist(v.to(DEV)).cpu().numpy()
+    _check_close(got, want)
+    assert np.array_equal(bz.pairdist(v.to(DEV)).cpu().numpy(), got)   # integer sums: the same bits every time
+    assert bz.pipeline_timeouts() == 0
+
+
+def test_scales_grow_in_mid_stream(monkeypatch):
+    # magnitudes that jump by orders of magnitude late in a row force new scales (and a read-back of
+    # the accumulators) in the middle of the stream
+    monkeypatch.setenv("BZ_PAIRDIST_PATH", "i8")
+    f, d = 49, 400_000
+    g = inputs.true_gradients(f, d, seed=5).numpy()
+    g[3, 150_000] = 3.0e4
+    g[3, 300_000] = -7.0e8
+    g[17, 222_222:222_300] *= 1.0e3
+    g[40] *= 1.0e-6
+    g[41] = g[40]
+    want = oracle.pairdist(g)
+    got = bz.pairdist(torch.from_numpy(g).to(DEV)).cpu().numpy()
+    _check_close(got, want)
+    assert bz.pipeline_timeouts() == 0
+
+
+def test_library_choice(monkeypatch):
+    _, v = _voted(7, 3, 5, 300_000, "alie")
+    v = v.to(DEV)
+    monkeypatch.setenv("BZ_PAIRDIST_PATH", "i8")
+    by_i8 = bz.pairdist(v).cpu().numpy()
+    monkeypatch.setenv("BZ_PAIRDIST_PATH", "fp32")
+    by_fp32 = bz.pairdist(v).cpu().numpy()
+    monkeypatch.delenv("BZ_PAIRDIST_PATH")
+    # ordinary gradients: the integer kernel's estimate is far below the tolerance, its result stands
+    assert np.array_equal(bz.pairdist(v).cpu().numpy(), by_i8)
+    want = oracle.pairdist(v.cpu().numpy())
+    _check_close(by_i8, want)
+    _check_close(by_fp32, want)
+    # two rows that differ by far less than a fixed-point step of their scale: the estimate must send
+    # the library to the binary32 kernel
+    w = v.clone()
+    w[1] = w[0]
+    w[1, ::1000] += 1.0e-7
+    monkeypatch.setenv("BZ_PAIRDIST_PATH", "fp32")
+    by_fp32 = bz.pairdist(w).cpu().numpy()
+    monkeypatch.delenv("BZ_PAIRDIST_PATH")
+    assert np.array_equal(bz.pairdist(w).cpu().numpy(), by_fp32)
+
+
+@pytest.mark.parametrize("bad", [float("inf"), float("nan"), 3.0e38])
+def test_values_without_a_fixed_point_scale(bad, monkeypatch):
+    # the integer kernel marks them and the binary32 kernel's answer is what the caller gets
+    v = inputs.true_gradients(25, 20_000, seed=9)
+    v[4, 12_345] = bad
+    got = bz.pairdist(v.to(DEV)).cpu().numpy()
+    monkeypatch.setenv("BZ_PAIRDIST_PATH", "fp32")
+    by_fp32 = bz.pairdist(v.to(DEV)).cpu().numpy()
+    assert np.array_equal(got, by_fp32, equal_nan=True)
+    want = oracle.pairdist(v.numpy())
+    if not np.isfinite(bad):
+        assert np.array_equal(np.isnan(got), np.isnan(want)) and np.array_equal(np.isinf(got), np.isinf(want))
+    clean = np.ones((25, 25), dtype=bool)
+    clean[4, :] = clean[:, 4] = False
+    clean &= ~np.eye(25, dtype=bool)
+    assert (np.abs(got[clean] - want[clean]) <= DIST_TOL * want[clean]).all()
+
+
+@pytest.mark.parametrize("l,r,q,attack,d", [(5, 3, 3, "reversed", 50004), (7, 3, 5, "alie", 100_000), (5, 5, 6, "constant", 40_000),
+                                            (7, 5, 5, "alie", 20_000), (7, 7, 4, "reversed", 20_000)])
+def test_vote_and_distances_in_one_pass(l, r, q, attack, d, monkeypatch):
+    monkeypatch.setenv("BZ_PAIRDIST_PATH", "i8")
+    rep, v = _voted(l, r, q, d, attack)
+    voted, dist = bz.vote_pairdist(rep.to(DEV))
+    assert np.array_equal(voted.cpu().numpy().view(np.uint32), v.numpy().view(np.uint32))
+    _check_close(dist.cpu().numpy(), oracle.pairdist(v.numpy()))
+    assert bz.pipeline_timeouts() == 0
