@@ -70,16 +70,29 @@ __global__ void __launch_bounds__(1024)
     if (tid == 0) flag[0] = (s_bad && !force) ? 1 : 0;
 }
 
-template <int F, int W, int R, int DEPTH>
-int launch_i8(const Rows<R>& rows, double* dist, double* tpart, int* info, int* flag, int force, cudaStream_t s) {
-    using S = I8Shape<F, W>;
-    const int64_t d = rows.d;
-    auto kern = pairdist_i8_kernel<F, W, R, DEPTH>;
+// rep: R = 1: rows [f][d] with leading dimension ld_file.  R > 1: replicas[r][f][d].
+// Returns 1 if the tensor map cannot express the shape.
+template <int F, int W, int R, int FC, int NS>
+int launch_i8(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted, double* dist,
+              double* tpart, int* info, int* flag, int force, cudaStream_t s) {
+    using S = I8Shape<F, W, R, FC, NS>;
+    EncodeTiledFn enc = encode_tiled();
+    if (enc == nullptr) return 1;
+    CUtensorMap map;
+    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(F), static_cast<cuuint64_t>(R)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(ld_file) * 4, static_cast<cuuint64_t>(R > 1 ? ld_rep : ld_file * F) * 4};
+    const cuuint32_t box[3] = {kTK, FC, R};
+    const cuuint32_t elem[3] = {1, 1, 1};
+    const CUresult cr = enc(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(rep), dims, strides, box, elem,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return 1;
+    auto kern = pairdist_i8_kernel<F, W, R, FC, NS>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kSmem);
     if (e != cudaSuccess) return cuda_failed(e);
     int64_t ctas = (d + kTK - 1) / kTK;
     if (ctas > kNumSMs) ctas = kNumSMs;
-    kern<<<static_cast<int>(ctas), S::kThreads, S::kSmem, s>>>(rows, tpart, info);
+    kern<<<static_cast<int>(ctas), S::kThreads, S::kSmem, s>>>(map, d, voted, ld_voted, tpart, info);
     note_launch();
     int st = check_launch();
     if (st != BZ_OK) return st;
@@ -121,32 +134,30 @@ size_t pairdist_i8_workspace(int f) {
 // dist holds the distances and *flag_out points at the device flag that is 1 if they must be
 // recomputed in binary32.
 int pairdist_i8(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, int force, int** flag_out, cudaStream_t s) {
-    if (!pairdist_i8_has(f) || !aligned16(v) || (ld % 4) != 0 || d < 64 * kTK) return 1;
+    if (!pairdist_i8_has(f) || !aligned16(v) || (ld % 4) != 0 || d < 64 * kTK || d >= (int64_t(1) << 31)) return 1;
     const Scratch sc = carve(ws, f);
     *flag_out = sc.flag;
-    const Rows<1> rows{v, ld, 0, d, nullptr, 0};
-    if (f == 25) return launch_i8<25, 13, 1, 3>(rows, dist, sc.tpart, sc.info, sc.flag, force, s);
-    return launch_i8<49, 13, 1, 3>(rows, dist, sc.tpart, sc.info, sc.flag, force, s);
+    // <rows, converter warps, copies, rows per box, boxes in the ring>
+    if (f == 25) return launch_i8<25, 13, 1, 25, 8>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
+    return launch_i8<49, 13, 1, 49, 3>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
 }
 
 // The same from the replicas: vote (Eq. 3) and distances in one pass; the winners go to `voted`.
 int vote_pairdist_i8(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted,
                      double* dist, void* ws, int force, int** flag_out, cudaStream_t s) {
     if (!pairdist_i8_has(f) || !aligned16(rep) || !aligned16(voted) || (ld_file % 4) != 0 || (ld_rep % 4) != 0 ||
-        (ld_voted % 4) != 0 || d < 64 * kTK)
+        (ld_voted % 4) != 0 || d < 64 * kTK || d >= (int64_t(1) << 31))
         return 1;
     const Scratch sc = carve(ws, f);
     *flag_out = sc.flag;
-#define BZ_I8_CASE(R_, F_, W_, DEPTH_)                                                          \
-    if (r == R_ && f == F_) {                                                                   \
-        const Rows<R_> rows{rep, ld_file, ld_rep, d, voted, ld_voted};                          \
-        return launch_i8<F_, W_, R_, DEPTH_>(rows, dist, sc.tpart, sc.info, sc.flag, force, s); \
-    }
-    BZ_I8_CASE(3, 25, 13, 1)
-    BZ_I8_CASE(3, 49, 13, 1)
-    BZ_I8_CASE(5, 25, 13, 1)
-    BZ_I8_CASE(5, 49, 13, 1)
-    BZ_I8_CASE(7, 49, 13, 1)
+#define BZ_I8_CASE(R_, F_, W_, FC_, NS_) \
+    if (r == R_ && f == F_)              \
+        return launch_i8<F_, W_, R_, FC_, NS_>(rep, d, ld_file, ld_rep, voted, ld_voted, dist, sc.tpart, sc.info, sc.flag, force, s);
+    BZ_I8_CASE(3, 25, 10, 5, 8)
+    BZ_I8_CASE(3, 49, 14, 7, 6)
+    BZ_I8_CASE(5, 25, 10, 5, 6)
+    BZ_I8_CASE(5, 49, 14, 7, 4)
+    BZ_I8_CASE(7, 49, 14, 7, 3)
 #undef BZ_I8_CASE
     return 1;
 }

@@ -26,15 +26,15 @@
 // estimate for every pair and raises a flag when it exceeds the library's distance tolerance; the
 // caller then runs the binary32 difference-form kernel, which starts by looking at that flag.
 //
-// Per 128-coordinate tile and SM: f*512 bytes from HBM, f*128 conversions, 4 or 8 MMA instructions;
-// shared memory carries the operand tile once in (ordinary stores) and the MMAs' reads of it.  The
-// rows go from global memory straight to registers: shared-memory bandwidth is what the MMAs need.
+// Per 128-coordinate tile and SM: f*512 bytes from HBM (r times that with the vote in front),
+// f*128 conversions, 4 or 8 MMA instructions.
 //
-// Roles in a CTA (one CTA per SM, tiles dealt round-robin): W converter warps own fixed rows (row r
-// belongs to warp r % W), hold the tiles in flight in registers, track the rows' scales and write the
-// operand tiles (K-major, 128-byte swizzle) of a ring; one thread issues the MMAs; four warps drain.
-// Every mbarrier wait is bounded; on expiry the CTA stops and g_i8_timeouts is raised.  No cluster
-// multicast is used.
+// Roles in a CTA (one CTA per SM, tiles dealt round-robin): one thread issues TMA loads of boxes
+// [R copies][FC rows][128 coordinates] into a ring of shared memory; W converter warps own fixed rows
+// (row r belongs to warp r % W), vote them if there are copies, track their scales and write the
+// operand tiles (K-major, 128-byte swizzle) of a second ring; one thread issues the MMAs; four warps
+// drain.  Every mbarrier wait is bounded; on expiry the CTA stops and g_i8_timeouts is raised.  No
+// cluster multicast is used.
 #pragma once
 
 #include "umma.cuh"
@@ -44,27 +44,34 @@ namespace bz {
 constexpr int kTK = 128;             // coordinates per tile = bytes per operand row
 constexpr int kDrainWarps = 4;       // warps 0-3: one per 32 lanes of tensor memory
 constexpr int kMmaWarp = 4;
-constexpr int kConvWarp0 = 5;
+constexpr int kTmaWarp = 5;
+constexpr int kConvWarp0 = 6;
 constexpr int kFlushTiles = 512;     // 2^9 tiles * 2^7 coordinates * 2^14 per product < 2^31
 constexpr int kENone = -1000, kELo = -64, kEHi = 64;
 constexpr int kCtlBytes = 2048;
 constexpr int kInfoStride = 72;      // ints per CTA: the rows' largest exponents, then the "bad" mark
 constexpr int kInfoBad = 64;
-constexpr int kPrefetchTiles = 8;    // how far ahead of the register loads the L2 prefetch runs
 
 __device__ unsigned int g_i8_timeouts = 0;
 
-template <int F, int W> struct I8Shape {
+// F rows, W converter warps, R copies per row (1: the rows are given), FC rows per box, NS boxes in the ring
+template <int F, int W, int R, int FC, int NS> struct I8Shape {
     static constexpr int RP = F <= 32 ? 32 : 64;          // rows of one slice in an operand tile (f padded)
     static constexpr int SPM = 128 / RP;                   // slices stacked along M in one MMA
     static constexpr int NMMA = 4 / SPM;                   // MMAs per 32 coordinates
     static constexpr int kOpStageBytes = 4 * RP * kTK;     // slices 3, 2, 1, 0 one after the other
     static constexpr int kOpStages = 4;
     static constexpr int kTmemCols = RP == 64 ? 512 : 128;
-    static constexpr int RW = (F + W - 1) / W;             // rows per converter warp
+    static constexpr int kChunks = F / FC;                 // boxes per tile
+    static constexpr int RWC = (FC + W - 1) / W;           // rows of a box one converter warp may own
+    static constexpr int kBoxFloats = R * FC * kTK;
+    static constexpr int kBoxBytes = kBoxFloats * 4;
     static constexpr int kThreads = (kConvWarp0 + W) * 32;
-    static constexpr int kSmem = 1024 + kOpStages * kOpStageBytes + kCtlBytes;
+    static constexpr int kSmem = 1024 + kOpStages * kOpStageBytes + NS * kBoxBytes + kCtlBytes;
     static_assert(F <= 64, "at most 64 rows");
+    static_assert(kChunks * FC == F, "FC must divide F");
+    static_assert(kBoxBytes % 128 == 0, "TMA destinations are 128-byte aligned");
+    static_assert(kSmem <= 227 * 1024, "shared memory");
     // MMA m covers slice indices m*SPM .. m*SPM+SPM-1 along M and m*SPM .. 3 along N
     static constexpr int mma_n(int m) { return (4 - m * SPM) * RP; }
     static constexpr int mma_col(int m) { return m == 0 ? 0 : 4 * RP; }
@@ -103,95 +110,35 @@ __device__ __forceinline__ float max_abs_nan(float a, float b) {
     return m;
 }
 
-// Asks the L2 cache to fetch `bytes` (a multiple of 16, 16-byte aligned) from global memory.
-__device__ __forceinline__ void prefetch_l2(const void* p, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
-}
-
-// Where the f rows come from.  R = 1: they are given (src[row*ld_file + j]).  R > 1: row `row` is the
-// vote (Eq. 3, element by element on bit patterns) over its R copies src[k*ld_rep + row*ld_file + j],
-// which is also written to voted[row*ld_voted + j].  All bases 16-byte aligned, all leading dimensions
-// multiples of 4.  interior: the whole tile lies below d (uniform over the warp); the ragged last
-// tile is handled element by element and coordinates past d count as zero.
-template <int R> struct Rows {
-    const float* src;
-    int64_t ld_file, ld_rep, d;
-    float* voted;
-    int64_t ld_voted;
-
-    // issued here and now (the values are used later): volatile, so that the compiler leaves them in place
-    __device__ __forceinline__ void load(int row, int64_t j, bool interior, uint4 (&x)[R]) const {
-#pragma unroll
-        for (int k = 0; k < R; ++k) {
-            const float* p = src + k * ld_rep + row * ld_file + j;
-            if (interior) {
-                asm volatile("ld.global.cs.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(x[k].x), "=r"(x[k].y), "=r"(x[k].z), "=r"(x[k].w) : "l"(p));
-            } else {
-                const uint32_t* q = reinterpret_cast<const uint32_t*>(p);
-                x[k] = make_uint4(0u, 0u, 0u, 0u);
-                if (j < d) x[k].x = q[0];
-                if (j + 1 < d) x[k].y = q[1];
-                if (j + 2 < d) x[k].z = q[2];
-                if (j + 3 < d) x[k].w = q[3];
-            }
-        }
-    }
-    __device__ __forceinline__ float4 finish(int row, int64_t j, bool interior, const uint4 (&x)[R]) const {
-        uint4 w;
-        if constexpr (R == 1) {
-            w = x[0];
-        } else {
-            uint32_t c[R];
-#pragma unroll
-            for (int k = 0; k < R; ++k) c[k] = x[k].x;
-            w.x = vote_bits<R>(c);
-#pragma unroll
-            for (int k = 0; k < R; ++k) c[k] = x[k].y;
-            w.y = vote_bits<R>(c);
-#pragma unroll
-            for (int k = 0; k < R; ++k) c[k] = x[k].z;
-            w.z = vote_bits<R>(c);
-#pragma unroll
-            for (int k = 0; k < R; ++k) c[k] = x[k].w;
-            w.w = vote_bits<R>(c);
-            uint32_t* q = reinterpret_cast<uint32_t*>(voted + row * ld_voted + j);
-            if (interior) {
-                __stcs(reinterpret_cast<uint4*>(q), w);
-            } else {
-                if (j < d) q[0] = w.x;
-                if (j + 1 < d) q[1] = w.y;
-                if (j + 2 < d) q[2] = w.z;
-                if (j + 3 < d) q[3] = w.w;
-            }
-        }
-        return make_float4(__uint_as_float(w.x), __uint_as_float(w.y), __uint_as_float(w.z), __uint_as_float(w.w));
-    }
-};
-
-// R = 1: distances of given rows.  R > 1: vote and distances in one pass over the replicas.
-// DEPTH: tiles a converter warp holds in registers (the one it works on and DEPTH - 1 in flight).
-template <int F, int W, int R, int DEPTH>
-__global__ void __launch_bounds__(I8Shape<F, W>::kThreads, 1)
-    pairdist_i8_kernel(const Rows<R> rows, double* __restrict__ tpart, int* __restrict__ info) {
-    using S = I8Shape<F, W>;
-    constexpr int RP = S::RP, SPM = S::SPM, NMMA = S::NMMA, NO = S::kOpStages, RW = S::RW;
-    const int64_t d = rows.d;
+// R = 1: distances of the rows of `map` ([f][d]).  R > 1: `map` covers replicas[r][f][d]; row i is the vote
+// (Eq. 3, element by element on bit patterns) over its R copies, which is also written to
+// voted[i*ld_voted + j] (16-byte aligned, ld_voted a multiple of 4).
+template <int F, int W, int R, int FC, int NS>
+__global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
+    pairdist_i8_kernel(const __grid_constant__ CUtensorMap map, int64_t d, float* __restrict__ voted, int64_t ld_voted,
+                       double* __restrict__ tpart, int* __restrict__ info) {
+    using S = I8Shape<F, W, R, FC, NS>;
+    constexpr int RP = S::RP, SPM = S::SPM, NMMA = S::NMMA, NO = S::kOpStages, CH = S::kChunks, RWC = S::RWC;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char* op = base;
-    unsigned char* ctl = base + NO * S::kOpStageBytes;
+    float* in = reinterpret_cast<float*>(base + NO * S::kOpStageBytes);
+    unsigned char* ctl = base + NO * S::kOpStageBytes + NS * S::kBoxBytes;
     uint64_t* op_full = reinterpret_cast<uint64_t*>(ctl);
     uint64_t* op_empty = op_full + NO;
-    uint64_t* acc_ready = op_empty + NO;
+    uint64_t* in_full = op_empty + NO;
+    uint64_t* in_empty = in_full + NS;
+    uint64_t* acc_ready = in_empty + NS;
     uint64_t* drain_go = acc_ready + 1;
     uint64_t* drained = drain_go + 1;
     volatile int* e_stage = reinterpret_cast<volatile int*>(drained + 1);  // [NO][64]: the rows' exponents BEFORE a tile
-    int* op_flush = const_cast<int*>(e_stage) + NO * 64;                     // [NO]: some row's scale changes with this tile
+    volatile int* e_cur = e_stage + NO * 64;                                 // [64]: the rows' exponents now
+    int* op_flush = const_cast<int*>(e_cur) + 64;                            // [NO]: some row's scale changes with this tile
     volatile int* drain_stage = op_flush + NO;                               // which e_stage row a drain uses
     volatile int* drain_final = drain_stage + 1;                             // is it the last drain
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(drain_final) + 1);
     volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    static_assert((2 * NO + 3) * 8 + (NO * 64 + NO + 4) * 4 <= kCtlBytes, "control block");
+    static_assert((2 * NO + 2 * NS + 3) * 8 + (NO * 64 + 64 + NO + 4) * 4 <= kCtlBytes, "control block");
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int64_t n_tiles = (d + kTK - 1) / kTK;
@@ -205,6 +152,10 @@ __global__ void __launch_bounds__(I8Shape<F, W>::kThreads, 1)
             mbar_init(&op_empty[o], 1);
             op_flush[o] = 0;
         }
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(&in_full[s], 1);
+            mbar_init(&in_empty[s], W);
+        }
         mbar_init(acc_ready, 1);
         mbar_init(drain_go, 1);
         mbar_init(drained, kDrainWarps);
@@ -212,6 +163,7 @@ __global__ void __launch_bounds__(I8Shape<F, W>::kThreads, 1)
         info[blockIdx.x * kInfoStride + kInfoBad] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (tid < 64) e_cur[tid] = kENone;
     // rows f .. RP-1 of every slice stay zero for the whole run
     for (int e = tid; e < NO * S::kOpStageBytes / 16; e += S::kThreads) reinterpret_cast<uint4*>(op)[e] = make_uint4(0, 0, 0, 0);
     for (int e = tid; e < F * F; e += S::kThreads) tp[e] = 0.0;
@@ -320,117 +272,158 @@ __global__ void __launch_bounds__(I8Shape<F, W>::kThreads, 1)
             }
             if (!ok) atomicAdd(&g_i8_timeouts, 1u);
         }
-    } else {
-        // ------------------------------------------------------------------ converters: global -> registers -> operand tiles
-        const int cw = warp - kConvWarp0;
-        int E[RW], e_max[RW];
-#pragma unroll
-        for (int i = 0; i < RW; ++i) {
-            E[i] = kENone;
-            e_max[i] = kELo;
+    } else if (warp == kTmaWarp) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const int64_t n_boxes = my_tiles * CH;
+            int64_t issued = 0;
+            bool ok = true;
+            for (; issued < n_boxes; ++issued) {
+                const int s = static_cast<int>(issued % NS);
+                const uint32_t round = static_cast<uint32_t>(issued / NS);
+                if (round > 0 && !mbar_wait_live(&in_empty[s], (round - 1) & 1, dead)) {
+                    ok = false;
+                    break;
+                }
+                const int64_t tile = blockIdx.x + (issued / CH) * gridDim.x;
+                const int chunk = static_cast<int>(issued % CH);
+                mbar_expect_tx(&in_full[s], S::kBoxBytes);
+                tma_load_3d(in + static_cast<size_t>(s) * S::kBoxFloats, &map, &in_full[s], static_cast<int>(tile * kTK), chunk * FC, 0);
+            }
+            if (!ok) {
+                atomicAdd(&g_i8_timeouts, 1u);
+                // shared memory must outlive the loads already issued
+                for (int64_t b = issued > NS ? issued - NS : 0; b < issued; ++b)
+                    mbar_wait(&in_full[b % NS], static_cast<uint32_t>(b / NS) & 1);
+            }
         }
+    } else {
+        // ------------------------------------------------------------------ converters: boxes -> operand tiles
+        const int cw = warp - kConvWarp0;
         int unrepresentable = 0;
         bool ok = true;
-        uint4 buf[DEPTH][RW][R];
-
-        // With few tiles in flight in registers the loads cover the latency of L2, not that of HBM:
-        // every copy of the rows of tile it + kPrefetchTiles is then requested into L2 now (one lane
-        // per row and copy).
-        auto prefetch_tile = [&](int64_t it) {
-            if constexpr (DEPTH >= 3) return;  // enough in flight without it
-            const int64_t tile = blockIdx.x + it * gridDim.x;
-            const int i = lane / R, k = lane % R;
-            if (it < my_tiles && i < RW && cw + W * i < F && (tile + 1) * kTK <= d)
-                prefetch_l2(rows.src + k * rows.ld_rep + (cw + W * i) * rows.ld_file + tile * kTK, kTK * 4);
-        };
-        auto load_tile = [&](uint4(&dst)[RW][R], int64_t it) {
-            prefetch_tile(it + kPrefetchTiles);
-            if (it < my_tiles) {
-                const int64_t tile = blockIdx.x + it * gridDim.x;
-                const int64_t j = tile * kTK + 4 * lane;
-                const bool interior = (tile + 1) * kTK <= d;
-#pragma unroll
-                for (int i = 0; i < RW; ++i) {
-                    const int r = cw + W * i;
-                    if (r < F) rows.load(r, j, interior, dst[i]);
-                }
-            }
-        };
-        // this lane's byte offset inside a slice, for each of the warp's rows:
-        // row r = 8-row group r/8, row r%8 in it, 16-byte chunk (lane/4) ^ (r%8)
-        uint32_t row_off[RW];
-#pragma unroll
-        for (int i = 0; i < RW; ++i) {
-            const int r = cw + W * i;
-            row_off[i] = (r >> 3) * 1024 + (r & 7) * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | ((lane & 3) << 2));
-        }
-        auto convert_tile = [&](const uint4(&raw)[RW][R], int64_t it) -> bool {
+        int64_t box = 0;
+        for (int64_t it = 0; it < my_tiles && ok; ++it) {
             const int o = static_cast<int>(it % NO);
-            float4 val[RW];
-            {
-                const int64_t tile = blockIdx.x + it * gridDim.x;
-                const int64_t j = tile * kTK + 4 * lane;
-                const bool interior = (tile + 1) * kTK <= d;
-#pragma unroll
-                for (int i = 0; i < RW; ++i)
-                    if (cw + W * i < F) val[i] = rows.finish(cw + W * i, j, interior, raw[i]);
-            }
-            // Scale with the rows' current exponents and look at the largest result: below 2^30 (and no
-            // NaN) the tile converts as it is - nearly always.  Otherwise the rows' largest magnitudes are
-            // found exactly, exponents grow, and the tile is scaled again.
-            int old[RW];
-            float4 t[RW];
-            float m = (it == 0) ? __int_as_float(0x7f800000) : 0.f;  // no exponents yet on the first tile
-#pragma unroll
-            for (int i = 0; i < RW; ++i) {
-                old[i] = E[i];
-                if (cw + W * i < F) {
-                    const float scale = __int_as_float((30 - E[i] + 127) << 23);
-                    t[i] = make_float4(val[i].x * scale, val[i].y * scale, val[i].z * scale, val[i].w * scale);
-                    m = max_abs_nan(max_abs_nan(m, t[i].x), max_abs_nan(t[i].y, max_abs_nan(t[i].z, t[i].w)));
+            const int64_t j = (blockIdx.x + it * gridDim.x) * kTK + 4 * lane;
+            unsigned char* tile = op + static_cast<size_t>(o) * S::kOpStageBytes;
+            bool raise = false, have_slot = false;
+#pragma unroll 1
+            for (int c = 0; c < CH && ok; ++c, ++box) {
+                const int s = static_cast<int>(box % NS);
+                if (!mbar_wait_live(&in_full[s], static_cast<uint32_t>(box / NS) & 1, dead)) {
+                    ok = false;
+                    break;
                 }
-            }
-            bool raise = false;
-            if (__any_sync(0xffffffffu, !(fabsf(m) < 1073741824.0f))) {
+                const uint32_t* src = reinterpret_cast<const uint32_t*>(in + static_cast<size_t>(s) * S::kBoxFloats);
+                // rows of this box that belong to this warp: c*FC + off + W*i
+                const int off = ((cw - c * FC) % W + W) % W;
+                float4 val[RWC];
+                int E[RWC];
 #pragma unroll
-                for (int i = 0; i < RW; ++i) {
-                    if (cw + W * i < F) {
-                        const uint32_t m4 = max(max(__float_as_uint(val[i].x) & 0x7fffffffu, __float_as_uint(val[i].y) & 0x7fffffffu),
-                                                max(__float_as_uint(val[i].z) & 0x7fffffffu, __float_as_uint(val[i].w) & 0x7fffffffu));
-                        const int need = static_cast<int>(__reduce_max_sync(0xffffffffu, m4) >> 23) - 126;  // |v| < 2^need
-                        if (need > 60) unrepresentable = 1;  // infinities, NaNs, magnitudes beyond 2^60
-                        if (E[i] == kENone || need > E[i]) {   // |v| * 2^(30 - E) may reach 2^30
-                            raise = raise || E[i] != kENone;
-                            E[i] = clamp_e(need + 2);
-                            e_max[i] = max(e_max[i], E[i]);
+                for (int i = 0; i < RWC; ++i) {
+                    const int fi = off + W * i;
+                    if (fi < FC) {
+                        uint4 w;
+                        if constexpr (R == 1) {
+                            w = *reinterpret_cast<const uint4*>(src + fi * kTK + 4 * lane);
+                        } else {
+                            uint4 x[R];
+#pragma unroll
+                            for (int k = 0; k < R; ++k) x[k] = *reinterpret_cast<const uint4*>(src + (k * FC + fi) * kTK + 4 * lane);
+                            uint32_t cp[R];
+#pragma unroll
+                            for (int k = 0; k < R; ++k) cp[k] = x[k].x;
+                            w.x = vote_bits<R>(cp);
+#pragma unroll
+                            for (int k = 0; k < R; ++k) cp[k] = x[k].y;
+                            w.y = vote_bits<R>(cp);
+#pragma unroll
+                            for (int k = 0; k < R; ++k) cp[k] = x[k].z;
+                            w.z = vote_bits<R>(cp);
+#pragma unroll
+                            for (int k = 0; k < R; ++k) cp[k] = x[k].w;
+                            w.w = vote_bits<R>(cp);
+                            uint32_t* q = reinterpret_cast<uint32_t*>(voted + (c * FC + fi) * ld_voted + j);
+                            if (j + 3 < d) {
+                                __stcs(reinterpret_cast<uint4*>(q), w);
+                            } else {  // ragged end
+                                if (j < d) q[0] = w.x;
+                                if (j + 1 < d) q[1] = w.y;
+                                if (j + 2 < d) q[2] = w.z;
+                            }
                         }
-                        const float scale = __int_as_float((30 - E[i] + 127) << 23);
+                        val[i] = make_float4(__uint_as_float(w.x), __uint_as_float(w.y), __uint_as_float(w.z), __uint_as_float(w.w));
+                        E[i] = e_cur[c * FC + fi];
+                    }
+                }
+                // the box is in registers: hand it back
+                __syncwarp();
+                if (lane == 0) mbar_arrive_relaxed(&in_empty[s]);
+                // Scale with the rows' current exponents and look at the largest result: below 2^30 (and
+                // no NaN) the rows convert as they are - nearly always.  Otherwise the rows' largest
+                // magnitudes are found exactly, exponents grow, and the rows are scaled again.
+                int old[RWC];
+                float4 t[RWC];
+                float m = 0.f;
+#pragma unroll
+                for (int i = 0; i < RWC; ++i) {
+                    if (off + W * i < FC) {
+                        old[i] = E[i];
+                        if (E[i] == kENone) m = __int_as_float(0x7f800000);  // no exponent yet (first tile)
+                        const float scale = __int_as_float((30 - (E[i] == kENone ? 0 : E[i]) + 127) << 23);
                         t[i] = make_float4(val[i].x * scale, val[i].y * scale, val[i].z * scale, val[i].w * scale);
+                        m = max_abs_nan(max_abs_nan(m, t[i].x), max_abs_nan(t[i].y, max_abs_nan(t[i].z, t[i].w)));
+                    }
+                }
+                if (__any_sync(0xffffffffu, !(fabsf(m) < 1073741824.0f))) {
+#pragma unroll
+                    for (int i = 0; i < RWC; ++i) {
+                        if (off + W * i < FC) {
+                            const uint32_t m4 = max(max(__float_as_uint(val[i].x) & 0x7fffffffu, __float_as_uint(val[i].y) & 0x7fffffffu),
+                                                    max(__float_as_uint(val[i].z) & 0x7fffffffu, __float_as_uint(val[i].w) & 0x7fffffffu));
+                            const int need = static_cast<int>(__reduce_max_sync(0xffffffffu, m4) >> 23) - 126;  // |v| < 2^need
+                            if (need > 60) unrepresentable = 1;  // infinities, NaNs, magnitudes beyond 2^60
+                            if (E[i] == kENone || need > E[i]) {   // |v| * 2^(30 - E) may reach 2^30
+                                raise = raise || E[i] != kENone;
+                                E[i] = clamp_e(need + 2);
+                                if (lane == 0) e_cur[c * FC + off + W * i] = E[i];
+                            }
+                            const float scale = __int_as_float((30 - E[i] + 127) << 23);
+                            t[i] = make_float4(val[i].x * scale, val[i].y * scale, val[i].z * scale, val[i].w * scale);
+                        }
+                    }
+                }
+                // the operand slot is free once the MMAs of tile it - NO are done
+                if (!have_slot) {
+                    if (it >= NO && !mbar_wait_live(&op_empty[o], (static_cast<uint32_t>(it / NO) - 1) & 1, dead)) {
+                        ok = false;
+                        break;
+                    }
+                    have_slot = true;
+                }
+#pragma unroll
+                for (int i = 0; i < RWC; ++i) {
+                    const int fi = off + W * i;
+                    if (fi < FC) {
+                        const int r = c * FC + fi;
+                        // a row whose scale changes hands its old exponent to the drain that comes before this tile
+                        if (lane == 0) e_stage[o * 64 + r] = old[i] == kENone ? E[i] : old[i];
+                        uint32_t w[4];
+                        slice4(t[i], w);
+                        // row r of a slice: 8-row group r/8, row r%8 in it, 16-byte chunk (lane/4) ^ (r%8)
+                        unsigned char* dst = tile + (r >> 3) * 1024 + (r & 7) * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | ((lane & 3) << 2));
+                        *reinterpret_cast<uint32_t*>(dst + 0 * RP * kTK) = w[3];
+                        *reinterpret_cast<uint32_t*>(dst + 1 * RP * kTK) = w[2];
+                        *reinterpret_cast<uint32_t*>(dst + 2 * RP * kTK) = w[1];
+                        *reinterpret_cast<uint32_t*>(dst + 3 * RP * kTK) = w[0];
                     }
                 }
             }
-            // The slot is free once the MMAs of tile it - NO are done.  A row whose scale changes hands
-            // its old exponent to the drain that comes before this tile.
-            {
-                if (it >= NO && !mbar_wait_live(&op_empty[o], (static_cast<uint32_t>(it / NO) - 1) & 1, dead)) return false;
-                int mine = 0;
-#pragma unroll
-                for (int i = 0; i < RW; ++i)
-                    if (lane == i) mine = old[i] == kENone ? E[i] : old[i];
-                if (lane < RW && cw + W * lane < F) e_stage[o * 64 + cw + W * lane] = mine;
-            }
-            unsigned char* tile = op + static_cast<size_t>(o) * S::kOpStageBytes;
-#pragma unroll
-            for (int i = 0; i < RW; ++i) {
-                if (cw + W * i < F) {
-                    uint32_t w[4];
-                    slice4(t[i], w);
-                    unsigned char* dst = tile + row_off[i];
-                    *reinterpret_cast<uint32_t*>(dst + 0 * RP * kTK) = w[3];
-                    *reinterpret_cast<uint32_t*>(dst + 1 * RP * kTK) = w[2];
-                    *reinterpret_cast<uint32_t*>(dst + 2 * RP * kTK) = w[1];
-                    *reinterpret_cast<uint32_t*>(dst + 3 * RP * kTK) = w[0];
-                }
+            if (!ok) break;
+            if (!have_slot && it >= NO && !mbar_wait_live(&op_empty[o], (static_cast<uint32_t>(it / NO) - 1) & 1, dead)) {
+                ok = false;
+                break;
             }
             fence_async_smem();
             __syncwarp();
@@ -438,42 +431,23 @@ __global__ void __launch_bounds__(I8Shape<F, W>::kThreads, 1)
                 if (raise) atomicOr(&op_flush[o], 1);
                 mbar_arrive_relaxed(&op_full[o]);
             }
-            return true;
-        };
-
-        for (int64_t it = DEPTH - 1; it < kPrefetchTiles; ++it) prefetch_tile(it);
-#pragma unroll
-        for (int k = 0; k < DEPTH - 1; ++k) load_tile(buf[k], k);
-        for (int64_t it = 0; it < my_tiles && ok; it += DEPTH) {
-#pragma unroll
-            for (int k = 0; k < DEPTH; ++k) {
-                if (ok && it + k < my_tiles) {
-                    load_tile(buf[(k + DEPTH - 1) % DEPTH], it + k + DEPTH - 1);
-                    ok = convert_tile(buf[k], it + k);
-                }
-            }
         }
         if (ok) {
             // the stage after the last tile: current exponents, nothing to multiply
             const int o = static_cast<int>(my_tiles % NO);
             if (my_tiles >= NO && !mbar_wait_live(&op_empty[o], (static_cast<uint32_t>(my_tiles / NO) - 1) & 1, dead)) ok = false;
             if (ok) {
-                int mine = 0;
-#pragma unroll
-                for (int i = 0; i < RW; ++i)
-                    if (lane == i) mine = E[i];
-                if (lane < RW && cw + W * lane < F) e_stage[o * 64 + cw + W * lane] = mine;
+                if (lane == 0)
+                    for (int r = cw; r < F; r += W) e_stage[o * 64 + r] = e_cur[r];
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&op_full[o]);
             }
         }
         if (!ok && lane == 0) atomicAdd(&g_i8_timeouts, 1u);
-        int mine = kELo;
-#pragma unroll
-        for (int i = 0; i < RW; ++i)
-            if (lane == i) mine = e_max[i];
-        if (lane < RW && cw + W * lane < F) info[blockIdx.x * kInfoStride + cw + W * lane] = mine;
-        if (lane == 0 && (unrepresentable || !ok)) atomicOr(&info[blockIdx.x * kInfoStride + kInfoBad], 1);
+        if (lane == 0) {
+            for (int r = cw; r < F; r += W) info[blockIdx.x * kInfoStride + r] = e_cur[r];
+            if (unrepresentable || !ok) atomicOr(&info[blockIdx.x * kInfoStride + kInfoBad], 1);
+        }
     }
     tc_fence_before_sync();
     __syncthreads();
