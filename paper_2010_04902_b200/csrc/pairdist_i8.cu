@@ -1,5 +1,6 @@
 // Pairwise squared distances of the Krum family (Sec. 1.2; cost in Appendix A.1) on the tensor cores,
 // in exact integer arithmetic.  Host side; the kernel is in pairdist_i8_kernel.cuh.
+#include <cstdlib>
 #include "pairdist_i8_kernel.cuh"
 
 namespace bz {
@@ -138,7 +139,13 @@ int pairdist_i8(const float* v, int f, int64_t d, int64_t ld, double* dist, void
     const Scratch sc = carve(ws, f);
     *flag_out = sc.flag;
     // <rows, converter warps, copies, rows per box, boxes in the ring>
-    if (f == 25) return launch_i8<25, 13, 1, 25, 8>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
+    const char* we = std::getenv("BZ_I8_W");
+    const int w = we ? std::atoi(we) : 0;
+#define TRY(F_, W_, NS_) if (f == F_ && w == W_) return launch_i8<F_, W_, 1, F_, NS_>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
+    TRY(49, 16, 3) TRY(49, 20, 3) TRY(49, 12, 3) TRY(49, 8, 3)
+    TRY(25, 8, 8) TRY(25, 12, 8) TRY(25, 16, 8) TRY(25, 20, 8)
+#undef TRY
+    if (f == 25) return launch_i8<25, 25, 1, 25, 8>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
     return launch_i8<49, 13, 1, 49, 3>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
 }
 

@@ -29,6 +29,10 @@
 // Per 128-coordinate tile and SM: f*512 bytes from HBM (r times that with the vote in front),
 // f*128 conversions, 4 or 8 MMA instructions.
 //
+// Every warp of a CTA sees every tile, so what a warp spends per tile on waiting, signalling and
+// bookkeeping bounds the CTA's rate whatever the number of warps: the unit of work between two
+// signals is therefore a step of two tiles.
+//
 // Roles in a CTA (one CTA per SM, tiles dealt round-robin): one thread issues TMA loads of boxes
 // [R copies][FC rows][128 coordinates] into a ring of shared memory; W converter warps own fixed rows
 // (row r belongs to warp r % W), vote them if there are copies, track their scales and write the
@@ -59,15 +63,16 @@ template <int F, int W, int R, int FC, int NS> struct I8Shape {
     static constexpr int RP = F <= 32 ? 32 : 64;          // rows of one slice in an operand tile (f padded)
     static constexpr int SPM = 128 / RP;                   // slices stacked along M in one MMA
     static constexpr int NMMA = 4 / SPM;                   // MMAs per 32 coordinates
-    static constexpr int kOpStageBytes = 4 * RP * kTK;     // slices 3, 2, 1, 0 one after the other
-    static constexpr int kOpStages = 4;
+    static constexpr int kOpStageBytes = 4 * RP * kTK;     // one tile: slices 3, 2, 1, 0 one after the other
+    static constexpr int kSlotBytes = 2 * kOpStageBytes;   // a step = two tiles
+    static constexpr int kSlots = 2;
     static constexpr int kTmemCols = RP == 64 ? 512 : 128;
     static constexpr int kChunks = F / FC;                 // boxes per tile
     static constexpr int RWC = (FC + W - 1) / W;           // rows of a box one converter warp may own
     static constexpr int kBoxFloats = R * FC * kTK;
     static constexpr int kBoxBytes = kBoxFloats * 4;
     static constexpr int kThreads = (kConvWarp0 + W) * 32;
-    static constexpr int kSmem = 1024 + kOpStages * kOpStageBytes + NS * kBoxBytes + kCtlBytes;
+    static constexpr int kSmem = 1024 + kSlots * kSlotBytes + NS * kBoxBytes + kCtlBytes;
     static_assert(F <= 64, "at most 64 rows");
     static_assert(kChunks * FC == F, "FC must divide F");
     static_assert(kBoxBytes % 128 == 0, "TMA destinations are 128-byte aligned");
@@ -118,12 +123,12 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
     pairdist_i8_kernel(const __grid_constant__ CUtensorMap map, int64_t d, float* __restrict__ voted, int64_t ld_voted,
                        double* __restrict__ tpart, int* __restrict__ info) {
     using S = I8Shape<F, W, R, FC, NS>;
-    constexpr int RP = S::RP, SPM = S::SPM, NMMA = S::NMMA, NO = S::kOpStages, CH = S::kChunks, RWC = S::RWC;
+    constexpr int RP = S::RP, SPM = S::SPM, NMMA = S::NMMA, NO = S::kSlots, CH = S::kChunks, RWC = S::RWC;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char* op = base;
-    float* in = reinterpret_cast<float*>(base + NO * S::kOpStageBytes);
-    unsigned char* ctl = base + NO * S::kOpStageBytes + NS * S::kBoxBytes;
+    float* in = reinterpret_cast<float*>(base + NO * S::kSlotBytes);
+    unsigned char* ctl = base + NO * S::kSlotBytes + NS * S::kBoxBytes;
     uint64_t* op_full = reinterpret_cast<uint64_t*>(ctl);
     uint64_t* op_empty = op_full + NO;
     uint64_t* in_full = op_empty + NO;
@@ -131,9 +136,9 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
     uint64_t* acc_ready = in_empty + NS;
     uint64_t* drain_go = acc_ready + 1;
     uint64_t* drained = drain_go + 1;
-    volatile int* e_stage = reinterpret_cast<volatile int*>(drained + 1);  // [NO][64]: the rows' exponents BEFORE a tile
+    volatile int* e_stage = reinterpret_cast<volatile int*>(drained + 1);  // [NO][64]: the rows' exponents BEFORE a step
     volatile int* e_cur = e_stage + NO * 64;                                 // [64]: the rows' exponents now
-    int* op_flush = const_cast<int*>(e_cur) + 64;                            // [NO]: some row's scale changes with this tile
+    volatile int* op_flush = e_cur + 64;                                     // [NO]: some row's scale changes with this step
     volatile int* drain_stage = op_flush + NO;                               // which e_stage row a drain uses
     volatile int* drain_final = drain_stage + 1;                             // is it the last drain
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(drain_final) + 1);
@@ -144,6 +149,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
     const int64_t n_tiles = (d + kTK - 1) / kTK;
     // tiles are dealt round-robin, so that at any moment the CTAs read neighbouring pieces of each row
     const int64_t my_tiles = (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x;  // at least 1: the grid never exceeds n_tiles
+    const int64_t my_steps = (my_tiles + 1) / 2;                                   // the last step may hold one tile
     double* tp = tpart + static_cast<size_t>(blockIdx.x) * F * F;
 
     if (tid == 0) {
@@ -165,7 +171,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
     }
     if (tid < 64) e_cur[tid] = kENone;
     // rows f .. RP-1 of every slice stay zero for the whole run
-    for (int e = tid; e < NO * S::kOpStageBytes / 16; e += S::kThreads) reinterpret_cast<uint4*>(op)[e] = make_uint4(0, 0, 0, 0);
+    for (int e = tid; e < NO * S::kSlotBytes / 16; e += S::kThreads) reinterpret_cast<uint4*>(op)[e] = make_uint4(0, 0, 0, 0);
     for (int e = tid; e < F * F; e += S::kThreads) tp[e] = 0.0;
     fence_async_smem();
     if (warp == kMmaWarp) tmem_alloc(tmem_slot, S::kTmemCols);
@@ -232,17 +238,23 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
             uint32_t n_flush = 0, have_acc = 0;
             int since = 0;
             bool ok = true;
-            // tile my_tiles carries no data: it hands over the final exponents for the last drain
-            for (int64_t it = 0; it <= my_tiles && ok; ++it) {
-                const int o = static_cast<int>(it % NO);
-                if (!mbar_wait_live(&op_full[o], static_cast<uint32_t>(it / NO) & 1, dead)) {
+            uint64_t desc0[NO];
+#pragma unroll
+            for (int o = 0; o < NO; ++o) desc0[o] = smem_desc_k128(smem_u32(op + static_cast<size_t>(o) * S::kSlotBytes));
+            int o = 0;
+            uint32_t phase = 0;
+            // step my_steps carries no data: it hands over the final exponents for the last drain
+            for (int64_t step = 0; step <= my_steps && ok; ++step) {
+                if (!mbar_wait_live(&op_full[o], phase, dead)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after_sync();
-                const bool last = it == my_tiles;
-                const int wants = atomicExch(&op_flush[o], 0);
-                if (have_acc && (wants || since == kFlushTiles || last)) {
+                const bool last = step == my_steps;
+                // every converter has arrived, so nobody writes the flag until the slot is handed back
+                const int wants = op_flush[o];
+                if (wants) op_flush[o] = 0;
+                if (have_acc && (wants || since >= kFlushTiles - 1 || last)) {
                     *drain_stage = o;
                     *drain_final = last ? 1 : 0;
                     mma_commit(acc_ready);
@@ -257,38 +269,62 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
                     since = 0;
                 }
                 if (last) break;
-                const uint32_t op_addr = smem_u32(op + static_cast<size_t>(o) * S::kOpStageBytes);
+                uint64_t slot_desc = desc0[0];
 #pragma unroll
-                for (int ks = 0; ks < kTK / 32; ++ks) {
+                for (int k = 1; k < NO; ++k)
+                    if (o == k) slot_desc = desc0[k];
+                const int n_sub = (2 * step + 1 < my_tiles) ? 2 : 1;
+                for (int sub = 0; sub < n_sub; ++sub) {
 #pragma unroll
-                    for (int m = 0; m < NMMA; ++m) {
-                        const uint64_t desc = smem_desc_k128(op_addr + m * SPM * RP * kTK + ks * 32);
-                        mma_s8(tmem_base + S::mma_col(m), desc, desc, idesc_s8(128, S::mma_n(m)), have_acc | (ks > 0));
+                    for (int ks = 0; ks < kTK / 32; ++ks) {
+#pragma unroll
+                        for (int m = 0; m < NMMA; ++m) {
+                            // the start-address field counts 16-byte units and cannot carry out of its 14 bits
+                            const uint64_t desc = slot_desc + static_cast<uint64_t>((sub * S::kOpStageBytes + m * SPM * RP * kTK + ks * 32) >> 4);
+                            mma_s8(tmem_base + S::mma_col(m), desc, desc, idesc_s8(128, S::mma_n(m)), have_acc | (sub > 0) | (ks > 0));
+                        }
                     }
                 }
                 mma_commit(&op_empty[o]);
                 have_acc = 1;
-                ++since;
+                since += n_sub;
+                if (++o == NO) {
+                    o = 0;
+                    phase ^= 1;
+                }
             }
             if (!ok) atomicAdd(&g_i8_timeouts, 1u);
         }
     } else if (warp == kTmaWarp) {
         // ------------------------------------------------------------------ TMA producer
+        // box order: step by step, box-row by box-row, first the earlier tile of the step then the later
         if (lane == 0) {
-            const int64_t n_boxes = my_tiles * CH;
-            int64_t issued = 0;
             bool ok = true;
-            for (; issued < n_boxes; ++issued) {
-                const int s = static_cast<int>(issued % NS);
-                const uint32_t round = static_cast<uint32_t>(issued / NS);
-                if (round > 0 && !mbar_wait_live(&in_empty[s], (round - 1) & 1, dead)) {
-                    ok = false;
-                    break;
+            int s = 0, filled = 0;
+            uint32_t phase = 0;
+            int64_t issued = 0;
+            for (int64_t step = 0; step < my_steps && ok; ++step) {
+                const int n_sub = (2 * step + 1 < my_tiles) ? 2 : 1;
+                for (int c = 0; c < CH && ok; ++c) {
+                    for (int sub = 0; sub < n_sub; ++sub) {
+                        if (filled == NS) {
+                            if (!mbar_wait_live(&in_empty[s], phase ^ 1, dead)) {
+                                ok = false;
+                                break;
+                            }
+                        } else {
+                            ++filled;
+                        }
+                        const int64_t tile = blockIdx.x + (2 * step + sub) * gridDim.x;
+                        mbar_expect_tx(&in_full[s], S::kBoxBytes);
+                        tma_load_3d(in + static_cast<size_t>(s) * S::kBoxFloats, &map, &in_full[s], static_cast<int>(tile * kTK), c * FC, 0);
+                        ++issued;
+                        if (++s == NS) {
+                            s = 0;
+                            phase ^= 1;
+                        }
+                    }
                 }
-                const int64_t tile = blockIdx.x + (issued / CH) * gridDim.x;
-                const int chunk = static_cast<int>(issued % CH);
-                mbar_expect_tx(&in_full[s], S::kBoxBytes);
-                tma_load_3d(in + static_cast<size_t>(s) * S::kBoxFloats, &map, &in_full[s], static_cast<int>(tile * kTK), chunk * FC, 0);
             }
             if (!ok) {
                 atomicAdd(&g_i8_timeouts, 1u);
@@ -302,87 +338,108 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
         const int cw = warp - kConvWarp0;
         int unrepresentable = 0;
         bool ok = true;
-        int64_t box = 0;
-        for (int64_t it = 0; it < my_tiles && ok; ++it) {
-            const int o = static_cast<int>(it % NO);
-            const int64_t j = (blockIdx.x + it * gridDim.x) * kTK + 4 * lane;
-            unsigned char* tile = op + static_cast<size_t>(o) * S::kOpStageBytes;
+        int s = 0, o = 0;
+        uint32_t in_phase = 0, op_phase = 0;
+        for (int64_t step = 0; step < my_steps && ok; ++step) {
+            const int n_sub = (2 * step + 1 < my_tiles) ? 2 : 1;
+            const int64_t j0 = (blockIdx.x + 2 * step * gridDim.x) * kTK + 4 * lane;  // this lane's coordinates in the earlier tile
+            unsigned char* slot = op + static_cast<size_t>(o) * S::kSlotBytes;
             bool raise = false, have_slot = false;
 #pragma unroll 1
-            for (int c = 0; c < CH && ok; ++c, ++box) {
-                const int s = static_cast<int>(box % NS);
-                if (!mbar_wait_live(&in_full[s], static_cast<uint32_t>(box / NS) & 1, dead)) {
-                    ok = false;
-                    break;
-                }
-                const uint32_t* src = reinterpret_cast<const uint32_t*>(in + static_cast<size_t>(s) * S::kBoxFloats);
-                // rows of this box that belong to this warp: c*FC + off + W*i
+            for (int c = 0; c < CH && ok; ++c) {
+                // rows of this box-row that belong to this warp: c*FC + off + W*i
                 const int off = ((cw - c * FC) % W + W) % W;
-                float4 val[RWC];
+                float4 val[2][RWC];
                 int E[RWC];
 #pragma unroll
-                for (int i = 0; i < RWC; ++i) {
-                    const int fi = off + W * i;
-                    if (fi < FC) {
-                        uint4 w;
-                        if constexpr (R == 1) {
-                            w = *reinterpret_cast<const uint4*>(src + fi * kTK + 4 * lane);
-                        } else {
-                            uint4 x[R];
+                for (int sub = 0; sub < 2; ++sub) {
+                    if (sub < n_sub) {
+                        if (!mbar_wait_live(&in_full[s], in_phase, dead)) {
+                            ok = false;
+                            break;
+                        }
+                        const uint32_t* src = reinterpret_cast<const uint32_t*>(in + static_cast<size_t>(s) * S::kBoxFloats);
+                        const int64_t j = j0 + sub * static_cast<int64_t>(gridDim.x) * kTK;
 #pragma unroll
-                            for (int k = 0; k < R; ++k) x[k] = *reinterpret_cast<const uint4*>(src + (k * FC + fi) * kTK + 4 * lane);
-                            uint32_t cp[R];
+                        for (int i = 0; i < RWC; ++i) {
+                            const int fi = off + W * i;
+                            if (fi < FC) {
+                                uint4 w;
+                                if constexpr (R == 1) {
+                                    w = *reinterpret_cast<const uint4*>(src + fi * kTK + 4 * lane);
+                                } else {
+                                    uint4 x[R];
 #pragma unroll
-                            for (int k = 0; k < R; ++k) cp[k] = x[k].x;
-                            w.x = vote_bits<R>(cp);
+                                    for (int k = 0; k < R; ++k) x[k] = *reinterpret_cast<const uint4*>(src + (k * FC + fi) * kTK + 4 * lane);
+                                    uint32_t cp[R];
 #pragma unroll
-                            for (int k = 0; k < R; ++k) cp[k] = x[k].y;
-                            w.y = vote_bits<R>(cp);
+                                    for (int k = 0; k < R; ++k) cp[k] = x[k].x;
+                                    w.x = vote_bits<R>(cp);
 #pragma unroll
-                            for (int k = 0; k < R; ++k) cp[k] = x[k].z;
-                            w.z = vote_bits<R>(cp);
+                                    for (int k = 0; k < R; ++k) cp[k] = x[k].y;
+                                    w.y = vote_bits<R>(cp);
 #pragma unroll
-                            for (int k = 0; k < R; ++k) cp[k] = x[k].w;
-                            w.w = vote_bits<R>(cp);
-                            uint32_t* q = reinterpret_cast<uint32_t*>(voted + (c * FC + fi) * ld_voted + j);
-                            if (j + 3 < d) {
-                                __stcs(reinterpret_cast<uint4*>(q), w);
-                            } else {  // ragged end
-                                if (j < d) q[0] = w.x;
-                                if (j + 1 < d) q[1] = w.y;
-                                if (j + 2 < d) q[2] = w.z;
+                                    for (int k = 0; k < R; ++k) cp[k] = x[k].z;
+                                    w.z = vote_bits<R>(cp);
+#pragma unroll
+                                    for (int k = 0; k < R; ++k) cp[k] = x[k].w;
+                                    w.w = vote_bits<R>(cp);
+                                    uint32_t* q = reinterpret_cast<uint32_t*>(voted + (c * FC + fi) * ld_voted + j);
+                                    if (j + 3 < d) {
+                                        __stcs(reinterpret_cast<uint4*>(q), w);
+                                    } else {  // ragged end
+                                        if (j < d) q[0] = w.x;
+                                        if (j + 1 < d) q[1] = w.y;
+                                        if (j + 2 < d) q[2] = w.z;
+                                    }
+                                }
+                                val[sub][i] = make_float4(__uint_as_float(w.x), __uint_as_float(w.y), __uint_as_float(w.z), __uint_as_float(w.w));
                             }
                         }
-                        val[i] = make_float4(__uint_as_float(w.x), __uint_as_float(w.y), __uint_as_float(w.z), __uint_as_float(w.w));
-                        E[i] = e_cur[c * FC + fi];
+                        // the box is in registers: hand it back
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_relaxed(&in_empty[s]);
+                        if (++s == NS) {
+                            s = 0;
+                            in_phase ^= 1;
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < RWC; ++i) val[sub][i] = make_float4(0.f, 0.f, 0.f, 0.f);
                     }
                 }
-                // the box is in registers: hand it back
-                __syncwarp();
-                if (lane == 0) mbar_arrive_relaxed(&in_empty[s]);
+                if (!ok) break;
                 // Scale with the rows' current exponents and look at the largest result: below 2^30 (and
                 // no NaN) the rows convert as they are - nearly always.  Otherwise the rows' largest
-                // magnitudes are found exactly, exponents grow, and the rows are scaled again.
+                // magnitudes are found exactly, exponents grow, and the rows are scaled again.  Both tiles
+                // of the step take the same exponents.
                 int old[RWC];
-                float4 t[RWC];
+                float4 t[2][RWC];
                 float m = 0.f;
 #pragma unroll
                 for (int i = 0; i < RWC; ++i) {
                     if (off + W * i < FC) {
+                        E[i] = e_cur[c * FC + off + W * i];
                         old[i] = E[i];
-                        if (E[i] == kENone) m = __int_as_float(0x7f800000);  // no exponent yet (first tile)
+                        if (E[i] == kENone) m = __int_as_float(0x7f800000);  // no exponent yet (first step)
                         const float scale = __int_as_float((30 - (E[i] == kENone ? 0 : E[i]) + 127) << 23);
-                        t[i] = make_float4(val[i].x * scale, val[i].y * scale, val[i].z * scale, val[i].w * scale);
-                        m = max_abs_nan(max_abs_nan(m, t[i].x), max_abs_nan(t[i].y, max_abs_nan(t[i].z, t[i].w)));
+#pragma unroll
+                        for (int sub = 0; sub < 2; ++sub) {
+                            t[sub][i] = make_float4(val[sub][i].x * scale, val[sub][i].y * scale, val[sub][i].z * scale, val[sub][i].w * scale);
+                            m = max_abs_nan(max_abs_nan(m, t[sub][i].x), max_abs_nan(t[sub][i].y, max_abs_nan(t[sub][i].z, t[sub][i].w)));
+                        }
                     }
                 }
                 if (__any_sync(0xffffffffu, !(fabsf(m) < 1073741824.0f))) {
 #pragma unroll
                     for (int i = 0; i < RWC; ++i) {
                         if (off + W * i < FC) {
-                            const uint32_t m4 = max(max(__float_as_uint(val[i].x) & 0x7fffffffu, __float_as_uint(val[i].y) & 0x7fffffffu),
-                                                    max(__float_as_uint(val[i].z) & 0x7fffffffu, __float_as_uint(val[i].w) & 0x7fffffffu));
-                            const int need = static_cast<int>(__reduce_max_sync(0xffffffffu, m4) >> 23) - 126;  // |v| < 2^need
+                            uint32_t m8 = 0;
+#pragma unroll
+                            for (int sub = 0; sub < 2; ++sub)
+                                m8 = max(m8, max(max(__float_as_uint(val[sub][i].x) & 0x7fffffffu, __float_as_uint(val[sub][i].y) & 0x7fffffffu),
+                                                 max(__float_as_uint(val[sub][i].z) & 0x7fffffffu, __float_as_uint(val[sub][i].w) & 0x7fffffffu)));
+                            const int need = static_cast<int>(__reduce_max_sync(0xffffffffu, m8) >> 23) - 126;  // |v| < 2^need
                             if (need > 60) unrepresentable = 1;  // infinities, NaNs, magnitudes beyond 2^60
                             if (E[i] == kENone || need > E[i]) {   // |v| * 2^(30 - E) may reach 2^30
                                 raise = raise || E[i] != kENone;
@@ -390,13 +447,15 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
                                 if (lane == 0) e_cur[c * FC + off + W * i] = E[i];
                             }
                             const float scale = __int_as_float((30 - E[i] + 127) << 23);
-                            t[i] = make_float4(val[i].x * scale, val[i].y * scale, val[i].z * scale, val[i].w * scale);
+#pragma unroll
+                            for (int sub = 0; sub < 2; ++sub)
+                                t[sub][i] = make_float4(val[sub][i].x * scale, val[sub][i].y * scale, val[sub][i].z * scale, val[sub][i].w * scale);
                         }
                     }
                 }
-                // the operand slot is free once the MMAs of tile it - NO are done
+                // the operand slot is free once the MMAs of step - NO are done
                 if (!have_slot) {
-                    if (it >= NO && !mbar_wait_live(&op_empty[o], (static_cast<uint32_t>(it / NO) - 1) & 1, dead)) {
+                    if (step >= NO && !mbar_wait_live(&op_empty[o], op_phase ^ 1, dead)) {
                         ok = false;
                         break;
                     }
@@ -407,35 +466,43 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
                     const int fi = off + W * i;
                     if (fi < FC) {
                         const int r = c * FC + fi;
-                        // a row whose scale changes hands its old exponent to the drain that comes before this tile
+                        // a row whose scale changes hands its old exponent to the drain that comes before this step
                         if (lane == 0) e_stage[o * 64 + r] = old[i] == kENone ? E[i] : old[i];
-                        uint32_t w[4];
-                        slice4(t[i], w);
-                        // row r of a slice: 8-row group r/8, row r%8 in it, 16-byte chunk (lane/4) ^ (r%8)
-                        unsigned char* dst = tile + (r >> 3) * 1024 + (r & 7) * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | ((lane & 3) << 2));
-                        *reinterpret_cast<uint32_t*>(dst + 0 * RP * kTK) = w[3];
-                        *reinterpret_cast<uint32_t*>(dst + 1 * RP * kTK) = w[2];
-                        *reinterpret_cast<uint32_t*>(dst + 2 * RP * kTK) = w[1];
-                        *reinterpret_cast<uint32_t*>(dst + 3 * RP * kTK) = w[0];
+                        // row r of a slice: 128 bytes per row, 16-byte chunk (lane/4) ^ (r%8) within it
+                        unsigned char* dst = slot + r * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | ((lane & 3) << 2));
+#pragma unroll
+                        for (int sub = 0; sub < 2; ++sub) {
+                            if (sub < n_sub) {
+                                uint32_t w[4];
+                                slice4(t[sub][i], w);
+                                *reinterpret_cast<uint32_t*>(dst + sub * S::kOpStageBytes + 0 * RP * kTK) = w[3];
+                                *reinterpret_cast<uint32_t*>(dst + sub * S::kOpStageBytes + 1 * RP * kTK) = w[2];
+                                *reinterpret_cast<uint32_t*>(dst + sub * S::kOpStageBytes + 2 * RP * kTK) = w[1];
+                                *reinterpret_cast<uint32_t*>(dst + sub * S::kOpStageBytes + 3 * RP * kTK) = w[0];
+                            }
+                        }
                     }
                 }
             }
             if (!ok) break;
-            if (!have_slot && it >= NO && !mbar_wait_live(&op_empty[o], (static_cast<uint32_t>(it / NO) - 1) & 1, dead)) {
+            if (!have_slot && step >= NO && !mbar_wait_live(&op_empty[o], op_phase ^ 1, dead)) {
                 ok = false;
                 break;
             }
             fence_async_smem();
             __syncwarp();
             if (lane == 0) {
-                if (raise) atomicOr(&op_flush[o], 1);
+                if (raise) atomicOr(const_cast<int*>(&op_flush[o]), 1);
                 mbar_arrive_relaxed(&op_full[o]);
+            }
+            if (++o == NO) {
+                o = 0;
+                op_phase ^= 1;
             }
         }
         if (ok) {
-            // the stage after the last tile: current exponents, nothing to multiply
-            const int o = static_cast<int>(my_tiles % NO);
-            if (my_tiles >= NO && !mbar_wait_live(&op_empty[o], (static_cast<uint32_t>(my_tiles / NO) - 1) & 1, dead)) ok = false;
+            // the slot after the last step: current exponents, nothing to multiply
+            if (my_steps >= NO && !mbar_wait_live(&op_empty[o], op_phase ^ 1, dead)) ok = false;
             if (ok) {
                 if (lane == 0)
                     for (int r = cw; r < F; r += W) e_stage[o * 64 + r] = e_cur[r];
