@@ -283,6 +283,14 @@ def extra_paths(bz, inputs, torch, device):
         gbs = nbytes / (ms * 1e-3) / 1e9
         return {"achieved_GBs": gbs, "frac_of_measured_hbm": gbs / peak}
 
+    def timed_fp32(fn):
+        """The same call with the distances kept on the binary32 kernels (the library reads the variable per call)."""
+        os.environ["BZ_PAIRDIST_PATH"] = "fp32"
+        try:
+            return timed(torch, fn, 5, 2)
+        finally:
+            del os.environ["BZ_PAIRDIST_PATH"]
+
     # vote -> multi-Krum: K=21, r=3, l=7, f=49, d=11.2M, q=5 ALIE, c=5, m=44
     cfg = dict(l=7, r=3, q=5, d=11_200_000, attack="alie", seed=0)
     rep, fw, byz, cmax = make_inputs(bz, inputs, cfg, device)
@@ -293,20 +301,24 @@ def extra_paths(bz, inputs, torch, device):
     sel44 = torch.arange(44, dtype=torch.int32, device=device)
     t_vote = timed(torch, lambda: bz.vote(rep, voted), 5, 2)
     t_pd = timed(torch, lambda: bz.pairdist(voted, ws), 5, 2)
+    t_pd32 = timed_fp32(lambda: bz.pairdist(voted, ws))
     t_mean = timed(torch, lambda: bz.mean_rows(voted, sel44, out), 5, 2)
     t_mk = timed(torch, lambda: bz.multikrum(voted, 5, 44, workspace=ws, out=out), 5, 2)
     t_vm = timed(torch, lambda: bz.vote_median(rep, out), 5, 2)
     t_med = timed(torch, lambda: bz.median(voted, out), 5, 2)
     t_vpd = timed(torch, lambda: bz.vote_pairdist(rep, voted, ws), 5, 2)
+    t_vpd32 = timed_fp32(lambda: bz.vote_pairdist(rep, voted, ws))
     t_vmk = timed(torch, lambda: bz.vote_multikrum(rep, 5, 44, voted=voted, workspace=ws, out=out), 5, 2)
     bytes_pipeline = (4 * r * f + 4 * f + 4 * f + 4 * 44 + 4) * d
     res["vote+multikrum"] = dict(
         workload="K=21 r=3 l=7 f=49 d=11.2M, q=5 ALIE, c=5 m=44", c_max=cmax,
         coordinates_per_s=d / ((t_vote + t_mk) * 1e-3), ms_vote=t_vote, ms_multikrum=t_mk, ms_pairdist=t_pd,
-        ms_mean_rows=t_mean, pairdist_fma_lane_ops_per_s=2 * (f * (f - 1) // 2) * d / (t_pd * 1e-3),
+        ms_mean_rows=t_mean, ms_pairdist_fp32=t_pd32, pairdist_fp32_fma_lane_ops_per_s=2 * (f * (f - 1) // 2) * d / (t_pd32 * 1e-3),
+        pairdist=dict(kernel="integer MMA (tcgen05 kind::i8)", **hbm(4 * f * d, t_pd)),
         vote=hbm((4 * r * f + 4 * f) * d, t_vote), mean_rows=hbm((4 * 44 + 4) * d, t_mean),
         pipeline=hbm(bytes_pipeline, t_vote + t_mk),
-        single_pass=dict(ms_vote_pairdist=t_vpd, ms_vote_multikrum=t_vmk, coordinates_per_s=d / (t_vmk * 1e-3),
+        single_pass=dict(ms_vote_pairdist=t_vpd, ms_vote_pairdist_fp32=t_vpd32, vote_pairdist=hbm((4 * r * f + 4 * f) * d, t_vpd),
+                         ms_vote_multikrum=t_vmk, coordinates_per_s=d / (t_vmk * 1e-3),
                          **hbm((4 * r * f + 4 * f + 4 * 44 + 4) * d, t_vmk)))
     res["vote+median f=49"] = dict(workload="same replicas, fused vote+median", ms=t_vm, coordinates_per_s=d / (t_vm * 1e-3),
                                    **hbm((4 * r * f + 4) * d, t_vm))
@@ -325,6 +337,7 @@ def extra_paths(bz, inputs, torch, device):
     sel17 = torch.arange(17, dtype=torch.int32, device=device)
     t_vote = timed(torch, lambda: bz.vote(rep, voted), 5, 2)
     t_pd = timed(torch, lambda: bz.pairdist(voted, ws), 5, 2)
+    t_pd32 = timed_fp32(lambda: bz.pairdist(voted, ws))
     t_tm = timed(torch, lambda: bz.trimmed_mean(voted, sel17, 9, out), 5, 2)
     t_bu = timed(torch, lambda: bz.bulyan(voted, 4, workspace=ws, out=out), 5, 2)
     t_vm = timed(torch, lambda: bz.vote_median(rep, out), 5, 2)
@@ -334,7 +347,7 @@ def extra_paths(bz, inputs, torch, device):
     res["vote+bulyan"] = dict(
         workload="K=25 r=5 l=5 f=25 d=25M (1% Student-t coordinates), q=6 constant, c=4 (theta=17, beta=9)",
         c_max=cmax, coordinates_per_s=d / ((t_vote + t_bu) * 1e-3), ms_vote=t_vote, ms_bulyan=t_bu, ms_pairdist=t_pd,
-        ms_trimmed_mean=t_tm, vote=hbm((4 * r * f + 4 * f) * d, t_vote), pairdist=hbm(4 * f * d, t_pd),
+        ms_pairdist_fp32=t_pd32, ms_trimmed_mean=t_tm, vote=hbm((4 * r * f + 4 * f) * d, t_vote), pairdist=hbm(4 * f * d, t_pd),
         trimmed_mean=hbm((4 * theta + 4) * d, t_tm), pipeline=hbm(bytes_pipeline, t_vote + t_bu),
         single_pass=dict(ms_vote_bulyan=t_vbu, coordinates_per_s=d / (t_vbu * 1e-3),
                          **hbm((4 * r * f + 4 * f + 4 * theta + 4) * d, t_vbu)))

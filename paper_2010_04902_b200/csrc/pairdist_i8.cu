@@ -1,6 +1,5 @@
 // Pairwise squared distances of the Krum family (Sec. 1.2; cost in Appendix A.1) on the tensor cores,
 // in exact integer arithmetic.  Host side; the kernel is in pairdist_i8_kernel.cuh.
-#include <cstdlib>
 #include "pairdist_i8_kernel.cuh"
 
 namespace bz {
@@ -73,10 +72,10 @@ __global__ void __launch_bounds__(1024)
 
 // rep: R = 1: rows [f][d] with leading dimension ld_file.  R > 1: replicas[r][f][d].
 // Returns 1 if the tensor map cannot express the shape.
-template <int F, int W, int R, int FC, int NS>
+template <int F, int W, int R, int FC, int NS, int TS>
 int launch_i8(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted, double* dist,
               double* tpart, int* info, int* flag, int force, cudaStream_t s) {
-    using S = I8Shape<F, W, R, FC, NS>;
+    using S = I8Shape<F, W, R, FC, NS, TS>;
     EncodeTiledFn enc = encode_tiled();
     if (enc == nullptr) return 1;
     CUtensorMap map;
@@ -88,7 +87,7 @@ int launch_i8(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, floa
                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (cr != CUDA_SUCCESS) return 1;
-    auto kern = pairdist_i8_kernel<F, W, R, FC, NS>;
+    auto kern = pairdist_i8_kernel<F, W, R, FC, NS, TS>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kSmem);
     if (e != cudaSuccess) return cuda_failed(e);
     int64_t ctas = (d + kTK - 1) / kTK;
@@ -138,15 +137,9 @@ int pairdist_i8(const float* v, int f, int64_t d, int64_t ld, double* dist, void
     if (!pairdist_i8_has(f) || !aligned16(v) || (ld % 4) != 0 || d < 64 * kTK || d >= (int64_t(1) << 31)) return 1;
     const Scratch sc = carve(ws, f);
     *flag_out = sc.flag;
-    // <rows, converter warps, copies, rows per box, boxes in the ring>
-    const char* we = std::getenv("BZ_I8_W");
-    const int w = we ? std::atoi(we) : 0;
-#define TRY(F_, W_, NS_) if (f == F_ && w == W_) return launch_i8<F_, W_, 1, F_, NS_>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
-    TRY(49, 16, 3) TRY(49, 20, 3) TRY(49, 12, 3) TRY(49, 8, 3)
-    TRY(25, 8, 8) TRY(25, 12, 8) TRY(25, 16, 8) TRY(25, 20, 8)
-#undef TRY
-    if (f == 25) return launch_i8<25, 25, 1, 25, 8>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
-    return launch_i8<49, 13, 1, 49, 3>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
+    // <rows, converter warps, copies, rows per box, boxes in the ring, tiles per step>
+    if (f == 25) return launch_i8<25, 13, 1, 25, 6, 4>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
+    return launch_i8<49, 13, 1, 49, 3, 2>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
 }
 
 // The same from the replicas: vote (Eq. 3) and distances in one pass; the winners go to `voted`.
@@ -157,14 +150,14 @@ int vote_pairdist_i8(const float* rep, int r, int f, int64_t d, int64_t ld_file,
         return 1;
     const Scratch sc = carve(ws, f);
     *flag_out = sc.flag;
-#define BZ_I8_CASE(R_, F_, W_, FC_, NS_) \
-    if (r == R_ && f == F_)              \
-        return launch_i8<F_, W_, R_, FC_, NS_>(rep, d, ld_file, ld_rep, voted, ld_voted, dist, sc.tpart, sc.info, sc.flag, force, s);
-    BZ_I8_CASE(3, 25, 10, 5, 8)
-    BZ_I8_CASE(3, 49, 14, 7, 6)
-    BZ_I8_CASE(5, 25, 10, 5, 6)
-    BZ_I8_CASE(5, 49, 14, 7, 4)
-    BZ_I8_CASE(7, 49, 14, 7, 3)
+#define BZ_I8_CASE(R_, F_, W_, FC_, NS_, TS_) \
+    if (r == R_ && f == F_)                   \
+        return launch_i8<F_, W_, R_, FC_, NS_, TS_>(rep, d, ld_file, ld_rep, voted, ld_voted, dist, sc.tpart, sc.info, sc.flag, force, s);
+    BZ_I8_CASE(3, 25, 10, 5, 8, 4)
+    BZ_I8_CASE(3, 49, 14, 7, 6, 2)
+    BZ_I8_CASE(5, 25, 10, 5, 6, 4)
+    BZ_I8_CASE(5, 49, 14, 7, 4, 2)
+    BZ_I8_CASE(7, 49, 14, 7, 3, 2)
 #undef BZ_I8_CASE
     return 1;
 }

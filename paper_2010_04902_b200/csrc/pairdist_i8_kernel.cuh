@@ -31,7 +31,7 @@
 //
 // Every warp of a CTA sees every tile, so what a warp spends per tile on waiting, signalling and
 // bookkeeping bounds the CTA's rate whatever the number of warps: the unit of work between two
-// signals is therefore a step of two tiles.
+// signals is therefore a step of TS tiles (2 to 4, as many as shared memory holds).
 //
 // Roles in a CTA (one CTA per SM, tiles dealt round-robin): one thread issues TMA loads of boxes
 // [R copies][FC rows][128 coordinates] into a ring of shared memory; W converter warps own fixed rows
@@ -58,13 +58,14 @@ constexpr int kInfoBad = 64;
 
 __device__ unsigned int g_i8_timeouts = 0;
 
-// F rows, W converter warps, R copies per row (1: the rows are given), FC rows per box, NS boxes in the ring
-template <int F, int W, int R, int FC, int NS> struct I8Shape {
+// F rows, W converter warps, R copies per row (1: the rows are given), FC rows per box, NS boxes in the ring,
+// TS tiles per step
+template <int F, int W, int R, int FC, int NS, int TS> struct I8Shape {
     static constexpr int RP = F <= 32 ? 32 : 64;          // rows of one slice in an operand tile (f padded)
     static constexpr int SPM = 128 / RP;                   // slices stacked along M in one MMA
     static constexpr int NMMA = 4 / SPM;                   // MMAs per 32 coordinates
     static constexpr int kOpStageBytes = 4 * RP * kTK;     // one tile: slices 3, 2, 1, 0 one after the other
-    static constexpr int kSlotBytes = 2 * kOpStageBytes;   // a step = two tiles
+    static constexpr int kSlotBytes = TS * kOpStageBytes;  // a step = TS tiles
     static constexpr int kSlots = 2;
     static constexpr int kTmemCols = RP == 64 ? 512 : 128;
     static constexpr int kChunks = F / FC;                 // boxes per tile
@@ -118,11 +119,11 @@ __device__ __forceinline__ float max_abs_nan(float a, float b) {
 // R = 1: distances of the rows of `map` ([f][d]).  R > 1: `map` covers replicas[r][f][d]; row i is the vote
 // (Eq. 3, element by element on bit patterns) over its R copies, which is also written to
 // voted[i*ld_voted + j] (16-byte aligned, ld_voted a multiple of 4).
-template <int F, int W, int R, int FC, int NS>
-__global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
+template <int F, int W, int R, int FC, int NS, int TS>
+__global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
     pairdist_i8_kernel(const __grid_constant__ CUtensorMap map, int64_t d, float* __restrict__ voted, int64_t ld_voted,
                        double* __restrict__ tpart, int* __restrict__ info) {
-    using S = I8Shape<F, W, R, FC, NS>;
+    using S = I8Shape<F, W, R, FC, NS, TS>;
     constexpr int RP = S::RP, SPM = S::SPM, NMMA = S::NMMA, NO = S::kSlots, CH = S::kChunks, RWC = S::RWC;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -149,7 +150,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
     const int64_t n_tiles = (d + kTK - 1) / kTK;
     // tiles are dealt round-robin, so that at any moment the CTAs read neighbouring pieces of each row
     const int64_t my_tiles = (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x;  // at least 1: the grid never exceeds n_tiles
-    const int64_t my_steps = (my_tiles + 1) / 2;                                   // the last step may hold one tile
+    const int64_t my_steps = (my_tiles + TS - 1) / TS;                             // the last step may hold fewer tiles
     double* tp = tpart + static_cast<size_t>(blockIdx.x) * F * F;
 
     if (tid == 0) {
@@ -254,7 +255,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
                 // every converter has arrived, so nobody writes the flag until the slot is handed back
                 const int wants = op_flush[o];
                 if (wants) op_flush[o] = 0;
-                if (have_acc && (wants || since >= kFlushTiles - 1 || last)) {
+                if (have_acc && (wants || since > kFlushTiles - TS || last)) {
                     *drain_stage = o;
                     *drain_final = last ? 1 : 0;
                     mma_commit(acc_ready);
@@ -273,7 +274,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
 #pragma unroll
                 for (int k = 1; k < NO; ++k)
                     if (o == k) slot_desc = desc0[k];
-                const int n_sub = (2 * step + 1 < my_tiles) ? 2 : 1;
+                const int n_sub = static_cast<int>(my_tiles - TS * step < TS ? my_tiles - TS * step : TS);
                 for (int sub = 0; sub < n_sub; ++sub) {
 #pragma unroll
                     for (int ks = 0; ks < kTK / 32; ++ks) {
@@ -304,7 +305,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
             uint32_t phase = 0;
             int64_t issued = 0;
             for (int64_t step = 0; step < my_steps && ok; ++step) {
-                const int n_sub = (2 * step + 1 < my_tiles) ? 2 : 1;
+                const int n_sub = static_cast<int>(my_tiles - TS * step < TS ? my_tiles - TS * step : TS);
                 for (int c = 0; c < CH && ok; ++c) {
                     for (int sub = 0; sub < n_sub; ++sub) {
                         if (filled == NS) {
@@ -315,7 +316,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
                         } else {
                             ++filled;
                         }
-                        const int64_t tile = blockIdx.x + (2 * step + sub) * gridDim.x;
+                        const int64_t tile = blockIdx.x + (TS * step + sub) * gridDim.x;
                         mbar_expect_tx(&in_full[s], S::kBoxBytes);
                         tma_load_3d(in + static_cast<size_t>(s) * S::kBoxFloats, &map, &in_full[s], static_cast<int>(tile * kTK), c * FC, 0);
                         ++issued;
@@ -341,18 +342,18 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
         int s = 0, o = 0;
         uint32_t in_phase = 0, op_phase = 0;
         for (int64_t step = 0; step < my_steps && ok; ++step) {
-            const int n_sub = (2 * step + 1 < my_tiles) ? 2 : 1;
-            const int64_t j0 = (blockIdx.x + 2 * step * gridDim.x) * kTK + 4 * lane;  // this lane's coordinates in the earlier tile
+            const int n_sub = static_cast<int>(my_tiles - TS * step < TS ? my_tiles - TS * step : TS);
+            const int64_t j0 = (blockIdx.x + TS * step * gridDim.x) * kTK + 4 * lane;  // this lane's coordinates in the first tile
             unsigned char* slot = op + static_cast<size_t>(o) * S::kSlotBytes;
             bool raise = false, have_slot = false;
 #pragma unroll 1
             for (int c = 0; c < CH && ok; ++c) {
                 // rows of this box-row that belong to this warp: c*FC + off + W*i
                 const int off = ((cw - c * FC) % W + W) % W;
-                float4 val[2][RWC];
+                float4 val[TS][RWC];
                 int E[RWC];
 #pragma unroll
-                for (int sub = 0; sub < 2; ++sub) {
+                for (int sub = 0; sub < TS; ++sub) {
                     if (sub < n_sub) {
                         if (!mbar_wait_live(&in_full[s], in_phase, dead)) {
                             ok = false;
@@ -411,10 +412,10 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
                 if (!ok) break;
                 // Scale with the rows' current exponents and look at the largest result: below 2^30 (and
                 // no NaN) the rows convert as they are - nearly always.  Otherwise the rows' largest
-                // magnitudes are found exactly, exponents grow, and the rows are scaled again.  Both tiles
+                // magnitudes are found exactly, exponents grow, and the rows are scaled again.  All tiles
                 // of the step take the same exponents.
                 int old[RWC];
-                float4 t[2][RWC];
+                float4 t[TS][RWC];
                 float m = 0.f;
 #pragma unroll
                 for (int i = 0; i < RWC; ++i) {
@@ -424,7 +425,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
                         if (E[i] == kENone) m = __int_as_float(0x7f800000);  // no exponent yet (first step)
                         const float scale = __int_as_float((30 - (E[i] == kENone ? 0 : E[i]) + 127) << 23);
 #pragma unroll
-                        for (int sub = 0; sub < 2; ++sub) {
+                        for (int sub = 0; sub < TS; ++sub) {
                             t[sub][i] = make_float4(val[sub][i].x * scale, val[sub][i].y * scale, val[sub][i].z * scale, val[sub][i].w * scale);
                             m = max_abs_nan(max_abs_nan(m, t[sub][i].x), max_abs_nan(t[sub][i].y, max_abs_nan(t[sub][i].z, t[sub][i].w)));
                         }
@@ -436,7 +437,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
                         if (off + W * i < FC) {
                             uint32_t m8 = 0;
 #pragma unroll
-                            for (int sub = 0; sub < 2; ++sub)
+                            for (int sub = 0; sub < TS; ++sub)
                                 m8 = max(m8, max(max(__float_as_uint(val[sub][i].x) & 0x7fffffffu, __float_as_uint(val[sub][i].y) & 0x7fffffffu),
                                                  max(__float_as_uint(val[sub][i].z) & 0x7fffffffu, __float_as_uint(val[sub][i].w) & 0x7fffffffu)));
                             const int need = static_cast<int>(__reduce_max_sync(0xffffffffu, m8) >> 23) - 126;  // |v| < 2^need
@@ -448,7 +449,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
                             }
                             const float scale = __int_as_float((30 - E[i] + 127) << 23);
 #pragma unroll
-                            for (int sub = 0; sub < 2; ++sub)
+                            for (int sub = 0; sub < TS; ++sub)
                                 t[sub][i] = make_float4(val[sub][i].x * scale, val[sub][i].y * scale, val[sub][i].z * scale, val[sub][i].w * scale);
                         }
                     }
@@ -471,7 +472,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS>::kThreads, 1)
                         // row r of a slice: 128 bytes per row, 16-byte chunk (lane/4) ^ (r%8) within it
                         unsigned char* dst = slot + r * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | ((lane & 3) << 2));
 #pragma unroll
-                        for (int sub = 0; sub < 2; ++sub) {
+                        for (int sub = 0; sub < TS; ++sub) {
                             if (sub < n_sub) {
                                 uint32_t w[4];
                                 slice4(t[sub][i], w);
