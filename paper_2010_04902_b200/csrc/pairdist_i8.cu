@@ -6,42 +6,54 @@ namespace bz {
 
 namespace {
 
-// D from the CTAs' partial matrices, then the error estimate of the conversion.
+// D from the CTAs' partial matrices, then the error estimate of the conversion (two small kernels).
 // flag[0] = 1 asks for the binary32 kernel (estimate above the tolerance, or values the fixed-point
 // scale cannot hold); with force != 0 the flag stays 0 whatever the estimate says.
 // Estimate for a pair: each value is rounded to a multiple of its row's step, an unbiased error of
 // standard deviation 0.29 step; over d coordinates that moves D by about 2 sqrt(D var) + d var.
 constexpr double kRelTol = 5e-9;
 
+// One warp per pair a <= b: lane l takes CTAs l, l+32, ... in order, then the lanes are added in a fixed
+// tree.  Identical rows meet identical numbers in the same order and get identical distances.
 template <int F>
-__global__ void __launch_bounds__(1024)
-    pairdist_i8_reduce_kernel(const double* __restrict__ tpart, const int* __restrict__ info, int n_ctas, int64_t d, int force,
-                              double* __restrict__ dist, int* __restrict__ flag) {
-    __shared__ double D[F * F];
+__global__ void __launch_bounds__(256)
+    pairdist_i8_reduce_kernel(const double* __restrict__ tpart, int n_ctas, double* __restrict__ dist) {
+    const int pair = blockIdx.x * (blockDim.x / 32) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (pair >= F * F) return;
+    const int a = pair / F, b = pair % F;
+    if (a > b) return;
+    double s = 0.0;
+    if (a < b) {
+        for (int c = lane; c < n_ctas; c += 32) {
+            const double* T = tpart + static_cast<size_t>(c) * F * F;
+            s += (T[a * F + a] + T[b * F + b]) - (T[a * F + b] + T[b * F + a]);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xffffffffu, s, o);
+    }
+    if (lane == 0) {
+        dist[a * F + b] = s;
+        dist[b * F + a] = s;
+    }
+}
+
+// The error estimate.  flag[0] = 1 asks for the binary32 kernel.
+template <int F>
+__global__ void __launch_bounds__(64)
+    pairdist_i8_check_kernel(const double* __restrict__ dist, const int* __restrict__ info, int n_ctas, int64_t d, int force,
+                             int* __restrict__ flag) {
     __shared__ int s_emax[F];
     __shared__ int s_bad;
     const int tid = threadIdx.x;
-    if (tid < F) s_emax[tid] = kELo;
     if (tid == 0) s_bad = 0;
-    __syncthreads();
-    for (int e = tid; e < n_ctas * kInfoStride; e += blockDim.x) {
-        const int a = e % kInfoStride;
-        if (a < F) atomicMax(&s_emax[a], info[e]);
-        if (a == kInfoBad && info[e]) atomicOr(&s_bad, 1);
-    }
-    for (int p = tid; p < F * F; p += blockDim.x) {
-        const int a = p / F, b = p % F;
-        if (a > b) continue;
-        double s = 0.0;
-        if (a < b)
-            for (int c = 0; c < n_ctas; ++c) {
-                const double* T = tpart + static_cast<size_t>(c) * F * F;
-                s += (T[a * F + a] + T[b * F + b]) - (T[a * F + b] + T[b * F + a]);
-            }
-        D[a * F + b] = s;
-        D[b * F + a] = s;
+    if (tid < F) {
+        int e = kELo;
+        for (int c = 0; c < n_ctas; ++c) e = max(e, info[c * kInfoStride + tid]);
+        s_emax[tid] = e;
     }
     __syncthreads();
+    for (int c = tid; c < n_ctas; c += blockDim.x)
+        if (info[c * kInfoStride + kInfoBad]) atomicOr(&s_bad, 1);
     if (tid < F) {
         const int a = tid;
         const double step_a = __longlong_as_double(static_cast<long long>(1023 + s_emax[a] - 30) << 52);
@@ -51,7 +63,7 @@ __global__ void __launch_bounds__(1024)
             if (b == a) continue;
             const double step_b = __longlong_as_double(static_cast<long long>(1023 + s_emax[b] - 30) << 52);
             const double var = 0.0841 * (step_a * step_a + step_b * step_b);
-            const double v = D[a * F + b];
+            const double v = dist[a * F + b];
             if (v > 0.0) {
                 if (2.0 * sqrt(var / v) + static_cast<double>(d) * var / v > kRelTol) bad = true;
                 min_nz = fmin(min_nz, v);
@@ -66,7 +78,6 @@ __global__ void __launch_bounds__(1024)
         if (bad) atomicOr(&s_bad, 1);
     }
     __syncthreads();
-    for (int p = tid; p < F * F; p += blockDim.x) dist[p] = D[p];
     if (tid == 0) flag[0] = (s_bad && !force) ? 1 : 0;
 }
 
@@ -96,7 +107,11 @@ int launch_i8(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, floa
     note_launch();
     int st = check_launch();
     if (st != BZ_OK) return st;
-    pairdist_i8_reduce_kernel<F><<<1, 1024, 0, s>>>(tpart, info, static_cast<int>(ctas), d, force, dist, flag);
+    pairdist_i8_reduce_kernel<F><<<(F * F + 7) / 8, 256, 0, s>>>(tpart, static_cast<int>(ctas), dist);
+    note_launch();
+    st = check_launch();
+    if (st != BZ_OK) return st;
+    pairdist_i8_check_kernel<F><<<1, 64, 0, s>>>(dist, info, static_cast<int>(ctas), d, force, flag);
     note_launch();
     return check_launch();
 }
