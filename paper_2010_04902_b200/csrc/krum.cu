@@ -17,23 +17,41 @@ namespace {
 // ------------------------------------------------------------------------------------------------
 // Selection kernels: one CTA, thread a owns row a.
 
-// Krum score of row a inside the rows flagged in `active`: the nb smallest distances to the other
-// active rows, added in ascending order.  (Insertion sort in local memory; f <= BZ_MAX_F.)
-__device__ double krum_score_row(const double* dist, int f, const unsigned char* active, int a, int nb) {
-    double buf[BZ_MAX_F];
+// Row a's distances to the other rows, ascending (insertion sort in local memory; f <= BZ_MAX_F).
+// The loads are issued first, all independent; the order of a row never changes afterwards.
+struct SortedRow {
+    double val[BZ_MAX_F];
+    unsigned char idx[BZ_MAX_F];
+    int n;
+};
+__device__ void sort_row(const double* __restrict__ dist, int f, int a, SortedRow& row) {
+    for (int b = 0; b < f; ++b) row.val[b] = dist[a * f + b];
     int n = 0;
+    // in place: entries 0 .. n-1 are sorted, entry b is still raw (b >= n always holds)
     for (int b = 0; b < f; ++b) {
-        if (b == a || !active[b]) continue;
-        const double x = dist[a * f + b];
+        if (b == a) continue;
+        const double x = row.val[b];
         int pos = n++;
-        while (pos > 0 && buf[pos - 1] > x) {
-            buf[pos] = buf[pos - 1];
+        while (pos > 0 && row.val[pos - 1] > x) {
+            row.val[pos] = row.val[pos - 1];
+            row.idx[pos] = row.idx[pos - 1];
             --pos;
         }
-        buf[pos] = x;
+        row.val[pos] = x;
+        row.idx[pos] = static_cast<unsigned char>(b);
     }
+    row.n = n;
+}
+// Krum score inside the rows flagged in `active`: the nb smallest distances to the other active rows,
+// added in ascending order.
+__device__ double krum_score(const SortedRow& row, const unsigned char* active, int nb) {
     double s = 0.0;
-    for (int t = 0; t < nb; ++t) s += buf[t];
+    int taken = 0;
+    for (int t = 0; t < row.n && taken < nb; ++t)
+        if (active[row.idx[t]]) {
+            s += row.val[t];
+            ++taken;
+        }
     return s;
 }
 
@@ -44,7 +62,11 @@ __global__ void __launch_bounds__(BZ_MAX_F) krum_select_kernel(const double* __r
     const int a = threadIdx.x;
     if (a < f) active[a] = 1;
     __syncthreads();
-    if (a < f) score[a] = krum_score_row(dist, f, active, a, f - c - 2);
+    if (a < f) {
+        SortedRow row;
+        sort_row(dist, f, a, row);
+        score[a] = krum_score(row, active, f - c - 2);
+    }
     __syncthreads();
     if (a < f) {
         int rank = 0;
@@ -59,6 +81,9 @@ __global__ void __launch_bounds__(BZ_MAX_F) bulyan_select_kernel(const double* _
     __shared__ unsigned char active[BZ_MAX_F];
     const int a = threadIdx.x;
     if (a < f) active[a] = 1;
+    SortedRow row;
+    row.n = 0;
+    if (a < f) sort_row(dist, f, a, row);
     __syncthreads();
     const int theta = f - 2 * c;
     for (int t = 0; t < theta; ++t) {
@@ -66,7 +91,7 @@ __global__ void __launch_bounds__(BZ_MAX_F) bulyan_select_kernel(const double* _
         int nb = n - c - 2;
         if (nb < 1) nb = 1;
         if (nb > n - 1) nb = n - 1;
-        if (a < f && active[a]) score[a] = (n > 1) ? krum_score_row(dist, f, active, a, nb) : 0.0;
+        if (a < f && active[a]) score[a] = (n > 1) ? krum_score(row, active, nb) : 0.0;
         __syncthreads();
         bool win = false;
         if (a < f && active[a]) {

@@ -39,21 +39,21 @@ __global__ void __launch_bounds__(256)
 
 // The error estimate.  flag[0] = 1 asks for the binary32 kernel.
 template <int F>
-__global__ void __launch_bounds__(64)
+__global__ void __launch_bounds__(256)
     pairdist_i8_check_kernel(const double* __restrict__ dist, const int* __restrict__ info, int n_ctas, int64_t d, int force,
                              int* __restrict__ flag) {
     __shared__ int s_emax[F];
     __shared__ int s_bad;
     const int tid = threadIdx.x;
     if (tid == 0) s_bad = 0;
-    if (tid < F) {
-        int e = kELo;
-        for (int c = 0; c < n_ctas; ++c) e = max(e, info[c * kInfoStride + tid]);
-        s_emax[tid] = e;
+    if (tid < F) s_emax[tid] = kELo;
+    __syncthreads();
+    for (int e = tid; e < n_ctas * kInfoStride; e += blockDim.x) {
+        const int a = e % kInfoStride;
+        if (a < F) atomicMax(&s_emax[a], info[e]);
+        if (a == kInfoBad && info[e]) atomicOr(&s_bad, 1);
     }
     __syncthreads();
-    for (int c = tid; c < n_ctas; c += blockDim.x)
-        if (info[c * kInfoStride + kInfoBad]) atomicOr(&s_bad, 1);
     if (tid < F) {
         const int a = tid;
         const double step_a = __longlong_as_double(static_cast<long long>(1023 + s_emax[a] - 30) << 52);
@@ -111,7 +111,7 @@ int launch_i8(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, floa
     note_launch();
     st = check_launch();
     if (st != BZ_OK) return st;
-    pairdist_i8_check_kernel<F><<<1, 64, 0, s>>>(dist, info, static_cast<int>(ctas), d, force, flag);
+    pairdist_i8_check_kernel<F><<<1, 256, 0, s>>>(dist, info, static_cast<int>(ctas), d, force, flag);
     note_launch();
     return check_launch();
 }
