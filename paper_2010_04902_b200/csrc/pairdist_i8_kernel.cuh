@@ -16,7 +16,7 @@
 // are read back ("drained") only when some row's scale changes or 512 tiles have gone by (32-bit
 // headroom); a drain combines the blocks in binary64 and adds
 //     T[a][b] += 2^(E_a + E_b - 60) * sum_blocks weight * S_i S_j^T [a][b]
-// to the CTA's partial matrix.  A last kernel forms, per CTA and then over CTAs in a fixed order,
+// to the CTA's partial matrix (in shared memory, written out once).  A last kernel forms, per CTA and then over CTAs in a fixed order,
 //     D[a][b] = (T[a][a] + T[b][b]) - (T[a][b] + T[b][a]).
 // Identical rows give identical integers and therefore exactly equal distances and D = 0.
 //
@@ -73,7 +73,8 @@ template <int F, int W, int R, int FC, int NS, int TS> struct I8Shape {
     static constexpr int kBoxFloats = R * FC * kTK;
     static constexpr int kBoxBytes = kBoxFloats * 4;
     static constexpr int kThreads = (kConvWarp0 + W) * 32;
-    static constexpr int kSmem = 1024 + kSlots * kSlotBytes + NS * kBoxBytes + kCtlBytes;
+    static constexpr int kPartialBytes = (F * F * 8 + 15) / 16 * 16;   // the CTA's partial matrix T
+    static constexpr int kSmem = 1024 + kSlots * kSlotBytes + NS * kBoxBytes + kCtlBytes + kPartialBytes;
     static_assert(F <= 64, "at most 64 rows");
     static_assert(kChunks * FC == F, "FC must divide F");
     static_assert(kBoxBytes % 128 == 0, "TMA destinations are 128-byte aligned");
@@ -130,6 +131,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
     unsigned char* op = base;
     float* in = reinterpret_cast<float*>(base + NO * S::kSlotBytes);
     unsigned char* ctl = base + NO * S::kSlotBytes + NS * S::kBoxBytes;
+    double* tp_s = reinterpret_cast<double*>(ctl + kCtlBytes);
     uint64_t* op_full = reinterpret_cast<uint64_t*>(ctl);
     uint64_t* op_empty = op_full + NO;
     uint64_t* in_full = op_empty + NO;
@@ -173,7 +175,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
     if (tid < 64) e_cur[tid] = kENone;
     // rows f .. RP-1 of every slice stay zero for the whole run
     for (int e = tid; e < NO * S::kSlotBytes / 16; e += S::kThreads) reinterpret_cast<uint4*>(op)[e] = make_uint4(0, 0, 0, 0);
-    for (int e = tid; e < F * F; e += S::kThreads) tp[e] = 0.0;
+    for (int e = tid; e < F * F; e += S::kThreads) tp_s[e] = 0.0;
     fence_async_smem();
     if (warp == kMmaWarp) tmem_alloc(tmem_slot, S::kTmemCols);
     tc_fence_before_sync();
@@ -198,35 +200,45 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
             const int e_a = a < F ? e_row[a] : 0;
             for (int ph = 0; ph < SPM; ++ph) {
                 if (g == ph) {  // uniform over the warp
+                    constexpr int NBLK = (NMMA == 1) ? 4 : 6;  // blocks a lane meets: 4 - m*SPM over the MMAs
                     for (int b0 = 0; b0 < F; b0 += 8) {
+                        int32_t x[NBLK][8];
+                        {
+                            int q = 0;
+#pragma unroll
+                            for (int m = 0; m < NMMA; ++m)
+#pragma unroll
+                                for (int h = 0; h < 4 - m * SPM; ++h, ++q) tmem_ld8(lane_base + S::mma_col(m) + h * RP + b0, x[q]);
+                        }
+                        tmem_ld_wait();
                         double val[8];
 #pragma unroll
                         for (int c = 0; c < 8; ++c) val[c] = 0.0;
+                        {
+                            int q = 0;
 #pragma unroll
-                        for (int m = 0; m < NMMA; ++m) {
-                            const int si = m * SPM + g;
+                            for (int m = 0; m < NMMA; ++m)
 #pragma unroll
-                            for (int h = 0; h < 4 - m * SPM; ++h) {
-                                int32_t x[8];
-                                tmem_ld8(lane_base + S::mma_col(m) + h * RP + b0, x);
-                                tmem_ld_wait();
-                                const double w = block_weight<SPM>(si, m * SPM + h);
+                                for (int h = 0; h < 4 - m * SPM; ++h, ++q) {
+                                    const double w = block_weight<SPM>(m * SPM + g, m * SPM + h);
 #pragma unroll
-                                for (int c = 0; c < 8; ++c) val[c] += w * static_cast<double>(x[c]);
-                            }
+                                    for (int c = 0; c < 8; ++c) val[c] += w * static_cast<double>(x[q][c]);
+                                }
                         }
                         if (a < F) {
 #pragma unroll
                             for (int c = 0; c < 8; ++c)
                                 if (b0 + c < F) {
                                     const double sc = __longlong_as_double(static_cast<long long>(1023 + e_a + e_row[b0 + c] - 60) << 52);
-                                    tp[a * F + b0 + c] += val[c] * sc;
+                                    tp_s[a * F + b0 + c] += val[c] * sc;
                                 }
                         }
                     }
                 }
                 asm volatile("bar.sync 1, %0;" ::"n"(kDrainWarps * 32) : "memory");
             }
+            if (last)  // the barrier above has ordered the last additions
+                for (int e = tid; e < F * F; e += kDrainWarps * 32) tp[e] = tp_s[e];
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(drained);
@@ -443,8 +455,10 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                             const int need = static_cast<int>(__reduce_max_sync(0xffffffffu, m8) >> 23) - 126;  // |v| < 2^need
                             if (need > 60) unrepresentable = 1;  // infinities, NaNs, magnitudes beyond 2^60
                             if (E[i] == kENone || need > E[i]) {   // |v| * 2^(30 - E) may reach 2^30
+                                // two bits of headroom at first, four once a row has shown that it grows
+                                // (every change of scale costs a read-back of the accumulators)
                                 raise = raise || E[i] != kENone;
-                                E[i] = clamp_e(need + 2);
+                                E[i] = clamp_e(need + (E[i] == kENone ? 2 : 4));
                                 if (lane == 0) e_cur[c * FC + off + W * i] = E[i];
                             }
                             const float scale = __int_as_float((30 - E[i] + 127) << 23);
