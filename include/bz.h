@@ -145,10 +145,21 @@ int bz_vote_median_host(const float* replicas_host, int r, int f, int64_t d, flo
 /*
  * Squared Euclidean distances between all pairs of voted gradients, the O(f^2 d) part of the
  * Krum family (Sec. 1.2; cost in Appendix A.1): dist[a][b] = sum_j (v_a[j] - v_b[j])^2.
- * Differences and squares are formed in binary32, added in binary32 inside blocks of at most 1024
- * coordinates (as interleaved partial sums of at most 128 terms) and in binary64 across blocks, in
- * a fixed order (results are reproducible from run to run).
- *   dist  device, double [f][f], symmetric with a zero diagonal.
+ * Two kernels compute it; results are reproducible from run to run with either.
+ *   - Tensor cores (f = 25 or 49, d >= 8192, 16-byte aligned rows, ld a multiple of 4): every row
+ *     is converted to 31-bit fixed point on a power-of-two scale of its own, the Gram matrix of
+ *     the integers is formed exactly by 8-bit integer MMAs, and dist = |a|^2 + |b|^2 - 2ab is taken
+ *     in binary64.  The only error is the rounding of a value to a multiple of its row's step
+ *     2^(E-30), 2^E bounding the row's magnitudes.  The library estimates that error for every pair
+ *     and, where it exceeds 5e-9 relative, or where a row holds infinities, NaNs or magnitudes
+ *     beyond 2^60, recomputes with the second kernel (decided on the device; the call stays
+ *     asynchronous).
+ *   - Binary32 difference form (every other shape): differences and squares in binary32, added in
+ *     binary32 inside blocks of at most 1024 coordinates (interleaved partial sums of at most 128
+ *     terms) and in binary64 across blocks, in a fixed order.
+ * Environment: BZ_PAIRDIST_PATH=fp32 keeps every call on the second kernel; =i8 takes the first
+ * kernel's result whatever its estimate says (for testing it); read at every call.
+ *   dist  device, double [f][f], symmetric with a zero diagonal; identical rows give exactly 0.
  *   workspace  device, bz_workspace_bytes(BZ_OP_PAIRDIST, 0, f, d, 0, 0) bytes, 256-byte aligned.
  */
 int bz_pairdist(const float* voted, int f, int64_t d, int64_t ld, double* dist, void* workspace,
@@ -163,8 +174,9 @@ int bz_pairdist(const float* voted, int f, int64_t d, int64_t ld, double* dist, 
  * inputs and outputs only; the partial sums go to an array of BZ_STATIC_SCRATCH_BYTES that is part
  * of the library image, so every GPU that loads the library holds those 4 MiB until the process
  * exits.  The call itself allocates and frees nothing.
- *   - Results are those of bz_pairdist (same kernels, same summation order).
- *   - Shapes whose scratch need, bz_workspace_bytes(BZ_OP_PAIRDIST, 0, f, d, 0, 0), exceeds the
+ *   - Results are those of bz_pairdist's binary32 difference-form kernel (the only one this call
+ *     uses; same summation order).
+ *   - Shapes whose partial sums exceed the
  *     array are refused with BZ_ERR_STATIC_LIMIT before anything runs: f = 25 (0.9 MB) and f = 49
  *     (1.6 MB) fit, any other f fits up to 84; f from 85 to BZ_MAX_F is refused.
  *   - The first call on each device looks up the array's device address (the device must be
@@ -231,7 +243,9 @@ int bz_bulyan(const float* voted, int f, int64_t d, int64_t ld, int c, float* ou
  * bz_vote and bz_pairdist in one pass over the replicas: the winners of Eq. (3) are written to
  * `voted` and enter the distance sums of Sec. 1.2 from on-chip memory, so the voted rows are not
  * read back (4*f of the 4*(r*f + 2*f) bytes per coordinate the two calls move are saved).
- * voted is bit-identical to bz_vote's; dist is summed as in bz_pairdist.  Shapes without a fused
+ * voted is bit-identical to bz_vote's; dist is computed as in bz_pairdist (f = 49: the vote runs in
+ * front of the tensor-core kernel, with the same estimate and fall-back; f = 25: the vote runs in
+ * front of the binary32 kernel, the faster pass there).  Shapes without a fused
  * kernel (r*f outside {3,5}x{25,49} and 7x49, unaligned or short arrays) run the two calls.
  *   replicas, ld_file, ld_replica as bz_vote;  voted device [f][d] with ld_voted (written);
  *   dist device double [f][f];  workspace as bz_pairdist.
