@@ -123,3 +123,27 @@ def test_vote_and_distances_in_one_pass(l, r, q, attack, d, monkeypatch):
     assert np.array_equal(voted.cpu().numpy().view(np.uint32), v.numpy().view(np.uint32))
     _check_close(dist.cpu().numpy(), oracle.pairdist(v.numpy()))
     assert bz.pipeline_timeouts() == 0
+
+
+def test_full_size_on_sampled_rows():
+    # the benchmark's multi-Krum shape (r = 3, f = 49, d = 11.2 M) in the library's default configuration:
+    # the oracle computes the distances among a sample of rows from copies of the same bytes
+    l, r, q, d = 7, 3, 5, 11_200_000
+    wf, fw, _ = oracle.assign(l, r)
+    byz = oracle.worst_case(wf, l * l, r, q)[1]
+    g = inputs.true_gradients(l * l, d, seed=0, device=DEV)
+    rep = inputs.build_replicas(g, fw, byz, "alie")
+    del g
+    distorted = sorted({int(i) for i in range(l * l) if sum(int(w) in set(int(b) for b in byz) for w in fw[i]) >= 2})
+    rows = sorted(set([0, 1, 17, 30, 48] + distorted[:2]))
+    voted, dist = bz.vote_pairdist(rep)                      # vote in front of the integer kernel
+    alone = bz.pairdist(voted)                               # the integer kernel on given rows
+    torch.cuda.synchronize()
+    sample = voted[rows].cpu().numpy()
+    assert np.array_equal(sample.view(np.uint32), oracle.vote(rep[:, rows].cpu().numpy()).view(np.uint32))
+    want = oracle.pairdist(sample)
+    for got in (dist, alone):
+        sub = got.cpu().numpy()[np.ix_(rows, rows)]
+        _check_close(sub, want)
+    assert np.array_equal(dist.cpu().numpy(), alone.cpu().numpy())   # same integers either way
+    assert bz.pipeline_timeouts() == 0
