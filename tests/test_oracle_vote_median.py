@@ -199,3 +199,57 @@ def test_inputs_are_seeded():
     dev = (h - h.median(dim=0).values).abs().max(dim=0).values
     frac_wide = float((dev > 0.6).float().mean())   # 6 sigma: only heavy-tailed coordinates get there
     assert 0.002 < frac_wide < 0.012
+
+
+# ---- Eq. (3) on whole vectors (the paper's own statement of the vote) --------------------------------
+
+def test_vectorwise_vote_hand_cases():
+    # file 0: copies (A, B, A) -> A wins, first at k = 0;  file 1: (A, B, B) -> k = 1;
+    # file 2: three different vectors -> every count is 1, the earliest copy wins
+    A = np.array([1.0, 2.0, 3.0, 4.0], np.float32)
+    B = np.array([1.0, 2.0, 3.0, 4.5], np.float32)   # differs from A in the last coordinate only
+    C = np.array([9.0, 2.0, 3.0, 4.0], np.float32)   # differs in the first coordinate only
+    rep = np.stack([np.stack([A, A, A]), np.stack([B, B, B]), np.stack([A, B, C])])   # [k][file]
+    assert oracle.vote_vectorwise(rep).tolist() == [0, 1, 0]
+    # r = 5: (A, B, B, A, C) is a 2-2 tie -> the vector seen first (k = 0); (C, B, B, A, B) -> B at k = 1
+    rep5 = np.stack([np.stack([A, C]), np.stack([B, B]), np.stack([B, B]), np.stack([A, A]), np.stack([C, B])])
+    assert oracle.vote_vectorwise(rep5).tolist() == [0, 1]
+    # equality is on bit patterns: +0 and -0 are different vectors, a NaN equals itself
+    Z = np.array([0.0, 1.0], np.float32)
+    N = np.array([-0.0, 1.0], np.float32)
+    Q = np.array([np.nan, 1.0], np.float32)
+    rep3 = np.stack([np.stack([Z, Q]), np.stack([N, Q]), np.stack([N, Z])])
+    assert oracle.vote_vectorwise(rep3).tolist() == [1, 0]
+
+
+def test_vectorwise_vote_against_counter():
+    # brute force: the most common byte string among a file's copies, ties to the one seen first
+    from collections import Counter
+    rng = np.random.default_rng(11)
+    for r, f, d in [(3, 6, 5), (5, 9, 3), (7, 4, 2)]:
+        pool = rng.integers(-2, 3, size=(3, d)).astype(np.float32)    # few distinct vectors -> many agreements
+        pick = rng.integers(0, 3, size=(r, f))
+        rep = pool[pick]
+        win = oracle.vote_vectorwise(rep)
+        for i in range(f):
+            keys = [rep[k, i].tobytes() for k in range(r)]
+            cnt = Counter(keys)
+            best = max(cnt.values())
+            first = next(k for k in range(r) if cnt[keys[k]] == best)
+            assert win[i] == first
+
+
+def test_vectorwise_and_elementwise_votes_differ_only_without_an_agreeing_majority():
+    # A file with honest copies in the minority and Byzantine copies that disagree among themselves:
+    # element by element the honest value can still win coordinates where two attackers happen to
+    # agree with it, while no whole vector has a majority (the case Sec. 2 leaves open).
+    g = np.array([[1.0, 2.0, 3.0]], np.float32)
+    b1 = np.array([[1.0, 7.0, 8.0]], np.float32)
+    b2 = np.array([[5.0, 2.0, 9.0]], np.float32)
+    rep = np.stack([b1, b2, g])                      # k = 0, 1 Byzantine, k = 2 honest
+    assert oracle.vote_vectorwise(rep).tolist() == [0]           # all counts 1: first copy
+    assert oracle.vote(rep)[0].tolist() == [1.0, 2.0, 8.0]       # per coordinate: 1 (b1, g), 2 (b2, g), tie -> first
+    # with a true majority both rules return the honest vector
+    rep = np.stack([g, b2, g])
+    assert oracle.vote_vectorwise(rep).tolist() == [0]
+    assert np.array_equal(oracle.vote(rep)[0], g[0])
