@@ -300,6 +300,8 @@ def extra_paths(bz, inputs, torch, device):
     ws = bz.alloc_workspace(bz.OP_MULTIKRUM, 0, f, d, 5, 44, device=device)
     sel44 = torch.arange(44, dtype=torch.int32, device=device)
     t_vote = timed(torch, lambda: bz.vote(rep, voted), 5, 2)
+    ws_vw = bz.alloc_workspace(bz.OP_VOTE_VECTORWISE, r, f, d, device=device)
+    t_vw = timed(torch, lambda: bz.vote_vectorwise(rep, voted, ws_vw), 5, 2)
     t_pd = timed(torch, lambda: bz.pairdist(voted, ws), 5, 2)
     t_pd32 = timed_fp32(lambda: bz.pairdist(voted, ws))
     t_mean = timed(torch, lambda: bz.mean_rows(voted, sel44, out), 5, 2)
@@ -317,6 +319,7 @@ def extra_paths(bz, inputs, torch, device):
         pairdist=dict(kernel="integer MMA (tcgen05 kind::i8)", **hbm(4 * f * d, t_pd)),
         vote=hbm((4 * r * f + 4 * f) * d, t_vote), mean_rows=hbm((4 * 44 + 4) * d, t_mean),
         pipeline=hbm(bytes_pipeline, t_vote + t_mk),
+        vote_vectorwise=dict(ms=t_vw, **hbm((4 * r * f + 8 * f) * d, t_vw)),
         single_pass=dict(ms_vote_pairdist=t_vpd, ms_vote_pairdist_fp32=t_vpd32, vote_pairdist=hbm((4 * r * f + 4 * f) * d, t_vpd),
                          ms_vote_multikrum=t_vmk, coordinates_per_s=d / (t_vmk * 1e-3),
                          **hbm((4 * r * f + 4 * f + 4 * 44 + 4) * d, t_vmk)))
@@ -433,6 +436,7 @@ def profile_op(args):
         fn = {
             "vote_median": lambda: bz.vote_median(rep, out),
             "vote": lambda: bz.vote(rep, voted),
+            "vote_vectorwise": lambda: bz.vote_vectorwise(rep, voted),
             "median": lambda: bz.median(voted, out),
             "pairdist": lambda: bz.pairdist(voted, ws),
             "vote_pairdist": lambda: bz.vote_pairdist(rep, voted, ws),
@@ -498,7 +502,7 @@ def main():
     ap.add_argument("--coords", type=int, default=0, help="profiling only: override the number of coordinates d")
     ap.add_argument("--no-e2e", action="store_true", help="profiling only: skip the host-buffer leg")
     ap.add_argument("--no-cpu", action="store_true", help="profiling only: skip the CPU baseline / parity leg")
-    ap.add_argument("--op", default="", help="profiling only: run a single entry point (vote_median, vote, median, "
+    ap.add_argument("--op", default="", help="profiling only: run a single entry point (vote_median, vote, vote_vectorwise, median, "
                     "pairdist, vote_pairdist, vote_median_update, multikrum, bulyan, mean_rows, trimmed_mean, worst_case, "
                     "worst_case_mols) instead of the benchmark")
     ap.add_argument("--shape", default="5,3,3", help="profiling only: l,r,q of the cluster for --op")

@@ -57,6 +57,7 @@ extern "C" {
 #define BZ_OP_WORST_CASE 4
 #define BZ_OP_VOTE_MEDIAN_HOST 5
 #define BZ_OP_WORST_CASE_MOLS 6
+#define BZ_OP_VOTE_VECTORWISE 7
 
 /*
  * Task assignment (Algorithm 2; Sec. 4.1.1 for the squares L_alpha(i,j) = alpha*i + j over F_l).
@@ -131,6 +132,21 @@ int bz_vote_median_update(const float* replicas, int r, int f, int64_t d, int64_
  * outputs).  g must not overlap w or velocity.
  */
 int bz_model_update(const float* g, int64_t d, float* w, float* velocity, float eta, float mu, void* stream);
+
+/*
+ * Eq. (3) as the paper states it (Sec. 2, "Training Protocol"): the vote on WHOLE gradients.  For
+ * every file the copy whose complete vector (exact match on bit patterns) occurs most often among
+ * the file's r copies wins; among equally frequent vectors the one whose first copy has the lowest
+ * k.  bz_vote applies the same rule coordinate by coordinate; the two give the same rows whenever
+ * a majority of a file's copies is identical (always, with at most r' - 1 Byzantine holders, and
+ * whenever the attackers collude).  They differ only when no vector has a majority.
+ *   replicas, ld_file, ld_replica as bz_vote.
+ *   voted   device [f][d] with ld_voted: the winning copies (may be NULL if only `winner` is wanted).
+ *   winner  device int32 [f]: index k of the winning copy of each file (may be NULL).
+ *   workspace device, bz_workspace_bytes(BZ_OP_VOTE_VECTORWISE, r, f, d, 0, 0) bytes, 256-byte aligned.
+ */
+int bz_vote_vectorwise(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica, float* voted,
+                       int64_t ld_voted, int32_t* winner, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * The same aggregation for a caller whose gradients sit in HOST memory (ideally page-locked):

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG, "libbz.so")
 
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_PRECONDITION, ERR_WORKSPACE, ERR_BUDGET, ERR_CUDA = -1, -2, -3, -4, -5, -6
-OP_PAIRDIST, OP_MULTIKRUM, OP_BULYAN, OP_WORST_CASE, OP_VOTE_MEDIAN_HOST, OP_WORST_CASE_MOLS = 1, 2, 3, 4, 5, 6
+OP_PAIRDIST, OP_MULTIKRUM, OP_BULYAN, OP_WORST_CASE, OP_VOTE_MEDIAN_HOST, OP_WORST_CASE_MOLS, OP_VOTE_VECTORWISE = 1, 2, 3, 4, 5, 6, 7
 MAX_R, MAX_F = 15, 128
 
 
@@ -39,6 +39,7 @@ _SIGNATURES = {
     "bz_assign_mols": (_c_int, [_c_int, _c_int, _c_vp, _c_vp, _c_vp]),
     "bz_assign_ramanujan": (_c_int, [_c_int, _c_int, _c_vp, _c_vp, _c_vp]),
     "bz_vote": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_i64, _c_vp]),
+    "bz_vote_vectorwise": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_i64, _c_vp, _c_vp, _c_sz, _c_vp]),
     "bz_median": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_vp]),
     "bz_vote_median": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_vp]),
     "bz_vote_median_host": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_vp, _c_vp, _c_sz, _c_vp]),
@@ -223,6 +224,23 @@ def vote(replicas: torch.Tensor, voted: torch.Tensor | None = None) -> torch.Ten
                        _dev(voted, torch.float32, "voted"), ld_v, _stream())
     _check(st, "bz_vote")
     return voted
+
+
+def vote_vectorwise(replicas: torch.Tensor, voted: torch.Tensor | None = None, workspace: torch.Tensor | None = None):
+    """bz_vote_vectorwise: the vote of Eq. (3) on whole gradients.  Returns (voted[f][d], winner[f])."""
+    r, f, d, ld_file, ld_rep = _replicas(replicas)
+    if voted is None:
+        voted = torch.empty((f, d), dtype=torch.float32, device=replicas.device)
+    vf, vd, ld_v = _rows(voted, "voted")
+    if (vf, vd) != (f, d):
+        raise ValueError("voted must be [%d][%d]" % (f, d))
+    ws = workspace if workspace is not None else alloc_workspace(OP_VOTE_VECTORWISE, r, f, d, device=replicas.device)
+    winner = torch.empty(f, dtype=torch.int32, device=replicas.device)
+    st = lib().bz_vote_vectorwise(_dev(replicas, torch.float32, "replicas"), r, f, d, ld_file, ld_rep,
+                                  _dev(voted, torch.float32, "voted"), ld_v, winner.data_ptr(), ws.data_ptr(), ws.numel(),
+                                  _stream())
+    _check(st, "bz_vote_vectorwise")
+    return voted, winner
 
 
 def median(voted: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:

@@ -11,6 +11,7 @@ namespace bz {
 size_t krum_workspace_bytes(int op, int f);   // krum.cu
 size_t worst_case_workspace_bytes();          // worst_case.cu
 size_t worst_case_mols_workspace_bytes(int l, int r);  // worst_case_mols.cu
+size_t vote_vectorwise_workspace(int f);      // vote_vectorwise.cu
 int pipeline_timeouts(unsigned int* count);   // vote_median_tma.cu
 int vote_pairdist_timeouts(unsigned int* count);  // vote_pairdist.cu
 int pairdist_i8_timeouts(unsigned int* count);    // pairdist_i8.cu
@@ -107,6 +108,7 @@ extern "C" size_t bz_workspace_bytes(int op, int r, int f, int64_t d, int c, int
         case BZ_OP_MULTIKRUM:
         case BZ_OP_BULYAN: return krum_workspace_bytes(op, f);
         case BZ_OP_WORST_CASE: return worst_case_workspace_bytes();
+        case BZ_OP_VOTE_VECTORWISE: return vote_vectorwise_workspace(f);
         case BZ_OP_WORST_CASE_MOLS: {
             int l = 2;
             while (l * l < f) ++l;

@@ -1,0 +1,173 @@
+// Eq. (3) as the paper states it (Sec. 2, "Training Protocol"): per file, the WHOLE gradient that
+// most of its r copies agree on, exact match on bit patterns; among equally frequent gradients the
+// one whose first copy has the lowest index.  (bz_vote applies the same rule coordinate by
+// coordinate; the two agree whenever a majority of a file's copies is identical.)
+//
+// Three kernels: (1) one streaming pass over the replicas that ORs, per file, a bit for every pair
+// of copies that differ anywhere; (2) a tiny kernel that turns the pair bits into the winner's index;
+// (3) a gather of the winning copies into `voted`.  Bytes per coordinate: 4rf read, then 4f read and
+// 4f written: bound by HBM.
+#include "bz_common.cuh"
+
+namespace bz {
+
+namespace {
+
+constexpr int kMaxPairs = BZ_MAX_R * (BZ_MAX_R - 1) / 2;   // 105: two 64-bit words per file
+constexpr int kMaskWords = 2;
+
+__device__ __forceinline__ bool differ(const uint4& a, const uint4& b) { return ((a.x ^ b.x) | (a.y ^ b.y) | (a.z ^ b.z) | (a.w ^ b.w)) != 0; }
+__device__ __forceinline__ bool differ(uint32_t a, uint32_t b) { return a != b; }
+
+// pair (k, k2), k < k2, -> bit index, row-major over the strict upper triangle
+__host__ __device__ __forceinline__ int pair_index(int r, int k, int k2) { return k * r - k * (k + 1) / 2 + (k2 - k - 1); }
+
+// grid = (chunks, f).  V = uint4: n counts groups of 4 coordinates and leading dimensions are in groups.
+template <int R, typename V>
+__global__ void __launch_bounds__(256) copies_differ_kernel(const V* __restrict__ rep, int64_t n, int64_t ld_file, int64_t ld_rep,
+                                                            unsigned long long* __restrict__ mask) {
+    const int file = blockIdx.y;
+    const V* base = rep + file * ld_file;
+    uint32_t bits = 0;  // R <= 7: 21 pairs
+    for (int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < n; j += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        V c[R];
+#pragma unroll
+        for (int k = 0; k < R; ++k) c[k] = ld_stream(base + k * ld_rep + j);
+        int p = 0;
+#pragma unroll
+        for (int k = 0; k < R; ++k)
+#pragma unroll
+            for (int k2 = k + 1; k2 < R; ++k2, ++p) bits |= differ(c[k], c[k2]) ? (1u << p) : 0u;
+    }
+    bits = __reduce_or_sync(0xffffffffu, bits);
+    if ((threadIdx.x & 31) == 0 && bits != 0) atomicOr(&mask[file * kMaskWords], static_cast<unsigned long long>(bits));
+}
+
+// any odd r <= BZ_MAX_R, any alignment
+__global__ void __launch_bounds__(256) copies_differ_generic_kernel(const uint32_t* __restrict__ rep, int r, int64_t d, int64_t ld_file,
+                                                                    int64_t ld_rep, unsigned long long* __restrict__ mask) {
+    const int file = blockIdx.y;
+    const uint32_t* base = rep + file * ld_file;
+    unsigned long long lo = 0, hi = 0;
+    for (int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < d; j += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        uint32_t c[BZ_MAX_R];
+        for (int k = 0; k < r; ++k) c[k] = base[k * ld_rep + j];
+        int p = 0;
+        for (int k = 0; k < r; ++k)
+            for (int k2 = k + 1; k2 < r; ++k2, ++p)
+                if (c[k] != c[k2]) {
+                    if (p < 64) lo |= 1ull << p;
+                    else hi |= 1ull << (p - 64);
+                }
+    }
+    if (lo) atomicOr(&mask[file * kMaskWords], lo);
+    if (hi) atomicOr(&mask[file * kMaskWords + 1], hi);
+}
+
+// thread i: winner of file i from its pair bits
+__global__ void __launch_bounds__(BZ_MAX_F) winner_kernel(const unsigned long long* __restrict__ mask, int r, int f,
+                                                          int32_t* __restrict__ winner) {
+    const int i = threadIdx.x;
+    if (i >= f) return;
+    const unsigned long long lo = mask[i * kMaskWords], hi = mask[i * kMaskWords + 1];
+    auto same = [&](int k, int k2) {
+        if (k == k2) return true;
+        const int p = k < k2 ? pair_index(r, k, k2) : pair_index(r, k2, k);
+        return ((p < 64 ? lo >> p : hi >> (p - 64)) & 1ull) == 0;
+    };
+    int best = 0, best_count = 0;
+    for (int k = 0; k < r; ++k) {
+        int count = 0;
+        for (int k2 = 0; k2 < r; ++k2) count += same(k, k2) ? 1 : 0;
+        if (count > best_count) {
+            best_count = count;
+            best = k;
+        }
+    }
+    winner[i] = best;
+}
+
+template <typename V>
+__global__ void __launch_bounds__(256) gather_winners_kernel(const V* __restrict__ rep, int64_t n, int64_t ld_file, int64_t ld_rep,
+                                                             const int32_t* __restrict__ winner, V* __restrict__ voted, int64_t ld_voted) {
+    const int file = blockIdx.y;
+    const V* src = rep + winner[file] * ld_rep + file * ld_file;
+    V* dst = voted + file * ld_voted;
+    for (int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < n; j += static_cast<int64_t>(gridDim.x) * blockDim.x)
+        dst[j] = ld_stream(src + j);
+}
+
+int chunks_for(int64_t n, int f) {
+    // enough CTAs to fill the SMs a few times over, never more than the work
+    int64_t per_file = (static_cast<int64_t>(kNumSMs) * 8 + f - 1) / f;
+    const int64_t most = (n + 255) / 256;
+    if (per_file > most) per_file = most;
+    if (per_file < 1) per_file = 1;
+    return static_cast<int>(per_file);
+}
+
+template <int R>
+int launch_differ_vec(const float* rep, int f, int64_t d, int64_t ld_file, int64_t ld_rep, unsigned long long* mask, cudaStream_t s) {
+    const int64_t n = d / 4;
+    const dim3 grid(chunks_for(n, f), f);
+    copies_differ_kernel<R, uint4><<<grid, 256, 0, s>>>(reinterpret_cast<const uint4*>(rep), n, ld_file / 4, ld_rep / 4, mask);
+    note_launch();
+    return check_launch();
+}
+
+}  // namespace
+
+size_t vote_vectorwise_workspace(int f) { return round_up(static_cast<size_t>(f) * (kMaskWords * 8 + 4), 256); }
+
+}  // namespace bz
+
+using namespace bz;
+
+extern "C" int bz_vote_vectorwise(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica, float* voted,
+                                  int64_t ld_voted, int32_t* winner, void* workspace, size_t workspace_bytes, void* stream) {
+    // the argument rules of bz_vote
+    if (d < 0 || r < 1 || f < 1 || (r % 2) == 0) return BZ_ERR_INVALID_ARG;
+    if (replicas == nullptr && d > 0) return BZ_ERR_INVALID_ARG;
+    if (r > BZ_MAX_R || f > BZ_MAX_F) return BZ_ERR_UNSUPPORTED;
+    if (ld_file < d || (r > 1 && ld_replica < d)) return BZ_ERR_INVALID_ARG;
+    int st = BZ_OK;
+    if (voted == nullptr && winner == nullptr) return BZ_ERR_INVALID_ARG;
+    if (voted != nullptr && ld_voted < d) return BZ_ERR_INVALID_ARG;
+    if (workspace == nullptr || !aligned256(workspace) || workspace_bytes < vote_vectorwise_workspace(f)) return BZ_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned long long* mask = static_cast<unsigned long long*>(workspace);
+    int32_t* win = winner != nullptr ? winner : reinterpret_cast<int32_t*>(mask + static_cast<size_t>(f) * kMaskWords);
+    cudaError_t e = cudaMemsetAsync(mask, 0, static_cast<size_t>(f) * kMaskWords * 8, s);  // every call starts from "all copies agree"
+    if (e != cudaSuccess) return cuda_failed(e);
+    if (d > 0 && r > 1) {
+        const bool vec = aligned16(replicas) && (ld_file % 4 == 0) && (ld_replica % 4 == 0) && (d % 4 == 0) && (r == 3 || r == 5 || r == 7);
+        if (vec) {
+            st = r == 3 ? launch_differ_vec<3>(replicas, f, d, ld_file, ld_replica, mask, s)
+                        : (r == 5 ? launch_differ_vec<5>(replicas, f, d, ld_file, ld_replica, mask, s)
+                                  : launch_differ_vec<7>(replicas, f, d, ld_file, ld_replica, mask, s));
+        } else {
+            const dim3 grid(chunks_for(d, f), f);
+            copies_differ_generic_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const uint32_t*>(replicas), r, d, ld_file, ld_replica, mask);
+            note_launch();
+            st = check_launch();
+        }
+        if (st != BZ_OK) return st;
+    }
+    winner_kernel<<<1, BZ_MAX_F, 0, s>>>(mask, r, f, win);
+    note_launch();
+    st = check_launch();
+    if (st != BZ_OK || voted == nullptr || d == 0) return st;
+    const bool vec = aligned16(replicas) && aligned16(voted) && (ld_file % 4 == 0) && (ld_voted % 4 == 0) && (d % 4 == 0) &&
+                     (r == 1 || ld_replica % 4 == 0);
+    if (vec) {
+        const dim3 grid(chunks_for(d / 4, f), f);
+        gather_winners_kernel<uint4><<<grid, 256, 0, s>>>(reinterpret_cast<const uint4*>(replicas), d / 4, ld_file / 4, ld_replica / 4, win,
+                                                          reinterpret_cast<uint4*>(voted), ld_voted / 4);
+    } else {
+        const dim3 grid(chunks_for(d, f), f);
+        gather_winners_kernel<uint32_t><<<grid, 256, 0, s>>>(reinterpret_cast<const uint32_t*>(replicas), d, ld_file, ld_replica, win,
+                                                             reinterpret_cast<uint32_t*>(voted), ld_voted);
+    }
+    note_launch();
+    return check_launch();
+}

@@ -81,6 +81,7 @@ def test_workspace_sizes(lib):
         bu = bz.workspace_bytes(bz.OP_BULYAN, 0, f, 1000, 1)
         assert pd > 0 and pd % 256 == 0 and mk >= pd + f * f * 8 and bu == mk
     assert bz.workspace_bytes(bz.OP_WORST_CASE, 3, 25) > 0
+    assert bz.workspace_bytes(bz.OP_VOTE_VECTORWISE, 3, 25, 1000) >= 25 * 20
     small = bz.workspace_bytes(bz.OP_VOTE_MEDIAN_HOST, 3, 25, 1000)
     big = bz.workspace_bytes(bz.OP_VOTE_MEDIAN_HOST, 3, 25, 10 ** 7)
     assert 76 * 1000 * 4 <= small <= big <= 76 * 65536 * 4 + 256
@@ -104,6 +105,16 @@ def test_validation_runs_before_any_launch(lib):
     assert L.bz_vote(fake, 3, 25, 10, 10, 250, None, 10, None) == bz.ERR_INVALID_ARG
     assert L.bz_vote(fake, 3, 25, 10, 10, 250, fake, 9, None) == bz.ERR_INVALID_ARG
     assert L.bz_vote(fake, 3, 25, 0, 0, 0, fake, 0, None) == bz.OK
+    # whole-vector vote: bz_vote's rules, then its outputs and workspace
+    assert L.bz_vote_vectorwise(None, 3, 25, 10, 10, 250, fake, 10, fake, fake, 1 << 20, None) == bz.ERR_INVALID_ARG
+    assert L.bz_vote_vectorwise(fake, 4, 25, 10, 10, 250, fake, 10, fake, fake, 1 << 20, None) == bz.ERR_INVALID_ARG
+    assert L.bz_vote_vectorwise(fake, 17, 25, 10, 10, 250, fake, 10, fake, fake, 1 << 20, None) == bz.ERR_UNSUPPORTED
+    assert L.bz_vote_vectorwise(fake, 3, 25, 10, 10, 5, fake, 10, fake, fake, 1 << 20, None) == bz.ERR_INVALID_ARG
+    assert L.bz_vote_vectorwise(fake, 3, 25, 10, 10, 250, None, 10, None, fake, 1 << 20, None) == bz.ERR_INVALID_ARG   # no output
+    assert L.bz_vote_vectorwise(fake, 3, 25, 10, 10, 250, fake, 9, fake, fake, 1 << 20, None) == bz.ERR_INVALID_ARG    # ld_voted < d
+    assert L.bz_vote_vectorwise(fake, 3, 25, 10, 10, 250, fake, 10, fake, None, 1 << 20, None) == bz.ERR_WORKSPACE
+    assert L.bz_vote_vectorwise(fake, 3, 25, 10, 10, 250, fake, 10, fake, fake, 16, None) == bz.ERR_WORKSPACE
+    assert L.bz_vote_vectorwise(fake, 3, 25, 10, 10, 250, fake, 10, fake, ctypes.c_void_p(264), 1 << 20, None) == bz.ERR_WORKSPACE
     assert L.bz_median(None, 25, 10, 10, fake, None) == bz.ERR_INVALID_ARG
     assert L.bz_median(fake, 0, 10, 10, fake, None) == bz.ERR_INVALID_ARG
     assert L.bz_median(fake, 25, 0, 0, fake, None) == bz.OK

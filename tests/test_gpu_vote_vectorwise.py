@@ -1,0 +1,119 @@
+"""GPU parity of the whole-vector vote (Eq. 3 as stated in Sec. 2) against the CPU oracle: winners and
+voted rows bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2010_04902_b200 import binding as bz
+from paper_2010_04902_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda"
+
+
+def _bits(a):
+    if isinstance(a, torch.Tensor):
+        a = a.detach().cpu().numpy()
+    return np.ascontiguousarray(a, np.float32).view(np.uint32)
+
+
+def _check(rep):
+    want_win = oracle.vote_vectorwise(rep.numpy())
+    voted, win = bz.vote_vectorwise(rep.to(DEV))
+    assert win.cpu().tolist() == want_win.tolist()
+    want = np.stack([rep.numpy()[want_win[i], i] for i in range(rep.shape[1])])
+    assert np.array_equal(_bits(voted), _bits(want))
+    return voted, win
+
+
+@pytest.mark.parametrize("l,r,q,attack,d", [(5, 3, 3, "reversed", 40_000), (7, 3, 5, "alie", 30_001), (5, 5, 6, "constant", 20_002),
+                                            (7, 5, 5, "independent", 10_003), (7, 7, 4, "reversed", 8_000), (3, 3, 2, "alie", 7)])
+def test_clusters(l, r, q, attack, d):
+    wf, fw, _ = oracle.assign(l, r)
+    byz = oracle.worst_case(wf, l * l, r, q)[1]
+    g = inputs.true_gradients(l * l, d, seed=l + r)
+    rep = inputs.build_replicas(g, fw, byz, attack)
+    voted, _ = _check(rep)
+    if attack != "independent":
+        # colluding attackers: the paper's whole-vector vote and the element-wise vote give the same rows
+        assert np.array_equal(_bits(voted), _bits(bz.vote(rep.to(DEV))))
+
+
+def test_copies_that_differ_in_one_coordinate():
+    # the difference sits in the first, a middle or the very last coordinate (tail of an odd length)
+    rng = np.random.default_rng(0)
+    r, f, d = 5, 6, 100_003
+    g = rng.standard_normal((f, d)).astype(np.float32)
+    rep = np.repeat(g[None], r, axis=0).copy()
+    rep[0, 0, 0] += 1.0                    # file 0: copy 0 alone differs -> copies 1..4 agree, winner k = 1
+    rep[1, 1, d // 2] += 1.0               # file 1: copy 1 alone
+    rep[4, 2, d - 1] += 1.0                # file 2: copy 4 alone, last coordinate
+    rep[0, 3, 5] = 7.0
+    rep[1, 3, 5] = 7.0                     # file 3: copies (0, 1) agree, (2, 3, 4) agree -> k = 2
+    rep[0, 4, 9] = 1.0
+    rep[1, 4, 9] = 2.0
+    rep[2, 4, 9] = 3.0
+    rep[3, 4, 9] = 4.0                     # file 4: all five differ -> k = 0
+    rep[:, 5, 77] = np.float32(-0.0)
+    rep[2, 5, 77] = np.float32(0.0)        # file 5: +0 against four -0: bit patterns differ
+    _, win = _check(torch.from_numpy(rep))
+    assert win.cpu().tolist() == [1, 0, 0, 2, 0, 0]
+
+
+def test_other_r_and_layouts():
+    rng = np.random.default_rng(5)
+    # r = 9 and r = 11: the generic kernel (more than 32 pairs of copies)
+    for r, f, d in [(9, 4, 5_000), (11, 3, 2_001), (1, 5, 300)]:
+        pool = rng.standard_normal((3, f, d)).astype(np.float32)
+        pick = rng.integers(0, 3, size=(r, f))
+        rep = np.stack([np.stack([pool[pick[k, i], i] for i in range(f)]) for k in range(r)])
+        _check(torch.from_numpy(rep))
+    # padded rows and an unaligned start (leading dimensions not multiples of 4)
+    g = torch.from_numpy(rng.standard_normal((25, 1001)).astype(np.float32))
+    rep = g[None].repeat(3, 1, 1).clone()
+    rep[2, 7] = -rep[2, 7]
+    rep[0, 8] = 0.5
+    rep[1, 8] = 0.5
+    big = torch.zeros((3, 25, 1007), dtype=torch.float32, device=DEV)
+    big[:, :, 3:1004] = rep.to(DEV)
+    voted, win = bz.vote_vectorwise(big[:, :, 3:1004])
+    want_win = oracle.vote_vectorwise(rep.numpy())
+    assert win.cpu().tolist() == want_win.tolist()
+    assert np.array_equal(_bits(voted), _bits(np.stack([rep.numpy()[want_win[i], i] for i in range(25)])))
+
+
+def test_two_calls_share_the_workspace():
+    # the pair bits of one call must not leak into the next
+    g = inputs.true_gradients(25, 4096, seed=1)
+    rep_a = g[None].repeat(3, 1, 1).clone()
+    rep_a[0] += 1.0                                   # copy 0 differs everywhere -> winners k = 1
+    rep_b = g[None].repeat(3, 1, 1).clone()           # all agree -> winners k = 0
+    ws = bz.alloc_workspace(bz.OP_VOTE_VECTORWISE, 3, 25, 4096)
+    _, win_a = bz.vote_vectorwise(rep_a.to(DEV), workspace=ws)
+    _, win_b = bz.vote_vectorwise(rep_b.to(DEV), workspace=ws)
+    assert win_a.cpu().tolist() == [1] * 25 and win_b.cpu().tolist() == [0] * 25
+
+
+def test_full_size_cluster():
+    # K = 15, r = 3, f = 25, d = 11.2 M on the device; the oracle checks the winners from the worker
+    # placement (a file's winner is its first honest copy when at most one holder is Byzantine, else
+    # the first Byzantine copy: colluders send one vector) and sampled columns of the voted rows
+    l, r, q, d = 5, 3, 3, 11_200_000
+    wf, fw, _ = oracle.assign(l, r)
+    byz = set(int(u) for u in oracle.worst_case(wf, l * l, r, q)[1])
+    g = inputs.true_gradients(l * l, d, seed=0, device=DEV)
+    rep = inputs.build_replicas(g, fw, sorted(byz), "reversed")
+    voted, win = bz.vote_vectorwise(rep)
+    torch.cuda.synchronize()
+    want_win = []
+    for i in range(l * l):
+        bad = [int(fw[i][k]) in byz for k in range(r)]
+        want_win.append(bad.index(True) if sum(bad) >= 2 else bad.index(False))
+    assert win.cpu().tolist() == want_win
+    idx = torch.from_numpy(np.unique(np.concatenate([np.arange(0, 64), np.arange(d - 64, d),
+                                                     np.random.default_rng(2).integers(0, d, 5000)]))).to(DEV)
+    sample = rep[:, :, idx].cpu().numpy()
+    assert oracle.vote_vectorwise(sample).tolist() == want_win      # the sample separates the copies as well
+    assert np.array_equal(_bits(voted[:, idx]), _bits(np.stack([sample[want_win[i], i] for i in range(l * l)])))
