@@ -56,6 +56,16 @@ def assign(l: int, r: int):
     return wf, fw, (mask if f <= 64 else None)
 
 
+def field_tables(l: int):
+    """Addition and multiplication tables [l][l] of the finite field with l = p^k elements."""
+    lib = _load()
+    add = np.zeros((l, l), np.int32)
+    mul = np.zeros((l, l), np.int32)
+    if lib.orc_field_tables(ctypes.c_int(l), _p(add, _i32p), _p(mul, _i32p)) != 0:
+        raise ValueError("no field with %d elements" % l)
+    return add, mul
+
+
 def ramanujan_dims(m: int, s: int):
     """(K, f, l, r) of Eq. (7)."""
     return (m * s, s * s, s, m) if m < s else (s * s, m * s, m, s)

@@ -14,7 +14,7 @@
 // the paper, closed forms, brute force on tiny inputs or reductions to library routines, except
 // where a header comment says "parity unpinned".
 //
-//   orc_assign            Algorithm 2 (MOLS placement) + Sec. 4.2.1 (Ramanujan Case 2, m = s = l)
+//   orc_assign            Algorithm 2 (MOLS placement; prime and prime-power l, Sec. 4.1.1) + Sec. 4.2.1 (Ramanujan Case 2, m = s = l)
 //   orc_assign_ramanujan  Sec. 4.2.1 Steps 1-3 and Eq. (7): the array-code matrix B, H = B or B^T
 //   orc_vote              Eq. (3): per-file majority over the r returned copies
 //   orc_vote_vectorwise   Eq. (3) read on whole vectors (Sec. 2, "Training Protocol")
@@ -54,6 +54,87 @@ float float_of(uint32_t u) {
     std::memcpy(&x, &u, 4);
     return x;
 }
+
+// The finite field with l = p^k elements (Sec. 4.1.1: "pick a prime power l ... addition is over F_l").
+// An element is the integer whose base-p digits are the coefficients of a polynomial of degree < k over
+// Z_p (digit t = coefficient of x^t).  Sums add coefficients mod p; products are polynomial products
+// reduced modulo a monic irreducible polynomial of degree k - the first one when the candidates are
+// listed by the integer value of their lower coefficients.  For a prime l (k = 1) this is arithmetic mod l.
+struct Field {
+    int p = 0, k = 0, l = 0;
+    std::vector<int> irr;   // irr[0..k], irr[k] = 1
+
+    std::vector<int> digits(int a, int n) const {
+        std::vector<int> c(n, 0);
+        for (int t = 0; t < n && a > 0; ++t, a /= p) c[t] = a % p;
+        return c;
+    }
+    int number(const std::vector<int>& c) const {
+        int a = 0;
+        for (int t = (int)c.size() - 1; t >= 0; --t) a = a * p + c[t];
+        return a;
+    }
+    // remainder of the polynomial c (any degree) on division by the monic polynomial m of degree dm
+    std::vector<int> remainder(std::vector<int> c, const std::vector<int>& m, int dm) const {
+        for (int t = (int)c.size() - 1; t >= dm; --t) {
+            const int q = c[t];
+            if (q == 0) continue;
+            for (int u = 0; u <= dm; ++u) c[t - dm + u] = ((c[t - dm + u] - q * m[u]) % p + p) % p;
+        }
+        c.resize(dm);
+        return c;
+    }
+    bool irreducible(const std::vector<int>& m) const {
+        // no monic polynomial of degree 1 .. k/2 divides m
+        for (int dg = 1; dg <= k / 2; ++dg) {
+            int count = 1;
+            for (int t = 0; t < dg; ++t) count *= p;
+            for (int low = 0; low < count; ++low) {
+                std::vector<int> g = digits(low, dg + 1);
+                g[dg] = 1;
+                std::vector<int> rem = remainder(m, g, dg);
+                bool zero = true;
+                for (int v : rem) zero = zero && v == 0;
+                if (zero) return false;
+            }
+        }
+        return true;
+    }
+    bool init(int size) {
+        if (size < 2) return false;
+        int q = 2;
+        while (size % q != 0) ++q;   // smallest prime factor
+        int kk = 0, rest = size;
+        while (rest % q == 0) {
+            rest /= q;
+            ++kk;
+        }
+        if (rest != 1) return false;
+        p = q;
+        k = kk;
+        l = size;
+        for (int low = 0; low < l; ++low) {
+            std::vector<int> m = digits(low, k + 1);
+            m[k] = 1;
+            if (k == 1 || irreducible(m)) {
+                irr = m;
+                return true;
+            }
+        }
+        return false;
+    }
+    int add(int a, int b) const {
+        std::vector<int> x = digits(a, k), y = digits(b, k);
+        for (int t = 0; t < k; ++t) x[t] = (x[t] + y[t]) % p;
+        return number(x);
+    }
+    int mul(int a, int b) const {
+        std::vector<int> x = digits(a, k), y = digits(b, k), c(2 * k - 1 > 0 ? 2 * k - 1 : 1, 0);
+        for (int t = 0; t < k; ++t)
+            for (int u = 0; u < k; ++u) c[t + u] = (c[t + u] + x[t] * y[u]) % p;
+        return number(remainder(c, irr, k));
+    }
+};
 
 // IEEE-754 total order as an unsigned key: negatives have all bits flipped, non-negatives have
 // the sign bit set.  -NaN < -inf < ... < -0 < +0 < ... < +inf < +NaN.
@@ -101,14 +182,17 @@ int orc_num_threads(void) {
 // worker_files[K][l] ascending; file_workers[f][r] indexed by class k; worker_mask[K] bit x set
 // iff the worker holds file x (only when f <= 64; may be null).
 int orc_assign(int l, int r, int32_t* worker_files, int32_t* file_workers, uint64_t* worker_mask) {
-    if (!is_prime(l) || r < 1 || r > l) return -1;
+    const bool prime = is_prime(l);
+    Field F;
+    if (!prime && !F.init(l)) return -1;                 // neither a prime nor a prime power
+    if (r < 1 || r > l || (!prime && r > l - 1)) return -1;   // Algorithm 2 has l - 1 squares; r = l only via the bigraph (prime l)
     const int K = r * l, f = l * l;
     std::vector<std::vector<int>> held(K);
     for (int k = 0; k < r; ++k) {
         const int alpha = (r == l) ? k : k + 1;
         for (int i = 0; i < l; ++i)
             for (int j = 0; j < l; ++j) {
-                const int s = (alpha * i + j) % l;
+                const int s = prime ? (alpha * i + j) % l : F.add(F.mul(alpha, i), j);
                 const int file = i * l + j, worker = k * l + s;
                 held[worker].push_back(file);
                 file_workers[file * r + k] = worker;
@@ -124,6 +208,18 @@ int orc_assign(int l, int r, int32_t* worker_files, int32_t* file_workers, uint6
             worker_mask[u] = m;
         }
     }
+    return 0;
+}
+
+// The field's addition and multiplication tables ([l][l] each), for tests of the field itself.
+int orc_field_tables(int l, int32_t* add, int32_t* mul) {
+    Field F;
+    if (!F.init(l)) return -1;
+    for (int a = 0; a < l; ++a)
+        for (int b = 0; b < l; ++b) {
+            add[a * l + b] = F.add(a, b);
+            mul[a * l + b] = F.mul(a, b);
+        }
     return 0;
 }
 
