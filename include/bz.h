@@ -64,7 +64,10 @@ extern "C" {
  * Square k = 0..r-1 uses alpha = k+1 when r < l.  When r == l the l parallel classes are those of
  * the Ramanujan Case 2 graph with m = s = l (Sec. 4.2.1), i.e. alpha = k.  File i*l + j is given
  * to worker k*l + L(i, j).  Host only, synchronous.
- *   l              prime; r in [1, l]
+ *   l              a prime with r in [1, l], or a prime power p^k <= 1024 with r in [1, l-1]: then
+ *                  F_l is the field of polynomials over Z_p modulo the first monic irreducible
+ *                  polynomial of degree k (candidates ordered by their lower coefficients read as
+ *                  a base-p number), element = integer whose base-p digits are the coefficients
  *   worker_files   host, int32 [r*l][l]: files of each worker, ascending        (may be NULL)
  *   file_workers   host, int32 [l*l][r]: holder of each file in class k         (may be NULL)
  *   worker_mask    host, uint64 [r*l]: bit x set iff the worker holds file x; requires l*l <= 64

@@ -26,6 +26,90 @@ bool is_prime(int n) {
         if (n % t == 0) return false;
     return true;
 }
+
+// Arithmetic of the finite field with l = p^k elements (Sec. 4.1.1).  Elements are the integers
+// 0 .. l-1 read in base p (digit t = coefficient of x^t).  Products are built digit by digit from the
+// top ("multiply the running value by x, reduce, add a times the digit"), with x^k replaced through the
+// first monic irreducible polynomial of degree k when the candidates are ordered by their lower
+// coefficients read as a base-p number.
+class GaloisField {
+public:
+    bool init(int l) {
+        if (l < 2) return false;
+        p_ = 2;
+        while (l % p_ != 0) ++p_;
+        k_ = 0;
+        int rest = l;
+        while (rest % p_ == 0) {
+            rest /= p_;
+            ++k_;
+        }
+        if (rest != 1) return false;
+        l_ = l;
+        top_ = l / p_;  // p^(k-1): the weight of the leading digit
+        if (k_ == 1) {
+            low_ = 0;
+            return true;
+        }
+        for (low_ = 0; low_ < l; ++low_)
+            if (has_no_factor(low_)) return true;
+        return false;
+    }
+    int add(int a, int b) const {
+        int sum = 0, w = 1;
+        for (int t = 0; t < k_; ++t, w *= p_, a /= p_, b /= p_) sum += ((a % p_ + b % p_) % p_) * w;
+        return sum;
+    }
+    int scale(int a, int c) const {  // a times the constant c of Z_p
+        int out = 0, w = 1;
+        for (int t = 0; t < k_; ++t, w *= p_, a /= p_) out += ((a % p_) * c % p_) * w;
+        return out;
+    }
+    int times_x(int a) const {       // a * x with x^k = -(lower part of the modulus)
+        const int lead = a / top_;
+        const int shifted = (a % top_) * p_;
+        return add(shifted, scale(low_, (p_ - lead) % p_));
+    }
+    int mul(int a, int b) const {
+        if (k_ == 1) return static_cast<int>(static_cast<long long>(a) * b % l_);
+        int acc = 0;
+        for (int w = top_; w >= 1; w /= p_) {
+            acc = times_x(acc);
+            acc = add(acc, scale(a, (b / w) % p_));
+        }
+        return acc;
+    }
+
+private:
+    // is x^k + low(x) free of monic factors of degree 1 .. k/2?  Tested through arithmetic modulo the
+    // candidate itself: g divides m iff some nonzero h of degree < k - deg g has g*h = 0 mod m; here simply
+    // by evaluating the product of g with every cofactor of the right degree.
+    bool has_no_factor(int low) const {
+        const int full = l_ + low;  // the monic candidate as a number with k+1 digits
+        for (int dg = 1; dg <= k_ / 2; ++dg) {
+            int ng = 1, nh = 1;
+            for (int t = 0; t < dg; ++t) ng *= p_;
+            for (int t = 0; t < k_ - dg; ++t) nh *= p_;
+            for (int g = ng; g < 2 * ng; ++g)          // monic of degree dg: leading digit 1
+                for (int h = nh; h < 2 * nh; ++h)      // monic of degree k - dg
+                    if (plain_product(g, h) == full) return false;
+        }
+        return true;
+    }
+    int plain_product(int g, int h) const {  // polynomial product over Z_p without reduction
+        int digits_g[16], digits_h[16], out[32] = {0};
+        int ng = 0, nh = 0;
+        for (; g > 0; g /= p_) digits_g[ng++] = g % p_;
+        for (; h > 0; h /= p_) digits_h[nh++] = h % p_;
+        for (int t = 0; t < ng; ++t)
+            for (int u = 0; u < nh; ++u) out[t + u] = (out[t + u] + digits_g[t] * digits_h[u]) % p_;
+        int v = 0;
+        for (int t = ng + nh - 2; t >= 0; --t) v = v * p_ + out[t];
+        return v;
+    }
+    int p_ = 0, k_ = 0, l_ = 0, top_ = 0, low_ = 0;
+};
+
 }  // namespace
 
 void note_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
@@ -45,7 +129,11 @@ int check_launch() {
 using namespace bz;
 
 extern "C" int bz_assign_mols(int l, int r, int32_t* worker_files, int32_t* file_workers, uint64_t* worker_mask) {
-    if (l < 2 || l > 46340 || !is_prime(l) || r < 1 || r > l) return BZ_ERR_INVALID_ARG;
+    if (l < 2 || l > 46340 || r < 1 || r > l) return BZ_ERR_INVALID_ARG;
+    const bool prime = is_prime(l);
+    GaloisField field;
+    if (!prime && (l > 1024 || !field.init(l))) return BZ_ERR_INVALID_ARG;  // neither a prime nor a (small) prime power
+    if (!prime && r > l - 1) return BZ_ERR_INVALID_ARG;  // l - 1 squares exist; r = l only through the bigraph (prime l)
     const int64_t f = static_cast<int64_t>(l) * l;
     if (worker_mask != nullptr && f > 64) return BZ_ERR_INVALID_ARG;
     const int K = r * l;
@@ -59,7 +147,15 @@ extern "C" int bz_assign_mols(int l, int r, int32_t* worker_files, int32_t* file
         for (int s = 0; s < l; ++s) {
             const int u = k * l + s;
             for (int i = 0; i < l; ++i) {
-                const int j = static_cast<int>(((s - static_cast<int64_t>(alpha) * i) % l + l) % l);
+                // the column j with alpha*i + j = s
+                int j;
+                if (prime) {
+                    j = static_cast<int>(((s - static_cast<int64_t>(alpha) * i) % l + l) % l);
+                } else {
+                    const int ai = field.mul(alpha, i);
+                    j = 0;
+                    while (field.add(ai, j) != s) ++j;
+                }
                 const int file = i * l + j;
                 if (worker_files) worker_files[static_cast<int64_t>(u) * l + i] = file;
                 if (file_workers) file_workers[static_cast<int64_t>(file) * r + k] = u;

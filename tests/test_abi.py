@@ -51,7 +51,9 @@ def test_assign_matches_printed_table_and_oracle(lib):
     wf, fw, mask = bz.assign_mols(5, 3)
     for row in read_golden_rows("assignment_l5_r3.txt"):
         assert list(wf[int(row[0])]) == [int(x) for x in row[1:]]
-    for l, r in [(3, 2), (5, 3), (5, 5), (7, 3), (7, 5), (7, 7), (11, 4), (13, 13)]:
+    # primes, and prime powers over F_l (the library and the checker build the field in different ways)
+    for l, r in [(3, 2), (5, 3), (5, 5), (7, 3), (7, 5), (7, 7), (11, 4), (13, 13),
+                 (4, 3), (8, 3), (8, 7), (9, 5), (16, 15), (25, 4), (27, 3), (32, 5), (49, 2), (81, 3)]:
         wf, fw, mask = bz.assign_mols(l, r)
         owf, ofw, omask = oracle.assign(l, r)
         assert np.array_equal(wf, owf) and np.array_equal(fw, ofw)
@@ -61,7 +63,7 @@ def test_assign_matches_printed_table_and_oracle(lib):
             assert mask is None
 
 
-@pytest.mark.parametrize("l,r", [(4, 2), (6, 3), (9, 2), (5, 6), (5, 7), (5, 0), (1, 1), (0, 0), (-3, 1)])
+@pytest.mark.parametrize("l,r", [(4, 4), (6, 3), (9, 9), (10, 2), (2048, 3), (5, 6), (5, 7), (5, 0), (1, 1), (0, 0), (-3, 1)])
 def test_assign_rejects(lib, l, r):
     with pytest.raises(bz.BzError) as e:
         bz.assign_mols(l, r)

@@ -91,6 +91,31 @@ def test_ramanujan_clusters():
     assert np.linalg.norm(out.cpu().numpy().astype(np.float64) - want_out) <= 1e-5 * np.linalg.norm(want_out)
 
 
+@pytest.mark.parametrize("l,r,q", [(4, 3, 3), (8, 3, 4), (8, 5, 5)])
+def test_prime_power_clusters(l, r, q):
+    # squares over the field F_l (Sec. 4.1.1): f = 16 and f = 64 files
+    K, f, d = l * r, l * l, 20_001
+    wf, fw, mask = bz.assign_mols(l, r)
+    owf, ofw, _ = oracle.assign(l, r)
+    assert np.array_equal(wf, owf) and np.array_equal(fw, ofw)
+    cmax, byz, n = bz.worst_case(mask, f, r, q)
+    ocmax, obyz, on = oracle.worst_case(owf, f, r, q)
+    assert (cmax, n, byz.tolist()) == (ocmax, on, obyz.tolist())
+    g = inputs.true_gradients(f, d, seed=l)
+    rep = inputs.build_replicas(g, fw, byz, "alie")
+    want_voted = oracle.vote(rep.numpy())
+    assert sum(not np.array_equal(_bits(want_voted[i]), _bits(g[i])) for i in range(f)) == cmax   # Sec. 2 / Sec. 5.3.2
+    assert np.array_equal(_bits(bz.vote(rep.to(DEV))), _bits(want_voted))
+    assert np.array_equal(_bits(bz.vote_median(rep.to(DEV))), _bits(oracle.median(want_voted)))   # even f: two middle values
+    voted, win = bz.vote_vectorwise(rep.to(DEV))
+    assert np.array_equal(_bits(voted), _bits(want_voted)) and win.cpu().tolist() == oracle.vote_vectorwise(rep.numpy()).tolist()
+    c = cmax
+    out, sel = bz.multikrum(torch.from_numpy(want_voted).to(DEV), c, f - c)
+    want_out, want_sel, _ = oracle.multikrum(want_voted, c, f - c)
+    assert sel.cpu().tolist() == want_sel.tolist()
+    assert np.linalg.norm(out.cpu().numpy().astype(np.float64) - want_out) <= 1e-5 * np.linalg.norm(want_out)
+
+
 def test_hundred_million_coordinates():
     # (l, r) = (5, 3), d = 1e8: 30 GB of replicas, 7.5e9 elements - offsets need 64 bits
     l, r, q, d = 5, 3, 3, 100_000_000
