@@ -106,6 +106,18 @@ def vote_vectorwise(replicas):
     return win
 
 
+def vote_clusters(replicas, abs_tol: float, rel_tol: float):
+    """replicas [r][f][d] -> winner[f]: the copy that agrees with the most copies of its file, where two copies
+    agree iff |a - b| <= abs_tol + rel_tol * max(|a|, |b|) at every coordinate (or the bits are equal)."""
+    lib = _load()
+    rep = _f32(replicas)
+    r, f, d = rep.shape
+    win = np.empty(f, np.int32)
+    lib.orc_vote_clusters(_p(rep, _f32p), ctypes.c_int(r), ctypes.c_int(f), ctypes.c_int64(d), ctypes.c_float(abs_tol),
+                          ctypes.c_float(rel_tol), _p(win, _i32p))
+    return win
+
+
 def median(voted):
     """voted [f][d] -> out[d], coordinate-wise median by IEEE total order."""
     lib = _load()

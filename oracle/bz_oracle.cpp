@@ -18,6 +18,7 @@
 //   orc_assign_ramanujan  Sec. 4.2.1 Steps 1-3 and Eq. (7): the array-code matrix B, H = B or B^T
 //   orc_vote              Eq. (3): per-file majority over the r returned copies
 //   orc_vote_vectorwise   Eq. (3) read on whole vectors (Sec. 2, "Training Protocol")
+//   orc_vote_clusters     the same vote with agreement up to a tolerance (Sec. 2; reading of the builder: parity otherwise unpinned by the paper)
 //   orc_median            coordinate-wise median of the f winners (Sec. 2 / Sec. 6.1)
 //   orc_pairdist ... orc_mean_rows      Krum / Multi-Krum (Sec. 1.2, Sec. 6.1)
 //   orc_bulyan_select, orc_trimmed_mean Bulyan (Sec. 1.2 trimmed mean, Sec. 6.1)
@@ -315,6 +316,39 @@ void orc_vote_vectorwise(const float* replicas, int r, int f, int64_t d, int32_t
             for (int k2 = 0; k2 < r; ++k2) {
                 const float* v2 = replicas + ((size_t)k2 * f + i) * d;
                 if (std::memcmp(vk, v2, (size_t)d * 4) == 0) ++count;
+            }
+            if (count > best_count) {
+                best_count = count;
+                best_k = k;
+            }
+        }
+        winner[i] = best_k;
+    }
+}
+
+// The vote on whole vectors with agreement up to a tolerance (Sec. 2: "potential precision issues can
+// easily be handled by deciding the majority by defining appropriate clusters amongst the returned
+// gradients"; the paper defines no rule - this is the reading taken).  Two copies of a file agree iff
+// at every coordinate their bit patterns are equal or |a - b| <= abs_tol + rel_tol * max(|a|, |b|),
+// the bound formed in binary32 with one fused multiply-add (the precision the decision is taken in on
+// the GPU as well).  The winner is the copy that agrees with the most copies (itself included); ties
+// go to the lowest k.  With both tolerances 0 this is orc_vote_vectorwise.
+void orc_vote_clusters(const float* replicas, int r, int f, int64_t d, float abs_tol, float rel_tol, int32_t* winner) {
+    for (int i = 0; i < f; ++i) {
+        int best_k = 0, best_count = 0;
+        for (int k = 0; k < r; ++k) {
+            const float* vk = replicas + ((size_t)k * f + i) * d;
+            int count = 0;
+            for (int k2 = 0; k2 < r; ++k2) {
+                const float* v2 = replicas + ((size_t)k2 * f + i) * d;
+                bool agree = true;
+                for (int64_t j = 0; j < d && agree; ++j) {
+                    if (bits_of(vk[j]) == bits_of(v2[j])) continue;
+                    const float gap = std::fabs(vk[j] - v2[j]);
+                    const float bound = std::fmaf(rel_tol, std::fmax(std::fabs(vk[j]), std::fabs(v2[j])), abs_tol);
+                    if (!(gap <= bound)) agree = false;
+                }
+                if (agree) ++count;
             }
             if (count > best_count) {
                 best_count = count;

@@ -253,3 +253,72 @@ def test_vectorwise_and_elementwise_votes_differ_only_without_an_agreeing_majori
     rep = np.stack([g, b2, g])
     assert oracle.vote_vectorwise(rep).tolist() == [0]
     assert np.array_equal(oracle.vote(rep)[0], g[0])
+
+
+# ---- agreement up to a tolerance (Sec. 2: "defining appropriate clusters") --------------------------
+
+def test_cluster_vote_reduces_to_the_exact_vote():
+    rng = np.random.default_rng(3)
+    pool = rng.standard_normal((3, 6)).astype(np.float32)
+    rep = pool[rng.integers(0, 3, size=(5, 8))]
+    assert oracle.vote_clusters(rep, 0.0, 0.0).tolist() == oracle.vote_vectorwise(rep).tolist()
+
+
+def test_cluster_vote_hand_cases():
+    one = np.float32(1.0)
+    up = np.nextafter(one, np.float32(2.0))          # 1 + 2^-23
+    A = np.array([1.0, 100.0], np.float32)
+    A1 = np.array([up, 100.0], np.float32)           # A with one ulp of noise
+    Bz = np.array([1.0, -100.0], np.float32)
+    # exact vote: three different vectors -> first copy; with a relative tolerance of 1e-6 the two honest
+    # copies agree and the earlier of them wins although the Byzantine copy comes first
+    rep = np.stack([Bz, A, A1])[:, None, :]
+    assert oracle.vote_vectorwise(rep).tolist() == [0]
+    assert oracle.vote_clusters(rep, 0.0, 1e-6).tolist() == [1]
+    assert oracle.vote_clusters(rep, 0.0, 1e-8).tolist() == [0]      # tolerance below one ulp: nothing agrees
+    # agreement is not transitive: 0.0 ~ 0.6 ~ 1.2 with abs_tol 0.7, but 0.0 !~ 1.2 -> the middle copy agrees with all
+    rep = np.array([[[0.0]], [[1.2]], [[0.6]]], np.float32)
+    assert oracle.vote_clusters(rep, 0.7, 0.0).tolist() == [2]
+    # the bound is abs_tol + rel_tol * max(|a|, |b|): 10 vs 11 agree at rel_tol 0.1 (bound 1.1), not at 0.05;
+    # with abs_tol 0.5 added the second bound is 1.05 and they agree again
+    rep = np.array([[[10.0]], [[11.0]], [[50.0]]], np.float32)
+    assert oracle.vote_clusters(rep, 0.0, 0.1).tolist() == [0]
+    rep3 = np.array([[[50.0]], [[10.0]], [[11.0]]], np.float32)
+    assert oracle.vote_clusters(rep3, 0.0, 0.1).tolist() == [1]
+    assert oracle.vote_clusters(rep3, 0.0, 0.05).tolist() == [0]
+    assert oracle.vote_clusters(rep3, 0.5, 0.05).tolist() == [1]
+    # one coordinate out of tolerance breaks the agreement of the whole vector
+    C = np.array([1.0, 2.0, 3.0], np.float32)
+    C1 = np.array([1.0, 2.0, 3.5], np.float32)
+    rep = np.stack([C1, C, C])[:, None, :]
+    assert oracle.vote_clusters(rep, 0.1, 0.0).tolist() == [1]
+    # NaN agrees only with the same bit pattern; infinities of equal sign are equal bit patterns
+    N = np.array([np.nan, 1.0], np.float32)
+    I = np.array([np.inf, 1.0], np.float32)
+    rep = np.stack([N, I, I])[:, None, :]
+    assert oracle.vote_clusters(rep, 1.0, 1.0).tolist() == [1]
+    rep = np.stack([N, N, I])[:, None, :]
+    assert oracle.vote_clusters(rep, 1.0, 1.0).tolist() == [0]
+
+
+def test_cluster_vote_recovers_noisy_honest_copies():
+    # honest copies differ by rounding noise (a few ulps), Byzantine copies collude: the exact vote is
+    # lost on every file (all copies differ), the cluster vote picks an honest copy wherever honest copies
+    # are in the majority - the guarantee of Sec. 2 carried over
+    wf, fw, _ = oracle.assign(5, 3)
+    byz = oracle.worst_case(wf, 25, 3, 3)[1]
+    g = inputs.true_gradients(25, 300, seed=4)
+    rep = inputs.build_replicas(g, fw, byz, "reversed").numpy().copy()
+    rng = np.random.default_rng(0)
+    noise = (1.0 + rng.integers(-2, 3, size=rep.shape) * 2.0 ** -23).astype(np.float32)
+    honest = np.ones(rep.shape[:2], bool)
+    for i in range(25):
+        for k in range(3):
+            honest[k, i] = int(fw[i][k]) not in set(int(b) for b in byz)
+    rep = np.where(honest[:, :, None], rep * noise, rep)
+    win = oracle.vote_clusters(rep, 0.0, 1e-5)
+    for i in range(25):
+        if honest[:, i].sum() >= 2:
+            assert honest[win[i], i] and win[i] == int(np.argmax(honest[:, i]))
+        else:
+            assert not honest[win[i], i]
