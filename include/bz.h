@@ -152,6 +152,21 @@ int bz_vote_vectorwise(const float* replicas, int r, int f, int64_t d, int64_t l
                        int64_t ld_voted, int32_t* winner, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * bz_vote_vectorwise with agreement up to a tolerance, for clusters whose honest workers do not return
+ * bit-identical gradients (Sec. 2: "potential precision issues can easily be handled by deciding
+ * the majority by defining appropriate clusters amongst the returned gradients"; the paper gives no
+ * rule, this one is the library's).  Two copies of a file agree iff at every coordinate their bit
+ * patterns are equal or |a - b| <= abs_tol + rel_tol * max(|a|, |b|) (binary32, one fused
+ * multiply-add for the bound; a NaN agrees only with its own bit pattern).  The winner is the copy
+ * that agrees with the most copies of its file, itself included (agreement need not be transitive);
+ * ties go to the lowest k.  The winning COPY is returned, not an average.  abs_tol = rel_tol = 0
+ * is bz_vote_vectorwise.  BZ_ERR_INVALID_ARG for negative or NaN tolerances.
+ */
+int bz_vote_clusters(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica, float abs_tol,
+                     float rel_tol, float* voted, int64_t ld_voted, int32_t* winner, void* workspace, size_t workspace_bytes,
+                     void* stream);
+
+/*
  * The same aggregation for a caller whose gradients sit in HOST memory (ideally page-locked):
  * coordinate slabs are copied to the device workspace, aggregated there and the result is copied
  * back; the call returns after out_host is complete.  replicas_host is contiguous [r][f][d],

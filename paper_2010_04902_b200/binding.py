@@ -40,6 +40,7 @@ _SIGNATURES = {
     "bz_assign_ramanujan": (_c_int, [_c_int, _c_int, _c_vp, _c_vp, _c_vp]),
     "bz_vote": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_i64, _c_vp]),
     "bz_vote_vectorwise": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_i64, _c_vp, _c_vp, _c_sz, _c_vp]),
+    "bz_vote_clusters": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, ctypes.c_float, ctypes.c_float, _c_vp, _c_i64, _c_vp, _c_vp, _c_sz, _c_vp]),
     "bz_median": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_vp]),
     "bz_vote_median": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_vp]),
     "bz_vote_median_host": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_vp, _c_vp, _c_sz, _c_vp]),
@@ -240,6 +241,24 @@ def vote_vectorwise(replicas: torch.Tensor, voted: torch.Tensor | None = None, w
                                   _dev(voted, torch.float32, "voted"), ld_v, winner.data_ptr(), ws.data_ptr(), ws.numel(),
                                   _stream())
     _check(st, "bz_vote_vectorwise")
+    return voted, winner
+
+
+def vote_clusters(replicas: torch.Tensor, abs_tol: float, rel_tol: float, voted: torch.Tensor | None = None,
+                  workspace: torch.Tensor | None = None):
+    """bz_vote_clusters: the whole-vector vote with agreement up to a tolerance.  Returns (voted[f][d], winner[f])."""
+    r, f, d, ld_file, ld_rep = _replicas(replicas)
+    if voted is None:
+        voted = torch.empty((f, d), dtype=torch.float32, device=replicas.device)
+    vf, vd, ld_v = _rows(voted, "voted")
+    if (vf, vd) != (f, d):
+        raise ValueError("voted must be [%d][%d]" % (f, d))
+    ws = workspace if workspace is not None else alloc_workspace(OP_VOTE_VECTORWISE, r, f, d, device=replicas.device)
+    winner = torch.empty(f, dtype=torch.int32, device=replicas.device)
+    st = lib().bz_vote_clusters(_dev(replicas, torch.float32, "replicas"), r, f, d, ld_file, ld_rep, float(abs_tol),
+                                float(rel_tol), _dev(voted, torch.float32, "voted"), ld_v, winner.data_ptr(), ws.data_ptr(),
+                                ws.numel(), _stream())
+    _check(st, "bz_vote_clusters")
     return voted, winner
 
 

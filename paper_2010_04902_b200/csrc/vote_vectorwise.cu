@@ -16,8 +16,27 @@ namespace {
 constexpr int kMaxPairs = BZ_MAX_R * (BZ_MAX_R - 1) / 2;   // 105: two 64-bit words per file
 constexpr int kMaskWords = 2;
 
-__device__ __forceinline__ bool differ(const uint4& a, const uint4& b) { return ((a.x ^ b.x) | (a.y ^ b.y) | (a.z ^ b.z) | (a.w ^ b.w)) != 0; }
-__device__ __forceinline__ bool differ(uint32_t a, uint32_t b) { return a != b; }
+// When do two copies of a coordinate agree?  Exactly (bit patterns), or - for clusters whose honest
+// members may differ by rounding (Sec. 2: "deciding the majority by defining appropriate clusters") -
+// within |a - b| <= abs_tol + rel_tol * max(|a|, |b|), evaluated in binary32 with one fused
+// multiply-add; identical bit patterns always agree (so equal NaNs and infinities do).
+struct Agreement {
+    float abs_tol, rel_tol;
+    int exact;
+};
+__device__ __forceinline__ bool differ1(uint32_t a, uint32_t b, const Agreement& g) {
+    if (a == b) return false;
+    if (g.exact) return true;
+    const float x = __uint_as_float(a), y = __uint_as_float(b);
+    const float gap = fabsf(__fsub_rn(x, y));
+    const float bound = __fmaf_rn(g.rel_tol, fmaxf(fabsf(x), fabsf(y)), g.abs_tol);
+    return !(gap <= bound);   // a NaN on either side differs
+}
+__device__ __forceinline__ bool differ(const uint4& a, const uint4& b, const Agreement& g) {
+    if (g.exact) return ((a.x ^ b.x) | (a.y ^ b.y) | (a.z ^ b.z) | (a.w ^ b.w)) != 0;
+    return differ1(a.x, b.x, g) || differ1(a.y, b.y, g) || differ1(a.z, b.z, g) || differ1(a.w, b.w, g);
+}
+__device__ __forceinline__ bool differ(uint32_t a, uint32_t b, const Agreement& g) { return differ1(a, b, g); }
 
 // pair (k, k2), k < k2, -> bit index, row-major over the strict upper triangle
 __host__ __device__ __forceinline__ int pair_index(int r, int k, int k2) { return k * r - k * (k + 1) / 2 + (k2 - k - 1); }
@@ -25,7 +44,7 @@ __host__ __device__ __forceinline__ int pair_index(int r, int k, int k2) { retur
 // grid = (chunks, f).  V = uint4: n counts groups of 4 coordinates and leading dimensions are in groups.
 template <int R, typename V>
 __global__ void __launch_bounds__(256) copies_differ_kernel(const V* __restrict__ rep, int64_t n, int64_t ld_file, int64_t ld_rep,
-                                                            unsigned long long* __restrict__ mask) {
+                                                            unsigned long long* __restrict__ mask, const Agreement agree) {
     const int file = blockIdx.y;
     const V* base = rep + file * ld_file;
     uint32_t bits = 0;  // R <= 7: 21 pairs
@@ -37,7 +56,7 @@ __global__ void __launch_bounds__(256) copies_differ_kernel(const V* __restrict_
 #pragma unroll
         for (int k = 0; k < R; ++k)
 #pragma unroll
-            for (int k2 = k + 1; k2 < R; ++k2, ++p) bits |= differ(c[k], c[k2]) ? (1u << p) : 0u;
+            for (int k2 = k + 1; k2 < R; ++k2, ++p) bits |= differ(c[k], c[k2], agree) ? (1u << p) : 0u;
     }
     bits = __reduce_or_sync(0xffffffffu, bits);
     if ((threadIdx.x & 31) == 0 && bits != 0) atomicOr(&mask[file * kMaskWords], static_cast<unsigned long long>(bits));
@@ -45,7 +64,8 @@ __global__ void __launch_bounds__(256) copies_differ_kernel(const V* __restrict_
 
 // any odd r <= BZ_MAX_R, any alignment
 __global__ void __launch_bounds__(256) copies_differ_generic_kernel(const uint32_t* __restrict__ rep, int r, int64_t d, int64_t ld_file,
-                                                                    int64_t ld_rep, unsigned long long* __restrict__ mask) {
+                                                                    int64_t ld_rep, unsigned long long* __restrict__ mask,
+                                                                    const Agreement agree) {
     const int file = blockIdx.y;
     const uint32_t* base = rep + file * ld_file;
     unsigned long long lo = 0, hi = 0;
@@ -55,7 +75,7 @@ __global__ void __launch_bounds__(256) copies_differ_generic_kernel(const uint32
         int p = 0;
         for (int k = 0; k < r; ++k)
             for (int k2 = k + 1; k2 < r; ++k2, ++p)
-                if (c[k] != c[k2]) {
+                if (differ1(c[k], c[k2], agree)) {
                     if (p < 64) lo |= 1ull << p;
                     else hi |= 1ull << (p - 64);
                 }
@@ -107,10 +127,11 @@ int chunks_for(int64_t n, int f) {
 }
 
 template <int R>
-int launch_differ_vec(const float* rep, int f, int64_t d, int64_t ld_file, int64_t ld_rep, unsigned long long* mask, cudaStream_t s) {
+int launch_differ_vec(const float* rep, int f, int64_t d, int64_t ld_file, int64_t ld_rep, unsigned long long* mask,
+                      const Agreement& agree, cudaStream_t s) {
     const int64_t n = d / 4;
     const dim3 grid(chunks_for(n, f), f);
-    copies_differ_kernel<R, uint4><<<grid, 256, 0, s>>>(reinterpret_cast<const uint4*>(rep), n, ld_file / 4, ld_rep / 4, mask);
+    copies_differ_kernel<R, uint4><<<grid, 256, 0, s>>>(reinterpret_cast<const uint4*>(rep), n, ld_file / 4, ld_rep / 4, mask, agree);
     note_launch();
     return check_launch();
 }
@@ -123,8 +144,9 @@ size_t vote_vectorwise_workspace(int f) { return round_up(static_cast<size_t>(f)
 
 using namespace bz;
 
-extern "C" int bz_vote_vectorwise(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica, float* voted,
-                                  int64_t ld_voted, int32_t* winner, void* workspace, size_t workspace_bytes, void* stream) {
+static int vote_whole_vectors(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica, float* voted,
+                              int64_t ld_voted, int32_t* winner, void* workspace, size_t workspace_bytes, const Agreement& agree,
+                              void* stream) {
     // the argument rules of bz_vote
     if (d < 0 || r < 1 || f < 1 || (r % 2) == 0) return BZ_ERR_INVALID_ARG;
     if (replicas == nullptr && d > 0) return BZ_ERR_INVALID_ARG;
@@ -142,12 +164,12 @@ extern "C" int bz_vote_vectorwise(const float* replicas, int r, int f, int64_t d
     if (d > 0 && r > 1) {
         const bool vec = aligned16(replicas) && (ld_file % 4 == 0) && (ld_replica % 4 == 0) && (d % 4 == 0) && (r == 3 || r == 5 || r == 7);
         if (vec) {
-            st = r == 3 ? launch_differ_vec<3>(replicas, f, d, ld_file, ld_replica, mask, s)
-                        : (r == 5 ? launch_differ_vec<5>(replicas, f, d, ld_file, ld_replica, mask, s)
-                                  : launch_differ_vec<7>(replicas, f, d, ld_file, ld_replica, mask, s));
+            st = r == 3 ? launch_differ_vec<3>(replicas, f, d, ld_file, ld_replica, mask, agree, s)
+                        : (r == 5 ? launch_differ_vec<5>(replicas, f, d, ld_file, ld_replica, mask, agree, s)
+                                  : launch_differ_vec<7>(replicas, f, d, ld_file, ld_replica, mask, agree, s));
         } else {
             const dim3 grid(chunks_for(d, f), f);
-            copies_differ_generic_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const uint32_t*>(replicas), r, d, ld_file, ld_replica, mask);
+            copies_differ_generic_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const uint32_t*>(replicas), r, d, ld_file, ld_replica, mask, agree);
             note_launch();
             st = check_launch();
         }
@@ -170,4 +192,18 @@ extern "C" int bz_vote_vectorwise(const float* replicas, int r, int f, int64_t d
     }
     note_launch();
     return check_launch();
+}
+
+extern "C" int bz_vote_vectorwise(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica, float* voted,
+                                  int64_t ld_voted, int32_t* winner, void* workspace, size_t workspace_bytes, void* stream) {
+    const Agreement exact{0.f, 0.f, 1};
+    return vote_whole_vectors(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, winner, workspace, workspace_bytes, exact, stream);
+}
+
+extern "C" int bz_vote_clusters(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica, float abs_tol,
+                                float rel_tol, float* voted, int64_t ld_voted, int32_t* winner, void* workspace,
+                                size_t workspace_bytes, void* stream) {
+    if (!(abs_tol >= 0.f) || !(rel_tol >= 0.f)) return BZ_ERR_INVALID_ARG;  // negative or NaN tolerances
+    const Agreement within{abs_tol, rel_tol, 0};
+    return vote_whole_vectors(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, winner, workspace, workspace_bytes, within, stream);
 }

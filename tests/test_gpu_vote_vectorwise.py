@@ -117,3 +117,51 @@ def test_full_size_cluster():
     sample = rep[:, :, idx].cpu().numpy()
     assert oracle.vote_vectorwise(sample).tolist() == want_win      # the sample separates the copies as well
     assert np.array_equal(_bits(voted[:, idx]), _bits(np.stack([sample[want_win[i], i] for i in range(l * l)])))
+
+
+# ---- agreement up to a tolerance ----------------------------------------------------------------------
+
+def _check_clusters(rep, abs_tol, rel_tol):
+    want_win = oracle.vote_clusters(rep.numpy(), abs_tol, rel_tol)
+    voted, win = bz.vote_clusters(rep.to(DEV), abs_tol, rel_tol)
+    assert win.cpu().tolist() == want_win.tolist()
+    assert np.array_equal(_bits(voted), _bits(np.stack([rep.numpy()[want_win[i], i] for i in range(rep.shape[1])])))
+    return win.cpu().tolist()
+
+
+@pytest.mark.parametrize("l,r,q,d", [(5, 3, 3, 30_000), (7, 3, 5, 10_001), (5, 5, 6, 8_002), (7, 7, 4, 4_000)])
+def test_noisy_honest_copies(l, r, q, d):
+    wf, fw, _ = oracle.assign(l, r)
+    byz = set(int(u) for u in oracle.worst_case(wf, l * l, r, q)[1])
+    g = inputs.true_gradients(l * l, d, seed=l * r)
+    rep = inputs.build_replicas(g, fw, sorted(byz), "reversed").numpy().copy()
+    rng = np.random.default_rng(l)
+    noise = (1.0 + rng.integers(-2, 3, size=rep.shape) * 2.0 ** -23).astype(np.float32)
+    honest = np.array([[int(fw[i][k]) not in byz for i in range(l * l)] for k in range(r)])
+    rep = torch.from_numpy(np.where(honest[:, :, None], rep * noise, rep).astype(np.float32))
+    win = _check_clusters(rep, 0.0, 1e-5)
+    rp = (r + 1) // 2
+    for i in range(l * l):
+        assert honest[win[i], i] == (honest[:, i].sum() >= rp)       # Sec. 2's guarantee, carried over
+    # tolerances on either side of the noise, and the exact vote as the zero-tolerance case
+    _check_clusters(rep, 0.0, 1e-8)
+    _check_clusters(rep, 1e-3, 0.0)
+    assert _check_clusters(rep, 0.0, 0.0) == oracle.vote_vectorwise(rep.numpy()).tolist()
+
+
+def test_cluster_vote_edge_values_and_generic_r():
+    rng = np.random.default_rng(9)
+    # values at the edge of the bound, NaN and infinities, r = 9 (generic kernel), odd length
+    r, f, d = 9, 5, 1_003
+    base = rng.standard_normal((f, d)).astype(np.float32)
+    rep = np.repeat(base[None], r, axis=0).copy()
+    rep[1:4, 0] += np.float32(0.25)                 # three copies shifted by exactly the absolute tolerance
+    rep[4:, 1] *= np.float32(1.0 + 2.0 ** -10)      # five copies scaled to the edge of the relative tolerance
+    rep[0, 2, 17] = np.nan
+    rep[1, 2, 17] = np.nan
+    rep[2, 3, 5] = np.inf
+    rep[3, 3, 5] = np.inf
+    rep[4, 3, 5] = -np.inf
+    rep = torch.from_numpy(rep)
+    for abs_tol, rel_tol in [(0.25, 0.0), (0.2499, 0.0), (0.0, 2.0 ** -10), (0.0, 2.0 ** -11), (0.1, 0.01)]:
+        _check_clusters(rep, abs_tol, rel_tol)
