@@ -137,6 +137,18 @@ int bz_vote_median_update(const float* replicas, int r, int f, int64_t d, int64_
 int bz_model_update(const float* g, int64_t d, float* w, float* velocity, float eta, float mu, void* stream);
 
 /*
+ * bz_vote_median and bz_vote for copies that do not sit in one strided array (Algorithm 1: the
+ * parameter server receives, from each of the K workers, the l gradients of that worker's files -
+ * K separate buffers).  rows is a DEVICE table of r*f device pointers: entry k*f + i is copy k of
+ * file i, i.e. the gradient worker file_workers[i][k] returned for file i, d floats.  Results are
+ * those of bz_vote_median / bz_vote on the same values.  128-bit loads are used when every row
+ * (and the output) is 16-byte aligned, which the kernels check themselves; any alignment works.
+ *   out    device [d];   voted  device [f][d] with ld_voted.
+ */
+int bz_vote_median_rows(const float* const* rows, int r, int f, int64_t d, float* out, void* stream);
+int bz_vote_rows(const float* const* rows, int r, int f, int64_t d, float* voted, int64_t ld_voted, void* stream);
+
+/*
  * Eq. (3) as the paper states it (Sec. 2, "Training Protocol"): the vote on WHOLE gradients.  For
  * every file the copy whose complete vector (exact match on bit patterns) occurs most often among
  * the file's r copies wins; among equally frequent vectors the one whose first copy has the lowest

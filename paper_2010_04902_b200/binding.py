@@ -39,6 +39,8 @@ _SIGNATURES = {
     "bz_assign_mols": (_c_int, [_c_int, _c_int, _c_vp, _c_vp, _c_vp]),
     "bz_assign_ramanujan": (_c_int, [_c_int, _c_int, _c_vp, _c_vp, _c_vp]),
     "bz_vote": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_i64, _c_vp]),
+    "bz_vote_median_rows": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_vp, _c_vp]),
+    "bz_vote_rows": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_vp, _c_i64, _c_vp]),
     "bz_vote_vectorwise": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_i64, _c_vp, _c_vp, _c_sz, _c_vp]),
     "bz_vote_clusters": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, ctypes.c_float, ctypes.c_float, _c_vp, _c_i64, _c_vp, _c_vp, _c_sz, _c_vp]),
     "bz_median": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_vp]),
@@ -224,6 +226,47 @@ def vote(replicas: torch.Tensor, voted: torch.Tensor | None = None) -> torch.Ten
     st = lib().bz_vote(_dev(replicas, torch.float32, "replicas"), r, f, d, ld_file, ld_rep,
                        _dev(voted, torch.float32, "voted"), ld_v, _stream())
     _check(st, "bz_vote")
+    return voted
+
+
+def row_table(worker_buffers, file_workers, worker_files) -> torch.Tensor:
+    """Device table of r*f row pointers for bz_vote_median_rows / bz_vote_rows from what the workers sent:
+    worker_buffers[u] is a CUDA float32 tensor [l][d] holding worker u's gradients in the order of
+    worker_files[u]; entry k*f + i of the table points at the gradient worker file_workers[i][k] returned
+    for file i.  The buffers must stay alive while the table is in use."""
+    f, r = len(file_workers), len(file_workers[0])
+    ptrs = []
+    for k in range(r):
+        for i in range(f):
+            u = int(file_workers[i][k])
+            slot = [int(x) for x in worker_files[u]].index(i)
+            row = worker_buffers[u][slot]
+            if row.dtype != torch.float32 or not row.is_cuda or row.stride(0) != 1:
+                raise ValueError("worker buffers must be CUDA float32 tensors with contiguous rows")
+            ptrs.append(row.data_ptr())
+    return torch.tensor(ptrs, dtype=torch.int64, device=worker_buffers[0].device)
+
+
+def vote_median_rows(table: torch.Tensor, r: int, f: int, d: int, out: torch.Tensor | None = None) -> torch.Tensor:
+    """bz_vote_median_rows on a table made by row_table()."""
+    if table.dtype != torch.int64 or not table.is_cuda or table.numel() != r * f:
+        raise ValueError("table must be a CUDA int64 tensor of r*f pointers")
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=table.device)
+    st = lib().bz_vote_median_rows(table.data_ptr(), r, f, d, _dev(out, torch.float32, "out"), _stream())
+    _check(st, "bz_vote_median_rows")
+    return out
+
+
+def vote_rows(table: torch.Tensor, r: int, f: int, d: int, voted: torch.Tensor | None = None) -> torch.Tensor:
+    """bz_vote_rows on a table made by row_table()."""
+    if table.dtype != torch.int64 or not table.is_cuda or table.numel() != r * f:
+        raise ValueError("table must be a CUDA int64 tensor of r*f pointers")
+    if voted is None:
+        voted = torch.empty((f, d), dtype=torch.float32, device=table.device)
+    _, _, ld_v = _rows(voted, "voted")
+    st = lib().bz_vote_rows(table.data_ptr(), r, f, d, _dev(voted, torch.float32, "voted"), ld_v, _stream())
+    _check(st, "bz_vote_rows")
     return voted
 
 

@@ -248,6 +248,120 @@ int vote_dispatch(const float* rep, int f, int64_t d, int64_t ld_file, int64_t l
     return launch_vote<R, uint32_t>(rep + 4 * n4, f, d - 4 * n4, ld_file, ld_rep, voted + 4 * n4, ld_voted, s);
 }
 
+// ------------------------------------------------------------------------------------------------
+// The same kernels for copies that do not sit in one strided array: `rows` is a device table of r*f
+// pointers, entry k*f + i = copy k of file i (d floats).  This is the layout of a parameter server
+// that keeps what each worker sent in that worker's own buffer (K buffers of l gradients, Algorithm 1).
+// Whether 128-bit loads may be used is decided on the device from the pointers themselves: the
+// vector kernel returns at once unless every row (and the output) is 16-byte aligned, and the scalar
+// kernel then takes either the tail or everything.
+__device__ __forceinline__ bool rows_aligned(const float* const* rows, int count, bool out_aligned) {
+    int ok = out_aligned ? 1 : 0;
+    for (int t = threadIdx.x; t < count; t += blockDim.x) ok &= (reinterpret_cast<uintptr_t>(rows[t]) & 15u) == 0;
+    return __syncthreads_and(ok) != 0;
+}
+
+template <int R, int F, typename V>
+__global__ void __launch_bounds__(kBlock) vote_median_rows_kernel(const float* const* __restrict__ rows, int64_t d,
+                                                                   float* __restrict__ out, int out_aligned) {
+    constexpr int VEC = Lanes<V>::n;
+    constexpr int B = files_per_batch<R, VEC>();
+    __shared__ const float* tab[R * F];
+    for (int t = threadIdx.x; t < R * F; t += kBlock) tab[t] = rows[t];
+    const bool aligned = rows_aligned(rows, R * F, out_aligned != 0);   // contains the barrier that publishes tab
+    int64_t begin, end;
+    if (VEC == 4) {
+        if (!aligned) return;
+        begin = 0;
+        end = d / 4;
+    } else {
+        begin = aligned ? (d / 4) * 4 : 0;
+        end = d;
+    }
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kBlock;
+    for (int64_t j = begin + static_cast<int64_t>(blockIdx.x) * kBlock + threadIdx.x; j < end; j += stride) {
+        int key[VEC][F];
+#pragma unroll
+        for (int i0 = 0; i0 < F; i0 += B) {
+            V x[B][R];
+#pragma unroll
+            for (int b = 0; b < B; ++b)
+#pragma unroll
+                for (int k = 0; k < R; ++k)
+                    if (i0 + b < F) x[b][k] = ld_stream(reinterpret_cast<const V*>(tab[k * F + i0 + b]) + j);
+#pragma unroll
+            for (int b = 0; b < B; ++b)
+                if (i0 + b < F) {
+#pragma unroll
+                    for (int c = 0; c < VEC; ++c) {
+                        uint32_t copies[R];
+#pragma unroll
+                        for (int k = 0; k < R; ++k) copies[k] = Lanes<V>::get(x[b][k], c);
+                        key[c][i0 + b] = order_key(vote_bits<R>(copies));
+                    }
+                }
+        }
+        uint32_t res[VEC];
+#pragma unroll
+        for (int c = 0; c < VEC; ++c) res[c] = key_bits(MedianNet<F>::run(key[c]));
+        reinterpret_cast<V*>(out)[j] = Lanes<V>::make(res);
+    }
+}
+
+// Any (r, f) within the limits and any alignment.  mode 0: vote only (writes voted), mode 1: vote + median.
+__global__ void __launch_bounds__(128) generic_rows_kernel(const float* const* __restrict__ rows, int r, int f, int64_t d,
+                                                           uint32_t* __restrict__ voted, int64_t ld_voted,
+                                                           float* __restrict__ out, int mode) {
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    for (int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < d; j += stride) {
+        int key[BZ_MAX_F];
+        for (int i = 0; i < f; ++i) {
+            uint32_t x[BZ_MAX_R];
+            for (int k = 0; k < r; ++k) x[k] = reinterpret_cast<const uint32_t*>(rows[k * f + i])[j];
+            const uint32_t w = vote_bits_dyn(x, r);
+            if (mode == 0)
+                voted[i * ld_voted + j] = w;
+            else
+                key[i] = order_key(w);
+        }
+        if (mode == 0) continue;
+        const int want_hi = f / 2, want_lo = (f - 1) / 2;
+        int k_lo = 0, k_hi = 0;
+        for (int i = 0; i < f; ++i) {
+            int rank = 0;
+            for (int t = 0; t < f; ++t) rank += (key[t] < key[i]) || (key[t] == key[i] && t < i);
+            if (rank == want_lo) k_lo = key[i];
+            if (rank == want_hi) k_hi = key[i];
+        }
+        out[j] = (f & 1) ? __uint_as_float(key_bits(k_lo))
+                         : __fadd_rn(__fmul_rn(0.5f, __uint_as_float(key_bits(k_lo))), __fmul_rn(0.5f, __uint_as_float(key_bits(k_hi))));
+    }
+}
+
+template <int R, int F>
+int launch_vm_rows(const float* const* rows, int64_t d, float* out, cudaStream_t s) {
+    const int out_aligned = aligned16(out) ? 1 : 0;
+    if (d >= 4) {
+        vote_median_rows_kernel<R, F, uint4><<<grid_for(d / 4, kBlock, 16), kBlock, 0, s>>>(rows, d, out, out_aligned);
+        note_launch();
+        const int st = check_launch();
+        if (st != BZ_OK) return st;
+    }
+    // the tail if the rows are aligned (at most 3 coordinates), everything otherwise: sized for the latter
+    vote_median_rows_kernel<R, F, uint32_t><<<grid_for(d, kBlock, 16), kBlock, 0, s>>>(rows, d, out, out_aligned);
+    note_launch();
+    return check_launch();
+}
+
+template <int R>
+int vm_rows_dispatch_f(const float* const* rows, int f, int64_t d, float* out, cudaStream_t s) {
+    switch (f) {
+        case 25: return launch_vm_rows<R, 25>(rows, d, out, s);
+        case 49: return launch_vm_rows<R, 49>(rows, d, out, s);
+        default: return 1;
+    }
+}
+
 int validate_replicas(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep) {
     if (d < 0 || r < 1 || f < 1 || (r % 2) == 0) return BZ_ERR_INVALID_ARG;
     if (rep == nullptr && d > 0) return BZ_ERR_INVALID_ARG;  // an empty array may have no address
@@ -378,6 +492,37 @@ extern "C" int bz_model_update(const float* g, int64_t d, float* w, float* veloc
     if (d == 0) return BZ_OK;
     const ModelUpdate upd = {w, velocity, eta, mu};
     model_update_kernel<<<grid_for(d, 256, 8), 256, 0, static_cast<cudaStream_t>(stream)>>>(g, d, upd);
+    note_launch();
+    return check_launch();
+}
+
+extern "C" int bz_vote_median_rows(const float* const* rows, int r, int f, int64_t d, float* out, void* stream) {
+    if (d < 0 || r < 1 || f < 1 || (r % 2) == 0 || rows == nullptr) return BZ_ERR_INVALID_ARG;
+    if (r > BZ_MAX_R || f > BZ_MAX_F) return BZ_ERR_UNSUPPORTED;
+    if (out == nullptr && d > 0) return BZ_ERR_INVALID_ARG;
+    if (d == 0) return BZ_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int st = 1;
+    switch (r) {
+        case 1: st = vm_rows_dispatch_f<1>(rows, f, d, out, s); break;
+        case 3: st = vm_rows_dispatch_f<3>(rows, f, d, out, s); break;
+        case 5: st = vm_rows_dispatch_f<5>(rows, f, d, out, s); break;
+        case 7: st = vm_rows_dispatch_f<7>(rows, f, d, out, s); break;
+        default: break;
+    }
+    if (st != 1) return st;
+    generic_rows_kernel<<<grid_for(d, 128, 8), 128, 0, s>>>(rows, r, f, d, nullptr, 0, out, 1);
+    note_launch();
+    return check_launch();
+}
+
+extern "C" int bz_vote_rows(const float* const* rows, int r, int f, int64_t d, float* voted, int64_t ld_voted, void* stream) {
+    if (d < 0 || r < 1 || f < 1 || (r % 2) == 0 || rows == nullptr) return BZ_ERR_INVALID_ARG;
+    if (r > BZ_MAX_R || f > BZ_MAX_F) return BZ_ERR_UNSUPPORTED;
+    if ((voted == nullptr && d > 0) || ld_voted < d) return BZ_ERR_INVALID_ARG;
+    if (d == 0) return BZ_OK;
+    generic_rows_kernel<<<grid_for(d, 128, 8), 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        rows, r, f, d, reinterpret_cast<uint32_t*>(voted), ld_voted, nullptr, 0);
     note_launch();
     return check_launch();
 }

@@ -120,6 +120,13 @@ def test_validation_runs_before_any_launch(lib):
     assert L.bz_vote_clusters(fake, 3, 25, 10, 10, 250, -1.0, 0.0, fake, 10, fake, fake, 1 << 20, None) == bz.ERR_INVALID_ARG
     assert L.bz_vote_clusters(fake, 3, 25, 10, 10, 250, 0.0, float('nan'), fake, 10, fake, fake, 1 << 20, None) == bz.ERR_INVALID_ARG
     assert L.bz_vote_clusters(fake, 3, 25, 10, 10, 250, 0.0, 1e-6, fake, 10, fake, None, 0, None) == bz.ERR_WORKSPACE
+    assert L.bz_vote_median_rows(None, 3, 25, 10, fake, None) == bz.ERR_INVALID_ARG
+    assert L.bz_vote_median_rows(fake, 2, 25, 10, fake, None) == bz.ERR_INVALID_ARG
+    assert L.bz_vote_median_rows(fake, 3, 25, 10, None, None) == bz.ERR_INVALID_ARG
+    assert L.bz_vote_median_rows(fake, 3, 200, 10, fake, None) == bz.ERR_UNSUPPORTED
+    assert L.bz_vote_median_rows(fake, 3, 25, 0, None, None) == bz.OK
+    assert L.bz_vote_rows(fake, 3, 25, 10, fake, 9, None) == bz.ERR_INVALID_ARG
+    assert L.bz_vote_rows(fake, 3, 25, 10, None, 10, None) == bz.ERR_INVALID_ARG
     assert L.bz_median(None, 25, 10, 10, fake, None) == bz.ERR_INVALID_ARG
     assert L.bz_median(fake, 0, 10, 10, fake, None) == bz.ERR_INVALID_ARG
     assert L.bz_median(fake, 25, 0, 0, fake, None) == bz.OK
