@@ -153,8 +153,8 @@ int pairdist_i8(const float* v, int f, int64_t d, int64_t ld, double* dist, void
     const Scratch sc = carve(ws, f);
     *flag_out = sc.flag;
     // <rows, converter warps, copies, rows per box, boxes in the ring, tiles per step>
-    if (f == 25) return launch_i8<25, 13, 1, 25, 6, 4>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
-    return launch_i8<49, 13, 1, 49, 3, 2>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
+    if (f == 25) return launch_i8<25, 25, 1, 25, 6, 4>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
+    return launch_i8<49, 25, 1, 49, 3, 2>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
 }
 
 // The same from the replicas: vote (Eq. 3) and distances in one pass; the winners go to `voted`.
@@ -168,7 +168,7 @@ int vote_pairdist_i8(const float* rep, int r, int f, int64_t d, int64_t ld_file,
 #define BZ_I8_CASE(R_, F_, W_, FC_, NS_, TS_) \
     if (r == R_ && f == F_)                   \
         return launch_i8<F_, W_, R_, FC_, NS_, TS_>(rep, d, ld_file, ld_rep, voted, ld_voted, dist, sc.tpart, sc.info, sc.flag, force, s);
-    BZ_I8_CASE(3, 25, 10, 5, 8, 4)
+    BZ_I8_CASE(3, 25, 15, 5, 8, 4)
     BZ_I8_CASE(3, 49, 14, 7, 6, 2)
     BZ_I8_CASE(5, 25, 10, 5, 6, 4)
     BZ_I8_CASE(5, 49, 14, 7, 4, 2)
