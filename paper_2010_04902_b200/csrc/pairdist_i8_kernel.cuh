@@ -353,15 +353,19 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
         bool ok = true;
         int s = 0, o = 0;
         uint32_t in_phase = 0, op_phase = 0;
-        for (int64_t step = 0; step < my_steps && ok; ++step) {
-            const int n_sub = static_cast<int>(my_tiles - TS * step < TS ? my_tiles - TS * step : TS);
-            const int64_t j0 = (blockIdx.x + TS * step * gridDim.x) * kTK + 4 * lane;  // this lane's coordinates in the first tile
-            unsigned char* slot = op + static_cast<size_t>(o) * S::kSlotBytes;
+        // this lane's place inside a row of a slice: 16-byte chunk lane/4 (swizzled with the row), word lane%4
+        const uint32_t lane_word = (lane & 3) << 2;
+        int tiles_left = static_cast<int>(my_tiles < (int64_t(1) << 30) ? my_tiles : (int64_t(1) << 30));
+        for (int64_t step = 0; step < my_steps && ok; ++step, tiles_left -= TS) {
+            const int n_sub = tiles_left < TS ? tiles_left : TS;
+            // this lane's coordinates in the first tile (only the vote writes to global memory)
+            const int64_t j0 = R > 1 ? (blockIdx.x + TS * step * gridDim.x) * kTK + 4 * lane : 0;
+            unsigned char* slot = op + static_cast<uint32_t>(o) * S::kSlotBytes;
             bool raise = false, have_slot = false;
 #pragma unroll 1
             for (int c = 0; c < CH && ok; ++c) {
                 // rows of this box-row that belong to this warp: c*FC + off + W*i
-                const int off = ((cw - c * FC) % W + W) % W;
+                const int off = CH == 1 ? cw : ((cw - c * FC) % W + W) % W;
                 float4 val[TS][RWC];
                 int E[RWC];
 #pragma unroll
@@ -371,7 +375,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                             ok = false;
                             break;
                         }
-                        const uint32_t* src = reinterpret_cast<const uint32_t*>(in + static_cast<size_t>(s) * S::kBoxFloats);
+                        const uint32_t* src = reinterpret_cast<const uint32_t*>(in) + static_cast<uint32_t>(s) * S::kBoxFloats;
                         const int64_t j = j0 + sub * static_cast<int64_t>(gridDim.x) * kTK;
 #pragma unroll
                         for (int i = 0; i < RWC; ++i) {
@@ -484,7 +488,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                         // a row whose scale changes hands its old exponent to the drain that comes before this step
                         if (lane == 0) e_stage[o * 64 + r] = old[i] == kENone ? E[i] : old[i];
                         // row r of a slice: 128 bytes per row, 16-byte chunk (lane/4) ^ (r%8) within it
-                        unsigned char* dst = slot + r * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | ((lane & 3) << 2));
+                        unsigned char* dst = slot + r * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | lane_word);
 #pragma unroll
                         for (int sub = 0; sub < TS; ++sub) {
                             if (sub < n_sub) {
