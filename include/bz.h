@@ -289,9 +289,9 @@ int bz_bulyan(const float* voted, int f, int64_t d, int64_t ld, int c, float* ou
  * bz_vote and bz_pairdist in one pass over the replicas: the winners of Eq. (3) are written to
  * `voted` and enter the distance sums of Sec. 1.2 from on-chip memory, so the voted rows are not
  * read back (4*f of the 4*(r*f + 2*f) bytes per coordinate the two calls move are saved).
- * voted is bit-identical to bz_vote's; dist is computed as in bz_pairdist (f = 49: the vote runs in
- * front of the tensor-core kernel, with the same estimate and fall-back; f = 25: the vote runs in
- * front of the binary32 kernel, the faster pass there).  Shapes without a fused
+ * voted is bit-identical to bz_vote's; dist is computed as in bz_pairdist (f = 25, 49 with r = 3, 5
+ * and 7 x 49: the vote runs in front of the tensor-core kernel, with the same estimate and fall-back;
+ * BZ_PAIRDIST_PATH=fp32 puts it in front of the binary32 kernel instead).  Shapes without a fused
  * kernel (r*f outside {3,5}x{25,49} and 7x49, unaligned or short arrays) run the two calls.
  *   replicas, ld_file, ld_replica as bz_vote;  voted device [f][d] with ld_voted (written);
  *   dist device double [f][f];  workspace as bz_pairdist.

@@ -168,11 +168,11 @@ int vote_pairdist_i8(const float* rep, int r, int f, int64_t d, int64_t ld_file,
 #define BZ_I8_CASE(R_, F_, W_, FC_, NS_, TS_) \
     if (r == R_ && f == F_)                   \
         return launch_i8<F_, W_, R_, FC_, NS_, TS_>(rep, d, ld_file, ld_rep, voted, ld_voted, dist, sc.tpart, sc.info, sc.flag, force, s);
-    BZ_I8_CASE(3, 25, 15, 5, 8, 4)
-    BZ_I8_CASE(3, 49, 14, 7, 6, 2)
-    BZ_I8_CASE(5, 25, 10, 5, 6, 4)
-    BZ_I8_CASE(5, 49, 14, 7, 4, 2)
-    BZ_I8_CASE(7, 49, 14, 7, 3, 2)
+    BZ_I8_CASE(3, 25, 25, 25, 3, 2)
+    BZ_I8_CASE(3, 49, 25, 25, 2, 2)
+    BZ_I8_CASE(5, 25, 25, 25, 2, 2)
+    BZ_I8_CASE(5, 49, 25, 25, 2, 1)
+    BZ_I8_CASE(7, 49, 13, 13, 2, 1)
 #undef BZ_I8_CASE
     return 1;
 }

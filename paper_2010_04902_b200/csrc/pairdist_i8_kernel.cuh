@@ -68,7 +68,7 @@ template <int F, int W, int R, int FC, int NS, int TS> struct I8Shape {
     static constexpr int kSlotBytes = TS * kOpStageBytes;  // a step = TS tiles
     static constexpr int kSlots = 2;
     static constexpr int kTmemCols = RP == 64 ? 512 : 128;
-    static constexpr int kChunks = F / FC;                 // boxes per tile
+    static constexpr int kChunks = (F + FC - 1) / FC;      // boxes per tile (rows past f in the last one are filled with zeros by the TMA unit and skipped)
     static constexpr int RWC = (FC + W - 1) / W;           // rows of a box one converter warp may own
     static constexpr int kBoxFloats = R * FC * kTK;
     static constexpr int kBoxBytes = kBoxFloats * 4;
@@ -76,7 +76,6 @@ template <int F, int W, int R, int FC, int NS, int TS> struct I8Shape {
     static constexpr int kPartialBytes = (F * F * 8 + 15) / 16 * 16;   // the CTA's partial matrix T
     static constexpr int kSmem = 1024 + kSlots * kSlotBytes + NS * kBoxBytes + kCtlBytes + kPartialBytes;
     static_assert(F <= 64, "at most 64 rows");
-    static_assert(kChunks * FC == F, "FC must divide F");
     static_assert(kBoxBytes % 128 == 0, "TMA destinations are 128-byte aligned");
     static_assert(kSmem <= 227 * 1024, "shared memory");
     // MMA m covers slice indices m*SPM .. m*SPM+SPM-1 along M and m*SPM .. 3 along N
@@ -380,7 +379,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
 #pragma unroll
                         for (int i = 0; i < RWC; ++i) {
                             const int fi = off + W * i;
-                            if (fi < FC) {
+                            if (fi < FC && c * FC + fi < F) {
                                 uint4 w;
                                 if constexpr (R == 1) {
                                     w = *reinterpret_cast<const uint4*>(src + fi * kTK + 4 * lane);
@@ -435,7 +434,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                 float m = 0.f;
 #pragma unroll
                 for (int i = 0; i < RWC; ++i) {
-                    if (off + W * i < FC) {
+                    if (off + W * i < FC && c * FC + off + W * i < F) {
                         E[i] = e_cur[c * FC + off + W * i];
                         old[i] = E[i];
                         if (E[i] == kENone) m = __int_as_float(0x7f800000);  // no exponent yet (first step)
@@ -450,7 +449,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                 if (__any_sync(0xffffffffu, !(fabsf(m) < 1073741824.0f))) {
 #pragma unroll
                     for (int i = 0; i < RWC; ++i) {
-                        if (off + W * i < FC) {
+                        if (off + W * i < FC && c * FC + off + W * i < F) {
                             uint32_t m8 = 0;
 #pragma unroll
                             for (int sub = 0; sub < TS; ++sub)
@@ -483,7 +482,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
 #pragma unroll
                 for (int i = 0; i < RWC; ++i) {
                     const int fi = off + W * i;
-                    if (fi < FC) {
+                    if (fi < FC && c * FC + fi < F) {
                         const int r = c * FC + fi;
                         // a row whose scale changes hands its old exponent to the drain that comes before this step
                         if (lane == 0) e_stage[o * 64 + r] = old[i] == kENone ? E[i] : old[i];

@@ -90,12 +90,11 @@ extern "C" int bz_vote_pairdist(const float* replicas, int r, int f, int64_t d, 
     if (ld_file < d || (r > 1 && ld_replica < d) || ld_voted < d) return BZ_ERR_INVALID_ARG;
     int st = check_workspace(workspace, workspace_bytes, krum_workspace_bytes(BZ_OP_PAIRDIST, f));
     if (st != BZ_OK) return st;
-    // Vote + integer distances on the tensor cores where that is the faster single pass (f = 49 as
-    // measured; every shape that has the kernel when BZ_PAIRDIST_PATH=i8).  The binary32
-    // distance kernel follows only if the integer kernel's error estimate asks for it: it reads the
-    // flag on the device.
+    // Vote + integer distances on the tensor cores wherever that kernel exists (it is the faster single
+    // pass on every shape measured).  The binary32 distance kernel follows only if the integer kernel's
+    // error estimate asks for it: it reads the flag on the device.
     const bool forced = pairdist_path_i8_forced() != 0;
-    if (d > 0 && r > 1 && (forced || (!pairdist_path_fp32_only() && f == 49))) {
+    if (d > 0 && r > 1 && !pairdist_path_fp32_only()) {
         int* flag = nullptr;
         st = vote_pairdist_i8(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, dist,
                               static_cast<char*>(workspace) + pairdist_workspace_fp32(f), forced ? 1 : 0, &flag,
