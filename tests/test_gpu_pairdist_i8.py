@@ -147,3 +147,36 @@ def test_full_size_on_sampled_rows():
         _check_close(sub, want)
     assert np.array_equal(dist.cpu().numpy(), alone.cpu().numpy())   # same integers either way
     assert bz.pipeline_timeouts() == 0
+
+
+def test_padded_rows_and_coordinate_slabs(monkeypatch):
+    # rows with a leading dimension larger than d, and a coordinate slab of a larger allocation (the way
+    # multi-GPU slabs and the 1e8-coordinate cells are passed): the kernel's conditions hold (16-byte
+    # aligned start, ld a multiple of 4), so it runs; an unaligned slab takes the binary32 kernel
+    monkeypatch.setenv("BZ_PAIRDIST_PATH", "i8")
+    f, d_all = 49, 60_000
+    g = inputs.true_gradients(f, d_all, seed=8)
+    g[5] = -100.0 * g[5]
+    buf = torch.zeros((f, d_all + 12), dtype=torch.float32, device=DEV)
+    buf[:, :d_all] = g.to(DEV)
+    for j0, d in [(0, 60_000), (4_000, 33_336), (8, 20_002)]:
+        slab = buf[:, j0:j0 + d]
+        want = oracle.pairdist(g[:, j0:j0 + d].contiguous().numpy())
+        _check_close(bz.pairdist(slab).cpu().numpy(), want)
+    # the same through the vote: replicas and voted rows as slabs of padded arrays
+    r = 3
+    rep_all = torch.zeros((r, f, d_all + 12), dtype=torch.float32, device=DEV)
+    rep_all[:, :, :d_all] = g.to(DEV)[None]
+    rep_all[0, 7, :d_all] = 3.0
+    rep_all[1, 7, :d_all] = 3.0
+    voted_all = torch.zeros((f, d_all + 12), dtype=torch.float32, device=DEV)
+    j0, d = 4_000, 33_336
+    voted, dist = bz.vote_pairdist(rep_all[:, :, j0:j0 + d], voted_all[:, j0:j0 + d])
+    want_voted = oracle.vote(rep_all[:, :, j0:j0 + d].cpu().numpy())
+    assert np.array_equal(voted.cpu().numpy().view(np.uint32), want_voted.view(np.uint32))
+    assert (voted_all[:, :j0] == 0).all() and (voted_all[:, j0 + d:] == 0).all()      # nothing written outside the slab
+    _check_close(dist.cpu().numpy(), oracle.pairdist(want_voted))
+    assert bz.pipeline_timeouts() == 0
+    monkeypatch.delenv("BZ_PAIRDIST_PATH")
+    odd = buf[:, 1:50_001]                                                            # starts 4 bytes off a 16-byte boundary
+    _check_close(bz.pairdist(odd).cpu().numpy(), oracle.pairdist(g[:, 1:50_001].contiguous().numpy()))
