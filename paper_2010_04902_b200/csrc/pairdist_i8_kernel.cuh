@@ -31,7 +31,8 @@
 //
 // Every warp of a CTA sees every tile, so what a warp spends per tile on waiting, signalling and
 // bookkeeping bounds the CTA's rate whatever the number of warps: the unit of work between two
-// signals is therefore a step of TS tiles (2 to 4, as many as shared memory holds).
+// signals is therefore a step of TS tiles (up to 4, as many as shared memory holds), and a box holds all the
+// rows (or, with copies, 13 to 25 of them).
 //
 // Roles in a CTA (one CTA per SM, tiles dealt round-robin): one thread issues TMA loads of boxes
 // [R copies][FC rows][128 coordinates] into a ring of shared memory; W converter warps own fixed rows

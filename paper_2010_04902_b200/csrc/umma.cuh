@@ -62,9 +62,10 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, int32_t (&x)[8]) {
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Arrival without release ordering.  A release would first wait for every memory operation the thread
-// has in flight - also the global loads it issued for later tiles.  What the arrival must order, the
-// thread's own earlier shared-memory stores, is covered: they are made visible to the tensor core by
-// fence_async_smem() before this, and shared-memory operations of one thread are performed in order.
+// has in flight - also its global stores of voted rows, which nobody in the CTA reads.  What the
+// arrival must order, the thread's own earlier shared-memory accesses, is covered: stores are made
+// visible to the tensor core by fence_async_smem() before this, loads have delivered their values
+// (they were consumed), and shared-memory operations of one thread are performed in order.
 __device__ __forceinline__ void mbar_arrive_relaxed(uint64_t* bar) {
     asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
