@@ -109,6 +109,125 @@ __global__ void __launch_bounds__(BZ_MAX_F) bulyan_select_kernel(const double* _
 }
 
 // ------------------------------------------------------------------------------------------------
+// The same selections for f <= 64 with the sorted rows in shared memory, one warp per row.
+// Sorting is by rank counting: the lanes hold the row's distances and each counts how many of them
+// precede its own (by value, then index).  A score is the sum of the first nb ACTIVE entries of the
+// sorted row, added one by one in ascending order - the same sums in the same order as in the kernels above.
+constexpr int kSelF = 64;
+
+__device__ __forceinline__ void sort_rows_shared(const double* __restrict__ dist, int f, double (*sval)[kSelF],
+                                                 unsigned char (*sidx)[kSelF]) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int a = warp; a < f; a += blockDim.x >> 5) {
+        const int b0 = lane, b1 = lane + 32;
+        const double v0 = b0 < f ? dist[a * f + b0] : 0.0, v1 = b1 < f ? dist[a * f + b1] : 0.0;
+        int rank0 = 0, rank1 = 0;
+        for (int b = 0; b < f; ++b) {
+            const double y = __shfl_sync(0xffffffffu, b < 32 ? v0 : v1, b & 31);
+            if (b == a) continue;
+            rank0 += (y < v0) || (y == v0 && b < b0);
+            rank1 += (y < v1) || (y == v1 && b < b1);
+        }
+        if (b0 < f && b0 != a) {
+            sval[a][rank0] = v0;
+            sidx[a][rank0] = static_cast<unsigned char>(b0);
+        }
+        if (b1 < f && b1 != a) {
+            sval[a][rank1] = v1;
+            sidx[a][rank1] = static_cast<unsigned char>(b1);
+        }
+    }
+}
+
+// warp-collective: score of row a among the active rows (the result is valid in lane 0).
+// The lanes compact the first nb active entries into `comp` (positions by prefix counts of the
+// ballots); lane 0 adds them in ascending order.
+constexpr int kSelWarps = 16;
+__device__ __forceinline__ double krum_score_warp(const double (*sval)[kSelF], const unsigned char (*sidx)[kSelF], int f, int a,
+                                                  const unsigned char* active, int nb, double* comp) {
+    const int lane = threadIdx.x & 31;
+    const int p0 = lane, p1 = lane + 32;
+    const bool act0 = p0 < f - 1 && active[sidx[a][p0]];
+    const bool act1 = p1 < f - 1 && active[sidx[a][p1]];
+    const unsigned m0 = __ballot_sync(0xffffffffu, act0), m1 = __ballot_sync(0xffffffffu, act1);
+    const unsigned below = (1u << lane) - 1u;
+    const int q0 = __popc(m0 & below), q1 = __popc(m0) + __popc(m1 & below);
+    if (act0 && q0 < nb) comp[q0] = sval[a][p0];
+    if (act1 && q1 < nb) comp[q1] = sval[a][p1];
+    __syncwarp();
+    double s = 0.0;
+    if (lane == 0) {
+        const int total = min(nb, __popc(m0) + __popc(m1));
+        for (int k = 0; k < total; ++k) s += comp[k];
+    }
+    __syncwarp();
+    return s;
+}
+
+// bulyan == 0: Multi-Krum (first m of the ranking); bulyan != 0: theta = f - 2c picks, one per round
+__global__ void __launch_bounds__(kSelWarps * 32) select_shared_kernel(const double* __restrict__ dist, int f, int c, int m, int bulyan,
+                                                             int32_t* __restrict__ selected) {
+    __shared__ double sval[kSelF][kSelF];
+    __shared__ unsigned char sidx[kSelF][kSelF];
+    __shared__ double comp[kSelWarps][kSelF];
+    __shared__ double score[kSelF];
+    __shared__ unsigned char active[kSelF];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid < f) active[tid] = 1;
+    sort_rows_shared(dist, f, sval, sidx);
+    __syncthreads();
+    if (!bulyan) {
+        for (int a = warp; a < f; a += kSelWarps) {
+            const double s = krum_score_warp(sval, sidx, f, a, active, f - c - 2, comp[warp]);
+            if (lane == 0) score[a] = s;
+        }
+        __syncthreads();
+        if (tid < f) {
+            int rank = 0;
+            for (int b = 0; b < f; ++b) rank += (score[b] < score[tid]) || (score[b] == score[tid] && b < tid);
+            if (rank < m) selected[rank] = tid;
+        }
+        return;
+    }
+    const int theta = f - 2 * c;
+    for (int t = 0; t < theta; ++t) {
+        const int n = f - t;
+        int nb = n - c - 2;
+        if (nb < 1) nb = 1;
+        if (nb > n - 1) nb = n - 1;
+        for (int a = warp; a < f; a += kSelWarps) {
+            if (!active[a]) continue;  // uniform over the warp
+            const double s = (n > 1) ? krum_score_warp(sval, sidx, f, a, active, nb, comp[warp]) : 0.0;
+            if (lane == 0) score[a] = s;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // smallest (score, index) among the active rows
+            double best = 0.0;
+            int who = -1;
+            for (int a = lane; a < f; a += 32)
+                if (active[a] && (who < 0 || score[a] < best)) {  // a grows: a tie keeps the lower index
+                    best = score[a];
+                    who = a;
+                }
+            for (int o = 16; o > 0; o >>= 1) {
+                const double ob = __shfl_down_sync(0xffffffffu, best, o);
+                const int ow = __shfl_down_sync(0xffffffffu, who, o);
+                if (ow >= 0 && (who < 0 || ob < best || (ob == best && ow < who))) {
+                    best = ob;
+                    who = ow;
+                }
+            }
+            if (lane == 0) {
+                selected[t] = who;
+                active[who] = 0;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Means over selected rows.
 
 template <typename V> struct FL;
@@ -293,7 +412,10 @@ extern "C" int bz_krum_select(const double* dist, int f, int c, int m, int32_t* 
     if (dist == nullptr || selected == nullptr || f < 1) return BZ_ERR_INVALID_ARG;
     if (f > BZ_MAX_F) return BZ_ERR_UNSUPPORTED;
     if (c < 0 || f < 2 * c + 3 || m < 1 || m > f) return BZ_ERR_PRECONDITION;
-    krum_select_kernel<<<1, BZ_MAX_F, 0, static_cast<cudaStream_t>(stream)>>>(dist, f, c, m, selected);
+    if (f <= kSelF)
+        select_shared_kernel<<<1, kSelWarps * 32, 0, static_cast<cudaStream_t>(stream)>>>(dist, f, c, m, 0, selected);
+    else
+        krum_select_kernel<<<1, BZ_MAX_F, 0, static_cast<cudaStream_t>(stream)>>>(dist, f, c, m, selected);
     note_launch();
     return check_launch();
 }
@@ -330,7 +452,10 @@ extern "C" int bz_bulyan_select(const double* dist, int f, int c, int32_t* selec
     if (dist == nullptr || selected == nullptr || f < 1) return BZ_ERR_INVALID_ARG;
     if (f > BZ_MAX_F) return BZ_ERR_UNSUPPORTED;
     if (c < 0 || f < 4 * c + 3) return BZ_ERR_PRECONDITION;
-    bulyan_select_kernel<<<1, BZ_MAX_F, 0, static_cast<cudaStream_t>(stream)>>>(dist, f, c, selected);
+    if (f <= kSelF)
+        select_shared_kernel<<<1, kSelWarps * 32, 0, static_cast<cudaStream_t>(stream)>>>(dist, f, c, 0, 1, selected);
+    else
+        bulyan_select_kernel<<<1, BZ_MAX_F, 0, static_cast<cudaStream_t>(stream)>>>(dist, f, c, selected);
     note_launch();
     return check_launch();
 }
