@@ -54,29 +54,43 @@ __global__ void __launch_bounds__(256)
         if (a == kInfoBad && info[e]) atomicOr(&s_bad, 1);
     }
     __syncthreads();
+    // 2 sqrt(x) + d x <= tol  <=>  x <= x_max with sqrt(x_max) = (sqrt(1 + d tol) - 1) / d: one square root
+    // per thread instead of one per pair
+    const double dd = static_cast<double>(d);
+    const double y_max = (sqrt(1.0 + dd * kRelTol) - 1.0) / dd;
+    const double x_max = y_max * y_max;
+    __shared__ double s_min_nz[F], s_zero_step[F];
     if (tid < F) {
-        const int a = tid;
-        const double step_a = __longlong_as_double(static_cast<long long>(1023 + s_emax[a] - 30) << 52);
-        double min_nz = 1e300, zero_step = 0.0;
-        bool bad = false;
-        for (int b = 0; b < F; ++b) {
-            if (b == a) continue;
-            const double step_b = __longlong_as_double(static_cast<long long>(1023 + s_emax[b] - 30) << 52);
-            const double var = 0.0841 * (step_a * step_a + step_b * step_b);
-            const double v = dist[a * F + b];
-            if (v > 0.0) {
-                if (2.0 * sqrt(var / v) + static_cast<double>(d) * var / v > kRelTol) bad = true;
-                min_nz = fmin(min_nz, v);
-            } else if (v == 0.0) {
-                zero_step = fmax(zero_step, fmax(step_a, step_b));
-            } else {
-                bad = true;
-            }
-        }
-        // rows that convert to the same integers may still differ by less than a step everywhere
-        if (zero_step > 0.0 && min_nz < 1e300 && static_cast<double>(d) * zero_step * zero_step > kRelTol * min_nz) bad = true;
-        if (bad) atomicOr(&s_bad, 1);
+        s_min_nz[tid] = 1e300;
+        s_zero_step[tid] = 0.0;
     }
+    __syncthreads();
+    bool bad = false;
+    for (int p = tid; p < F * F; p += blockDim.x) {
+        const int a = p / F, b = p % F;
+        if (a >= b) continue;
+        const double step_a = __longlong_as_double(static_cast<long long>(1023 + s_emax[a] - 30) << 52);
+        const double step_b = __longlong_as_double(static_cast<long long>(1023 + s_emax[b] - 30) << 52);
+        const double var = 0.0841 * (step_a * step_a + step_b * step_b);
+        const double v = dist[a * F + b];
+        if (v > 0.0) {
+            if (var > x_max * v) bad = true;
+            atomicMin(reinterpret_cast<unsigned long long*>(&s_min_nz[a]), static_cast<unsigned long long>(__double_as_longlong(v)));
+            atomicMin(reinterpret_cast<unsigned long long*>(&s_min_nz[b]), static_cast<unsigned long long>(__double_as_longlong(v)));
+        } else if (v == 0.0) {
+            const double z = fmax(step_a, step_b);
+            atomicMax(reinterpret_cast<unsigned long long*>(&s_zero_step[a]), static_cast<unsigned long long>(__double_as_longlong(z)));
+            atomicMax(reinterpret_cast<unsigned long long*>(&s_zero_step[b]), static_cast<unsigned long long>(__double_as_longlong(z)));
+        } else {
+            bad = true;
+        }
+    }
+    if (bad) atomicOr(&s_bad, 1);
+    __syncthreads();
+    // rows that convert to the same integers may still differ by less than a step everywhere
+    if (tid < F && s_zero_step[tid] > 0.0 && s_min_nz[tid] < 1e300 &&
+        dd * s_zero_step[tid] * s_zero_step[tid] > kRelTol * s_min_nz[tid])
+        atomicOr(&s_bad, 1);
     __syncthreads();
     if (tid == 0) flag[0] = (s_bad && !force) ? 1 : 0;
 }
