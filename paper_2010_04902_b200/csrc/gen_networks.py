@@ -148,6 +148,7 @@ def emit():
     lines = [
         "// GENERATED by gen_networks.py - do not edit.  Comparator networks on register arrays:",
         "// BZ_CE(a,b) orders wires a <= b; BZ_LO / BZ_HI keep only the min on a / the max on b.",
+        "// BZ_CM is a BZ_CE that run<true> may compute on the multiply-add pipe (every other full comparator).",
         "",
     ]
     for n in MEDIAN_SIZES:
@@ -156,10 +157,15 @@ def emit():
         ops = sum(int(x) + int(y) for _, _, x, y in net)
         lines.append("// median of %d: %d comparators, %d min/max operations" % (n, len(net), ops))
         lines.append("template <> struct MedianNet<%d> {" % n)
-        lines.append("    template <typename T> __device__ __forceinline__ static T run(T (&k)[%d]) {" % n)
+        lines.append("    template <bool MIX = false, typename T> __device__ __forceinline__ static T run(T (&k)[%d]) {" % n)
         body = []
+        full = 0
         for a, b, na, nb in net:
-            body.append(("BZ_CE(%d,%d)" if (na and nb) else ("BZ_LO(%d,%d)" if na else "BZ_HI(%d,%d)")) % (a, b))
+            if na and nb:
+                full += 1
+                body.append(("BZ_CM(%d,%d)" if full % 2 == 0 else "BZ_CE(%d,%d)") % (a, b))
+            else:
+                body.append(("BZ_LO(%d,%d)" if na else "BZ_HI(%d,%d)") % (a, b))
         for i in range(0, len(body), 8):
             lines.append("        " + " ".join(body[i:i + 8]))
         lines.append("        return k[%d];" % ((n - 1) // 2))
@@ -171,8 +177,8 @@ def emit():
         verify_sort(ces, n)
         lines.append("// sort of %d: %d comparators" % (n, len(ces)))
         lines.append("template <> struct SortNet<%d> {" % n)
-        lines.append("    template <typename T> __device__ __forceinline__ static void run(T (&k)[%d]) {" % n)
-        body = ["BZ_CE(%d,%d)" % (a, b) for a, b in ces]
+        lines.append("    template <bool MIX = false, typename T> __device__ __forceinline__ static void run(T (&k)[%d]) {" % n)
+        body = [("BZ_CM(%d,%d)" if i % 2 else "BZ_CE(%d,%d)") % (a, b) for i, (a, b) in enumerate(ces)]
         for i in range(0, len(body), 8):
             lines.append("        " + " ".join(body[i:i + 8]))
         lines.append("    }")

@@ -302,7 +302,7 @@ __global__ void __launch_bounds__(128) trimmed_mean_kernel(const float* __restri
         int k[THETA];
 #pragma unroll
         for (int t = 0; t < THETA; ++t) k[t] = order_key(__float_as_uint(__ldcs(v + sel[t] * ld + j)));
-        SortNet<THETA>::run(k);
+        SortNet<THETA>::template run<true>(k);  // bound by the ALU pipe: comparators on two pipes
         float s[THETA];
 #pragma unroll
         for (int t = 0; t < THETA; ++t) s[t] = __uint_as_float(key_bits(k[t]));
