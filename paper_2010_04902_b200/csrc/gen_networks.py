@@ -178,7 +178,7 @@ def emit():
         lines.append("// sort of %d: %d comparators" % (n, len(ces)))
         lines.append("template <> struct SortNet<%d> {" % n)
         lines.append("    template <bool MIX = false, typename T> __device__ __forceinline__ static void run(T (&k)[%d]) {" % n)
-        body = [("BZ_CM(%d,%d)" if i % 2 else "BZ_CE(%d,%d)") % (a, b) for i, (a, b) in enumerate(ces)]
+        body = [("BZ_CM(%d,%d)" if i % 3 else "BZ_CE(%d,%d)") % (a, b) for i, (a, b) in enumerate(ces)]
         for i in range(0, len(body), 8):
             lines.append("        " + " ".join(body[i:i + 8]))
         lines.append("    }")

@@ -290,25 +290,66 @@ template <int THETA, int BETA> __device__ __forceinline__ float window_mean(cons
     return static_cast<float>(sum / static_cast<double>(BETA));
 }
 
-template <int THETA, int BETA>
+// V coordinates per thread (V = 2, 4: 64- and 128-bit loads, rows aligned accordingly): the address arithmetic
+// and the load instructions are shared by the V coordinates.
+template <int THETA, int BETA, int V>
 __global__ void __launch_bounds__(128) trimmed_mean_kernel(const float* __restrict__ v, int64_t d, int64_t ld,
                                                            const int32_t* __restrict__ selected,
                                                            float* __restrict__ out) {
-    __shared__ int32_t sel[THETA];
-    for (int t = threadIdx.x; t < THETA; t += blockDim.x) sel[t] = selected[t];
+    __shared__ int64_t row[THETA];
+    for (int t = threadIdx.x; t < THETA; t += blockDim.x) row[t] = selected[t] * ld;
     __syncthreads();
+    const int64_t groups = (d + V - 1) / V;
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
-    for (int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < d; j += stride) {
-        int k[THETA];
+    for (int64_t g = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; g < groups; g += stride) {
+        const int64_t j = g * V;
+        int k[V][THETA];
+        const bool whole = j + V <= d;  // the last group may hold fewer coordinates
+        if (V == 4 && whole) {
 #pragma unroll
-        for (int t = 0; t < THETA; ++t) k[t] = order_key(__float_as_uint(__ldcs(v + sel[t] * ld + j)));
-        SortNet<THETA>::template run<true>(k);  // bound by the ALU pipe: comparators on two pipes
-        float s[THETA];
+            for (int t = 0; t < THETA; ++t) {
+                const float4 x = __ldcs(reinterpret_cast<const float4*>(v + row[t] + j));
+                k[0][t] = order_key(__float_as_uint(x.x));
+                k[V > 1 ? 1 : 0][t] = order_key(__float_as_uint(x.y));
+                k[V > 2 ? 2 : 0][t] = order_key(__float_as_uint(x.z));
+                k[V > 3 ? 3 : 0][t] = order_key(__float_as_uint(x.w));
+            }
+        } else if (V == 2 && whole) {
 #pragma unroll
-        for (int t = 0; t < THETA; ++t) s[t] = __uint_as_float(key_bits(k[t]));
-        out[j] = window_mean<THETA, BETA>(s);
+            for (int t = 0; t < THETA; ++t) {
+                const float2 x = __ldcs(reinterpret_cast<const float2*>(v + row[t] + j));
+                k[0][t] = order_key(__float_as_uint(x.x));
+                k[V > 1 ? 1 : 0][t] = order_key(__float_as_uint(x.y));
+            }
+        } else {
+#pragma unroll
+            for (int c = 0; c < V; ++c) {
+                const int64_t jc = j + c < d ? j + c : d - 1;  // past the end: the last coordinate once more
+#pragma unroll
+                for (int t = 0; t < THETA; ++t) k[c][t] = order_key(__float_as_uint(__ldcs(v + row[t] + jc)));
+            }
+        }
+        float res[V];
+#pragma unroll
+        for (int c = 0; c < V; ++c) {
+            SortNet<THETA>::template run<true>(k[c]);  // bound by the ALU pipe: comparators on two pipes
+            float s[THETA];
+#pragma unroll
+            for (int t = 0; t < THETA; ++t) s[t] = __uint_as_float(key_bits(k[c][t]));
+            res[c] = window_mean<THETA, BETA>(s);
+        }
+        if (V == 4 && whole) {
+            *reinterpret_cast<float4*>(out + j) = make_float4(res[0], res[V > 1 ? 1 : 0], res[V > 2 ? 2 : 0], res[V > 3 ? 3 : 0]);
+        } else if (V == 2 && whole) {
+            *reinterpret_cast<float2*>(out + j) = make_float2(res[0], res[V > 1 ? 1 : 0]);
+        } else {
+#pragma unroll
+            for (int c = 0; c < V; ++c)
+                if (j + c < d) out[j + c] = res[c];
+        }
     }
 }
+
 
 // run-time theta: insertion sort in local memory, explicit window growth
 __global__ void __launch_bounds__(128) trimmed_mean_generic_kernel(const float* __restrict__ v, int64_t d, int64_t ld,
@@ -377,9 +418,17 @@ int mean_rows_on_device(const float* v, int64_t d, int64_t ld, const int32_t* se
 
 template <int THETA, int BETA>
 int launch_trimmed(const float* v, int64_t d, int64_t ld, const int32_t* selected, float* out, cudaStream_t s) {
-    int64_t grid = (d + 127) / 128;
+    // widest loads the layout allows; four coordinates per thread only while their keys fit the registers
+    const uintptr_t bits = reinterpret_cast<uintptr_t>(v) | reinterpret_cast<uintptr_t>(out) | static_cast<uintptr_t>(ld * 4);
+    const int width = (THETA <= 25 && bits % 16 == 0) ? 4 : (bits % 8 == 0 ? 2 : 1);
+    int64_t grid = ((d + width - 1) / width + 127) / 128;
     if (grid > kNumSMs * 16) grid = kNumSMs * 16;
-    trimmed_mean_kernel<THETA, BETA><<<static_cast<int>(grid), 128, 0, s>>>(v, d, ld, selected, out);
+    if (width == 4)
+        trimmed_mean_kernel<THETA, BETA, (THETA <= 25 ? 4 : 2)><<<static_cast<int>(grid), 128, 0, s>>>(v, d, ld, selected, out);
+    else if (width == 2)
+        trimmed_mean_kernel<THETA, BETA, 2><<<static_cast<int>(grid), 128, 0, s>>>(v, d, ld, selected, out);
+    else
+        trimmed_mean_kernel<THETA, BETA, 1><<<static_cast<int>(grid), 128, 0, s>>>(v, d, ld, selected, out);
     note_launch();
     return check_launch();
 }

@@ -34,7 +34,7 @@ __global__ void __launch_bounds__(kThreads)
     vote_median_tma_kernel(const __grid_constant__ CUtensorMap map, int64_t d, float* __restrict__ out,
                            const ModelUpdate upd) {
     using S = Shape<R, F, FC>;
-    constexpr bool kMixPipes = (R == 1);
+    constexpr bool kMixPipes = (R == 1) || (R == 5 && F == 49);  // where the ALU pipe limits the kernel (measured)
     extern __shared__ __align__(128) unsigned char smem_raw[];
     float* stages = reinterpret_cast<float*>(smem_raw);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + static_cast<size_t>(STAGES) * S::kStageBytes);
@@ -115,7 +115,6 @@ __global__ void __launch_bounds__(kThreads)
                 if ((tid & 31) == 0) mbar_arrive(&empty[s]);  // this warp is done reading the stage
             }
             if (alive && j < d) {
-                // the median of given rows (R = 1) is bound by the ALU pipe: spread its comparators over two pipes
                 const float med = __uint_as_float(key_bits(MedianNet<F>::template run<kMixPipes>(key)));
                 if (out != nullptr) out[j] = med;
                 if (has_w) {

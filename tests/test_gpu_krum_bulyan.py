@@ -134,6 +134,34 @@ def test_trimmed_mean_parity(theta, beta):
     assert np.array_equal(got.cpu().numpy(), want)
 
 
+@pytest.mark.parametrize("theta,beta", [(17, 9), (23, 21), (39, 29), (49, 49)])
+@pytest.mark.parametrize("d,ld,shift,out_shift", [
+    (4100, 4100, 0, 0),   # 16-byte aligned rows: four coordinates per thread for theta <= 25
+    (4099, 4100, 0, 0),   # ... with three coordinates left for the last group
+    (4098, 4098, 0, 0),   # 8-byte aligned rows: two coordinates per thread
+    (4097, 4100, 0, 0),   # odd d in even rows: the last group holds one coordinate
+    (4097, 4100, 1, 0),   # rows start 4 bytes off: one coordinate per thread
+    (4098, 4100, 0, 1),   # output 4 bytes off
+    (4098, 4100, 2, 2),   # rows and output 8 bytes off
+    (1, 2, 0, 0), (2, 2, 0, 0), (3, 4, 0, 0),
+])
+def test_trimmed_mean_layouts(theta, beta, d, ld, shift, out_shift):
+    rng = np.random.default_rng(theta * 1000 + d + shift)
+    f = 49
+    v = rng.standard_normal((f, d)).astype(np.float32)
+    v[:, : d // 3] = np.round(v[:, : d // 3] * 2) / 2
+    sel = rng.permutation(f)[:theta].astype(np.int32)
+    want = oracle.trimmed_mean(v, sel, beta)
+    buf = torch.full((f * ld + 8,), float("nan"), dtype=torch.float32, device=DEV)
+    rows = buf[shift: shift + f * ld].view(f, ld)[:, :d]
+    rows.copy_(torch.from_numpy(v))
+    out_buf = torch.full((d + 4,), -7.0, dtype=torch.float32, device=DEV)
+    out = out_buf[out_shift: out_shift + d]
+    bz.trimmed_mean(rows, torch.from_numpy(sel).to(DEV), beta, out=out)
+    assert np.array_equal(out.cpu().numpy(), want)
+    assert (out_buf[:out_shift] == -7.0).all() and (out_buf[out_shift + d:] == -7.0).all()
+
+
 def test_preconditions_reported():
     v = torch.zeros((25, 16), dtype=torch.float32, device=DEV)
     with pytest.raises(bz.BzError) as e:
