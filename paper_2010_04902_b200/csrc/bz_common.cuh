@@ -41,7 +41,8 @@ __device__ __forceinline__ int kmax(int a, int b) { return max(a, b); }
 // comparator network.  max = a + b - min (exact modulo 2^32) as two integer multiply-adds moves one of a
 // comparator's two operations there; the multipliers are read from constant memory so that the compiler
 // cannot fold them into an addition (which would issue on the ALU pipe again).  A loop of comparators alone
-// runs 26 % faster with every other comparator done this way; only kernels bound by the ALU pipe ask for it.
+// runs 26 % faster with every other comparator done this way (the networks mark two of three, since the
+// kernels have other ALU work besides); only kernels bound by the ALU pipe ask for it.
 static __constant__ unsigned int kPipeOne = 1u, kPipeMinusOne = 0xffffffffu;
 #define BZ_CM(a, b)                                                                                               \
     {                                                                                                             \

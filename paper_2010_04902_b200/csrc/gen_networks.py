@@ -148,7 +148,7 @@ def emit():
     lines = [
         "// GENERATED by gen_networks.py - do not edit.  Comparator networks on register arrays:",
         "// BZ_CE(a,b) orders wires a <= b; BZ_LO / BZ_HI keep only the min on a / the max on b.",
-        "// BZ_CM is a BZ_CE that run<true> may compute on the multiply-add pipe (every other full comparator).",
+        "// BZ_CM is a BZ_CE that run<true> computes on the multiply-add pipe (two of three full comparators).",
         "",
     ]
     for n in MEDIAN_SIZES:
@@ -163,7 +163,7 @@ def emit():
         for a, b, na, nb in net:
             if na and nb:
                 full += 1
-                body.append(("BZ_CM(%d,%d)" if full % 2 == 0 else "BZ_CE(%d,%d)") % (a, b))
+                body.append(("BZ_CM(%d,%d)" if full % 3 else "BZ_CE(%d,%d)") % (a, b))
             else:
                 body.append(("BZ_LO(%d,%d)" if na else "BZ_HI(%d,%d)") % (a, b))
         for i in range(0, len(body), 8):

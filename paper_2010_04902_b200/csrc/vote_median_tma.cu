@@ -34,7 +34,7 @@ __global__ void __launch_bounds__(kThreads)
     vote_median_tma_kernel(const __grid_constant__ CUtensorMap map, int64_t d, float* __restrict__ out,
                            const ModelUpdate upd) {
     using S = Shape<R, F, FC>;
-    constexpr bool kMixPipes = (R == 1) || (R == 5 && F == 49);  // where the ALU pipe limits the kernel (measured)
+    constexpr bool kMixPipes = R == 1 || (R == 5 && F == 49);  // where the ALU pipe limits the kernel (measured)
     extern __shared__ __align__(128) unsigned char smem_raw[];
     float* stages = reinterpret_cast<float*>(smem_raw);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + static_cast<size_t>(STAGES) * S::kStageBytes);
