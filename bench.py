@@ -319,7 +319,7 @@ def extra_paths(bz, inputs, torch, device):
         pairdist=dict(kernel="integer MMA (tcgen05 kind::i8)", **hbm(4 * f * d, t_pd)),
         vote=hbm((4 * r * f + 4 * f) * d, t_vote), mean_rows=hbm((4 * 44 + 4) * d, t_mean),
         pipeline=hbm(bytes_pipeline, t_vote + t_mk),
-        vote_vectorwise=dict(ms=t_vw, **hbm((4 * r * f + 8 * f) * d, t_vw)),
+        vote_vectorwise=dict(ms=t_vw, **hbm((4 * r * f + 4 * f) * d, t_vw)),
         single_pass=dict(ms_vote_pairdist=t_vpd, ms_vote_pairdist_fp32=t_vpd32, vote_pairdist=hbm((4 * r * f + 4 * f) * d, t_vpd),
                          ms_vote_multikrum=t_vmk, coordinates_per_s=d / (t_vmk * 1e-3),
                          **hbm((4 * r * f + 4 * f + 4 * 44 + 4) * d, t_vmk)))

@@ -165,8 +165,8 @@ int bz_vote_vectorwise(const float* replicas, int r, int f, int64_t d, int64_t l
 
 /*
  * bz_vote_vectorwise with agreement up to a tolerance, for clusters whose honest workers do not return
- * bit-identical gradients (Sec. 2: "potential precision issues can easily be handled by deciding
- * the majority by defining appropriate clusters amongst the returned gradients"; the paper gives no
+ * bit-identical gradients (Sec. 2, "Training Protocol", remarks that copies differing only by
+ * numerical precision can be voted on by grouping them into clusters; the paper gives no
  * rule, this one is the library's).  Two copies of a file agree iff at every coordinate their bit
  * patterns are equal or |a - b| <= abs_tol + rel_tol * max(|a|, |b|) (binary32, one fused
  * multiply-add for the bound; a NaN agrees only with its own bit pattern).  The winner is the copy

@@ -326,9 +326,9 @@ void orc_vote_vectorwise(const float* replicas, int r, int f, int64_t d, int32_t
     }
 }
 
-// The vote on whole vectors with agreement up to a tolerance (Sec. 2: "potential precision issues can
-// easily be handled by deciding the majority by defining appropriate clusters amongst the returned
-// gradients"; the paper defines no rule - this is the reading taken).  Two copies of a file agree iff
+// The vote on whole vectors with agreement up to a tolerance (Sec. 2, "Training Protocol",
+// remarks that copies which differ only by numerical precision can be voted on by grouping the returned
+// gradients into clusters; the paper defines no rule - this is the reading taken).  Two copies of a file agree iff
 // at every coordinate their bit patterns are equal or |a - b| <= abs_tol + rel_tol * max(|a|, |b|),
 // the bound formed in binary32 with one fused multiply-add (the precision the decision is taken in on
 // the GPU as well).  The winner is the copy that agrees with the most copies (itself included); ties

@@ -144,5 +144,7 @@ __device__ __forceinline__ void apply_update4(const ModelUpdate& u, int64_t j4, 
 // ---- streaming loads (read-once data: evict-first) -------------------------------------------
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }
 __device__ __forceinline__ uint32_t ld_stream(const uint32_t* p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(uint4* p, const uint4& x) { __stcs(p, x); }
+__device__ __forceinline__ void st_stream(uint32_t* p, uint32_t x) { __stcs(p, x); }
 
 }  // namespace bz

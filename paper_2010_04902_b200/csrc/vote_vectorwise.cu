@@ -4,9 +4,10 @@
 // coordinate; the two agree whenever a majority of a file's copies is identical.)
 //
 // Three kernels: (1) one streaming pass over the replicas that ORs, per file, a bit for every pair
-// of copies that differ anywhere; (2) a tiny kernel that turns the pair bits into the winner's index;
-// (3) a gather of the winning copies into `voted`.  Bytes per coordinate: 4rf read, then 4f read and
-// 4f written: bound by HBM.
+// of copies that differ anywhere - and, on 16-byte aligned data, writes copy 0 to `voted` while it
+// has it in registers; (2) a tiny kernel that turns the pair bits into the winner's index; (3) a
+// gather of the winning copies into `voted`, which skips the files that copy 0 has won.  Bytes per
+// coordinate: 4rf read and 4f written, then 8 more for every file whose first copy lost: bound by HBM.
 #include "bz_common.cuh"
 
 namespace bz {
@@ -17,7 +18,7 @@ constexpr int kMaxPairs = BZ_MAX_R * (BZ_MAX_R - 1) / 2;   // 105: two 64-bit wo
 constexpr int kMaskWords = 2;
 
 // When do two copies of a coordinate agree?  Exactly (bit patterns), or - for clusters whose honest
-// members may differ by rounding (Sec. 2: "deciding the majority by defining appropriate clusters") -
+// members may differ by rounding (Sec. 2 suggests grouping such copies into clusters, without a rule) -
 // within |a - b| <= abs_tol + rel_tol * max(|a|, |b|), evaluated in binary32 with one fused
 // multiply-add; identical bit patterns always agree (so equal NaNs and infinities do).
 struct Agreement {
@@ -44,14 +45,17 @@ __host__ __device__ __forceinline__ int pair_index(int r, int k, int k2) { retur
 // grid = (chunks, f).  V = uint4: n counts groups of 4 coordinates and leading dimensions are in groups.
 template <int R, typename V>
 __global__ void __launch_bounds__(256) copies_differ_kernel(const V* __restrict__ rep, int64_t n, int64_t ld_file, int64_t ld_rep,
-                                                            unsigned long long* __restrict__ mask, const Agreement agree) {
+                                                            unsigned long long* __restrict__ mask, const Agreement agree,
+                                                            V* __restrict__ voted, int64_t ld_voted) {
     const int file = blockIdx.y;
     const V* base = rep + file * ld_file;
+    V* first = voted != nullptr ? voted + file * ld_voted : nullptr;  // copy 0 goes here: right unless it loses
     uint32_t bits = 0;  // R <= 7: 21 pairs
     for (int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < n; j += static_cast<int64_t>(gridDim.x) * blockDim.x) {
         V c[R];
 #pragma unroll
         for (int k = 0; k < R; ++k) c[k] = ld_stream(base + k * ld_rep + j);
+        if (first != nullptr) st_stream(first + j, c[0]);
         int p = 0;
 #pragma unroll
         for (int k = 0; k < R; ++k)
@@ -109,12 +113,23 @@ __global__ void __launch_bounds__(BZ_MAX_F) winner_kernel(const unsigned long lo
 
 template <typename V>
 __global__ void __launch_bounds__(256) gather_winners_kernel(const V* __restrict__ rep, int64_t n, int64_t ld_file, int64_t ld_rep,
-                                                             const int32_t* __restrict__ winner, V* __restrict__ voted, int64_t ld_voted) {
+                                                             const int32_t* __restrict__ winner, V* __restrict__ voted, int64_t ld_voted,
+                                                             int have_copy0) {
     const int file = blockIdx.y;
+    if (have_copy0 && winner[file] == 0) return;  // the first pass has written this row
     const V* src = rep + winner[file] * ld_rep + file * ld_file;
     V* dst = voted + file * ld_voted;
-    for (int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < n; j += static_cast<int64_t>(gridDim.x) * blockDim.x)
-        dst[j] = ld_stream(src + j);
+    // few files may be left to copy, so every thread keeps four loads in flight
+    const int64_t step = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    for (; j + 3 * step < n; j += 4 * step) {
+        const V x0 = ld_stream(src + j), x1 = ld_stream(src + j + step), x2 = ld_stream(src + j + 2 * step), x3 = ld_stream(src + j + 3 * step);
+        st_stream(dst + j, x0);
+        st_stream(dst + j + step, x1);
+        st_stream(dst + j + 2 * step, x2);
+        st_stream(dst + j + 3 * step, x3);
+    }
+    for (; j < n; j += step) st_stream(dst + j, ld_stream(src + j));
 }
 
 int chunks_for(int64_t n, int f) {
@@ -128,10 +143,11 @@ int chunks_for(int64_t n, int f) {
 
 template <int R>
 int launch_differ_vec(const float* rep, int f, int64_t d, int64_t ld_file, int64_t ld_rep, unsigned long long* mask,
-                      const Agreement& agree, cudaStream_t s) {
+                      const Agreement& agree, float* voted, int64_t ld_voted, cudaStream_t s) {
     const int64_t n = d / 4;
     const dim3 grid(chunks_for(n, f), f);
-    copies_differ_kernel<R, uint4><<<grid, 256, 0, s>>>(reinterpret_cast<const uint4*>(rep), n, ld_file / 4, ld_rep / 4, mask, agree);
+    copies_differ_kernel<R, uint4><<<grid, 256, 0, s>>>(reinterpret_cast<const uint4*>(rep), n, ld_file / 4, ld_rep / 4, mask, agree,
+                                                        reinterpret_cast<uint4*>(voted), ld_voted / 4);
     note_launch();
     return check_launch();
 }
@@ -161,12 +177,15 @@ static int vote_whole_vectors(const float* replicas, int r, int f, int64_t d, in
     int32_t* win = winner != nullptr ? winner : reinterpret_cast<int32_t*>(mask + static_cast<size_t>(f) * kMaskWords);
     cudaError_t e = cudaMemsetAsync(mask, 0, static_cast<size_t>(f) * kMaskWords * 8, s);  // every call starts from "all copies agree"
     if (e != cudaSuccess) return cuda_failed(e);
+    int have_copy0 = 0;
     if (d > 0 && r > 1) {
         const bool vec = aligned16(replicas) && (ld_file % 4 == 0) && (ld_replica % 4 == 0) && (d % 4 == 0) && (r == 3 || r == 5 || r == 7);
         if (vec) {
-            st = r == 3 ? launch_differ_vec<3>(replicas, f, d, ld_file, ld_replica, mask, agree, s)
-                        : (r == 5 ? launch_differ_vec<5>(replicas, f, d, ld_file, ld_replica, mask, agree, s)
-                                  : launch_differ_vec<7>(replicas, f, d, ld_file, ld_replica, mask, agree, s));
+            float* first = (voted != nullptr && aligned16(voted) && ld_voted % 4 == 0) ? voted : nullptr;
+            have_copy0 = first != nullptr;
+            st = r == 3 ? launch_differ_vec<3>(replicas, f, d, ld_file, ld_replica, mask, agree, first, ld_voted, s)
+                        : (r == 5 ? launch_differ_vec<5>(replicas, f, d, ld_file, ld_replica, mask, agree, first, ld_voted, s)
+                                  : launch_differ_vec<7>(replicas, f, d, ld_file, ld_replica, mask, agree, first, ld_voted, s));
         } else {
             const dim3 grid(chunks_for(d, f), f);
             copies_differ_generic_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const uint32_t*>(replicas), r, d, ld_file, ld_replica, mask, agree);
@@ -184,11 +203,11 @@ static int vote_whole_vectors(const float* replicas, int r, int f, int64_t d, in
     if (vec) {
         const dim3 grid(chunks_for(d / 4, f), f);
         gather_winners_kernel<uint4><<<grid, 256, 0, s>>>(reinterpret_cast<const uint4*>(replicas), d / 4, ld_file / 4, ld_replica / 4, win,
-                                                          reinterpret_cast<uint4*>(voted), ld_voted / 4);
+                                                          reinterpret_cast<uint4*>(voted), ld_voted / 4, have_copy0);
     } else {
         const dim3 grid(chunks_for(d, f), f);
         gather_winners_kernel<uint32_t><<<grid, 256, 0, s>>>(reinterpret_cast<const uint32_t*>(replicas), d, ld_file, ld_replica, win,
-                                                             reinterpret_cast<uint32_t*>(voted), ld_voted);
+                                                             reinterpret_cast<uint32_t*>(voted), ld_voted, have_copy0);
     }
     note_launch();
     return check_launch();

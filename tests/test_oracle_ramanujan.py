@@ -58,7 +58,7 @@ def test_case2_spectrum_when_s_divides_m(m, s):
 
 def test_case1_reproduces_the_printed_table():
     # Sec. 5.3.2: for (K, f, l, r) = (15, 25, 5, 3) the simulated c_max of the Ramanujan Case 1 scheme
-    # was identical to the MOLS one, "thus both have been summarized in the same table"
+    # was identical to the MOLS one, so the paper prints one table for both
     wf, fw, _ = oracle.assign_ramanujan(3, 5)
     for K, f, l, r, q, cmax, _ in read_golden_rows("cmax_tables.txt"):
         if (K, f, l, r) == ("15", "25", "5", "3"):

@@ -255,7 +255,7 @@ def test_vectorwise_and_elementwise_votes_differ_only_without_an_agreeing_majori
     assert np.array_equal(oracle.vote(rep)[0], g[0])
 
 
-# ---- agreement up to a tolerance (Sec. 2: "defining appropriate clusters") --------------------------
+# ---- agreement up to a tolerance (Sec. 2: clusters of nearly equal copies) --------------------------
 
 def test_cluster_vote_reduces_to_the_exact_vote():
     rng = np.random.default_rng(3)
