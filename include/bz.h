@@ -274,6 +274,8 @@ int bz_bulyan_select(const double* dist, int f, int c, int32_t* selected, void* 
  * total order) are averaged.  Closeness is |v - median| in binary32; the window grows from the
  * median outward, ties go to the lower side; the mean is a binary64 sum in ascending order
  * divided by beta, rounded once.   1 <= beta <= theta <= f.
+ *   Any alignment works; rows and out that are 16-byte (8-byte) aligned, with ld a multiple of 4 (2),
+ *   are read with 128-bit (64-bit) loads.
  */
 int bz_trimmed_mean(const float* voted, int f, int64_t d, int64_t ld, const int32_t* selected, int theta,
                     int beta, float* out, void* stream);
