@@ -38,12 +38,29 @@ __device__ __forceinline__ bool differ(const uint4& a, const uint4& b, const Agr
     return differ1(a.x, b.x, g) || differ1(a.y, b.y, g) || differ1(a.z, b.z, g) || differ1(a.w, b.w, g);
 }
 __device__ __forceinline__ bool differ(uint32_t a, uint32_t b, const Agreement& g) { return differ1(a, b, g); }
+// the same test out of line: the streaming kernel calls it only for pairs that its quick test could not pass
+__device__ __noinline__ bool differ_exactly(const uint4 a, const uint4 b, const Agreement g) { return differ(a, b, g); }
+__device__ __noinline__ bool differ_exactly(const uint32_t a, const uint32_t b, const Agreement g) { return differ1(a, b, g); }
+
+// the smaller of a and b; a NaN in either comes through
+__device__ __forceinline__ float min_nan(float a, float b) {
+    float m;
+    asm("min.NaN.f32 %0, %1, %2;" : "=f"(m) : "f"(a), "f"(b));
+    return m;
+}
+__device__ __forceinline__ void unpack(const uint4& v, float (&o)[4]) {
+    o[0] = __uint_as_float(v.x);
+    o[1] = __uint_as_float(v.y);
+    o[2] = __uint_as_float(v.z);
+    o[3] = __uint_as_float(v.w);
+}
+__device__ __forceinline__ void unpack(uint32_t v, float (&o)[1]) { o[0] = __uint_as_float(v); }
 
 // pair (k, k2), k < k2, -> bit index, row-major over the strict upper triangle
 __host__ __device__ __forceinline__ int pair_index(int r, int k, int k2) { return k * r - k * (k + 1) / 2 + (k2 - k - 1); }
 
 // grid = (chunks, f).  V = uint4: n counts groups of 4 coordinates and leading dimensions are in groups.
-template <int R, typename V>
+template <int R, typename V, bool EXACT>
 __global__ void __launch_bounds__(256) copies_differ_kernel(const V* __restrict__ rep, int64_t n, int64_t ld_file, int64_t ld_rep,
                                                             unsigned long long* __restrict__ mask, const Agreement agree,
                                                             V* __restrict__ voted, int64_t ld_voted) {
@@ -51,16 +68,47 @@ __global__ void __launch_bounds__(256) copies_differ_kernel(const V* __restrict_
     const V* base = rep + file * ld_file;
     V* first = voted != nullptr ? voted + file * ld_voted : nullptr;  // copy 0 goes here: right unless it loses
     uint32_t bits = 0;  // R <= 7: 21 pairs
+#pragma unroll 2
     for (int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < n; j += static_cast<int64_t>(gridDim.x) * blockDim.x) {
         V c[R];
 #pragma unroll
         for (int k = 0; k < R; ++k) c[k] = ld_stream(base + k * ld_rep + j);
         if (first != nullptr) st_stream(first + j, c[0]);
         int p = 0;
+        if constexpr (EXACT) {
 #pragma unroll
-        for (int k = 0; k < R; ++k)
+            for (int k = 0; k < R; ++k)
 #pragma unroll
-            for (int k2 = k + 1; k2 < R; ++k2, ++p) bits |= differ(c[k], c[k2], agree) ? (1u << p) : 0u;
+                for (int k2 = k + 1; k2 < R; ++k2, ++p) bits |= differ(c[k], c[k2], agree) ? (1u << p) : 0u;
+        } else {
+            // The bound abs_tol + rel_tol*max(|a|, |b|) is the larger of the two copies' own bounds (the
+            // multiply-add is monotone in |a|), so each copy's bound is formed once.  A pair passes at once
+            // if its smallest margin bound - |a - b| is >= 0; anything else (a real difference, or NaN /
+            // infinities, whose margin is NaN) goes to the exact test.  A pair this thread has already
+            // seen differ is not looked at again.
+            constexpr int VE = sizeof(V) / 4;
+            float x[R][VE], bound[R][VE];
+#pragma unroll
+            for (int k = 0; k < R; ++k) {
+                unpack(c[k], x[k]);
+#pragma unroll
+                for (int e = 0; e < VE; ++e) {
+                    bound[k][e] = __fmaf_rn(agree.rel_tol, fabsf(x[k][e]), agree.abs_tol);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < R; ++k)
+#pragma unroll
+                for (int k2 = k + 1; k2 < R; ++k2, ++p) {
+                    if (((bits >> p) & 1u) == 0) {
+                        float least = __int_as_float(0x7f800000);
+#pragma unroll
+                        for (int e = 0; e < VE; ++e)
+                            least = min_nan(least, __fsub_rn(fmaxf(bound[k][e], bound[k2][e]), fabsf(__fsub_rn(x[k][e], x[k2][e]))));
+                        if (!(least >= 0.f) && differ_exactly(c[k], c[k2], agree)) bits |= 1u << p;
+                    }
+                }
+        }
     }
     bits = __reduce_or_sync(0xffffffffu, bits);
     if ((threadIdx.x & 31) == 0 && bits != 0) atomicOr(&mask[file * kMaskWords], static_cast<unsigned long long>(bits));
@@ -146,8 +194,12 @@ int launch_differ_vec(const float* rep, int f, int64_t d, int64_t ld_file, int64
                       const Agreement& agree, float* voted, int64_t ld_voted, cudaStream_t s) {
     const int64_t n = d / 4;
     const dim3 grid(chunks_for(n, f), f);
-    copies_differ_kernel<R, uint4><<<grid, 256, 0, s>>>(reinterpret_cast<const uint4*>(rep), n, ld_file / 4, ld_rep / 4, mask, agree,
-                                                        reinterpret_cast<uint4*>(voted), ld_voted / 4);
+    if (agree.exact)
+        copies_differ_kernel<R, uint4, true><<<grid, 256, 0, s>>>(reinterpret_cast<const uint4*>(rep), n, ld_file / 4, ld_rep / 4, mask, agree,
+                                                                  reinterpret_cast<uint4*>(voted), ld_voted / 4);
+    else
+        copies_differ_kernel<R, uint4, false><<<grid, 256, 0, s>>>(reinterpret_cast<const uint4*>(rep), n, ld_file / 4, ld_rep / 4, mask, agree,
+                                                                   reinterpret_cast<uint4*>(voted), ld_voted / 4);
     note_launch();
     return check_launch();
 }

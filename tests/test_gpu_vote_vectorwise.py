@@ -165,3 +165,29 @@ def test_cluster_vote_edge_values_and_generic_r():
     rep = torch.from_numpy(rep)
     for abs_tol, rel_tol in [(0.25, 0.0), (0.2499, 0.0), (0.0, 2.0 ** -10), (0.0, 2.0 ** -11), (0.1, 0.01)]:
         _check_clusters(rep, abs_tol, rel_tol)
+
+
+@pytest.mark.parametrize("r", [3, 5, 7])
+def test_cluster_vote_edge_values_vector_kernels(r):
+    # the same edge cases through the 128-bit kernels (d a multiple of 4): bound met exactly, one step
+    # beyond it, equal and unequal NaNs, infinities of either sign, signed zeros, one bad coordinate per file
+    rng = np.random.default_rng(90 + r)
+    f, d = 12, 2_048
+    base = rng.standard_normal((f, d)).astype(np.float32)
+    rep = np.repeat(base[None], r, axis=0).copy()
+    rep[1, 0] += np.float32(0.25)                                   # exactly the absolute tolerance away
+    rep[1, 1] = np.nextafter(rep[1, 1] + np.float32(0.25), np.float32(np.inf))   # mostly one step beyond it
+    rep[r - 1, 2] *= np.float32(1.0 + 2.0 ** -10)                   # edge of the relative tolerance
+    rep[0, 3, 17] = np.nan                                          # a NaN in one copy only
+    rep[:, 4, 33] = np.nan                                          # the same NaN everywhere: copies agree
+    rep[0, 5, 5] = np.inf                                           # infinity against finite values
+    rep[:, 6, 6] = np.inf                                           # equal infinities agree
+    rep[0, 7, 7], rep[1:, 7, 7] = np.inf, -np.inf
+    rep[0, 8, 8], rep[1:, 8, 8] = 0.0, -0.0
+    rep[0, 9, 1023] = rep[0, 9, 1023] + np.float32(1.0)             # one coordinate off in copy 0
+    rep[r // 2, 10, 2047] = np.float32(3e38)                        # the last coordinate of the middle copy
+    rep[:, 11] = 0.0                                                # all zero
+    rep = torch.from_numpy(rep)
+    for abs_tol, rel_tol in [(0.25, 0.0), (0.2499, 0.0), (0.0, 2.0 ** -10), (0.0, 2.0 ** -11), (0.1, 0.01), (0.0, 0.0),
+                             (1e30, 0.0), (0.0, 1.0)]:
+        _check_clusters(rep, abs_tol, rel_tol)
