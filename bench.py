@@ -30,7 +30,7 @@ WORKLOAD = dict(l=5, r=3, q=3, d=11_200_000, attack="reversed", seed=0)
 
 # DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum, scaled to a full launch), or None when no capture of the current kernel exists.
-TRAFFIC_BYTES_PER_LAUNCH = 3_429_614_000  # (600.03 + 12.40) MB at d = 2 M, scaled by 5.6 to d = 11.2 M
+TRAFFIC_BYTES_PER_LAUNCH = 3_420_054_000  # (600.02 + 10.70) MB at d = 2 M, scaled by 5.6 to d = 11.2 M
 
 
 def workload_name(cfg):
