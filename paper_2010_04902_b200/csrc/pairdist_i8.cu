@@ -182,11 +182,13 @@ int vote_pairdist_i8(const float* rep, int r, int f, int64_t d, int64_t ld_file,
 #define BZ_I8_CASE(R_, F_, W_, FC_, NS_, TS_) \
     if (r == R_ && f == F_)                   \
         return launch_i8<F_, W_, R_, FC_, NS_, TS_>(rep, d, ld_file, ld_rep, voted, ld_voted, dist, sc.tpart, sc.info, sc.flag, force, s);
+    // with the copies in front the kernel is bound by HBM: where shared memory forces the choice, a third box in
+    // flight is worth more than a second tile per step (r = 3, f = 49: 1.45 -> 1.32 ms; r = 7: 2.95 -> 2.65 ms)
     BZ_I8_CASE(3, 25, 25, 25, 3, 2)
-    BZ_I8_CASE(3, 49, 25, 25, 2, 2)
+    BZ_I8_CASE(3, 49, 25, 25, 3, 1)
     BZ_I8_CASE(5, 25, 25, 25, 2, 2)
     BZ_I8_CASE(5, 49, 25, 25, 2, 1)
-    BZ_I8_CASE(7, 49, 13, 13, 2, 1)
+    BZ_I8_CASE(7, 49, 13, 13, 3, 1)
 #undef BZ_I8_CASE
     return 1;
 }

@@ -145,7 +145,11 @@ def test_full_size_on_sampled_rows():
     for got in (dist, alone):
         sub = got.cpu().numpy()[np.ix_(rows, rows)]
         _check_close(sub, want)
-    assert np.array_equal(dist.cpu().numpy(), alone.cpu().numpy())   # same integers either way
+    # the two kernels fix a row's scale per step and their steps differ in size, so a few early tiles are
+    # rounded on different grids: equal far below the tolerance, not bit for bit
+    a, b = dist.cpu().numpy(), alone.cpu().numpy()
+    assert np.array_equal(a == 0, b == 0)
+    assert (np.abs(a - b) <= 1e-10 * np.maximum(a, b)).all()
     assert bz.pipeline_timeouts() == 0
 
 
