@@ -12,8 +12,11 @@
  * Conventions
  *   - "device" pointers are CUDA global-memory addresses of the current device; "host" pointers
  *     are ordinary process memory.  The caller owns every buffer.  The library never allocates
- *     or frees device memory and keeps no device state between calls; scratch space is a
- *     caller-provided device workspace whose size bz_workspace_bytes() reports.
+ *     or frees device memory; scratch space is a caller-provided device workspace whose size
+ *     bz_workspace_bytes() reports.  Device state that outlives a call is limited to what is part
+ *     of the library image: three counters of expired waits (bz_pipeline_timeouts), the switch of
+ *     bz_debug_stall_pipeline and the built-in array of bz_pairdist_static.  None of it
+ *     influences a result.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls with
  *     device outputs only enqueue work on that stream and return; outputs are valid once the
  *     caller has synchronised it.  Calls with host outputs synchronise the stream themselves.
@@ -39,7 +42,7 @@ extern "C" {
 #endif
 
 #define BZ_OK 0
-#define BZ_ERR_INVALID_ARG (-1)  /* null pointer, size out of range, r even, l not prime, r > l ... */
+#define BZ_ERR_INVALID_ARG (-1)  /* null pointer, size out of range, r even, l no prime power, r > l */
 #define BZ_ERR_UNSUPPORTED (-2)  /* a shape outside the compiled limits                              */
 #define BZ_ERR_PRECONDITION (-3) /* f < 2c+3 (Multi-Krum) or f < 4c+3 (Bulyan), m outside [1, f]     */
 #define BZ_ERR_WORKSPACE (-4)    /* workspace missing, misaligned (256 B) or too small               */
@@ -110,6 +113,10 @@ int bz_median(const float* voted, int f, int64_t d, int64_t ld, float* out, void
 /*
  * ByzShield's aggregation in one pass: bz_median(bz_vote(replicas)) without materialising the
  * voted gradients.  Reads 4*r*f bytes and writes 4 bytes per coordinate.
+ * The staged kernel behind this call (and behind bz_median and bz_vote_median_update) bounds its
+ * waits; should one run out, the kernel stops and part of `out` (of w and velocity) is left
+ * unwritten while the call has long returned BZ_OK.  bz_pipeline_timeouts() is how a caller
+ * learns of it: the counter has moved.  It never has on a healthy device.
  */
 int bz_vote_median(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica,
                    float* out, void* stream);
@@ -205,11 +212,34 @@ int bz_vote_median_host(const float* replicas_host, int r, int f, int64_t d, flo
  *     terms) and in binary64 across blocks, in a fixed order.
  * Environment: BZ_PAIRDIST_PATH=fp32 keeps every call on the second kernel; =i8 takes the first
  * kernel's result whatever its estimate says (for testing it); read at every call.
+ * With =i8 the second kernel still answers for rows the fixed point cannot hold and after a
+ * kernel that stopped early (below).
+ * The tensor-core kernel bounds every wait.  If one runs out the kernel stops early, says so in
+ * the workspace, and the second kernel recomputes the whole matrix on the same stream: the result
+ * is complete either way, bz_pairdist_status() reports what happened and bz_pipeline_timeouts()
+ * counts it.
  *   dist  device, double [f][f], symmetric with a zero diagonal; identical rows give exactly 0.
  *   workspace  device, bz_workspace_bytes(BZ_OP_PAIRDIST, 0, f, d, 0, 0) bytes, 256-byte aligned.
  */
 int bz_pairdist(const float* voted, int f, int64_t d, int64_t ld, double* dist, void* workspace,
                 size_t workspace_bytes, void* stream);
+
+/*
+ * What the distance stage of the last call that used `workspace` did (bz_pairdist, bz_multikrum,
+ * bz_bulyan, bz_vote_pairdist, bz_vote_multikrum, bz_vote_bulyan with the same f).  Synchronises
+ * `stream`, then writes a combination of the bits below to *status (host):
+ *   BZ_STATUS_RECOMPUTED     the binary32 kernel's distances were returned although the tensor-core
+ *                            kernel ran (its error estimate, values without a fixed-point scale,
+ *                            or an early stop asked for it)
+ *   BZ_STATUS_STOPPED_EARLY  a bounded wait of the tensor-core kernel ran out; its distances were
+ *                            recomputed and, in the calls that vote first, the voted rows were
+ *                            rebuilt by the vote kernel.  Outputs are complete and correct, the
+ *                            call was slow; a device that does this is not healthy.
+ * 0 when the tensor-core kernel's result stands or that kernel did not run.
+ */
+#define BZ_STATUS_RECOMPUTED 1
+#define BZ_STATUS_STOPPED_EARLY 2
+int bz_pairdist_status(const void* workspace, int f, int32_t* status, void* stream);
 
 /*
  * bz_pairdist for callers that have no device workspace to offer and may not allocate one.
@@ -226,7 +256,9 @@ int bz_pairdist(const float* voted, int f, int64_t d, int64_t ld, double* dist, 
  *     array are refused with BZ_ERR_STATIC_LIMIT before anything runs: f = 25 (0.9 MB) and f = 49
  *     (1.6 MB) fit, any other f fits up to 84; f from 85 to BZ_MAX_F is refused.
  *   - The first call on each device looks up the array's device address (the device must be
- *     current, as for every call).  Make that first call outside any stream capture.
+ *     current, as for every call).  Make that first call outside any stream capture.  The
+ *     address is kept per device for the life of the process: after cudaDeviceReset() on a
+ *     device this entry point must not be used on it again.
  *   - All calls share the one array and it keeps the previous call's contents.  The kernels
  *     overwrite or clear every element before reading it, so successive calls on one stream are
  *     independent; two calls that overlap on the GPU (different streams, several host threads)
@@ -295,6 +327,11 @@ int bz_bulyan(const float* voted, int f, int64_t d, int64_t ld, int c, float* ou
  * and 7 x 49: the vote runs in front of the tensor-core kernel, with the same estimate and fall-back;
  * BZ_PAIRDIST_PATH=fp32 puts it in front of the binary32 kernel instead).  Shapes without a fused
  * kernel (r*f outside {3,5}x{25,49} and 7x49, unaligned or short arrays) run the two calls.
+ * Should a bounded wait of the single-pass kernel run out, `voted` and `dist` are incomplete when
+ * that kernel ends; the call has already enqueued the repair behind it (bz_vote's kernel, then the
+ * binary32 distances; both return at once when there is nothing to repair), so outputs are
+ * complete once the stream is synchronised.  bz_pairdist_status() and bz_pipeline_timeouts() tell.
+ * The same holds for bz_vote_multikrum and bz_vote_bulyan, which start with this call.
  *   replicas, ld_file, ld_replica as bz_vote;  voted device [f][d] with ld_voted (written);
  *   dist device double [f][f];  workspace as bz_pairdist.
  */
@@ -362,6 +399,34 @@ const char* bz_last_cuda_error(void);
  * counter (synchronously; 0 after any number of healthy launches) into *count (host).
  */
 int bz_pipeline_timeouts(unsigned int* count);
+
+/*
+ * Testing aid for the recovery described at bz_pairdist: while `on` is not 0, the loader threads of
+ * the tensor-core distance kernels (given rows and vote in front) issue no loads, so that every
+ * CTA's first bounded wait runs out after about a second and the call takes its repair path.
+ * Nothing faults or hangs.  Off when the library is loaded; a per-device switch (the current
+ * device's is set); not for production use.  Synchronous.
+ */
+int bz_debug_stall_pipeline(int on);
+
+/*
+ * Which kernel family the calling thread's last call dispatched to (vote, median, fused pass,
+ * distances and the calls built on them); for tests and tuning, results never depend on it.
+ *   BZ_PATH_STAGED      vote / median kernels fed by the TMA unit through shared memory
+ *   BZ_PATH_REGISTERS   the same arithmetic with loads straight into registers (any alignment)
+ *   BZ_PATH_GENERIC     run-time (r, f) kernels for shapes without a specialisation
+ *   BZ_PATH_TENSOR      integer distances on the tensor cores (the binary32 kernel queued behind them)
+ *   BZ_PATH_FP32        binary32 difference-form distances
+ *   BZ_PATH_FP32_FUSED  vote and binary32 distances in one pass
+ */
+#define BZ_PATH_NONE 0
+#define BZ_PATH_STAGED 1
+#define BZ_PATH_REGISTERS 2
+#define BZ_PATH_GENERIC 3
+#define BZ_PATH_TENSOR 4
+#define BZ_PATH_FP32 5
+#define BZ_PATH_FP32_FUSED 6
+int bz_last_path(void);
 
 /* Number of kernels this library has launched from the calling process since it was loaded. */
 uint64_t bz_kernel_launch_count(void);

@@ -20,6 +20,8 @@ OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_PRECONDITION, ERR_WORKSPACE, ERR_BUDGET, ERR_CUDA = -1, -2, -3, -4, -5, -6
 OP_PAIRDIST, OP_MULTIKRUM, OP_BULYAN, OP_WORST_CASE, OP_VOTE_MEDIAN_HOST, OP_WORST_CASE_MOLS, OP_VOTE_VECTORWISE = 1, 2, 3, 4, 5, 6, 7
 MAX_R, MAX_F = 15, 128
+STATUS_RECOMPUTED, STATUS_STOPPED_EARLY = 1, 2
+PATH_NONE, PATH_STAGED, PATH_REGISTERS, PATH_GENERIC, PATH_TENSOR, PATH_FP32, PATH_FP32_FUSED = range(7)
 
 
 class BzError(RuntimeError):
@@ -70,6 +72,9 @@ _SIGNATURES = {
     "bz_last_cuda_error": (ctypes.c_char_p, []),
     "bz_kernel_launch_count": (_c_u64, []),
     "bz_pipeline_timeouts": (_c_int, [_c_vp]),
+    "bz_pairdist_status": (_c_int, [_c_vp, _c_int, _c_vp, _c_vp]),
+    "bz_debug_stall_pipeline": (_c_int, [_c_int]),
+    "bz_last_path": (_c_int, []),
 }
 
 EXPORTS = sorted(_SIGNATURES)
@@ -108,6 +113,24 @@ def pipeline_timeouts() -> int:
     n = ctypes.c_uint(0)
     _check(lib().bz_pipeline_timeouts(ctypes.addressof(n)), "bz_pipeline_timeouts")
     return int(n.value)
+
+
+def last_path() -> int:
+    """PATH_* of the kernel family this thread's last call dispatched to."""
+    return int(lib().bz_last_path())
+
+
+def pairdist_status(workspace: torch.Tensor, f: int) -> int:
+    """STATUS_* bits of the distance stage of the last call that used `workspace` (synchronises the stream)."""
+    st = ctypes.c_int32(0)
+    _check(lib().bz_pairdist_status(_dev(workspace, torch.uint8, "workspace"), f, ctypes.addressof(st), _stream()),
+           "bz_pairdist_status")
+    return int(st.value)
+
+
+def debug_stall_pipeline(on: bool) -> None:
+    """Testing aid: make the tensor-core distance kernels' bounded waits run out (see bz.h)."""
+    _check(lib().bz_debug_stall_pipeline(1 if on else 0), "bz_debug_stall_pipeline")
 
 
 def _check(status: int, what: str):
@@ -486,8 +509,9 @@ def vote_pairdist(replicas: torch.Tensor, voted: torch.Tensor | None = None, wor
 
 
 def vote_multikrum(replicas: torch.Tensor, c: int, m: int, voted: torch.Tensor | None = None,
-                   workspace: torch.Tensor | None = None, out: torch.Tensor | None = None):
-    """bz_vote_multikrum: returns (out[d], selected[m], voted[f][d])."""
+                   workspace: torch.Tensor | None = None, out: torch.Tensor | None = None,
+                   dist: torch.Tensor | None = None):
+    """bz_vote_multikrum: returns (out[d], selected[m], voted[f][d]); the distance matrix goes to `dist` if given."""
     r, f, d, ld_file, ld_rep, voted, ld_v = _voted_for(replicas, voted)
     ws = workspace if workspace is not None else alloc_workspace(OP_MULTIKRUM, 0, f, d, c, m, device=replicas.device)
     if out is None:
@@ -495,7 +519,8 @@ def vote_multikrum(replicas: torch.Tensor, c: int, m: int, voted: torch.Tensor |
     sel = torch.empty(max(m, 1), dtype=torch.int32, device=replicas.device)
     st = lib().bz_vote_multikrum(_dev(replicas, torch.float32, "replicas"), r, f, d, ld_file, ld_rep, c, m,
                                  _dev(voted, torch.float32, "voted"), ld_v, _dev(out, torch.float32, "out"),
-                                 sel.data_ptr(), None, ws.data_ptr(), ws.numel(), _stream())
+                                 sel.data_ptr(), None if dist is None else _dev(dist, torch.float64, "dist"),
+                                 ws.data_ptr(), ws.numel(), _stream())
     _check(st, "bz_vote_multikrum")
     return out, sel[:m], voted
 

@@ -15,6 +15,8 @@ size_t vote_vectorwise_workspace(int f);      // vote_vectorwise.cu
 int pipeline_timeouts(unsigned int* count);   // vote_median_tma.cu
 int vote_pairdist_timeouts(unsigned int* count);  // vote_pairdist.cu
 int pairdist_i8_timeouts(unsigned int* count);    // pairdist_i8.cu
+int pairdist_i8_stall(int on);
+int* pairdist_status_words(void* ws, int f);      // pairdist.cu
 
 namespace {
 std::atomic<uint64_t> g_launches{0};
@@ -113,6 +115,9 @@ private:
 }  // namespace
 
 void note_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+thread_local int g_last_path = BZ_PATH_NONE;
+void note_path(int path) { g_last_path = path; }
 
 int cuda_failed(cudaError_t e) {
     std::snprintf(g_cuda_msg, sizeof(g_cuda_msg), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
@@ -245,6 +250,23 @@ extern "C" int bz_pipeline_timeouts(unsigned int* count) {
     *count = a + b + c;
     return st;
 }
+
+extern "C" int bz_pairdist_status(const void* workspace, int f, int32_t* status, void* stream) {
+    if (workspace == nullptr || status == nullptr || f < 1) return BZ_ERR_INVALID_ARG;
+    if (f > BZ_MAX_F) return BZ_ERR_UNSUPPORTED;
+    int words[2] = {0, 0};
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(words, pairdist_status_words(const_cast<void*>(workspace), f), sizeof(words),
+                                    cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_failed(e);
+    *status = (words[0] ? BZ_STATUS_RECOMPUTED : 0) | (words[1] ? BZ_STATUS_STOPPED_EARLY : 0);
+    return BZ_OK;
+}
+
+extern "C" int bz_debug_stall_pipeline(int on) { return pairdist_i8_stall(on); }
+
+extern "C" int bz_last_path(void) { return g_last_path; }
 
 extern "C" const char* bz_last_cuda_error(void) { return g_cuda_msg; }
 

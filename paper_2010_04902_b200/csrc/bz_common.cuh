@@ -14,6 +14,7 @@ constexpr int kNumSMs = 148;  // B200: 2 dies x 74 SMs; grids are sized in multi
 void note_launch();                       // counts one kernel launch
 int cuda_failed(cudaError_t e);           // records the message, returns BZ_ERR_CUDA
 int check_launch();                       // cudaGetLastError() after a launch -> status
+void note_path(int path);                 // which kernel family a call dispatched to (BZ_PATH_*), per host thread
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }

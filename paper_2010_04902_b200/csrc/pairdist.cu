@@ -1,11 +1,14 @@
 // Pairwise squared distances between the f voted gradients - the O(f^2 d) part of the Krum family
-// (Sec. 1.2; cost in Appendix A.1).
+// (Sec. 1.2; cost in Appendix A.1): the binary32 kernels, the dispatch between them and the integer
+// tensor-core kernel (pairdist_i8_kernel.cuh, the default for f = 25 and 49), and the entry point that
+// keeps its scratch in a built-in array.
 //
-// The distances are accumulated in the difference form sum_j (v_a[j] - v_b[j])^2: its accuracy
-// does not depend on a common offset of the rows (gradients share a large per-coordinate mean)
-// nor on the size of an attacker's payload in other rows, which the Gram form |a|^2 + |b|^2 - 2ab
-// - and with it a tensor-core contraction - cannot offer at the precision the selection needs.
-// The work is therefore bound by the FP32 pipe: f(f-1) add/fma lane-operations per coordinate.
+// The kernels here accumulate the difference form sum_j (v_a[j] - v_b[j])^2 in binary32: its accuracy
+// does not depend on a common offset of the rows (gradients share a large per-coordinate mean) nor on
+// the size of an attacker's payload in other rows.  They are bound by the FP32 pipe (f(f-1) add/fma
+// lane-operations per coordinate) and serve every shape the integer kernel does not take, its fall-back
+// when its own error estimate or a row's values ask for one, and bz_pairdist_static.
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
 
@@ -214,7 +217,7 @@ int pairdist_path() {
 
 bool pairdist_i8_has(int f);                  // pairdist_i8.cu
 size_t pairdist_i8_workspace(int f);
-int pairdist_i8(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, int force, int** flag_out, cudaStream_t s);
+int pairdist_i8(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, int* flag, int force, cudaStream_t s);
 
 int pairdist_path_fp32_only() { return pairdist_path() == kPathFp32; }
 int pairdist_path_i8_forced() { return pairdist_path() == kPathI8; }
@@ -232,25 +235,37 @@ size_t pairdist_workspace_fp32(int f) {
     return round_up(doubles * sizeof(double), 256);
 }
 
-// binary32 partial sums, then the integer kernel's partial matrices
-size_t pairdist_workspace(int f) { return pairdist_workspace_fp32(f) + pairdist_i8_workspace(f); }
+// binary32 partial sums, the call's two status words (256 bytes), then the integer kernel's partial matrices
+constexpr size_t kStatusBytes = 256;
+size_t pairdist_workspace(int f) { return pairdist_workspace_fp32(f) + kStatusBytes + pairdist_i8_workspace(f); }
+int* pairdist_status_words(void* ws, int f) { return reinterpret_cast<int*>(static_cast<char*>(ws) + pairdist_workspace_fp32(f)); }
+void* pairdist_i8_part(void* ws, int f) { return static_cast<char*>(ws) + pairdist_workspace_fp32(f) + kStatusBytes; }
+// a call on which the integer kernel does not run clears the status words
+int pairdist_clear_status(void* ws, int f, cudaStream_t s) {
+    const cudaError_t e = cudaMemsetAsync(pairdist_status_words(ws, f), 0, 2 * sizeof(int), s);
+    return e == cudaSuccess ? BZ_OK : cuda_failed(e);
+}
 
 // The binary32 difference-form kernels.  gate != nullptr (only after the integer kernel ran, so on a
 // shape with a tiled kernel): they run only if *gate (device) is not 0.
 int pairdist_fp32(const float* v, int f, int64_t d, int64_t ld, double* dist, double* partial, const int* gate, cudaStream_t s);
 
-// tensor_cores: the workspace has room for the integer kernel (pairdist_workspace, not _fp32)
+// tensor_cores: the workspace has room for the status words and the integer kernel (pairdist_workspace, not _fp32)
 int pairdist_on_device(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, cudaStream_t s, bool tensor_cores) {
     double* partial = static_cast<double*>(ws);
     const int* gate = nullptr;
     const int path = pairdist_path();
-    if (tensor_cores && path != kPathFp32) {
-        int* flag = nullptr;
-        const int st = pairdist_i8(v, f, d, ld, dist, static_cast<char*>(ws) + pairdist_workspace_fp32(f), path == kPathI8, &flag, s);
+    if (tensor_cores) {
+        int* flag = pairdist_status_words(ws, f);
+        int st = 1;
+        if (path != kPathFp32) st = pairdist_i8(v, f, d, ld, dist, pairdist_i8_part(ws, f), flag, path == kPathI8, s);
         if (st == BZ_OK) {
-            if (path == kPathI8) return BZ_OK;
             gate = flag;  // the binary32 kernels below run only if the flag asks for them
-        } else if (st != 1) {
+            note_path(BZ_PATH_TENSOR);
+        } else if (st == 1) {
+            st = pairdist_clear_status(ws, f, s);
+            if (st != BZ_OK) return st;
+        } else {
             return st;
         }
     }
@@ -258,6 +273,7 @@ int pairdist_on_device(const float* v, int f, int64_t d, int64_t ld, double* dis
 }
 
 int pairdist_fp32(const float* v, int f, int64_t d, int64_t ld, double* dist, double* partial, const int* gate, cudaStream_t s) {
+    if (gate == nullptr) note_path(BZ_PATH_FP32);
     const bool vec = aligned16(v) && (ld % 4 == 0);
     if (vec && f == 25) return launch_pairdist_tiled<BZ_PD_25>(v, d, ld, dist, partial, gate, s);
     if (vec && f == 49) return launch_pairdist_tiled<BZ_PD_49>(v, d, ld, dist, partial, gate, s);
@@ -320,7 +336,11 @@ constexpr size_t kStaticScratchBytes = BZ_STATIC_SCRATCH_BYTES;  // 4 MiB
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 constexpr int kMaxDevices = 64;
-void* g_static_scratch_addr[kMaxDevices] = {};  // device address of the array on each device, once resolved
+// device address of the array on each device, once resolved.  Host threads may make a device's first call
+// at the same time: they all store the same address, atomically.  cudaDeviceReset() invalidates the address
+// (the next context maps the image anew); a process that resets a device must not call this entry point on
+// it afterwards.
+std::atomic<void*> g_static_scratch_addr[kMaxDevices];
 
 // The array's name is only a handle on the host side; kernels need its device address, which the
 // runtime hands out per device.
@@ -329,14 +349,14 @@ int static_scratch(void** ptr) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_failed(e);
     if (dev < 0 || dev >= kMaxDevices) return BZ_ERR_UNSUPPORTED;
-    if (g_static_scratch_addr[dev] == nullptr) {
-        void* p = nullptr;
+    void* p = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+    if (p == nullptr) {
         e = cudaGetSymbolAddress(&p, g_static_scratch);
         if (e != cudaSuccess) return cuda_failed(e);
         if (p == nullptr || !aligned256(p)) return BZ_ERR_WORKSPACE;
-        g_static_scratch_addr[dev] = p;
+        g_static_scratch_addr[dev].store(p, std::memory_order_release);
     }
-    *ptr = g_static_scratch_addr[dev];
+    *ptr = p;
     return BZ_OK;
 }
 

@@ -7,8 +7,10 @@ namespace bz {
 namespace {
 
 // D from the CTAs' partial matrices, then the error estimate of the conversion (two small kernels).
-// flag[0] = 1 asks for the binary32 kernel (estimate above the tolerance, or values the fixed-point
-// scale cannot hold); with force != 0 the flag stays 0 whatever the estimate says.
+// flag[0] = 1 asks for the binary32 kernel: the estimate is above the tolerance (ignored with force != 0),
+// a row holds values the fixed-point scale cannot carry, or a CTA stopped early.  flag[1] = 1 says the
+// latter: a bounded wait ran out, the partial matrices are incomplete and so are the voted rows of the
+// kernel with the vote in front.
 // Estimate for a pair: each value is rounded to a multiple of its row's step, an unbiased error of
 // standard deviation 0.29 step; over d coordinates that moves D by about 2 sqrt(D var) + d var.
 constexpr double kRelTol = 5e-9;
@@ -37,21 +39,21 @@ __global__ void __launch_bounds__(256)
     }
 }
 
-// The error estimate.  flag[0] = 1 asks for the binary32 kernel.
+// The error estimate and the CTAs' marks -> flag[0], flag[1].
 template <int F>
 __global__ void __launch_bounds__(256)
     pairdist_i8_check_kernel(const double* __restrict__ dist, const int* __restrict__ info, int n_ctas, int64_t d, int force,
                              int* __restrict__ flag) {
     __shared__ int s_emax[F];
-    __shared__ int s_bad;
+    __shared__ int s_bad, s_marks;
     const int tid = threadIdx.x;
-    if (tid == 0) s_bad = 0;
+    if (tid == 0) s_bad = s_marks = 0;
     if (tid < F) s_emax[tid] = kELo;
     __syncthreads();
     for (int e = tid; e < n_ctas * kInfoStride; e += blockDim.x) {
         const int a = e % kInfoStride;
         if (a < F) atomicMax(&s_emax[a], info[e]);
-        if (a == kInfoBad && info[e]) atomicOr(&s_bad, 1);
+        if (a == kInfoBad && info[e]) atomicOr(&s_marks, info[e]);
     }
     __syncthreads();
     // 2 sqrt(x) + d x <= tol  <=>  x <= x_max with sqrt(x_max) = (sqrt(1 + d tol) - 1) / d: one square root
@@ -92,7 +94,10 @@ __global__ void __launch_bounds__(256)
         dd * s_zero_step[tid] * s_zero_step[tid] > kRelTol * s_min_nz[tid])
         atomicOr(&s_bad, 1);
     __syncthreads();
-    if (tid == 0) flag[0] = (s_bad && !force) ? 1 : 0;
+    if (tid == 0) {
+        flag[0] = ((s_bad && !force) || s_marks) ? 1 : 0;
+        flag[1] = (s_marks & kBadStopped) ? 1 : 0;
+    }
 }
 
 // rep: R = 1: rows [f][d] with leading dimension ld_file.  R > 1: replicas[r][f][d].
@@ -136,7 +141,6 @@ size_t info_bytes() { return round_up(static_cast<size_t>(kNumSMs) * kInfoStride
 struct Scratch {
     double* tpart;
     int* info;
-    int* flag;
 };
 Scratch carve(void* ws, int f) {
     char* p = static_cast<char*>(ws);
@@ -144,8 +148,6 @@ Scratch carve(void* ws, int f) {
     s.tpart = reinterpret_cast<double*>(p);
     p += tpart_bytes(f);
     s.info = reinterpret_cast<int*>(p);
-    p += info_bytes();
-    s.flag = reinterpret_cast<int*>(p);
     return s;
 }
 
@@ -153,35 +155,33 @@ Scratch carve(void* ws, int f) {
 
 bool pairdist_i8_has(int f) { return f == 25 || f == 49; }
 
-// bytes of the partial matrices, the per-CTA records and the flag
+// bytes of the partial matrices and the per-CTA records
 size_t pairdist_i8_workspace(int f) {
     if (!pairdist_i8_has(f)) return 0;
-    return tpart_bytes(f) + info_bytes() + 256;
+    return tpart_bytes(f) + info_bytes();
 }
 
 // Returns BZ_OK / an error, or 1 when this path does not apply (shape, alignment, size).  On BZ_OK
-// dist holds the distances and *flag_out points at the device flag that is 1 if they must be
-// recomputed in binary32.
-int pairdist_i8(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, int force, int** flag_out, cudaStream_t s) {
+// dist holds the distances, flag[0] (device) is 1 if they must be recomputed in binary32 and flag[1] is 1
+// if the kernel stopped early.
+int pairdist_i8(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, int* flag, int force, cudaStream_t s) {
     if (!pairdist_i8_has(f) || !aligned16(v) || (ld % 4) != 0 || d < 64 * kTK || d >= (int64_t(1) << 31)) return 1;
     const Scratch sc = carve(ws, f);
-    *flag_out = sc.flag;
     // <rows, converter warps, copies, rows per box, boxes in the ring, tiles per step>
-    if (f == 25) return launch_i8<25, 25, 1, 25, 6, 4>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
-    return launch_i8<49, 25, 1, 49, 3, 2>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, sc.flag, force, s);
+    if (f == 25) return launch_i8<25, 25, 1, 25, 6, 4>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, flag, force, s);
+    return launch_i8<49, 25, 1, 49, 3, 2>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, flag, force, s);
 }
 
 // The same from the replicas: vote (Eq. 3) and distances in one pass; the winners go to `voted`.
 int vote_pairdist_i8(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted,
-                     double* dist, void* ws, int force, int** flag_out, cudaStream_t s) {
+                     double* dist, void* ws, int* flag, int force, cudaStream_t s) {
     if (!pairdist_i8_has(f) || !aligned16(rep) || !aligned16(voted) || (ld_file % 4) != 0 || (ld_rep % 4) != 0 ||
         (ld_voted % 4) != 0 || d < 64 * kTK || d >= (int64_t(1) << 31))
         return 1;
     const Scratch sc = carve(ws, f);
-    *flag_out = sc.flag;
 #define BZ_I8_CASE(R_, F_, W_, FC_, NS_, TS_) \
     if (r == R_ && f == F_)                   \
-        return launch_i8<F_, W_, R_, FC_, NS_, TS_>(rep, d, ld_file, ld_rep, voted, ld_voted, dist, sc.tpart, sc.info, sc.flag, force, s);
+        return launch_i8<F_, W_, R_, FC_, NS_, TS_>(rep, d, ld_file, ld_rep, voted, ld_voted, dist, sc.tpart, sc.info, flag, force, s);
     // with the copies in front the kernel is bound by HBM: where shared memory forces the choice, a third box in
     // flight is worth more than a second tile per step (r = 3, f = 49: 1.45 -> 1.32 ms; r = 7: 2.95 -> 2.65 ms)
     BZ_I8_CASE(3, 25, 25, 25, 3, 2)
@@ -191,6 +191,12 @@ int vote_pairdist_i8(const float* rep, int r, int f, int64_t d, int64_t ld_file,
     BZ_I8_CASE(7, 49, 13, 13, 3, 1)
 #undef BZ_I8_CASE
     return 1;
+}
+
+int pairdist_i8_stall(int on) {
+    const int v = on ? 1 : 0;
+    const cudaError_t e = cudaMemcpyToSymbol(g_i8_stall, &v, sizeof(int));
+    return e == cudaSuccess ? BZ_OK : cuda_failed(e);
 }
 
 int pairdist_i8_timeouts(unsigned int* count) {

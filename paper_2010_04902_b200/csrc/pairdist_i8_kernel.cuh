@@ -56,8 +56,13 @@ constexpr int kENone = -1000, kELo = -64, kEHi = 64;
 constexpr int kCtlBytes = 2048;
 constexpr int kInfoStride = 72;      // ints per CTA: the rows' largest exponents, then the "bad" mark
 constexpr int kInfoBad = 64;
+constexpr int kBadValues = 1;        // bits of the mark: a row holds values no fixed-point scale can carry
+constexpr int kBadStopped = 2;       //                   a wait ran out and the CTA stopped early
 
 __device__ unsigned int g_i8_timeouts = 0;
+// Testing aid (bz_debug_stall_pipeline): while not 0 the loader threads issue nothing, so the first bounded
+// wait of every CTA runs out and the launch ends the way it would after a lost load.
+__device__ int g_i8_stall = 0;
 
 // F rows, W converter warps, R copies per row (1: the rows are given), FC rows per box, NS boxes in the ring,
 // TS tiles per step
@@ -77,6 +82,7 @@ template <int F, int W, int R, int FC, int NS, int TS> struct I8Shape {
     static constexpr int kPartialBytes = (F * F * 8 + 15) / 16 * 16;   // the CTA's partial matrix T
     static constexpr int kSmem = 1024 + kSlots * kSlotBytes + NS * kBoxBytes + kCtlBytes + kPartialBytes;
     static_assert(F <= 64, "at most 64 rows");
+    static_assert(TS == 1 || TS == 2 || TS == 4, "step sizes that are tested");
     static_assert(kBoxBytes % 128 == 0, "TMA destinations are 128-byte aligned");
     static_assert(kSmem <= 227 * 1024, "shared memory");
     // MMA m covers slice indices m*SPM .. m*SPM+SPM-1 along M and m*SPM .. 3 along N
@@ -316,7 +322,8 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
             int s = 0, filled = 0;
             uint32_t phase = 0;
             int64_t issued = 0;
-            for (int64_t step = 0; step < my_steps && ok; ++step) {
+            const int64_t steps_to_load = *const_cast<volatile int*>(&g_i8_stall) ? 0 : my_steps;
+            for (int64_t step = 0; step < steps_to_load && ok; ++step) {
                 const int n_sub = static_cast<int>(my_tiles - TS * step < TS ? my_tiles - TS * step : TS);
                 for (int c = 0; c < CH && ok; ++c) {
                     for (int sub = 0; sub < n_sub; ++sub) {
@@ -401,21 +408,33 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
 #pragma unroll
                                     for (int k = 0; k < R; ++k) cp[k] = x[k].w;
                                     w.w = vote_bits<R>(cp);
-                                    uint32_t* q = reinterpret_cast<uint32_t*>(voted + (c * FC + fi) * ld_voted + j);
+                                }
+                                val[sub][i] = make_float4(__uint_as_float(w.x), __uint_as_float(w.y), __uint_as_float(w.z), __uint_as_float(w.w));
+                            }
+                        }
+                        // The box is in registers: hand it back.  The arrival is a release (the loads above are
+                        // ordered before the producer's next write into the box), so it comes BEFORE this tile's
+                        // global stores: a release waits for the stores its thread has in flight, and stores
+                        // issued after it have the whole conversion to drain before the step's next arrival.
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&in_empty[s]);
+                        if constexpr (R > 1) {
+#pragma unroll
+                            for (int i = 0; i < RWC; ++i) {
+                                const int fi = off + W * i;
+                                if (fi < FC && c * FC + fi < F) {
+                                    const float4 w = val[sub][i];
+                                    float* q = voted + (c * FC + fi) * ld_voted + j;
                                     if (j + 3 < d) {
-                                        __stcs(reinterpret_cast<uint4*>(q), w);
+                                        __stcs(reinterpret_cast<float4*>(q), w);
                                     } else {  // ragged end
                                         if (j < d) q[0] = w.x;
                                         if (j + 1 < d) q[1] = w.y;
                                         if (j + 2 < d) q[2] = w.z;
                                     }
                                 }
-                                val[sub][i] = make_float4(__uint_as_float(w.x), __uint_as_float(w.y), __uint_as_float(w.z), __uint_as_float(w.w));
                             }
                         }
-                        // the box is in registers: hand it back
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive_relaxed(&in_empty[s]);
                         if (++s == NS) {
                             s = 0;
                             in_phase ^= 1;
@@ -512,7 +531,9 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
             __syncwarp();
             if (lane == 0) {
                 if (raise) atomicOr(const_cast<int*>(&op_flush[o]), 1);
-                mbar_arrive_relaxed(&op_full[o]);
+                // release: this warp's operand tiles, exponents and flush request are ordered before whatever
+                // the MMA thread (and, through its own arrivals, the drain warps) does after its wait
+                mbar_arrive(&op_full[o]);
             }
             if (++o == NO) {
                 o = 0;
@@ -532,11 +553,14 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
         if (!ok && lane == 0) atomicAdd(&g_i8_timeouts, 1u);
         if (lane == 0) {
             for (int r = cw; r < F; r += W) info[blockIdx.x * kInfoStride + r] = e_cur[r];
-            if (unrepresentable || !ok) atomicOr(&info[blockIdx.x * kInfoStride + kInfoBad], 1);
+            if (unrepresentable) atomicOr(&info[blockIdx.x * kInfoStride + kInfoBad], kBadValues);
         }
     }
     tc_fence_before_sync();
     __syncthreads();
+    // whichever role's wait ran out first has raised `dead`: the CTA's partial matrix (and, with the vote in
+    // front, its share of the voted rows) is incomplete
+    if (tid == 0 && *dead) atomicOr(&info[blockIdx.x * kInfoStride + kInfoBad], kBadStopped);
     if (warp == kMmaWarp) tmem_dealloc(tmem_base, S::kTmemCols);
 }
 

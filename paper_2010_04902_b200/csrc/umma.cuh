@@ -61,15 +61,6 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, int32_t (&x)[8]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Arrival without release ordering.  A release would first wait for every memory operation the thread
-// has in flight - also its global stores of voted rows, which nobody in the CTA reads.  What the
-// arrival must order, the thread's own earlier shared-memory accesses, is covered: stores are made
-// visible to the tensor core by fence_async_smem() before this, loads have delivered their values
-// (they were consumed), and shared-memory operations of one thread are performed in order.
-__device__ __forceinline__ void mbar_arrive_relaxed(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-
 // ---- bounded waits that give up early once another thread of the CTA has ---------------------------
 // Each probe lets the hardware suspend the thread for up to `nap_ns` nanoseconds, so a warp that waits
 // takes no issue slots from the warps that work.  At most `probes` probes.

@@ -104,10 +104,13 @@ __global__ void __launch_bounds__(kBlock) vote_median_kernel(const V* __restrict
     }
 }
 
-// grid.y = file, grid.x strides over coordinate groups
+// grid.y = file, grid.x strides over coordinate groups.  gate != nullptr: the kernel runs only if *gate is
+// not 0 (the repair of voted rows after a single-pass kernel that stopped early).
 template <int R, typename V>
 __global__ void __launch_bounds__(256) vote_kernel(const V* __restrict__ rep, int64_t n, int64_t ld_file,
-                                                   int64_t ld_rep, V* __restrict__ voted, int64_t ld_voted) {
+                                                   int64_t ld_rep, V* __restrict__ voted, int64_t ld_voted,
+                                                   const int* __restrict__ gate) {
+    if (gate != nullptr && *gate == 0) return;
     constexpr int VEC = Lanes<V>::n;
     constexpr int U = (12 / R) < 1 ? 1 : (12 / R);  // coordinate groups per thread and trip: ~12 loads in flight
     const int i = blockIdx.y;
@@ -223,7 +226,7 @@ int launch_generic(const float* rep, int r, int f, int64_t d, int64_t ld_file, i
 
 template <int R, typename V>
 int launch_vote(const float* rep, int f, int64_t n, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted,
-                cudaStream_t s) {
+                const int* gate, cudaStream_t s) {
     if (n <= 0) return BZ_OK;
     constexpr int VEC = Lanes<V>::n;
     // about 8 CTAs per SM over the whole (coordinate group, file) grid
@@ -233,19 +236,19 @@ int launch_vote(const float* rep, int f, int64_t n, int64_t ld_file, int64_t ld_
     if (gx < 1) gx = 1;
     dim3 grid(static_cast<unsigned>(gx), f);
     vote_kernel<R, V><<<grid, 256, 0, s>>>(reinterpret_cast<const V*>(rep), n, ld_file / VEC, ld_rep / VEC,
-                                           reinterpret_cast<V*>(voted), ld_voted / VEC);
+                                           reinterpret_cast<V*>(voted), ld_voted / VEC, gate);
     note_launch();
     return check_launch();
 }
 
 template <int R>
 int vote_dispatch(const float* rep, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted,
-                  bool vec, cudaStream_t s) {
-    if (!vec) return launch_vote<R, uint32_t>(rep, f, d, ld_file, ld_rep, voted, ld_voted, s);
+                  bool vec, cudaStream_t s, const int* gate = nullptr) {
+    if (!vec) return launch_vote<R, uint32_t>(rep, f, d, ld_file, ld_rep, voted, ld_voted, gate, s);
     const int64_t n4 = d / 4;
-    int st = launch_vote<R, uint4>(rep, f, n4, ld_file, ld_rep, voted, ld_voted, s);
+    int st = launch_vote<R, uint4>(rep, f, n4, ld_file, ld_rep, voted, ld_voted, gate, s);
     if (st != BZ_OK) return st;
-    return launch_vote<R, uint32_t>(rep + 4 * n4, f, d - 4 * n4, ld_file, ld_rep, voted + 4 * n4, ld_voted, s);
+    return launch_vote<R, uint32_t>(rep + 4 * n4, f, d - 4 * n4, ld_file, ld_rep, voted + 4 * n4, ld_voted, gate, s);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -381,8 +384,12 @@ int vote_median_on_device(const float* rep, int r, int f, int64_t d, int64_t ld_
     int st = 1;
     if (staged_path_enabled()) {
         st = vote_median_tma(rep, r, f, d, ld_file, ld_rep, out, upd, s);
-        if (st != 1) return st;
+        if (st != 1) {
+            note_path(BZ_PATH_STAGED);
+            return st;
+        }
     }
+    note_path(BZ_PATH_REGISTERS);
     switch (r) {
         case 1: st = vm_dispatch_f<1>(rep, f, d, ld_file, ld_rep, out, upd, vec, s); break;
         case 3: st = vm_dispatch_f<3>(rep, f, d, ld_file, ld_rep, out, upd, vec, s); break;
@@ -390,7 +397,10 @@ int vote_median_on_device(const float* rep, int r, int f, int64_t d, int64_t ld_
         case 7: st = vm_dispatch_f<7>(rep, f, d, ld_file, ld_rep, out, upd, vec, s); break;
         default: break;
     }
-    if (st == 1) st = launch_generic(rep, r, f, d, ld_file, ld_rep, nullptr, 0, out, 1, upd, s);
+    if (st == 1) {
+        note_path(BZ_PATH_GENERIC);
+        st = launch_generic(rep, r, f, d, ld_file, ld_rep, nullptr, 0, out, 1, upd, s);
+    }
     return st;
 }
 
@@ -424,6 +434,7 @@ extern "C" int bz_vote(const float* replicas, int r, int f, int64_t d, int64_t l
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool vec = aligned16(replicas) && aligned16(voted) && (ld_file % 4 == 0) && (ld_voted % 4 == 0) &&
                      (r == 1 || ld_replica % 4 == 0);
+    note_path(r == 1 || r == 3 || r == 5 || r == 7 ? BZ_PATH_REGISTERS : BZ_PATH_GENERIC);
     switch (r) {
         case 1: return vote_dispatch<1>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, vec, s);
         case 3: return vote_dispatch<3>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, vec, s);
@@ -432,6 +443,20 @@ extern "C" int bz_vote(const float* replicas, int r, int f, int64_t d, int64_t l
         default: return launch_generic(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, nullptr, 0, kNoUpdate, s);
     }
 }
+
+namespace bz {
+// bz_vote on the device's say-so: the vote kernels are enqueued and return at once unless *gate (device) is
+// not 0.  Only for arrays the 128-bit kernels accept and r in {3, 5, 7} (the shapes of the single-pass kernels).
+int vote_if(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica, float* voted,
+            int64_t ld_voted, const int* gate, cudaStream_t s) {
+    switch (r) {
+        case 3: return vote_dispatch<3>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, true, s, gate);
+        case 5: return vote_dispatch<5>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, true, s, gate);
+        case 7: return vote_dispatch<7>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, true, s, gate);
+        default: return BZ_ERR_UNSUPPORTED;
+    }
+}
+}  // namespace bz
 
 extern "C" int bz_vote_median_host(const float* replicas_host, int r, int f, int64_t d, float* out_host,
                                    void* workspace, size_t workspace_bytes, void* stream) {

@@ -16,7 +16,12 @@ int pairdist_fp32(const float* v, int f, int64_t d, int64_t ld, double* dist, do
 int pairdist_path_fp32_only();
 int pairdist_path_i8_forced();
 int vote_pairdist_i8(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted,
-                     double* dist, void* ws, int force, int** flag_out, cudaStream_t s);  // pairdist_i8.cu
+                     double* dist, void* ws, int* flag, int force, cudaStream_t s);  // pairdist_i8.cu
+int* pairdist_status_words(void* ws, int f);   // pairdist.cu
+void* pairdist_i8_part(void* ws, int f);
+int pairdist_clear_status(void* ws, int f, cudaStream_t s);
+int vote_if(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica, float* voted,
+            int64_t ld_voted, const int* gate, cudaStream_t s);  // vote_median.cu
 size_t krum_workspace_bytes(int op, int f);
 int check_workspace(void* ws, size_t have, size_t need);
 
@@ -91,23 +96,30 @@ extern "C" int bz_vote_pairdist(const float* replicas, int r, int f, int64_t d, 
     int st = check_workspace(workspace, workspace_bytes, krum_workspace_bytes(BZ_OP_PAIRDIST, f));
     if (st != BZ_OK) return st;
     // Vote + integer distances on the tensor cores wherever that kernel exists (it is the faster single
-    // pass on every shape measured).  The binary32 distance kernel follows only if the integer kernel's
-    // error estimate asks for it: it reads the flag on the device.
-    const bool forced = pairdist_path_i8_forced() != 0;
+    // pass on every shape measured).  Two repairs follow, both decided on the device from the kernel's flag
+    // words and both returning at once in the ordinary case: the vote alone if the kernel stopped early (its
+    // voted rows are then incomplete), and the binary32 distance kernel if it stopped early or its error
+    // estimate asks for it.
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (d > 0 && r > 1 && !pairdist_path_fp32_only()) {
-        int* flag = nullptr;
-        st = vote_pairdist_i8(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, dist,
-                              static_cast<char*>(workspace) + pairdist_workspace_fp32(f), forced ? 1 : 0, &flag,
-                              static_cast<cudaStream_t>(stream));
+        int* flag = pairdist_status_words(workspace, f);
+        st = vote_pairdist_i8(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, dist, pairdist_i8_part(workspace, f), flag,
+                              pairdist_path_i8_forced(), s);
         if (st == BZ_OK) {
-            if (forced) return BZ_OK;
-            return pairdist_fp32(voted, f, d, ld_voted, dist, static_cast<double*>(workspace), flag, static_cast<cudaStream_t>(stream));
+            note_path(BZ_PATH_TENSOR);
+            st = vote_if(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, flag + 1, s);
+            if (st != BZ_OK) return st;
+            return pairdist_fp32(voted, f, d, ld_voted, dist, static_cast<double*>(workspace), flag, s);
         }
         if (st != 1) return st;
     }
     if (d > 0 && r > 1) {
         st = vote_pairdist_fused(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, dist,
-                                 static_cast<double*>(workspace), static_cast<cudaStream_t>(stream));
+                                 static_cast<double*>(workspace), s);
+        if (st == BZ_OK) {
+            note_path(BZ_PATH_FP32_FUSED);
+            return pairdist_clear_status(workspace, f, s);
+        }
         if (st != 1) return st;
     }
     // shapes without a fused kernel: the two calls this one stands for

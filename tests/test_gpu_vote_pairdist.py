@@ -48,7 +48,27 @@ def test_voted_rows_and_distances(l, r, d, attack):
     # the two-call path sums the same terms; it may group them differently across CTAs
     D2 = bz.pairdist(bz.vote(rep.to(DEV)))
     assert np.allclose(D.cpu().numpy(), D2.cpu().numpy(), rtol=2e-7, atol=0)
-    assert bz.pipeline_timeouts() == 0
+
+
+@pytest.mark.parametrize("l,r,d,attack", [(5, 3, 100_004, "reversed"), (7, 3, 50_000, "alie"), (5, 5, 70_000, "constant"),
+                                          (7, 5, 30_012, "reversed"), (7, 7, 20_000, "alie"), (5, 3, 2_000_000, "alie")])
+def test_binary32_single_pass_on_every_compiled_shape(l, r, d, attack, monkeypatch):
+    # BZ_PAIRDIST_PATH=fp32 puts the vote in front of the binary32 distance kernel (the default is the integer one)
+    monkeypatch.setenv("BZ_PAIRDIST_PATH", "fp32")
+    rep, _, _ = _case(l, r, d, seed=d % 89, attack=attack)
+    want_voted = oracle.vote(rep.numpy())
+    want_D = oracle.pairdist(want_voted)
+    ws = bz.alloc_workspace(bz.OP_PAIRDIST, 0, l * l, d)
+    voted, D = bz.vote_pairdist(rep.to(DEV), workspace=ws)
+    assert bz.last_path() == bz.PATH_FP32_FUSED
+    assert bz.pairdist_status(ws, l * l) == 0
+    assert np.array_equal(_bits(voted), _bits(want_voted))
+    assert _dist_close(D, want_D)
+    assert np.array_equal(D.cpu().numpy(), D.cpu().numpy().T) and (np.diag(D.cpu().numpy()) == 0).all()
+    monkeypatch.delenv("BZ_PAIRDIST_PATH")
+    voted, D = bz.vote_pairdist(rep.to(DEV), workspace=ws)
+    assert bz.last_path() == bz.PATH_TENSOR
+    assert np.array_equal(_bits(voted), _bits(want_voted)) and _dist_close(D, want_D)
 
 
 def test_two_calls_in_a_row_agree_bit_for_bit():

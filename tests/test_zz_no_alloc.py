@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2010_04902_b200 import binding as bz
 from paper_2010_04902_b200 import inputs
 
@@ -23,9 +24,15 @@ DIST_TOL = 1e-7   # the relative tolerance the distance tests use
 
 
 def _close(got, want):
-    got, want = got.cpu().numpy(), want.cpu().numpy()
+    got = got.cpu().numpy()
+    want = want.cpu().numpy() if isinstance(want, torch.Tensor) else want
     assert np.array_equal(got, got.T) and (np.diag(got) == 0).all()
     assert (np.abs(got - want) <= DIST_TOL * np.abs(want)).all()
+
+
+def _free_bytes():
+    torch.cuda.synchronize()
+    return torch.cuda.mem_get_info()[0]
 
 
 def test_two_calls_in_a_row_match_the_workspace_entry_point():
@@ -38,15 +45,20 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
     v2 = inputs.integer_gradients(25, 517, seed=22).to(DEV)
     want2 = bz.pairdist(v2)
     got2 = torch.empty((25, 25), dtype=torch.float64, device=DEV)
-    torch.cuda.synchronize()
-    before = torch.cuda.memory_allocated()
+    warm = torch.empty((25, 25), dtype=torch.float64, device=DEV)
+    bz.pairdist_static(v1, warm)                                      # the device's first call resolves the array's address
+    bz.pairdist_static(v2, warm)                                      # (and the runtime has loaded both kernels' code)
+    before_torch, before_free = torch.cuda.memory_allocated(), _free_bytes()
     bz.pairdist_static(v1, got1)
     bz.pairdist_static(v2, got2)
-    torch.cuda.synchronize()
-    assert torch.cuda.memory_allocated() == before                    # nothing was allocated through torch
+    # neither through torch's allocator nor behind its back: the device's free memory is what it was
+    assert torch.cuda.memory_allocated() == before_torch and _free_bytes() == before_free
     _close(got1, want1)
     _close(got2, want2)
     assert torch.equal(got2, want2)                                   # integer rows: exact on both paths
+    # and against the CPU oracle, not only against the library's other entry point
+    _close(got1, oracle.pairdist(v1.cpu().numpy()))
+    assert np.array_equal(got2.cpu().numpy(), oracle.pairdist(v2.cpu().numpy()))
 
 
 def test_other_shapes_and_a_third_call():
@@ -56,6 +68,7 @@ def test_other_shapes_and_a_third_call():
         got = torch.empty((f, f), dtype=torch.float64, device=DEV)
         bz.pairdist_static(v, got)
         _close(got, bz.pairdist(v))
+        _close(got, oracle.pairdist(v.cpu().numpy()))
     buf = torch.zeros((25, 2100), dtype=torch.float32, device=DEV)
     buf[:, 1:2002] = inputs.true_gradients(25, 2001, seed=5).to(DEV)
     got = torch.empty((25, 25), dtype=torch.float64, device=DEV)
