@@ -38,8 +38,11 @@
 // [R copies][FC rows][128 coordinates] into a ring of shared memory; W converter warps own fixed rows
 // (row r belongs to warp r % W), vote them if there are copies, track their scales and write the
 // operand tiles (K-major, 128-byte swizzle) of a second ring; one thread issues the MMAs; four warps
-// drain.  Every mbarrier wait is bounded; on expiry the CTA stops and g_i8_timeouts is raised.  No
-// cluster multicast is used.
+// drain.  Every mbarrier wait is bounded; on expiry the CTA stops, marks its record (the host side then
+// repairs the result with the binary32 kernel) and g_i8_timeouts is raised.  Loads are plain per-CTA loads.
+// Every hand-off of shared memory between roles is an mbarrier arrival with release semantics paired with the
+// waiter's acquire: converter -> loader (box read), converter -> MMA thread (operand tiles, exponents, flush
+// request), MMA thread -> drain warps -> MMA thread.
 #pragma once
 
 #include "umma.cuh"

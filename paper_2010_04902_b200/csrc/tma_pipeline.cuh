@@ -1,5 +1,5 @@
 // mbarrier and TMA (cp.async.bulk.tensor) primitives for the staged kernels, and the host lookup of
-// the driver's tensor-map encoder.  Every wait is bounded.  No cluster multicast is used anywhere.
+// the driver's tensor-map encoder.  Every wait is bounded; every load is a plain per-CTA load.
 #pragma once
 
 #include <cuda.h>

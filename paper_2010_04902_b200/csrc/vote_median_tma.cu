@@ -6,7 +6,7 @@
 // files of a stage straight out of shared memory and keep the winners' order keys in registers.
 // After the last file chunk of a coordinate tile the median network runs and one float is stored.
 // The bytes in flight are set by the ring (stages x ~37 KB per CTA), not by registers, and every
-// replica byte is read from HBM exactly once.  No cluster multicast is used anywhere.
+// replica byte is read from HBM exactly once.  Every load is a plain per-CTA load of this GPU's own memory.
 //
 // Every mbarrier wait is bounded: on expiry the kernel raises g_pipeline_timeouts, stops taking
 // new tiles, drains the loads it has already issued (bounded as well) and returns.

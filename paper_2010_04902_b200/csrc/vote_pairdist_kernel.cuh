@@ -1,8 +1,8 @@
 // The kernel of the single-pass vote + pairwise distances.  Included by vote_pairdist.cu only.
 //
 // A producer thread streams boxes [R copies][FC files][kTD coordinates] of a rank-3 tensor map over
-// replicas[r][f][d] into a ring of stages (cp.async.bulk.tensor, one mbarrier pair per stage; no
-// cluster multicast).  All other warps do both jobs, tile after tile:
+// replicas[r][f][d] into a ring of stages (cp.async.bulk.tensor, plain per-CTA loads, one mbarrier pair
+// per stage).  All other warps do both jobs, tile after tile:
 //   vote     box by box, every thread takes one 16-byte slot (file, column group): it reads the R
 //            copies from the ring, votes them and writes the winner to the CTA's [F][kTD] tile in
 //            shared memory and to `voted`; each warp hands the box back as soon as it is through;
