@@ -401,6 +401,15 @@ const char* bz_last_cuda_error(void);
 int bz_pipeline_timeouts(unsigned int* count);
 
 /*
+ * Measurement aid (no counterpart in the paper): reads `bytes` bytes of device memory once with
+ * 128-bit streaming loads and leaves the XOR of all its 64-bit words in *checksum (device).  Timed
+ * on a buffer much larger than the L2 it gives the read-only bandwidth of this GPU, the second
+ * denominator (beside a copy) for the aggregation kernels, which read r*f words per word they
+ * write.   buf device, 16-byte aligned; bytes a multiple of 8;  checksum device uint64 [1].
+ */
+int bz_stream_probe(const void* buf, size_t bytes, uint64_t* checksum, void* stream);
+
+/*
  * Testing aid for the recovery described at bz_pairdist: while `on` is not 0, the loader threads of
  * the tensor-core distance kernels (given rows and vote in front) issue no loads, so that every
  * CTA's first bounded wait runs out after about a second and the call takes its repair path.

@@ -68,3 +68,24 @@ def bulyan(voted_slab: torch.Tensor, c: int, ops=None, group=None):
     sel = ops.bulyan_select(D, c)
     theta = voted_slab.shape[0] - 2 * c
     return ops.trimmed_mean(voted_slab, sel, theta - 2 * c), sel, D
+
+
+def vote_multikrum(replicas_slab: torch.Tensor, c: int, m: int, ops=None, group=None):
+    """Multi-Krum from the replicas over coordinate slabs: vote and partial distances in one pass over this
+    rank's slab [r][f][d_local], one all-reduce of the f x f matrix, replicated selection, mean of the selected
+    voted rows of the slab.  Returns (out_slab[d_local], selected[m], dist[f][f], voted_slab[f][d_local])."""
+    ops = _ops(ops)
+    voted, D = ops.vote_pairdist(replicas_slab)
+    allreduce_sum_(D, group)
+    sel = ops.krum_select(D, c, m)
+    return ops.mean_rows(voted, sel), sel, D, voted
+
+
+def vote_bulyan(replicas_slab: torch.Tensor, c: int, ops=None, group=None):
+    """Bulyan from the replicas over coordinate slabs.  Returns (out_slab, selected[f-2c], dist, voted_slab)."""
+    ops = _ops(ops)
+    voted, D = ops.vote_pairdist(replicas_slab)
+    allreduce_sum_(D, group)
+    sel = ops.bulyan_select(D, c)
+    theta = voted.shape[0] - 2 * c
+    return ops.trimmed_mean(voted, sel, theta - 2 * c), sel, D, voted

@@ -43,6 +43,36 @@ def _oracle_ops():
     )
 
 
+def _recording_ops(calls):
+    """The same stand-ins, but every call is first bound against the CUDA binding's own signature (so the
+    arguments the sharding layer passes are the ones the default `ops=None` wiring would hand to the kernels)
+    and its name is recorded."""
+    import inspect
+    from paper_2010_04902_b200 import binding
+    base = _oracle_ops()
+    base.vote_pairdist = lambda rep: (lambda v: (torch.from_numpy(v), torch.from_numpy(oracle.pairdist(v))))(oracle.vote(rep.numpy()))
+
+    def wrap(name):
+        fn = getattr(base, name)
+        sig = inspect.signature(getattr(binding, name))
+
+        def call(*a, **kw):
+            sig.bind(*a, **kw)
+            calls.append(name)
+            return fn(*a, **kw)
+        return call
+    return types.SimpleNamespace(**{n: wrap(n) for n in ("vote_median", "pairdist", "vote_pairdist", "krum_select", "mean_rows",
+                                                         "bulyan_select", "trimmed_mean")})
+
+
+def test_default_ops_is_the_cuda_binding():
+    from paper_2010_04902_b200 import binding
+    ops = sharding._ops(None)
+    assert ops is binding
+    for name in ("vote_median", "pairdist", "vote_pairdist", "krum_select", "mean_rows", "bulyan_select", "trimmed_mean"):
+        assert callable(getattr(ops, name))
+
+
 def _free_port():
     s = socket.socket()
     s.bind(("127.0.0.1", 0))
@@ -66,6 +96,18 @@ def _worker(rank, world, port, d, ret):
         voted_slab = torch.from_numpy(oracle.vote(rep_slab.numpy()))
         mk_out, mk_sel, D = sharding.multikrum(voted_slab, 3, 22, ops=ops)
         bu_out, bu_sel, _ = sharding.bulyan(voted_slab, 3, ops=ops)
+        # the single-pass forms, through stand-ins that check the binding's signatures and record the order
+        calls = []
+        rec = _recording_ops(calls)
+        v_out, v_sel, v_D, v_voted = sharding.vote_multikrum(rep_slab, 3, 22, ops=rec)
+        order_mk = list(calls)
+        del calls[:]
+        b_out, b_sel, _, _ = sharding.vote_bulyan(rep_slab, 3, ops=rec)
+        order_bu = list(calls)
+        assert order_mk == ["vote_pairdist", "krum_select", "mean_rows"]
+        assert order_bu == ["vote_pairdist", "bulyan_select", "trimmed_mean"]
+        assert torch.equal(v_voted, voted_slab) and torch.equal(v_sel, mk_sel) and torch.equal(v_out, mk_out)
+        assert torch.equal(v_D, D) and torch.equal(b_sel, bu_sel) and torch.equal(b_out, bu_out)
         ret[rank] = dict(j=(j0, j1), med=med.numpy(), mk_out=mk_out.numpy(), mk_sel=mk_sel.numpy(), D=D.numpy(),
                          bu_out=bu_out.numpy(), bu_sel=bu_sel.numpy())
     finally:
