@@ -6,93 +6,170 @@ namespace bz {
 
 namespace {
 
-// D from the CTAs' partial matrices, then the error estimate of the conversion (two small kernels).
-// flag[0] = 1 asks for the binary32 kernel: the estimate is above the tolerance (ignored with force != 0),
-// a row holds values the fixed-point scale cannot carry, or a CTA stopped early.  flag[1] = 1 says the
-// latter: a bounded wait ran out, the partial matrices are incomplete and so are the voted rows of the
-// kernel with the vote in front.
-// Estimate for a pair: each value is rounded to a multiple of its row's step, an unbiased error of
-// standard deviation 0.29 step; over d coordinates that moves D by about 2 sqrt(D var) + d var.
-constexpr double kRelTol = 5e-9;
+// After the main kernel: D^ from the CTAs' partial matrices, the exact contribution of the listed outlier
+// coordinates, then the bound on the conversion error and the CTAs' marks (three small kernels).
+// flag[0] = 1 asks for the binary32 kernel: the bound does not fit the tolerance (ignored with force != 0), a
+// row holds values the fixed-point scale cannot carry, an outlier list overflowed, or a CTA stopped early.
+// flag[1] = 1 says the latter: a bounded wait ran out, the partial matrices are incomplete and so are the voted
+// rows of the kernel with the vote in front.
+constexpr double kRelTol = 1e-7;   // the library's tolerance for a squared distance
 
 // One warp per pair a <= b: lane l takes CTAs l, l+32, ... in order, then the lanes are added in a fixed
-// tree.  Identical rows meet identical numbers in the same order and get identical distances.
+// tree.  Identical rows meet identical numbers in the same order and get identical distances.  The diagonal
+// pairs deliver |q_a|^2 (what the binary64 sums had to carry: the check kernel bounds their rounding with it).
 template <int F>
 __global__ void __launch_bounds__(256)
-    pairdist_i8_reduce_kernel(const double* __restrict__ tpart, int n_ctas, double* __restrict__ dist) {
+    pairdist_i8_reduce_kernel(const double* __restrict__ tpart, int n_ctas, double* __restrict__ dist, double* __restrict__ norm2) {
     const int pair = blockIdx.x * (blockDim.x / 32) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (pair >= F * F) return;
     const int a = pair / F, b = pair % F;
     if (a > b) return;
     double s = 0.0;
-    if (a < b) {
-        for (int c = lane; c < n_ctas; c += 32) {
-            const double* T = tpart + static_cast<size_t>(c) * F * F;
-            s += (T[a * F + a] + T[b * F + b]) - (T[a * F + b] + T[b * F + a]);
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xffffffffu, s, o);
+    for (int c = lane; c < n_ctas; c += 32) {
+        const double* T = tpart + static_cast<size_t>(c) * F * F;
+        s += a < b ? (T[a * F + a] + T[b * F + b]) - (T[a * F + b] + T[b * F + a]) : T[a * F + a];
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xffffffffu, s, o);
     if (lane == 0) {
-        dist[a * F + b] = s;
-        dist[b * F + a] = s;
+        if (a < b) {
+            dist[a * F + b] = s;
+            dist[b * F + a] = s;
+        } else {
+            dist[a * F + a] = 0.0;
+            norm2[a] = s;
+        }
     }
 }
 
-// The error estimate and the CTAs' marks -> flag[0], flag[1].
+// What the listed outlier coordinates contribute.  CTA a handles row a's lists, thread b the pair (a, b):
+//   corr[a][b] = sum over row a's outliers j of (v_a[j] - v_b[j])^2 - (0 - fed_b[j])^2
+// with fed_b[j] what row b fed the contraction at j: its value, or zero if it was an outlier there too (then
+// the pair is handled from the list of the lower row only).  Lists are walked CTA by CTA, entry by entry:
+// a fixed order.  The check kernel adds corr[a][b] + corr[b][a] to D^.
+template <int F>
+__global__ void __launch_bounds__(128)
+    pairdist_i8_outlier_kernel(const float* __restrict__ v, int64_t ld, const int* __restrict__ info, const int* __restrict__ olist,
+                               int n_ctas, double* __restrict__ corr) {
+    const int a = blockIdx.x, tid = threadIdx.x;
+    __shared__ int s_cnt[kNumSMs], s_off[kNumSMs + 1];
+    __shared__ int s_j[kNumSMs * kOutCap];
+    __shared__ short s_c[kNumSMs * kOutCap];
+    for (int c = tid; c < n_ctas; c += blockDim.x) {
+        const int n = info[c * kInfoStride + kInfoOut + a];
+        s_cnt[c] = n > kOutCap ? kOutCap : (n < 0 ? 0 : n);  // an overflowing list sends the caller to the binary32 kernel anyway
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int run = 0;
+        for (int c = 0; c < n_ctas; ++c) {
+            s_off[c] = run;
+            run += s_cnt[c];
+        }
+        s_off[n_ctas] = run;
+    }
+    __syncthreads();
+    const int total = s_off[n_ctas];
+    if (total == 0) {
+        if (tid < F) corr[a * F + tid] = 0.0;
+        return;
+    }
+    // row a's entries, CTA by CTA, in list order
+    for (int e = tid; e < n_ctas * kOutCap; e += blockDim.x) {
+        const int c = e / kOutCap, k = e % kOutCap;
+        if (k < s_cnt[c]) {
+            s_j[s_off[c] + k] = olist[(static_cast<size_t>(c) * 64 + a) * kOutCap + k];
+            s_c[s_off[c] + k] = static_cast<short>(c);
+        }
+    }
+    __syncthreads();
+    const int b = tid;
+    if (b >= F) return;
+    double sum = 0.0;
+    if (b != a) {
+#pragma unroll 4
+        for (int e = 0; e < total; ++e) {
+            const int64_t j = s_j[e];
+            const int e_b = info[s_c[e] * kInfoStride + kInfoE + b];
+            const float limit_b = __int_as_float((e_b + 127) << 23);  // 2^E_b: row b's outliers in that CTA start here
+            const float va = v[a * ld + j], vb = v[b * ld + j];
+            const bool b_out = !(fabsf(vb) < limit_b);
+            const double diff = static_cast<double>(va) - static_cast<double>(vb);
+            const double fed = b_out ? 0.0 : static_cast<double>(vb);
+            if (!(b_out && b < a)) sum += diff * diff - fed * fed;
+        }
+    }
+    corr[a * F + b] = sum;
+}
+
+// The bound and the marks -> final distances, flag[0], flag[1].
+//   N_a^2 = sum over CTAs of n_small * (step / 2)^2, step = 2^(E - 30): every rounded value moved by at most half a step
+//   |D^ - D~| <= 2 (N_a + N_b) sqrt(D^) + (N_a + N_b)^2, D~ the distance with the outliers as zeros (Cauchy-Schwarz)
+//   + 2^-39 (|q_a|^2 + |q_b|^2) for the binary64 sums behind D^ (a few thousand roundings of terms of that size)
+// must stay below kRelTol times the final distance D^ + corr.
 template <int F>
 __global__ void __launch_bounds__(256)
-    pairdist_i8_check_kernel(const double* __restrict__ dist, const int* __restrict__ info, int n_ctas, int64_t d, int force,
-                             int* __restrict__ flag) {
-    __shared__ int s_emax[F];
+    pairdist_i8_check_kernel(double* __restrict__ dist, const double* __restrict__ corr, const double* __restrict__ norm2,
+                             const int* __restrict__ info, int n_ctas, int force, int* __restrict__ flag) {
+    __shared__ double s_n2[F];
     __shared__ int s_bad, s_marks;
     const int tid = threadIdx.x;
     if (tid == 0) s_bad = s_marks = 0;
-    if (tid < F) s_emax[tid] = kELo;
     __syncthreads();
-    for (int e = tid; e < n_ctas * kInfoStride; e += blockDim.x) {
-        const int a = e % kInfoStride;
-        if (a < F) atomicMax(&s_emax[a], info[e]);
-        if (a == kInfoBad && info[e]) atomicOr(&s_marks, info[e]);
+    // four threads per row, each over every fourth CTA in order; the four sums are added in a fixed order
+    __shared__ double s_part[4][F];
+    if (tid < 4 * F) {
+        const int row = tid % F, part = tid / F;
+        double n2 = 0.0;
+        int over = 0;
+#pragma unroll 4
+        for (int c = part; c < n_ctas; c += 4) {
+            const int* rec = info + c * kInfoStride;
+            const double half_step = __longlong_as_double(static_cast<long long>(1023 + rec[kInfoE + row] - 31) << 52);
+            n2 += static_cast<double>(rec[kInfoSmall + row]) * half_step * half_step;
+            over |= rec[kInfoOut + row] > kOutCap;
+        }
+        s_part[part][row] = n2;
+        if (over) atomicOr(&s_marks, kBadValues);
     }
     __syncthreads();
-    // 2 sqrt(x) + d x <= tol  <=>  x <= x_max with sqrt(x_max) = (sqrt(1 + d tol) - 1) / d: one square root
-    // per thread instead of one per pair
-    const double dd = static_cast<double>(d);
-    const double y_max = (sqrt(1.0 + dd * kRelTol) - 1.0) / dd;
-    const double x_max = y_max * y_max;
-    __shared__ double s_min_nz[F], s_zero_step[F];
+    if (tid < F) s_n2[tid] = (s_part[0][tid] + s_part[1][tid]) + (s_part[2][tid] + s_part[3][tid]);
+    for (int c = tid; c < n_ctas; c += blockDim.x)
+        if (info[c * kInfoStride + kInfoBad]) atomicOr(&s_marks, info[c * kInfoStride + kInfoBad]);
+    __shared__ double s_min_nz[F], s_zero_n2[F];
     if (tid < F) {
         s_min_nz[tid] = 1e300;
-        s_zero_step[tid] = 0.0;
+        s_zero_n2[tid] = 0.0;
     }
     __syncthreads();
     bool bad = false;
     for (int p = tid; p < F * F; p += blockDim.x) {
         const int a = p / F, b = p % F;
         if (a >= b) continue;
-        const double step_a = __longlong_as_double(static_cast<long long>(1023 + s_emax[a] - 30) << 52);
-        const double step_b = __longlong_as_double(static_cast<long long>(1023 + s_emax[b] - 30) << 52);
-        const double var = 0.0841 * (step_a * step_a + step_b * step_b);
-        const double v = dist[a * F + b];
-        if (v > 0.0) {
-            if (var > x_max * v) bad = true;
-            atomicMin(reinterpret_cast<unsigned long long*>(&s_min_nz[a]), static_cast<unsigned long long>(__double_as_longlong(v)));
-            atomicMin(reinterpret_cast<unsigned long long*>(&s_min_nz[b]), static_cast<unsigned long long>(__double_as_longlong(v)));
-        } else if (v == 0.0) {
-            const double z = fmax(step_a, step_b);
-            atomicMax(reinterpret_cast<unsigned long long*>(&s_zero_step[a]), static_cast<unsigned long long>(__double_as_longlong(z)));
-            atomicMax(reinterpret_cast<unsigned long long*>(&s_zero_step[b]), static_cast<unsigned long long>(__double_as_longlong(z)));
-        } else {
+        const double dh = dist[a * F + b];
+        const double df = dh + (corr[a * F + b] + corr[b * F + a]);
+        const double n = sqrt(s_n2[a]) + sqrt(s_n2[b]);
+        if (!(dh >= 0.0) || !(df >= 0.0)) {
             bad = true;
+        } else {
+            const double err = 2.0 * n * sqrt(dh) + n * n + 1.8189894035458565e-12 * (norm2[a] + norm2[b]);
+            if (df > 0.0) {
+                if (err > kRelTol * df) bad = true;
+                atomicMin(reinterpret_cast<unsigned long long*>(&s_min_nz[a]), static_cast<unsigned long long>(__double_as_longlong(df)));
+                atomicMin(reinterpret_cast<unsigned long long*>(&s_min_nz[b]), static_cast<unsigned long long>(__double_as_longlong(df)));
+            } else {
+                // rows that convert to the same integers may still differ, by up to err: judged below against the
+                // smallest distance either row has to anything else
+                atomicMax(reinterpret_cast<unsigned long long*>(&s_zero_n2[a]), static_cast<unsigned long long>(__double_as_longlong(err)));
+                atomicMax(reinterpret_cast<unsigned long long*>(&s_zero_n2[b]), static_cast<unsigned long long>(__double_as_longlong(err)));
+            }
         }
+        dist[a * F + b] = df;
+        dist[b * F + a] = df;
     }
     if (bad) atomicOr(&s_bad, 1);
     __syncthreads();
-    // rows that convert to the same integers may still differ by less than a step everywhere
-    if (tid < F && s_zero_step[tid] > 0.0 && s_min_nz[tid] < 1e300 &&
-        dd * s_zero_step[tid] * s_zero_step[tid] > kRelTol * s_min_nz[tid])
-        atomicOr(&s_bad, 1);
+    if (tid < F && s_zero_n2[tid] > 0.0 && s_min_nz[tid] < 1e300 && s_zero_n2[tid] > kRelTol * s_min_nz[tid]) atomicOr(&s_bad, 1);
     __syncthreads();
     if (tid == 0) {
         flag[0] = ((s_bad && !force) || s_marks) ? 1 : 0;
@@ -102,9 +179,19 @@ __global__ void __launch_bounds__(256)
 
 // rep: R = 1: rows [f][d] with leading dimension ld_file.  R > 1: replicas[r][f][d].
 // Returns 1 if the tensor map cannot express the shape.
+struct Scratch {
+    double* tpart;
+    int* info;
+    int* olist;
+    double* corr;
+    double* norm2;
+};
+
+// rep: R = 1: rows [f][d] with leading dimension ld_file.  R > 1: replicas[r][f][d].
+// Returns 1 if the tensor map cannot express the shape.
 template <int F, int W, int R, int FC, int NS, int TS>
 int launch_i8(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted, double* dist,
-              double* tpart, int* info, int* flag, int force, cudaStream_t s) {
+              const Scratch& sc, int* flag, int force, cudaStream_t s) {
     using S = I8Shape<F, W, R, FC, NS, TS>;
     EncodeTiledFn enc = encode_tiled();
     if (enc == nullptr) return 1;
@@ -122,32 +209,44 @@ int launch_i8(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, floa
     if (e != cudaSuccess) return cuda_failed(e);
     int64_t ctas = (d + kTK - 1) / kTK;
     if (ctas > kNumSMs) ctas = kNumSMs;
-    kern<<<static_cast<int>(ctas), S::kThreads, S::kSmem, s>>>(map, d, voted, ld_voted, tpart, info);
+    kern<<<static_cast<int>(ctas), S::kThreads, S::kSmem, s>>>(map, d, voted, ld_voted, sc.tpart, sc.info, sc.olist);
     note_launch();
     int st = check_launch();
     if (st != BZ_OK) return st;
-    pairdist_i8_reduce_kernel<F><<<(F * F + 7) / 8, 256, 0, s>>>(tpart, static_cast<int>(ctas), dist);
+    pairdist_i8_reduce_kernel<F><<<(F * F + 7) / 8, 256, 0, s>>>(sc.tpart, static_cast<int>(ctas), dist, sc.norm2);
     note_launch();
     st = check_launch();
     if (st != BZ_OK) return st;
-    pairdist_i8_check_kernel<F><<<1, 256, 0, s>>>(dist, info, static_cast<int>(ctas), d, force, flag);
+    // the rows the contraction saw: the given ones, or the winners the kernel has just written
+    const float* rows = R > 1 ? voted : rep;
+    const int64_t ld_rows = R > 1 ? ld_voted : ld_file;
+    pairdist_i8_outlier_kernel<F><<<F, 128, 0, s>>>(rows, ld_rows, sc.info, sc.olist, static_cast<int>(ctas), sc.corr);
+    note_launch();
+    st = check_launch();
+    if (st != BZ_OK) return st;
+    pairdist_i8_check_kernel<F><<<1, 256, 0, s>>>(dist, sc.corr, sc.norm2, sc.info, static_cast<int>(ctas), force, flag);
     note_launch();
     return check_launch();
 }
 
 size_t tpart_bytes(int f) { return round_up(static_cast<size_t>(kNumSMs) * f * f * sizeof(double), 256); }
 size_t info_bytes() { return round_up(static_cast<size_t>(kNumSMs) * kInfoStride * sizeof(int), 256); }
+size_t olist_bytes() { return round_up(static_cast<size_t>(kNumSMs) * 64 * kOutCap * sizeof(int), 256); }
+size_t corr_bytes(int f) { return round_up(static_cast<size_t>(f) * f * sizeof(double), 256); }
+size_t norm_bytes() { return round_up(64 * sizeof(double), 256); }
 
-struct Scratch {
-    double* tpart;
-    int* info;
-};
 Scratch carve(void* ws, int f) {
     char* p = static_cast<char*>(ws);
     Scratch s;
     s.tpart = reinterpret_cast<double*>(p);
     p += tpart_bytes(f);
     s.info = reinterpret_cast<int*>(p);
+    p += info_bytes();
+    s.olist = reinterpret_cast<int*>(p);
+    p += olist_bytes();
+    s.corr = reinterpret_cast<double*>(p);
+    p += corr_bytes(f);
+    s.norm2 = reinterpret_cast<double*>(p);
     return s;
 }
 
@@ -155,10 +254,10 @@ Scratch carve(void* ws, int f) {
 
 bool pairdist_i8_has(int f) { return f == 25 || f == 49; }
 
-// bytes of the partial matrices and the per-CTA records
+// bytes of the partial matrices, the per-CTA records, the outlier lists and their corrections
 size_t pairdist_i8_workspace(int f) {
     if (!pairdist_i8_has(f)) return 0;
-    return tpart_bytes(f) + info_bytes();
+    return tpart_bytes(f) + info_bytes() + olist_bytes() + corr_bytes(f) + norm_bytes();
 }
 
 // Returns BZ_OK / an error, or 1 when this path does not apply (shape, alignment, size).  On BZ_OK
@@ -168,8 +267,8 @@ int pairdist_i8(const float* v, int f, int64_t d, int64_t ld, double* dist, void
     if (!pairdist_i8_has(f) || !aligned16(v) || (ld % 4) != 0 || d < 64 * kTK || d >= (int64_t(1) << 31)) return 1;
     const Scratch sc = carve(ws, f);
     // <rows, converter warps, copies, rows per box, boxes in the ring, tiles per step>
-    if (f == 25) return launch_i8<25, 25, 1, 25, 6, 4>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, flag, force, s);
-    return launch_i8<49, 25, 1, 49, 3, 2>(v, d, ld, 0, nullptr, 0, dist, sc.tpart, sc.info, flag, force, s);
+    if (f == 25) return launch_i8<25, 25, 1, 25, 6, 4>(v, d, ld, 0, nullptr, 0, dist, sc, flag, force, s);
+    return launch_i8<49, 25, 1, 49, 3, 2>(v, d, ld, 0, nullptr, 0, dist, sc, flag, force, s);
 }
 
 // The same from the replicas: vote (Eq. 3) and distances in one pass; the winners go to `voted`.
@@ -181,7 +280,7 @@ int vote_pairdist_i8(const float* rep, int r, int f, int64_t d, int64_t ld_file,
     const Scratch sc = carve(ws, f);
 #define BZ_I8_CASE(R_, F_, W_, FC_, NS_, TS_) \
     if (r == R_ && f == F_)                   \
-        return launch_i8<F_, W_, R_, FC_, NS_, TS_>(rep, d, ld_file, ld_rep, voted, ld_voted, dist, sc.tpart, sc.info, flag, force, s);
+        return launch_i8<F_, W_, R_, FC_, NS_, TS_>(rep, d, ld_file, ld_rep, voted, ld_voted, dist, sc, flag, force, s);
     // with the copies in front the kernel is bound by HBM: where shared memory forces the choice, a third box in
     // flight is worth more than a second tile per step (r = 3, f = 49: 1.45 -> 1.32 ms; r = 7: 2.95 -> 2.65 ms)
     BZ_I8_CASE(3, 25, 25, 25, 3, 2)
