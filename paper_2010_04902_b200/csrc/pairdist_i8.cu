@@ -44,8 +44,8 @@ __global__ void __launch_bounds__(256)
 
 // What the listed outlier coordinates contribute.  CTA a handles row a's lists, thread b the pair (a, b):
 //   corr[a][b] = sum over row a's outliers j of (v_a[j] - v_b[j])^2 - (0 - fed_b[j])^2
-// with fed_b[j] what row b fed the contraction at j: its value, or zero if it was an outlier there too (then
-// the pair is handled from the list of the lower row only).  Lists are walked CTA by CTA, entry by entry:
+// with fed_b[j] what row b fed the contraction at j: its value, or zero if j is on row b's list too (then the
+// pair is handled from the list of the lower row only).  Lists are walked CTA by CTA, entry by entry:
 // a fixed order.  The check kernel adds corr[a][b] + corr[b][a] to D^.
 template <int F>
 __global__ void __launch_bounds__(128)
@@ -90,10 +90,14 @@ __global__ void __launch_bounds__(128)
 #pragma unroll 4
         for (int e = 0; e < total; ++e) {
             const int64_t j = s_j[e];
-            const int e_b = info[s_c[e] * kInfoStride + kInfoE + b];
-            const float limit_b = __int_as_float((e_b + 127) << 23);  // 2^E_b: row b's outliers in that CTA start here
+            const int c = s_c[e];
             const float va = v[a * ld + j], vb = v[b * ld + j];
-            const bool b_out = !(fabsf(vb) < limit_b);
+            // did row b enter as zero at j as well?  Then j is on its list in the same CTA.
+            int n_b = info[c * kInfoStride + kInfoOut + b];
+            n_b = n_b > kOutCap ? kOutCap : n_b;
+            bool b_out = false;
+            const int* list_b = olist + (static_cast<size_t>(c) * 64 + b) * kOutCap;
+            for (int k = 0; k < n_b; ++k) b_out = b_out || list_b[k] == static_cast<int>(j);
             const double diff = static_cast<double>(va) - static_cast<double>(vb);
             const double fed = b_out ? 0.0 : static_cast<double>(vb);
             if (!(b_out && b < a)) sum += diff * diff - fed * fed;
@@ -103,7 +107,8 @@ __global__ void __launch_bounds__(128)
 }
 
 // The bound and the marks -> final distances, flag[0], flag[1].
-//   N_a^2 = sum over CTAs of n_small * (step / 2)^2, step = 2^(E - 30): every rounded value moved by at most half a step
+//   N_a^2 = sum over CTAs (and a row's successive scales) of n_small * (step / 2)^2, step = 2^(E - 30): every rounded
+//   value moved by at most half a step
 //   |D^ - D~| <= 2 (N_a + N_b) sqrt(D^) + (N_a + N_b)^2, D~ the distance with the outliers as zeros (Cauchy-Schwarz)
 //   + 2^-39 (|q_a|^2 + |q_b|^2) for the binary64 sums behind D^ (a few thousand roundings of terms of that size)
 // must stay below kRelTol times the final distance D^ + corr.
@@ -126,7 +131,7 @@ __global__ void __launch_bounds__(256)
         for (int c = part; c < n_ctas; c += 4) {
             const int* rec = info + c * kInfoStride;
             const double half_step = __longlong_as_double(static_cast<long long>(1023 + rec[kInfoE + row] - 31) << 52);
-            n2 += static_cast<double>(rec[kInfoSmall + row]) * half_step * half_step;
+            n2 += reinterpret_cast<const double*>(rec + kInfoN2)[row] + static_cast<double>(rec[kInfoSmall + row]) * half_step * half_step;
             over |= rec[kInfoOut + row] > kOutCap;
         }
         s_part[part][row] = n2;

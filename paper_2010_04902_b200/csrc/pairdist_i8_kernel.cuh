@@ -4,15 +4,16 @@
 // The f x f matrix of squared distances is a contraction over the d coordinates, but in floating
 // point only its difference form is accurate enough: gradients share a large per-coordinate mean, so
 // |a|^2 + |b|^2 - 2ab cancels most of its digits.  Integers do not round.  Every value of row a is
-// converted to 31-bit fixed point on the row's own power-of-two scale 2^(30 - E_a) (fixed per CTA and
-// row), the fixed-point word is cut into four balanced signed bytes
+// converted to 31-bit fixed point on the row's own power-of-two scale 2^(30 - E_a) (per CTA; it changes
+// only when the row outgrows it), the fixed-point word is cut into four balanced signed bytes
 //     q = s3*2^24 + s2*2^16 + s1*2^8 + s0,   -128 <= s_i <= 127,
 // and the Gram matrix of the q's is the sum over slice pairs (i, j) of 2^(8(i+j)) S_i S_j^T.  Each
 // S_i S_j^T is an 8-bit integer MMA (tcgen05, kind::i8) with 32-bit accumulators in tensor memory:
 // exact, and independent of the order of the coordinates.  The slices are stacked along M and N, so
 // one or two MMAs per 32 coordinates produce every block that is needed (a block whose transpose is
 // not produced is counted twice).  The accumulators stay in tensor memory and are read back ("drained")
-// every 512 tiles (32-bit headroom) and at the end; a drain combines the blocks in binary64 and adds
+// every 512 tiles (32-bit headroom), when a row changes its scale and at the end; a drain combines the
+// blocks in binary64 and adds
 //     T[a][b] += 2^(E_a + E_b - 60) * sum_blocks weight * S_i S_j^T [a][b]
 // to the CTA's partial matrix (in shared memory, written out once).  A last kernel forms, per CTA and then over CTAs in a fixed order,
 //     D[a][b] = (T[a][a] + T[b][b]) - (T[a][b] + T[b][a]).
@@ -21,16 +22,19 @@
 // What is not exact is the conversion: a value of row a is rounded to a multiple of 2^(E_a - 30).  A CTA
 // fixes E_a when it first meets the row: one bit above the power of two that bounds the magnitudes of
 // its first step.  Values whose binary exponent lies within 7 of E_a keep all 24 bits; smaller ones are
-// rounded, by at most half a step, and the converters count them (n_small).  With N_a^2 = sum over CTAs
-// of n_small * (step/2)^2 the computed distance obeys |D^ - D| <= 2 (N_a + N_b) sqrt(D^) + (N_a + N_b)^2
-// (Cauchy-Schwarz): a bound that holds for every input, also for rows whose rounding errors were
-// arranged to line up.  The last kernel compares it with the library's distance tolerance and raises a
-// flag when it does not fit; the caller then runs the binary32 difference-form kernel, which starts by
-// looking at that flag.
-// A later value that does not fit the row's scale (magnitude 2^E_a or more - an outlier of a heavy-tailed
-// row) does not change the scale: it enters the contraction as zero and its coordinate goes on a short
-// list kept per CTA and row; a small kernel then adds, in binary64 and in a fixed order, what those
-// coordinates really contribute to every pair.  A list that overflows asks for the binary32 kernel.
+// rounded, by at most half a step, and the converters count them (n_small).  With N_a^2 = sum of
+// n_small * (step/2)^2 over CTAs (and over a row's successive scales) the computed distance obeys
+// |D^ - D| <= 2 (N_a + N_b) sqrt(D^) + (N_a + N_b)^2 (Cauchy-Schwarz): a bound that holds for every
+// input, also for rows whose rounding errors were arranged to line up.  The last kernel compares it with
+// the library's distance tolerance and raises a flag when it does not fit; the caller then runs the
+// binary32 difference-form kernel, which starts by looking at that flag.
+// A later value that does not fit the row's scale (magnitude 2^E_a or more) is an outlier as long as the
+// CTA has met at most kOutCap of them in that row - the rare large values of a heavy-tailed row: it
+// enters the contraction as zero and its coordinate goes on a short list kept per CTA and row; a small
+// kernel then adds, in binary64 and in a fixed order, what those coordinates really contribute to every
+// pair.  Past kOutCap the row has outgrown its scale (gradients change magnitude from layer to layer):
+// E_a is set anew from the current step, and the accumulators are read back first, because tensor memory
+// holds integers on the old scale.
 //
 // Per 128-coordinate tile and SM: f*512 bytes from HBM (r times that with the vote in front),
 // f*128 conversions, 4 or 8 MMA instructions.
@@ -62,11 +66,12 @@ constexpr int kTmaWarp = 5;
 constexpr int kConvWarp0 = 6;
 constexpr int kFlushTiles = 512;     // 2^9 tiles * 2^7 coordinates * 2^14 per product < 2^31
 constexpr int kENone = -1000, kELo = -64, kEHi = 64;
-constexpr int kCtlBytes = 2048;
+constexpr int kCtlBytes = 3072;
 // ints per CTA in the record the converters leave: the rows' exponents, their counts of values that may have
 // been rounded, their counts of outliers, then the "bad" mark
-constexpr int kInfoE = 0, kInfoSmall = 64, kInfoOut = 128, kInfoBad = 192, kInfoStride = 200;
-constexpr int kOutCap = 8;           // listed outliers per CTA and row
+// (kInfoN2: 64 doubles - the squared rounding budget a row used up under earlier, finer scales)
+constexpr int kInfoE = 0, kInfoSmall = 64, kInfoOut = 128, kInfoN2 = 192, kInfoBad = 320, kInfoStride = 328;
+constexpr int kOutCap = 8;           // listed outliers per CTA and row; a row that has more gets a coarser scale
 constexpr int kBadValues = 1;        // bits of the mark: a row holds values no fixed-point scale can carry
 constexpr int kBadStopped = 2;       //                   a wait ran out and the CTA stopped early
 
@@ -158,13 +163,16 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
     uint64_t* drained = drain_go + 1;
     volatile int* e_stage = reinterpret_cast<volatile int*>(drained + 1);  // [NO][64]: the rows' exponents as of a step
     volatile int* e_cur = e_stage + NO * 64;                                 // [64]: the rows' exponents now
-    volatile int* drain_stage = e_cur + 64;                                  // which e_stage row a drain uses
+    volatile int* op_flush = e_cur + 64;                                     // [NO]: some row's scale changes with this step
+    volatile int* drain_stage = op_flush + NO;                               // which e_stage row a drain uses
     volatile int* drain_final = drain_stage + 1;                             // is it the last drain
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(drain_final) + 1);
     volatile int* dead = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* n_small = dead + 1;                                        // [64]: values of a row that may have been rounded
     volatile int* n_out = n_small + 64;                                      // [64]: outliers of a row
-    static_assert((2 * NO + 2 * NS + 3) * 8 + (NO * 64 + 64 + 4 + 128) * 4 <= kCtlBytes, "control block");
+    // [64]: sum of count * (half a step)^2 over the row's earlier scales (8-byte aligned: padded to an even number of ints before it)
+    volatile double* n2_done = reinterpret_cast<volatile double*>(n_out + 64 + (NO & 1));
+    static_assert((2 * NO + 2 * NS + 3) * 8 + (NO * 64 + 64 + NO + 6 + 128) * 4 + 64 * 8 <= kCtlBytes, "control block");
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int64_t n_tiles = (d + kTK - 1) / kTK;
@@ -177,6 +185,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
         for (int o = 0; o < NO; ++o) {
             mbar_init(&op_full[o], W);
             mbar_init(&op_empty[o], 1);
+            op_flush[o] = 0;
         }
         for (int s = 0; s < NS; ++s) {
             mbar_init(&in_full[s], 1);
@@ -193,6 +202,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
         e_cur[tid] = kENone;
         n_small[tid] = 0;
         n_out[tid] = 0;
+        n2_done[tid] = 0.0;
     }
     // rows f .. RP-1 of every slice stay zero for the whole run
     for (int e = tid; e < NO * S::kSlotBytes / 16; e += S::kThreads) reinterpret_cast<uint4*>(op)[e] = make_uint4(0, 0, 0, 0);
@@ -285,7 +295,10 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                 }
                 tc_fence_after_sync();
                 const bool last = step == my_steps;
-                if (have_acc && (since > kFlushTiles - TS || last)) {
+                // every converter has arrived, so nobody writes the flag until the slot is handed back
+                const int wants = op_flush[o];
+                if (wants) op_flush[o] = 0;
+                if (have_acc && (wants || since > kFlushTiles - TS || last)) {
                     *drain_stage = o;
                     *drain_final = last ? 1 : 0;
                     mma_commit(acc_ready);
@@ -375,12 +388,17 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
         // this lane's place inside a row of a slice: 16-byte chunk lane/4 (swizzled with the row), word lane%4
         const uint32_t lane_word = (lane & 3) << 2;
         int tiles_left = static_cast<int>(my_tiles < (int64_t(1) << 30) ? my_tiles : (int64_t(1) << 30));
+        // this lane's counts of possibly rounded values, one per row the warp owns (box-row cc, i-th row of it);
+        // they meet in shared memory when a row changes its scale and at the end
+        int small_acc[CH * RWC];
+#pragma unroll
+        for (int e = 0; e < CH * RWC; ++e) small_acc[e] = 0;
         for (int64_t step = 0; step < my_steps && ok; ++step, tiles_left -= TS) {
             const int n_sub = tiles_left < TS ? tiles_left : TS;
             // this lane's coordinates in the first tile of the step
             const int64_t j0 = (blockIdx.x + TS * step * gridDim.x) * kTK + 4 * lane;
             unsigned char* slot = op + static_cast<uint32_t>(o) * S::kSlotBytes;
-            bool have_slot = false;
+            bool raise = false, have_slot = false;
 #pragma unroll 1
             for (int c = 0; c < CH && ok; ++c) {
                 // rows of this box-row that belong to this warp: c*FC + off + W*i
@@ -461,12 +479,14 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                 // rows convert as they are - nearly always.  Otherwise either the row is new to this CTA (its
                 // exponent is fixed now, from the exact maximum of this step) or some values do not fit its
                 // scale (they are listed and enter as zero).  All tiles of a step take the same exponents.
+                int old[RWC];
                 float4 t[TS][RWC];
                 float m = 0.f;
 #pragma unroll
                 for (int i = 0; i < RWC; ++i) {
                     if (off + W * i < FC && c * FC + off + W * i < F) {
                         E[i] = e_cur[c * FC + off + W * i];
+                        old[i] = E[i];
                         if (E[i] == kENone) m = __int_as_float(0x7f800000);  // no exponent yet (first step)
                         const float scale = __int_as_float((30 - (E[i] == kENone ? 0 : E[i]) + 127) << 23);
 #pragma unroll
@@ -497,31 +517,66 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                                 for (int sub = 0; sub < TS; ++sub)
                                     t[sub][i] = make_float4(val[sub][i].x * scale, val[sub][i].y * scale, val[sub][i].z * scale, val[sub][i].w * scale);
                             } else if (need > E[i]) {
-                                // outliers, in the fixed order (tile, component, lane)
-                                int cnt = n_out[row];
+                                // values of magnitude 2^E or more: how many?
+                                int total = 0;
 #pragma unroll
                                 for (int sub = 0; sub < TS; ++sub) {
                                     if (sub < n_sub) {
-                                        float* tv = reinterpret_cast<float*>(&t[sub][i]);
+                                        const float* tv = reinterpret_cast<const float*>(&t[sub][i]);
 #pragma unroll
-                                        for (int k = 0; k < 4; ++k) {
-                                            const bool big = !(fabsf(tv[k]) < 1073741824.0f);
-                                            const unsigned mask = __ballot_sync(0xffffffffu, big);
-                                            if (mask) {
+                                        for (int k = 0; k < 4; ++k) total += !(fabsf(tv[k]) < 1073741824.0f);
+                                    }
+                                }
+                                total = __reduce_add_sync(0xffffffffu, total);
+                                int cnt = n_out[row];
+                                if (cnt + total <= kOutCap) {
+                                    // few: outliers.  They enter as zero and are listed in the fixed order (tile, component, lane)
+#pragma unroll
+                                    for (int sub = 0; sub < TS; ++sub) {
+                                        if (sub < n_sub) {
+                                            float* tv = reinterpret_cast<float*>(&t[sub][i]);
+#pragma unroll
+                                            for (int k = 0; k < 4; ++k) {
+                                                const bool big = !(fabsf(tv[k]) < 1073741824.0f);
+                                                const unsigned mask = __ballot_sync(0xffffffffu, big);
                                                 if (big) {
-                                                    const int pos = cnt + __popc(mask & ((1u << lane) - 1u));
-                                                    if (pos < kOutCap)
-                                                        olist[(static_cast<size_t>(blockIdx.x) * 64 + row) * kOutCap + pos] =
-                                                            static_cast<int>(j0 + sub * static_cast<int64_t>(gridDim.x) * kTK + k);
+                                                    olist[(static_cast<size_t>(blockIdx.x) * 64 + row) * kOutCap + cnt + __popc(mask & ((1u << lane) - 1u))] =
+                                                        static_cast<int>(j0 + sub * static_cast<int64_t>(gridDim.x) * kTK + k);
                                                     tv[k] = 0.f;
                                                 }
                                                 cnt += __popc(mask);
                                             }
                                         }
                                     }
+                                    __syncwarp();
+                                    if (lane == 0) n_out[row] = cnt;
+                                } else {
+                                    // many: the row has outgrown its scale (gradients change magnitude from layer to layer).
+                                    // New exponent from this step's exact maximum; the accumulators are read back before
+                                    // this step's products are added, and the roundings counted so far are charged at the
+                                    // old step.
+                                    int so_far = 0;
+#pragma unroll
+                                    for (int cc = 0; cc < CH; ++cc) {
+                                        if (cc == c) {
+                                            so_far = small_acc[cc * RWC + i];
+                                            small_acc[cc * RWC + i] = 0;
+                                        }
+                                    }
+                                    so_far = __reduce_add_sync(0xffffffffu, so_far);
+                                    if (lane == 0) {
+                                        const double half_step = __longlong_as_double(static_cast<long long>(1023 + E[i] - 31) << 52);
+                                        n2_done[row] += static_cast<double>(so_far) * half_step * half_step;
+                                    }
+                                    raise = true;
+                                    E[i] = clamp_e(need + 1);
+                                    if (lane == 0) e_cur[row] = E[i];
+                                    const float scale = __int_as_float((30 - E[i] + 127) << 23);
+#pragma unroll
+                                    for (int sub = 0; sub < TS; ++sub)
+                                        t[sub][i] = make_float4(val[sub][i].x * scale, val[sub][i].y * scale, val[sub][i].z * scale, val[sub][i].w * scale);
+                                    __syncwarp();
                                 }
-                                __syncwarp();
-                                if (lane == 0) n_out[row] = cnt;
                             }
                         }
                     }
@@ -539,7 +594,8 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                     const int fi = off + W * i;
                     if (fi < FC && c * FC + fi < F) {
                         const int r = c * FC + fi;
-                        if (lane == 0) e_stage[o * 64 + r] = E[i];
+                        // a row whose scale changes hands its old exponent to the drain that comes before this step
+                        if (lane == 0) e_stage[o * 64 + r] = old[i] == kENone ? E[i] : old[i];
                         // row r of a slice: 128 bytes per row, 16-byte chunk (lane/4) ^ (r%8) within it
                         unsigned char* dst = slot + r * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | lane_word);
                         int small = 0;
@@ -558,8 +614,9 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                                 small += __popc((z - 0x01010101u) & ~z & 0x80808080u);
                             }
                         }
-                        small = __reduce_add_sync(0xffffffffu, small);
-                        if (lane == 0) n_small[r] += small;
+#pragma unroll
+                        for (int cc = 0; cc < CH; ++cc)
+                            if (cc == c) small_acc[cc * RWC + i] += small;
                     }
                 }
             }
@@ -571,7 +628,8 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
             fence_async_smem();
             __syncwarp();
             if (lane == 0) {
-                // release: this warp's operand tiles and exponents are ordered before whatever
+                if (raise) atomicOr(const_cast<int*>(&op_flush[o]), 1);
+                // release: this warp's operand tiles, exponents and flush request are ordered before whatever
                 // the MMA thread (and, through its own arrivals, the drain warps) does after its wait
                 mbar_arrive(&op_full[o]);
             }
@@ -591,11 +649,22 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
             }
         }
         if (!ok && lane == 0) atomicAdd(&g_i8_timeouts, 1u);
+#pragma unroll
+        for (int cc = 0; cc < CH; ++cc) {
+            const int off = CH == 1 ? cw : ((cw - cc * FC) % W + W) % W;
+#pragma unroll
+            for (int i = 0; i < RWC; ++i) {
+                const int total = __reduce_add_sync(0xffffffffu, small_acc[cc * RWC + i]);
+                if (lane == 0 && off + W * i < FC && cc * FC + off + W * i < F) n_small[cc * FC + off + W * i] = total;
+            }
+        }
+        __syncwarp();
         if (lane == 0) {
             for (int r = cw; r < F; r += W) {
                 info[blockIdx.x * kInfoStride + kInfoE + r] = e_cur[r];
                 info[blockIdx.x * kInfoStride + kInfoSmall + r] = n_small[r];
                 info[blockIdx.x * kInfoStride + kInfoOut + r] = n_out[r];
+                reinterpret_cast<double*>(info + blockIdx.x * kInfoStride + kInfoN2)[r] = n2_done[r];
             }
             if (unrepresentable) atomicOr(&info[blockIdx.x * kInfoStride + kInfoBad], kBadValues);
         }

@@ -83,25 +83,20 @@ def test_outliers_late_in_a_row():
     _check_close(dist.cpu().numpy(), want)
 
 
-def test_more_outliers_than_a_list_holds():
-    # 78 large values inside one 128-coordinate tile of one row: the list of that CTA and row overflows and the
-    # binary32 kernel answers (whatever BZ_PAIRDIST_PATH=i8 says: it only overrides the error bound)
+def test_a_row_that_outgrows_its_scale():
+    # more large values than a list holds (78 inside one tile; and a whole stretch of the row 300 times larger, the
+    # way gradients change magnitude from layer to layer): the CTAs that meet them give the row a coarser scale
+    # and read the accumulators back; the integer kernel still answers
     f, d = 49, 400_000
     g = inputs.true_gradients(f, d, seed=5).numpy()
     g[17, 222_222:222_300] *= 1.0e3
+    g[:, 300_000:] *= 300.0
+    g[5, 100_000:] *= 1.0e-3
     want = oracle.pairdist(g)
-    for force in (False, True):
-        if force:
-            import os
-            os.environ["BZ_PAIRDIST_PATH"] = "i8"
-        try:
-            ws = bz.alloc_workspace(bz.OP_PAIRDIST, 0, f, d)
-            got = bz.pairdist(torch.from_numpy(g).to(DEV), workspace=ws).cpu().numpy()
-            assert bz.pairdist_status(ws, f) == bz.STATUS_RECOMPUTED
-        finally:
-            if force:
-                del os.environ["BZ_PAIRDIST_PATH"]
-        _check_close(got, want)
+    ws = bz.alloc_workspace(bz.OP_PAIRDIST, 0, f, d)
+    got = bz.pairdist(torch.from_numpy(g).to(DEV), workspace=ws).cpu().numpy()
+    assert bz.last_path() == bz.PATH_TENSOR and bz.pairdist_status(ws, f) == 0
+    _check_close(got, want)
 
 
 def test_rounding_errors_lined_up_by_an_attacker():
@@ -111,7 +106,7 @@ def test_rounding_errors_lined_up_by_an_attacker():
     # to one honest row the same way.  Independent rounding errors would cancel to ~1e-10; lined up they reach the
     # 1e-7 the library promises.  The bound the kernel evaluates (Cauchy-Schwarz over the values it actually rounded)
     # holds for this input too, does not fit the tolerance, and the binary32 kernel answers.
-    f, d = 49, 11_200_000 // 8
+    f, d = 49, 11_200_000
     g = inputs.true_gradients(f, d, seed=12).numpy()
     b = g[7]
     step = 2.0 ** (8 - 30)                                   # |v| < 128 in a row's first step -> E = 8
@@ -119,7 +114,7 @@ def test_rounding_errors_lined_up_by_an_attacker():
     frac = np.where(b > 0, 15.0 / 32.0, 17.0 / 32.0)         # rounds down where b is above, up where b is below
     a = ((k + frac) * step).astype(np.float32)
     assert np.array_equal(a.astype(np.float64), (k + frac) * step)   # representable: the attack is exact
-    a[::128] = 100.0
+    a[:296 * 128:128] = 100.0                                # the tiles of every CTA's first step (148 CTAs x 2 tiles)
     g[30] = a
     want = oracle.pairdist(g)
     ws = bz.alloc_workspace(bz.OP_PAIRDIST, 0, f, d)
@@ -153,15 +148,26 @@ def test_library_choice(monkeypatch):
     want = oracle.pairdist(v.cpu().numpy())
     _check_close(by_i8, want)
     _check_close(by_fp32, want)
-    # two rows that differ by far less than a fixed-point step of their scale: the estimate must send
-    # the library to the binary32 kernel
+    # Two rows that differ in the last place of 300 values: their squared distance (~1e-12) is below what a Gram
+    # matrix in binary64 can resolve next to squared norms of ~1e5.  The library either hands the pair to the
+    # binary32 kernel or reports 0 - the latter only when its bound on what the distance could be is below 1e-7 of
+    # the smallest other distance of the two rows, i.e. invisible in any Krum score.
     w = v.clone()
     w[1] = w[0]
     w[1, ::1000] += 1.0e-7
-    monkeypatch.setenv("BZ_PAIRDIST_PATH", "fp32")
-    by_fp32 = bz.pairdist(w).cpu().numpy()
-    monkeypatch.delenv("BZ_PAIRDIST_PATH")
-    assert np.array_equal(bz.pairdist(w).cpu().numpy(), by_fp32)
+    want = oracle.pairdist(w.cpu().numpy())
+    ws = bz.alloc_workspace(bz.OP_PAIRDIST, 0, 49, w.shape[1])
+    got = bz.pairdist(w, workspace=ws).cpu().numpy()
+    if bz.pairdist_status(ws, 49) & bz.STATUS_RECOMPUTED:
+        monkeypatch.setenv("BZ_PAIRDIST_PATH", "fp32")
+        assert np.array_equal(got, bz.pairdist(w).cpu().numpy())
+        monkeypatch.delenv("BZ_PAIRDIST_PATH")
+    else:
+        # (row 0 is one of the cluster's colluding copies, so row 1 is this close to all of them)
+        tiny = want < 1e-9
+        resolved = want[0][~tiny[0]].min()
+        assert (got[tiny] == 0.0).all() and want[tiny].max() <= DIST_TOL * resolved
+        assert (np.abs(got[~tiny] - want[~tiny]) <= DIST_TOL * want[~tiny]).all()
 
 
 @pytest.mark.parametrize("bad", [float("inf"), float("nan"), 3.0e38])
