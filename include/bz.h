@@ -203,15 +203,25 @@ int bz_vote_median_host(const float* replicas_host, int r, int f, int64_t d, flo
  *     is converted to 31-bit fixed point on a power-of-two scale of its own, the Gram matrix of
  *     the integers is formed exactly by 8-bit integer MMAs, and dist = |a|^2 + |b|^2 - 2ab is taken
  *     in binary64.  The only error is the rounding of a value to a multiple of its row's step
- *     2^(E-30), 2^E bounding the row's magnitudes.  The library estimates that error for every pair
- *     and, where it exceeds 5e-9 relative, or where a row holds infinities, NaNs or magnitudes
- *     beyond 2^60, recomputes with the second kernel (decided on the device; the call stays
- *     asynchronous).
+ *     2^(E-30), with 2^E one bit above the magnitudes the row showed first.  Rare larger values
+ *     (the tail of a heavy-tailed gradient) are taken out of the contraction and added exactly in
+ *     binary64; a row that keeps producing them gets a coarser step.  The kernel counts the
+ *     values it rounded and bounds, for every pair and for EVERY input - also one whose rounding
+ *     errors an attacker lined up - what the roundings can have done to the distance
+ *     (Cauchy-Schwarz).  Where the bound exceeds 1e-7 relative, or a row holds infinities, NaNs
+ *     or magnitudes beyond 2^60, the second kernel recomputes (decided on the device; the call
+ *     stays asynchronous).  On gradients like the benchmark's the bound is ~3e-8 and the actual
+ *     error ~1e-11.  Two rows closer than binary64 sums of their squared norms can resolve are
+ *     reported at distance 0 if the bound on their true distance is below 1e-7 of the smallest
+ *     non-zero distance either has; otherwise the second kernel answers.
  *   - Binary32 difference form (every other shape): differences and squares in binary32, added in
  *     binary32 inside blocks of at most 1024 coordinates (interleaved partial sums of at most 128
- *     terms) and in binary64 across blocks, in a fixed order.
+ *     terms) and in binary64 across blocks, in a fixed order.  Its rounding errors are those of
+ *     binary32 products and short binary32 sums: ~3e-9 relative on gradients, with no bound of
+ *     the first kernel's kind (a run of a few hundred very large values inside one block can
+ *     cost 1e-7 and more).
  * Environment: BZ_PAIRDIST_PATH=fp32 keeps every call on the second kernel; =i8 takes the first
- * kernel's result whatever its estimate says (for testing it); read at every call.
+ * kernel's result whatever its bound says (for testing it); read at every call.
  * With =i8 the second kernel still answers for rows the fixed point cannot hold and after a
  * kernel that stopped early (below).
  * The tensor-core kernel bounds every wait.  If one runs out the kernel stops early, says so in
@@ -229,7 +239,7 @@ int bz_pairdist(const float* voted, int f, int64_t d, int64_t ld, double* dist, 
  * bz_bulyan, bz_vote_pairdist, bz_vote_multikrum, bz_vote_bulyan with the same f).  Synchronises
  * `stream`, then writes a combination of the bits below to *status (host):
  *   BZ_STATUS_RECOMPUTED     the binary32 kernel's distances were returned although the tensor-core
- *                            kernel ran (its error estimate, values without a fixed-point scale,
+ *                            kernel ran (its error bound, values without a fixed-point scale,
  *                            or an early stop asked for it)
  *   BZ_STATUS_STOPPED_EARLY  a bounded wait of the tensor-core kernel ran out; its distances were
  *                            recomputed and, in the calls that vote first, the voted rows were
@@ -324,7 +334,7 @@ int bz_bulyan(const float* voted, int f, int64_t d, int64_t ld, int c, float* ou
  * `voted` and enter the distance sums of Sec. 1.2 from on-chip memory, so the voted rows are not
  * read back (4*f of the 4*(r*f + 2*f) bytes per coordinate the two calls move are saved).
  * voted is bit-identical to bz_vote's; dist is computed as in bz_pairdist (f = 25, 49 with r = 3, 5
- * and 7 x 49: the vote runs in front of the tensor-core kernel, with the same estimate and fall-back;
+ * and 7 x 49: the vote runs in front of the tensor-core kernel, with the same bound and fall-back;
  * BZ_PAIRDIST_PATH=fp32 puts it in front of the binary32 kernel instead).  Shapes without a fused
  * kernel (r*f outside {3,5}x{25,49} and 7x49, unaligned or short arrays) run the two calls.
  * Should a bounded wait of the single-pass kernel run out, `voted` and `dist` are incomplete when

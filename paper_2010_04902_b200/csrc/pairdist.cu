@@ -7,7 +7,7 @@
 // does not depend on a common offset of the rows (gradients share a large per-coordinate mean) nor on
 // the size of an attacker's payload in other rows.  They are bound by the FP32 pipe (f(f-1) add/fma
 // lane-operations per coordinate) and serve every shape the integer kernel does not take, its fall-back
-// when its own error estimate or a row's values ask for one, and bz_pairdist_static.
+// when its own error bound or a row's values ask for one, and bz_pairdist_static.
 #include <atomic>
 #include <cstdlib>
 #include <cstring>
@@ -203,7 +203,7 @@ int launch_pairdist_tiled(const float* v, int64_t d, int64_t ld, double* dist, d
 }
 
 // BZ_PAIRDIST_PATH=fp32 keeps the distances off the tensor cores; =i8 takes the integer kernel's
-// result even where its error estimate asks for the binary32 kernel (for tests of that kernel).
+// result even where its error bound asks for the binary32 kernel (for tests of that kernel).
 enum { kPathAuto = 0, kPathFp32 = 1, kPathI8 = 2 };
 int pairdist_path() {
     const char* e = std::getenv("BZ_PAIRDIST_PATH");

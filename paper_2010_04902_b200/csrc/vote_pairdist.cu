@@ -99,7 +99,7 @@ extern "C" int bz_vote_pairdist(const float* replicas, int r, int f, int64_t d, 
     // pass on every shape measured).  Two repairs follow, both decided on the device from the kernel's flag
     // words and both returning at once in the ordinary case: the vote alone if the kernel stopped early (its
     // voted rows are then incomplete), and the binary32 distance kernel if it stopped early or its error
-    // estimate asks for it.
+    // bound asks for it.
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (d > 0 && r > 1 && !pairdist_path_fp32_only()) {
         int* flag = pairdist_status_words(workspace, f);

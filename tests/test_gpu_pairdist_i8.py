@@ -1,6 +1,6 @@
 """GPU parity of the integer (tensor-core) distance kernel against the CPU oracle.
 
-BZ_PAIRDIST_PATH=i8 takes that kernel's result whatever its own error estimate says, =fp32 keeps the
+BZ_PAIRDIST_PATH=i8 takes that kernel's result whatever its own error bound says, =fp32 keeps the
 distances on the binary32 kernels; unset, the library decides.  Shapes here satisfy the kernel's
 conditions (f in {25, 49}, 16-byte aligned rows, d >= 8192), so "i8" really runs it."""
 import numpy as np
@@ -143,7 +143,7 @@ def test_library_choice(monkeypatch):
     monkeypatch.setenv("BZ_PAIRDIST_PATH", "fp32")
     by_fp32 = bz.pairdist(v).cpu().numpy()
     monkeypatch.delenv("BZ_PAIRDIST_PATH")
-    # ordinary gradients: the integer kernel's estimate is far below the tolerance, its result stands
+    # ordinary gradients: the integer kernel's error bound is below the tolerance, its result stands
     assert np.array_equal(bz.pairdist(v).cpu().numpy(), by_i8)
     want = oracle.pairdist(v.cpu().numpy())
     _check_close(by_i8, want)
