@@ -725,6 +725,8 @@ def profile_op(args):
             "vote_pairdist": lambda: bz.vote_pairdist(rep, voted, ws),
             "vote_median_update": lambda: bz.vote_median_update(rep, out, 0.01, voted[0], 0.9),
             "multikrum": lambda: bz.multikrum(voted, c, f - c, workspace=ws, out=out),
+            "vote_multikrum": lambda: bz.vote_multikrum(rep, c, f - c, voted=voted, workspace=ws, out=out),
+            "vote_bulyan": lambda: bz.vote_bulyan(rep, c, voted=voted, workspace=ws, out=out),
             "bulyan": lambda: bz.bulyan(voted, c, workspace=ws, out=out),
             "mean_rows": lambda: bz.mean_rows(voted, sel, out),
             "trimmed_mean": lambda: bz.trimmed_mean(voted, sel, theta - 2 * c, out),
@@ -799,7 +801,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="profiling only: skip the host-buffer leg")
     ap.add_argument("--no-cpu", action="store_true", help="profiling only: skip the CPU baseline / parity legs")
     ap.add_argument("--op", default="", help="profiling only: run a single entry point (vote_median, vote, vote_vectorwise, median, "
-                    "pairdist, vote_pairdist, vote_median_update, multikrum, bulyan, mean_rows, trimmed_mean, stream_probe, "
+                    "pairdist, vote_pairdist, vote_median_update, multikrum, vote_multikrum, bulyan, vote_bulyan, mean_rows, trimmed_mean, stream_probe, "
                     "worst_case, worst_case_mols) instead of the benchmark")
     ap.add_argument("--shape", default="5,3,3", help="profiling only: l,r,q of the cluster for --op")
     args = ap.parse_args()

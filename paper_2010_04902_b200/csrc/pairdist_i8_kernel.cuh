@@ -22,7 +22,8 @@
 // What is not exact is the conversion: a value of row a is rounded to a multiple of 2^(E_a - 30).  A CTA
 // fixes E_a when it first meets the row: one bit above the power of two that bounds the magnitudes of
 // its first step.  Values whose binary exponent lies within 7 of E_a keep all 24 bits; smaller ones are
-// rounded, by at most half a step, and the converters count them (n_small).  With N_a^2 = sum of
+// rounded, by at most half a step, and the converters count them (n_small: a superset, read off the top
+// bytes).  With N_a^2 = sum of
 // n_small * (step/2)^2 over CTAs (and over a row's successive scales) the computed distance obeys
 // |D^ - D| <= 2 (N_a + N_b) sqrt(D^) + (N_a + N_b)^2 (Cauchy-Schwarz): a bound that holds for every
 // input, also for rows whose rounding errors were arranged to line up.  The last kernel compares it with
@@ -395,7 +396,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
         for (int e = 0; e < CH * RWC; ++e) small_acc[e] = 0;
         for (int64_t step = 0; step < my_steps && ok; ++step, tiles_left -= TS) {
             const int n_sub = tiles_left < TS ? tiles_left : TS;
-            // this lane's coordinates in the first tile of the step
+            // this lane's coordinates in the first tile of the step (used by the vote's stores and the outlier lists)
             const int64_t j0 = (blockIdx.x + TS * step * gridDim.x) * kTK + 4 * lane;
             unsigned char* slot = op + static_cast<uint32_t>(o) * S::kSlotBytes;
             bool raise = false, have_slot = false;
@@ -608,9 +609,10 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                                 *reinterpret_cast<uint32_t*>(dst + sub * S::kOpStageBytes + 1 * RP * kTK) = w[2];
                                 *reinterpret_cast<uint32_t*>(dst + sub * S::kOpStageBytes + 2 * RP * kTK) = w[1];
                                 *reinterpret_cast<uint32_t*>(dst + sub * S::kOpStageBytes + 3 * RP * kTK) = w[0];
-                                // A value can only have been rounded if |q| <= 2^23, and then its top byte is
-                                // -1, 0 or 1.  Bytes in [-2, 1] are those whose bits 7..1 are all equal: count them.
-                                const uint32_t z = (w[3] ^ (w[3] << 1)) & 0xfcfcfcfcu;
+                                // A value can only have been rounded if |q| <= 2^23, and then its top byte (of
+                                // q + 0x808080) is 0 or 1: count the bytes of that word whose upper seven bits are
+                                // clear (a zero-byte test; the bytes tested are even, so it has no false positives).
+                                const uint32_t z = w[3] & 0xfefefefeu;
                                 small += __popc((z - 0x01010101u) & ~z & 0x80808080u);
                             }
                         }
