@@ -23,8 +23,9 @@
  *   - Leading dimensions (ld_*) are in elements.  Gradients are IEEE binary32.  Row layout:
  *     replicas[k][i][j] sits at replicas + k*ld_replica + i*ld_file + j, with k the parallel
  *     class (Latin square) of the worker that sent the copy, i the file, j the coordinate.
- *     The vectorised kernels need 16-byte aligned bases and leading dimensions that are
- *     multiples of 4; anything else takes a slower scalar path, never an error.
+ *     The fastest kernels need 16-byte aligned bases and leading dimensions that are
+ *     multiples of 4; 8-byte alignment with even leading dimensions still gets 64-bit loads;
+ *     anything else takes a slower scalar path, never an error.
  *   - Every function returns BZ_OK or a negative status.  Arguments are validated on the host
  *     before anything is launched; on a non-zero status no output has been written and nothing
  *     has been enqueued (BZ_ERR_CUDA excepted: the runtime's message is kept for

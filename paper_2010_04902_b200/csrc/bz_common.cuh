@@ -17,6 +17,7 @@ int check_launch();                       // cudaGetLastError() after a launch -
 void note_path(int path);                 // which kernel family a call dispatched to (BZ_PATH_*), per host thread
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned8(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 7u) == 0; }
 inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -144,8 +145,10 @@ __device__ __forceinline__ void apply_update4(const ModelUpdate& u, int64_t j4, 
 
 // ---- streaming loads (read-once data: evict-first) -------------------------------------------
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }
+__device__ __forceinline__ uint2 ld_stream(const uint2* p) { return __ldcs(p); }
 __device__ __forceinline__ uint32_t ld_stream(const uint32_t* p) { return __ldcs(p); }
 __device__ __forceinline__ void st_stream(uint4* p, const uint4& x) { __stcs(p, x); }
+__device__ __forceinline__ void st_stream(uint2* p, const uint2& x) { __stcs(p, x); }
 __device__ __forceinline__ void st_stream(uint32_t* p, uint32_t x) { __stcs(p, x); }
 
 }  // namespace bz

@@ -40,6 +40,15 @@ template <> struct Lanes<uint4> {
     __device__ __forceinline__ static uint4 make(const uint32_t (&a)[4]) { return make_uint4(a[0], a[1], a[2], a[3]); }
     __device__ __forceinline__ static void update(const ModelUpdate& u, int64_t j, const uint4& g) { apply_update4(u, j, g); }
 };
+template <> struct Lanes<uint2> {
+    static constexpr int n = 2;
+    __device__ __forceinline__ static uint32_t get(const uint2& v, int c) { return c == 0 ? v.x : v.y; }
+    __device__ __forceinline__ static uint2 make(const uint32_t (&a)[2]) { return make_uint2(a[0], a[1]); }
+    __device__ __forceinline__ static void update(const ModelUpdate& u, int64_t j, const uint2& g) {
+        apply_update(u, 2 * j, __uint_as_float(g.x));
+        apply_update(u, 2 * j + 1, __uint_as_float(g.y));
+    }
+};
 template <> struct Lanes<uint32_t> {
     static constexpr int n = 1;
     __device__ __forceinline__ static uint32_t get(const uint32_t& v, int) { return v; }
@@ -195,20 +204,23 @@ int launch_vm(const float* rep, int64_t n, int64_t ld_file, int64_t ld_rep, floa
     return check_launch();
 }
 
+// vec = coordinates per load the arrays' alignment allows: 4 (128-bit loads), 2 (64-bit) or 1; whatever is left
+// past the last full group goes through the scalar kernel
 template <int R, int F>
 int vm_dispatch_vec(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, float* out, const ModelUpdate& upd,
-                    bool vec, cudaStream_t s) {
-    if (!vec) return launch_vm<R, F, uint32_t>(rep, d, ld_file, ld_rep, out, upd, s);
-    const int64_t n4 = d / 4;
-    int st = launch_vm<R, F, uint4>(rep, n4, ld_file, ld_rep, out, upd, s);
+                    int vec, cudaStream_t s) {
+    if (vec == 1) return launch_vm<R, F, uint32_t>(rep, d, ld_file, ld_rep, out, upd, s);
+    const int64_t nv = d / vec;
+    int st = vec == 4 ? launch_vm<R, F, uint4>(rep, nv, ld_file, ld_rep, out, upd, s)
+                      : launch_vm<R, F, uint2>(rep, nv, ld_file, ld_rep, out, upd, s);
     if (st != BZ_OK) return st;
-    return launch_vm<R, F, uint32_t>(rep + 4 * n4, d - 4 * n4, ld_file, ld_rep, out != nullptr ? out + 4 * n4 : nullptr,
-                                     shifted(upd, 4 * n4), s);
+    return launch_vm<R, F, uint32_t>(rep + vec * nv, d - vec * nv, ld_file, ld_rep, out != nullptr ? out + vec * nv : nullptr,
+                                     shifted(upd, vec * nv), s);
 }
 
 template <int R>
 int vm_dispatch_f(const float* rep, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* out,
-                  const ModelUpdate& upd, bool vec, cudaStream_t s) {
+                  const ModelUpdate& upd, int vec, cudaStream_t s) {
     switch (f) {
         case 25: return vm_dispatch_vec<R, 25>(rep, d, ld_file, ld_rep, out, upd, vec, s);
         case 49: return vm_dispatch_vec<R, 49>(rep, d, ld_file, ld_rep, out, upd, vec, s);
@@ -243,12 +255,13 @@ int launch_vote(const float* rep, int f, int64_t n, int64_t ld_file, int64_t ld_
 
 template <int R>
 int vote_dispatch(const float* rep, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted,
-                  bool vec, cudaStream_t s, const int* gate = nullptr) {
-    if (!vec) return launch_vote<R, uint32_t>(rep, f, d, ld_file, ld_rep, voted, ld_voted, gate, s);
-    const int64_t n4 = d / 4;
-    int st = launch_vote<R, uint4>(rep, f, n4, ld_file, ld_rep, voted, ld_voted, gate, s);
+                  int vec, cudaStream_t s, const int* gate = nullptr) {
+    if (vec == 1) return launch_vote<R, uint32_t>(rep, f, d, ld_file, ld_rep, voted, ld_voted, gate, s);
+    const int64_t nv = d / vec;
+    int st = vec == 4 ? launch_vote<R, uint4>(rep, f, nv, ld_file, ld_rep, voted, ld_voted, gate, s)
+                      : launch_vote<R, uint2>(rep, f, nv, ld_file, ld_rep, voted, ld_voted, gate, s);
     if (st != BZ_OK) return st;
-    return launch_vote<R, uint32_t>(rep + 4 * n4, f, d - 4 * n4, ld_file, ld_rep, voted + 4 * n4, ld_voted, gate, s);
+    return launch_vote<R, uint32_t>(rep + vec * nv, f, d - vec * nv, ld_file, ld_rep, voted + vec * nv, ld_voted, gate, s);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -379,8 +392,11 @@ int validate_replicas(const float* rep, int r, int f, int64_t d, int64_t ld_file
 // out may be null when upd.w is not: then only the updated state is written.
 int vote_median_on_device(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* out,
                           const ModelUpdate& upd, cudaStream_t s) {
-    const bool vec = aligned16(rep) && aligned16(out) && aligned16(upd.w) && aligned16(upd.v) && (ld_file % 4 == 0) &&
-                     (r == 1 || ld_rep % 4 == 0);
+    int vec = 1;
+    if (aligned16(rep) && aligned16(out) && aligned16(upd.w) && aligned16(upd.v) && (ld_file % 4 == 0) && (r == 1 || ld_rep % 4 == 0))
+        vec = 4;
+    else if (aligned8(rep) && aligned8(out) && aligned8(upd.w) && aligned8(upd.v) && (ld_file % 2 == 0) && (r == 1 || ld_rep % 2 == 0))
+        vec = 2;
     int st = 1;
     if (staged_path_enabled()) {
         st = vote_median_tma(rep, r, f, d, ld_file, ld_rep, out, upd, s);
@@ -432,8 +448,11 @@ extern "C" int bz_vote(const float* replicas, int r, int f, int64_t d, int64_t l
     if ((voted == nullptr && d > 0) || ld_voted < d) return BZ_ERR_INVALID_ARG;
     if (d == 0) return BZ_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const bool vec = aligned16(replicas) && aligned16(voted) && (ld_file % 4 == 0) && (ld_voted % 4 == 0) &&
-                     (r == 1 || ld_replica % 4 == 0);
+    int vec = 1;
+    if (aligned16(replicas) && aligned16(voted) && (ld_file % 4 == 0) && (ld_voted % 4 == 0) && (r == 1 || ld_replica % 4 == 0))
+        vec = 4;
+    else if (aligned8(replicas) && aligned8(voted) && (ld_file % 2 == 0) && (ld_voted % 2 == 0) && (r == 1 || ld_replica % 2 == 0))
+        vec = 2;
     note_path(r == 1 || r == 3 || r == 5 || r == 7 ? BZ_PATH_REGISTERS : BZ_PATH_GENERIC);
     switch (r) {
         case 1: return vote_dispatch<1>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, vec, s);
@@ -450,9 +469,9 @@ namespace bz {
 int vote_if(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica, float* voted,
             int64_t ld_voted, const int* gate, cudaStream_t s) {
     switch (r) {
-        case 3: return vote_dispatch<3>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, true, s, gate);
-        case 5: return vote_dispatch<5>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, true, s, gate);
-        case 7: return vote_dispatch<7>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, true, s, gate);
+        case 3: return vote_dispatch<3>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, 4, s, gate);
+        case 5: return vote_dispatch<5>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, 4, s, gate);
+        case 7: return vote_dispatch<7>(replicas, f, d, ld_file, ld_replica, voted, ld_voted, 4, s, gate);
         default: return BZ_ERR_UNSUPPORTED;
     }
 }

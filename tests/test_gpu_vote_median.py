@@ -44,6 +44,19 @@ def test_parity_specialised_and_generic_shapes(l, r, q, attack, d):
     _check_all(_cluster(l, r, q, d, attack))
 
 
+@pytest.mark.parametrize("d", [2, 6, 1026, 70002])
+@pytest.mark.parametrize("l,r,q,attack", [(5, 3, 3, "reversed"), (5, 5, 6, "constant"), (7, 3, 5, "alie"), (7, 7, 5, "reversed")])
+def test_rows_on_8_byte_boundaries(l, r, q, attack, d):
+    # d = 2 (mod 4): contiguous rows start on 8-byte, not 16-byte boundaries - the 64-bit load kernels
+    rep = _cluster(l, r, q, d, attack)
+    _check_all(rep)
+    assert bz.last_path() == bz.PATH_REGISTERS
+    # the same values in a window that starts 8 bytes into a padded allocation
+    buf = torch.zeros((r, l * l, d + 10), dtype=torch.float32, device=DEV)
+    buf[:, :, 2:2 + d] = rep.to(DEV)
+    _check_all(rep, buf[:, :, 2:2 + d])
+
+
 def test_config1_vote_then_median():
     # K=15, r=3, l=5, f=25, d=100000, q=2 at the worst-case placement, ALIE with z=1
     _check_all(_cluster(5, 3, 2, 100000, "alie", seed=0))
