@@ -14,7 +14,7 @@
  *     are ordinary process memory.  The caller owns every buffer.  The library never allocates
  *     or frees device memory; scratch space is a caller-provided device workspace whose size
  *     bz_workspace_bytes() reports.  Device state that outlives a call is limited to what is part
- *     of the library image: three counters of expired waits (bz_pipeline_timeouts), the switch of
+ *     of the library image: four counters of expired waits (bz_pipeline_timeouts), the switch of
  *     bz_debug_stall_pipeline and the built-in array of bz_pairdist_static.  None of it
  *     influences a result.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls with
@@ -412,13 +412,15 @@ const char* bz_last_cuda_error(void);
 int bz_pipeline_timeouts(unsigned int* count);
 
 /*
- * Measurement aid (no counterpart in the paper): reads `bytes` bytes of device memory once with
- * 128-bit streaming loads and leaves the XOR of all its 64-bit words in *checksum (device).  Timed
- * on a buffer much larger than the L2 it gives the read-only bandwidth of this GPU, the second
- * denominator (beside a copy) for the aggregation kernels, which read r*f words per word they
- * write.   buf device, 16-byte aligned; bytes a multiple of 8;  checksum device uint64 [1].
+ * Measurement aid (no counterpart in the paper): reads `bytes` bytes of device memory once and
+ * leaves the XOR of all its 64-bit words in *checksum (device).  staged == 0: 128-bit streaming
+ * loads into registers; staged != 0: 32 KB chunks brought into shared memory by the bulk-copy
+ * engine, four in flight per SM, the way the staged aggregation kernels read.  Timed on a buffer
+ * much larger than the L2 it gives the read-only bandwidth of this GPU, the second denominator
+ * (beside a copy) for the aggregation kernels, which read r*f words per word they write.
+ *   buf device, 16-byte aligned; bytes a multiple of 8;  checksum device uint64 [1].
  */
-int bz_stream_probe(const void* buf, size_t bytes, uint64_t* checksum, void* stream);
+int bz_stream_probe(const void* buf, size_t bytes, int staged, uint64_t* checksum, void* stream);
 
 /*
  * Testing aid for the recovery described at bz_pairdist: while `on` is not 0, the loader threads of

@@ -75,7 +75,7 @@ _SIGNATURES = {
     "bz_pairdist_status": (_c_int, [_c_vp, _c_int, _c_vp, _c_vp]),
     "bz_debug_stall_pipeline": (_c_int, [_c_int]),
     "bz_last_path": (_c_int, []),
-    "bz_stream_probe": (_c_int, [_c_vp, _c_sz, _c_vp, _c_vp]),
+    "bz_stream_probe": (_c_int, [_c_vp, _c_sz, _c_int, _c_vp, _c_vp]),
 }
 
 EXPORTS = sorted(_SIGNATURES)
@@ -116,14 +116,15 @@ def pipeline_timeouts() -> int:
     return int(n.value)
 
 
-def stream_probe(buf: torch.Tensor, checksum: torch.Tensor | None = None) -> torch.Tensor:
-    """bz_stream_probe: XOR of the 64-bit words of `buf` (any dtype, contiguous), read once from device memory."""
+def stream_probe(buf: torch.Tensor, checksum: torch.Tensor | None = None, staged: bool = False) -> torch.Tensor:
+    """bz_stream_probe: XOR of the 64-bit words of `buf` (any dtype, contiguous), read once from device memory
+    (staged: through the bulk-copy engine and shared memory instead of plain loads)."""
     if not buf.is_cuda or not buf.is_contiguous():
         raise TypeError("buf must be a contiguous CUDA tensor")
     if checksum is None:
         checksum = torch.zeros(1, dtype=torch.int64, device=buf.device)
-    _check(lib().bz_stream_probe(buf.data_ptr(), buf.numel() * buf.element_size(), _dev(checksum, torch.int64, "checksum"),
-                                 _stream()), "bz_stream_probe")
+    _check(lib().bz_stream_probe(buf.data_ptr(), buf.numel() * buf.element_size(), 1 if staged else 0,
+                                 _dev(checksum, torch.int64, "checksum"), _stream()), "bz_stream_probe")
     return checksum
 
 

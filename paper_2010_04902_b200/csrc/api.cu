@@ -16,6 +16,7 @@ int pipeline_timeouts(unsigned int* count);   // vote_median_tma.cu
 int vote_pairdist_timeouts(unsigned int* count);  // vote_pairdist.cu
 int pairdist_i8_timeouts(unsigned int* count);    // pairdist_i8.cu
 int pairdist_i8_stall(int on);
+int probe_timeouts(unsigned int* count);          // probe.cu
 int* pairdist_status_words(void* ws, int f);      // pairdist.cu
 
 namespace {
@@ -243,11 +244,12 @@ extern "C" const char* bz_status_string(int status) {
 
 extern "C" int bz_pipeline_timeouts(unsigned int* count) {
     if (count == nullptr) return BZ_ERR_INVALID_ARG;
-    unsigned int a = 0, b = 0, c = 0;
+    unsigned int a = 0, b = 0, c = 0, p = 0;
     int st = pipeline_timeouts(&a);
     if (st == BZ_OK) st = vote_pairdist_timeouts(&b);
     if (st == BZ_OK) st = pairdist_i8_timeouts(&c);
-    *count = a + b + c;
+    if (st == BZ_OK) st = probe_timeouts(&p);
+    *count = a + b + c + p;
     return st;
 }
 
