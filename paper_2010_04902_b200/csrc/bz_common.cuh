@@ -71,10 +71,27 @@ template <int R> __device__ __forceinline__ uint32_t vote_bits(const uint32_t (&
     } else if constexpr (R == 3) {
         return (x[1] == x[2]) ? x[1] : x[0];
     } else {
+        // A pattern held by more than half of the copies is the winner whatever the order, and it shows up among
+        // any R/2 + 1 copies.  Honest copies are identical, so copy 0 wins at once unless it is a Byzantine one;
+        // then the next R/2 copies are tried together, without branches.
+        constexpr int kHalf = R / 2 + 1;
         int same0 = 1;
 #pragma unroll
         for (int k = 1; k < R; ++k) same0 += (x[k] == x[0]);
-        if (2 * same0 >= R) return x[0];  // nothing can be strictly more frequent than copy 0
+        if (same0 >= kHalf) return x[0];
+        uint32_t major = x[0];
+        bool found = false;
+#pragma unroll
+        for (int c = kHalf - 1; c >= 1; --c) {
+            int same = 0;
+#pragma unroll
+            for (int k = 0; k < R; ++k) same += (x[k] == x[c]);
+            const bool hit = same >= kHalf;
+            major = hit ? x[c] : major;
+            found = found || hit;
+        }
+        if (found) return major;
+        // no majority: plurality, the pattern first seen wins among equally frequent ones
         uint32_t best = x[0];
         int best_count = same0;
 #pragma unroll
