@@ -199,7 +199,7 @@ int bz_vote_median_host(const float* replicas_host, int r, int f, int64_t d, flo
 /*
  * Squared Euclidean distances between all pairs of voted gradients, the O(f^2 d) part of the
  * Krum family (Sec. 1.2; cost in Appendix A.1): dist[a][b] = sum_j (v_a[j] - v_b[j])^2.
- * Two kernels compute it; results are reproducible from run to run with either.
+ * Three kernels compute it; results are reproducible from run to run with each.
  *   - Tensor cores (f = 25 or 49, d >= 8192, 16-byte aligned rows, ld a multiple of 4): every row
  *     is converted to 31-bit fixed point on a power-of-two scale of its own, the Gram matrix of
  *     the integers is formed exactly by 8-bit integer MMAs, and dist = |a|^2 + |b|^2 - 2ab is taken
@@ -210,23 +210,27 @@ int bz_vote_median_host(const float* replicas_host, int r, int f, int64_t d, flo
  *     values it rounded and bounds, for every pair and for EVERY input - also one whose rounding
  *     errors an attacker lined up - what the roundings can have done to the distance
  *     (Cauchy-Schwarz).  Where the bound exceeds 1e-7 relative, or a row holds infinities, NaNs
- *     or magnitudes beyond 2^60, the second kernel recomputes (decided on the device; the call
- *     stays asynchronous).  On gradients like the benchmark's the bound is ~3e-8 and the actual
+ *     or magnitudes beyond 2^60, the binary64 kernel below recomputes (decided on the device; the
+ *     call stays asynchronous).  On gradients like the benchmark's the bound is ~3e-8 and the actual
  *     error ~1e-11.  Two rows closer than binary64 sums of their squared norms can resolve are
  *     reported at distance 0 if the bound on their true distance is below 1e-7 of the smallest
- *     non-zero distance either has; otherwise the second kernel answers.
- *   - Binary32 difference form (every other shape): differences and squares in binary32, added in
- *     binary32 inside blocks of at most 1024 coordinates (interleaved partial sums of at most 128
- *     terms) and in binary64 across blocks, in a fixed order.  Its rounding errors are those of
- *     binary32 products and short binary32 sums: ~3e-9 relative on gradients, with no bound of
- *     the first kernel's kind (a run of a few hundred very large values inside one block can
- *     cost 1e-7 and more).
- * Environment: BZ_PAIRDIST_PATH=fp32 keeps every call on the second kernel; =i8 takes the first
- * kernel's result whatever its bound says (for testing it); read at every call.
- * With =i8 the second kernel still answers for rows the fixed point cannot hold and after a
+ *     non-zero distance either has; otherwise the binary64 kernel answers.
+ *   - Binary64 difference form (same shapes; also rows shorter than 8192): differences, squares and
+ *     sums in double precision, the oracle's result to ~1e-15 whatever the data; about 2.5x the
+ *     time of the binary32 kernel.  It runs behind the first kernel, reads that kernel's flag and
+ *     returns at once unless asked.
+ *   - Binary32 difference form (every other shape, and bz_pairdist_static): differences and squares
+ *     in binary32, added in binary32 inside blocks of at most 1024 coordinates (interleaved partial
+ *     sums of at most 128 terms) and in binary64 across blocks, in a fixed order.  Its rounding
+ *     errors are those of binary32 products and short binary32 sums: ~3e-9 relative on gradients,
+ *     up to ~2e-6 on rows of a few hundred coordinates, with no bound of the first kernel's kind.
+ * Environment: BZ_PAIRDIST_PATH=fp32 / =fp64 keeps every call on that kernel (fp64: where it
+ * exists); =i8 takes the first kernel's result whatever its bound says (for testing it); read at
+ * every call.
+ * With =i8 the binary64 kernel still answers for rows the fixed point cannot hold and after a
  * kernel that stopped early (below).
  * The tensor-core kernel bounds every wait.  If one runs out the kernel stops early, says so in
- * the workspace, and the second kernel recomputes the whole matrix on the same stream: the result
+ * the workspace, and the binary64 kernel recomputes the whole matrix on the same stream: the result
  * is complete either way, bz_pairdist_status() reports what happened and bz_pipeline_timeouts()
  * counts it.
  *   dist  device, double [f][f], symmetric with a zero diagonal; identical rows give exactly 0.
@@ -239,7 +243,7 @@ int bz_pairdist(const float* voted, int f, int64_t d, int64_t ld, double* dist, 
  * What the distance stage of the last call that used `workspace` did (bz_pairdist, bz_multikrum,
  * bz_bulyan, bz_vote_pairdist, bz_vote_multikrum, bz_vote_bulyan with the same f).  Synchronises
  * `stream`, then writes a combination of the bits below to *status (host):
- *   BZ_STATUS_RECOMPUTED     the binary32 kernel's distances were returned although the tensor-core
+ *   BZ_STATUS_RECOMPUTED     the binary64 kernel's distances were returned although the tensor-core
  *                            kernel ran (its error bound, values without a fixed-point scale,
  *                            or an early stop asked for it)
  *   BZ_STATUS_STOPPED_EARLY  a bounded wait of the tensor-core kernel ran out; its distances were
@@ -340,7 +344,7 @@ int bz_bulyan(const float* voted, int f, int64_t d, int64_t ld, int c, float* ou
  * kernel (r*f outside {3,5}x{25,49} and 7x49, unaligned or short arrays) run the two calls.
  * Should a bounded wait of the single-pass kernel run out, `voted` and `dist` are incomplete when
  * that kernel ends; the call has already enqueued the repair behind it (bz_vote's kernel, then the
- * binary32 distances; both return at once when there is nothing to repair), so outputs are
+ * binary64 distances; both return at once when there is nothing to repair), so outputs are
  * complete once the stream is synchronised.  bz_pairdist_status() and bz_pipeline_timeouts() tell.
  * The same holds for bz_vote_multikrum and bz_vote_bulyan, which start with this call.
  *   replicas, ld_file, ld_replica as bz_vote;  voted device [f][d] with ld_voted (written);
@@ -437,9 +441,10 @@ int bz_debug_stall_pipeline(int on);
  *   BZ_PATH_STAGED      vote / median kernels fed by the TMA unit through shared memory
  *   BZ_PATH_REGISTERS   the same arithmetic with loads straight into registers (any alignment)
  *   BZ_PATH_GENERIC     run-time (r, f) kernels for shapes without a specialisation
- *   BZ_PATH_TENSOR      integer distances on the tensor cores (the binary32 kernel queued behind them)
+ *   BZ_PATH_TENSOR      integer distances on the tensor cores (the binary64 kernel queued behind them)
  *   BZ_PATH_FP32        binary32 difference-form distances
  *   BZ_PATH_FP32_FUSED  vote and binary32 distances in one pass
+ *   BZ_PATH_FP64        binary64 difference-form distances
  */
 #define BZ_PATH_NONE 0
 #define BZ_PATH_STAGED 1
@@ -448,6 +453,7 @@ int bz_debug_stall_pipeline(int on);
 #define BZ_PATH_TENSOR 4
 #define BZ_PATH_FP32 5
 #define BZ_PATH_FP32_FUSED 6
+#define BZ_PATH_FP64 7
 int bz_last_path(void);
 
 /* Number of kernels this library has launched from the calling process since it was loaded. */

@@ -21,7 +21,7 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_PRECONDITION, ERR_WORKSPACE, ERR_BUDGET, E
 OP_PAIRDIST, OP_MULTIKRUM, OP_BULYAN, OP_WORST_CASE, OP_VOTE_MEDIAN_HOST, OP_WORST_CASE_MOLS, OP_VOTE_VECTORWISE = 1, 2, 3, 4, 5, 6, 7
 MAX_R, MAX_F = 15, 128
 STATUS_RECOMPUTED, STATUS_STOPPED_EARLY = 1, 2
-PATH_NONE, PATH_STAGED, PATH_REGISTERS, PATH_GENERIC, PATH_TENSOR, PATH_FP32, PATH_FP32_FUSED = range(7)
+PATH_NONE, PATH_STAGED, PATH_REGISTERS, PATH_GENERIC, PATH_TENSOR, PATH_FP32, PATH_FP32_FUSED, PATH_FP64 = range(8)
 
 
 class BzError(RuntimeError):

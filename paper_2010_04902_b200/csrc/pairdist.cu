@@ -118,6 +118,99 @@ __global__ void __launch_bounds__(PairTile<F, T, G>::NT, tiled_ctas_per_sm<F, T,
 }
 
 // ------------------------------------------------------------------------------------------------
+// The same tiling in binary64: differences, squares and sums all in double precision, so the result is
+// the oracle's up to a few units of 2^-53 per term - whatever the data.  This is the kernel that answers
+// when the integer kernel's error bound does not fit the tolerance (it reads that flag and returns at once
+// otherwise), and for rows too short for the integer kernel.  Bound by the FP64 pipe: one add and one
+// multiply-add per pair and coordinate, about 2.5x the time of the binary32 kernel.
+// Every thread keeps its T x T sums for its whole share of the tiles; the G coordinate groups of a pair
+// are added in a fixed order at the end.  Partial sums have the layout of the binary32 kernel's.
+template <int F, int T, int G> constexpr size_t f64_smem_bytes() {
+    using PT = PairTile<F, T, G>;
+    return size_t(2) * F * kRowStride * 4 + size_t(PT::NT) * PT::TT * 8;
+}
+
+template <int F, int T, int G>
+__global__ void __launch_bounds__(PairTile<F, T, G>::NT, 1)
+    pairdist_f64_kernel(const float* __restrict__ v, int64_t d, int64_t ld, double* __restrict__ partial,
+                        const int* __restrict__ gate) {
+    using PT = PairTile<F, T, G>;
+    if (gate != nullptr && *gate == 0) return;  // the integer kernel's distances stand
+    constexpr int NB = PT::NB, NPB = PT::NPB, NT = PT::NT, TT = PT::TT;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* stage0 = reinterpret_cast<float*>(smem_raw);                              // 2 x [F][kRowStride]
+    double* red = reinterpret_cast<double*>(stage0 + 2 * F * kRowStride);            // [G][NPB][TT]
+    static_assert((2 * F * kRowStride * 4) % 8 == 0, "binary64 buffer alignment");
+
+    const int tid = threadIdx.x;
+    int bi, bj, g;
+    pair_of_thread<F, T, G>(tid, bi, bj, g);
+    const int pb = tid % NPB;
+
+    const int64_t n_tiles = (d + kTD - 1) / kTD;
+    auto load_tile = [&](int buf, int64_t tile) {
+        const int64_t j0 = tile * kTD;
+        constexpr int per_row = kTD / 4;
+        float* dst = stage0 + buf * F * kRowStride;
+        for (int idx = tid; idx < F * per_row; idx += NT) {
+            const int row = idx / per_row, c4 = idx - row * per_row;
+            const int64_t j = j0 + 4 * c4;
+            const int64_t left = d - j;
+            const int bytes = left >= 4 ? 16 : (left > 0 ? static_cast<int>(left) * 4 : 0);
+            const float* src = bytes ? v + row * ld + j : v;  // zero-byte requests still name a valid address
+            cp_async16(dst + row * kRowStride + 4 * c4, src, bytes);
+        }
+        cp_async_commit();
+    };
+
+    double acc[TT];
+#pragma unroll
+    for (int e = 0; e < TT; ++e) acc[e] = 0.0;
+
+    int64_t tile = blockIdx.x;
+    int buf = 0;
+    if (tile < n_tiles) load_tile(0, tile);
+    for (; tile < n_tiles; tile += gridDim.x) {
+        const int64_t next = tile + gridDim.x;
+        if (next < n_tiles) {
+            load_tile(buf ^ 1, next);
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        const float* base = stage0 + buf * F * kRowStride;
+#pragma unroll 1
+        for (int c = g; c < kTD; c += G) {
+            double b[T];
+#pragma unroll
+            for (int u = 0; u < T; ++u) b[u] = static_cast<double>(base[(bj + NB * u) * kRowStride + c]);
+#pragma unroll
+            for (int t = 0; t < T; ++t) {
+                const double a = static_cast<double>(base[(bi + NB * t) * kRowStride + c]);
+#pragma unroll
+                for (int u = 0; u < T; ++u) {
+                    const double e = a - b[u];
+                    acc[t * T + u] = fma(e, e, acc[t * T + u]);
+                }
+            }
+        }
+        __syncthreads();
+        buf ^= 1;
+    }
+#pragma unroll
+    for (int e = 0; e < TT; ++e) red[tid * TT + e] = acc[e];  // tid = g * NPB + pb
+    __syncthreads();
+    double* mine = partial + static_cast<size_t>(blockIdx.x) * NPB * TT;
+    for (int e = g; e < TT; e += G) {
+        double s = 0.0;
+#pragma unroll
+        for (int g2 = 0; g2 < G; ++g2) s += red[(g2 * NPB + pb) * TT + e];
+        mine[pb * TT + e] = s;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Any f, any alignment: a CTA stages kGT coordinates of all rows with scalar loads; pair p is
 // always summed by thread p % blockDim of the CTA, binary32 inside the stage, binary64 across.
 constexpr int kGT = 64;
@@ -202,14 +295,32 @@ int launch_pairdist_tiled(const float* v, int64_t d, int64_t ld, double* dist, d
     return check_launch();
 }
 
-// BZ_PAIRDIST_PATH=fp32 keeps the distances off the tensor cores; =i8 takes the integer kernel's
-// result even where its error bound asks for the binary32 kernel (for tests of that kernel).
-enum { kPathAuto = 0, kPathFp32 = 1, kPathI8 = 2 };
+template <int F, int T, int G>
+int launch_pairdist_f64(const float* v, int64_t d, int64_t ld, double* dist, double* partial, const int* gate, cudaStream_t s) {
+    constexpr int NT = PairTile<F, T, G>::NT;
+    constexpr int smem = static_cast<int>(f64_smem_bytes<F, T, G>());
+    cudaError_t e = cudaFuncSetAttribute(pairdist_f64_kernel<F, T, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return cuda_failed(e);
+    const int ctas = pairdist_ctas(d, kTD, 1);  // never more CTAs than the binary32 kernel's workspace provides for
+    pairdist_f64_kernel<F, T, G><<<ctas, NT, smem, s>>>(v, d, ld, partial, gate);
+    note_launch();
+    int st = check_launch();
+    if (st != BZ_OK) return st;
+    pairdist_tiled_reduce_kernel<F, T, G><<<(F * F + 127) / 128, 128, 0, s>>>(partial, ctas, dist, gate);
+    note_launch();
+    return check_launch();
+}
+
+// BZ_PAIRDIST_PATH=fp32 keeps the distances off the tensor cores and on the binary32 kernels; =fp64 on the
+// binary64 kernel (where it exists); =i8 takes the integer kernel's result even where its error bound asks
+// for the binary64 kernel (for tests of that kernel).
+enum { kPathAuto = 0, kPathFp32 = 1, kPathI8 = 2, kPathFp64 = 3 };
 int pairdist_path() {
     const char* e = std::getenv("BZ_PAIRDIST_PATH");
     if (e == nullptr) return kPathAuto;
     if (std::strcmp(e, "fp32") == 0) return kPathFp32;
     if (std::strcmp(e, "i8") == 0) return kPathI8;
+    if (std::strcmp(e, "fp64") == 0) return kPathFp64;
     return kPathAuto;
 }
 
@@ -221,6 +332,7 @@ int pairdist_i8(const float* v, int f, int64_t d, int64_t ld, double* dist, void
 
 int pairdist_path_fp32_only() { return pairdist_path() == kPathFp32; }
 int pairdist_path_i8_forced() { return pairdist_path() == kPathI8; }
+int pairdist_path_fp64_only() { return pairdist_path() == kPathFp64; }
 
 // the partial sums of the binary32 kernels alone (what bz_pairdist_static keeps in its array)
 size_t pairdist_workspace_fp32(int f) {
@@ -246,9 +358,16 @@ int pairdist_clear_status(void* ws, int f, cudaStream_t s) {
     return e == cudaSuccess ? BZ_OK : cuda_failed(e);
 }
 
-// The binary32 difference-form kernels.  gate != nullptr (only after the integer kernel ran, so on a
-// shape with a tiled kernel): they run only if *gate (device) is not 0.
+// The binary32 difference-form kernels.  gate != nullptr: they run only if *gate (device) is not 0.
 int pairdist_fp32(const float* v, int f, int64_t d, int64_t ld, double* dist, double* partial, const int* gate, cudaStream_t s);
+
+// The binary64 kernel exists for the shapes of the integer kernel: f = 25 or 49, rows the 128-bit copies accept.
+bool pairdist_f64_has(const float* v, int f, int64_t ld) { return (f == 25 || f == 49) && aligned16(v) && (ld % 4 == 0); }
+int pairdist_f64(const float* v, int f, int64_t d, int64_t ld, double* dist, double* partial, const int* gate, cudaStream_t s) {
+    if (gate == nullptr) note_path(BZ_PATH_FP64);
+    if (f == 25) return launch_pairdist_f64<BZ_PD_25>(v, d, ld, dist, partial, gate, s);
+    return launch_pairdist_f64<BZ_PD_49>(v, d, ld, dist, partial, gate, s);
+}
 
 // tensor_cores: the workspace has room for the status words and the integer kernel (pairdist_workspace, not _fp32)
 int pairdist_on_device(const float* v, int f, int64_t d, int64_t ld, double* dist, void* ws, cudaStream_t s, bool tensor_cores) {
@@ -258,13 +377,15 @@ int pairdist_on_device(const float* v, int f, int64_t d, int64_t ld, double* dis
     if (tensor_cores) {
         int* flag = pairdist_status_words(ws, f);
         int st = 1;
-        if (path != kPathFp32) st = pairdist_i8(v, f, d, ld, dist, pairdist_i8_part(ws, f), flag, path == kPathI8, s);
+        if (path != kPathFp32 && path != kPathFp64) st = pairdist_i8(v, f, d, ld, dist, pairdist_i8_part(ws, f), flag, path == kPathI8, s);
         if (st == BZ_OK) {
-            gate = flag;  // the binary32 kernels below run only if the flag asks for them
             note_path(BZ_PATH_TENSOR);
+            return pairdist_f64(v, f, d, ld, dist, partial, flag, s);  // runs only if the flag asks for it
         } else if (st == 1) {
             st = pairdist_clear_status(ws, f, s);
             if (st != BZ_OK) return st;
+            // rows too short for the integer kernel: binary64 costs nothing there and keeps the tolerance
+            if (path != kPathFp32 && d > 0 && pairdist_f64_has(v, f, ld)) return pairdist_f64(v, f, d, ld, dist, partial, nullptr, s);
         } else {
             return st;
         }

@@ -35,7 +35,8 @@
 // kernel then adds, in binary64 and in a fixed order, what those coordinates really contribute to every
 // pair.  Past kOutCap the row has outgrown its scale (gradients change magnitude from layer to layer):
 // E_a is set anew from the current step, and the accumulators are read back first, because tensor memory
-// holds integers on the old scale.
+// holds integers on the old scale.  The other way round, rows that have left three bits or more of their
+// scale unused for four steps get a finer one.
 //
 // Per 128-coordinate tile and SM: f*512 bytes from HBM (r times that with the vote in front),
 // f*128 conversions, 4 or 8 MMA instructions.
@@ -56,6 +57,8 @@
 // request), MMA thread -> drain warps -> MMA thread.
 #pragma once
 
+#include <type_traits>
+
 #include "umma.cuh"
 
 namespace bz {
@@ -72,6 +75,7 @@ constexpr int kCtlBytes = 3072;
 // been rounded, their counts of outliers, then the "bad" mark
 // (kInfoN2: 64 doubles - the squared rounding budget a row used up under earlier, finer scales)
 constexpr int kInfoE = 0, kInfoSmall = 64, kInfoOut = 128, kInfoN2 = 192, kInfoBad = 320, kInfoStride = 328;
+constexpr int kLookEvery = 4;        // steps between two looks at whether rows would fit a finer scale
 constexpr int kOutCap = 8;           // listed outliers per CTA and row; a row that has more gets a coarser scale
 constexpr int kBadValues = 1;        // bits of the mark: a row holds values no fixed-point scale can carry
 constexpr int kBadStopped = 2;       //                   a wait ran out and the CTA stopped early
@@ -394,7 +398,14 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
         int small_acc[CH * RWC];
 #pragma unroll
         for (int e = 0; e < CH * RWC; ++e) small_acc[e] = 0;
-        for (int64_t step = 0; step < my_steps && ok; ++step, tiles_left -= TS) {
+        // the largest scaled magnitude this lane has seen in each box-row since the last look
+        float m_run[CH];
+#pragma unroll
+        for (int e = 0; e < CH; ++e) m_run[e] = 0.f;
+        // One step.  FIRST: the CTA meets the rows for the first time and fixes their scales; kept apart from the
+        // steps that follow so that their code carries none of it.
+        auto convert_step = [&](auto first_tag, int64_t step) {
+            constexpr bool FIRST = decltype(first_tag)::value;
             const int n_sub = tiles_left < TS ? tiles_left : TS;
             // this lane's coordinates in the first tile of the step (used by the vote's stores and the outlier lists)
             const int64_t j0 = (blockIdx.x + TS * step * gridDim.x) * kTK + 4 * lane;
@@ -481,23 +492,72 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                 // exponent is fixed now, from the exact maximum of this step) or some values do not fit its
                 // scale (they are listed and enter as zero).  All tiles of a step take the same exponents.
                 int old[RWC];
+#pragma unroll
+                for (int i = 0; i < RWC; ++i)
+                    if (off + W * i < FC && c * FC + off + W * i < F) old[i] = FIRST ? static_cast<int>(kENone) : static_cast<int>(e_cur[c * FC + off + W * i]);
+                // Every kLookEvery-th step: did the warp's rows of this box-row leave three bits or more of their
+                // scales unused ever since the last look?  Then they get finer ones (a row's magnitude falls as well
+                // as rises from layer to layer, and a step that stays coarse costs precision for all the values that
+                // follow).  As with every change of scale, the accumulators are read back before this step's
+                // products are added.
+                if (!FIRST && (step & (kLookEvery - 1)) == kLookEvery - 1) {
+                    float seen = 0.f;
+#pragma unroll
+                    for (int cc = 0; cc < CH; ++cc) {
+                        if (cc == c) {
+                            seen = m_run[cc];
+                            m_run[cc] = 0.f;
+                        }
+                    }
+                    const uint32_t top = __reduce_max_sync(0xffffffffu, __float_as_uint(seen) & 0x7fffffffu);
+                    const int finer = 28 - (static_cast<int>(top >> 23) - 127);  // the largest scaled value stays below 2^29
+                    if (top != 0 && finer >= 3 && finer < 64) {
+#pragma unroll
+                        for (int i = 0; i < RWC; ++i) {
+                            if (off + W * i < FC && c * FC + off + W * i < F && old[i] - finer >= kELo) {
+                                const int row = c * FC + off + W * i;
+                                int so_far = 0;
+#pragma unroll
+                                for (int cc = 0; cc < CH; ++cc) {
+                                    if (cc == c) {
+                                        so_far = small_acc[cc * RWC + i];
+                                        small_acc[cc * RWC + i] = 0;
+                                    }
+                                }
+                                so_far = __reduce_add_sync(0xffffffffu, so_far);
+                                if (lane == 0) {
+                                    const double half_step = __longlong_as_double(static_cast<long long>(1023 + old[i] - 31) << 52);
+                                    n2_done[row] += static_cast<double>(so_far) * half_step * half_step;
+                                    e_cur[row] = old[i] - finer;
+                                }
+                                raise = true;
+                            }
+                        }
+                        __syncwarp();
+                    }
+                }
                 float4 t[TS][RWC];
                 float m = 0.f;
+                if constexpr (!FIRST) {
 #pragma unroll
-                for (int i = 0; i < RWC; ++i) {
-                    if (off + W * i < FC && c * FC + off + W * i < F) {
-                        E[i] = e_cur[c * FC + off + W * i];
-                        old[i] = E[i];
-                        if (E[i] == kENone) m = __int_as_float(0x7f800000);  // no exponent yet (first step)
-                        const float scale = __int_as_float((30 - (E[i] == kENone ? 0 : E[i]) + 127) << 23);
+                    for (int i = 0; i < RWC; ++i) {
+                        if (off + W * i < FC && c * FC + off + W * i < F) {
+                            E[i] = e_cur[c * FC + off + W * i];
+                            const float scale = __int_as_float((30 - E[i] + 127) << 23);
 #pragma unroll
-                        for (int sub = 0; sub < TS; ++sub) {
-                            t[sub][i] = make_float4(val[sub][i].x * scale, val[sub][i].y * scale, val[sub][i].z * scale, val[sub][i].w * scale);
-                            m = max_abs_nan(max_abs_nan(m, t[sub][i].x), max_abs_nan(t[sub][i].y, max_abs_nan(t[sub][i].z, t[sub][i].w)));
+                            for (int sub = 0; sub < TS; ++sub) {
+                                t[sub][i] = make_float4(val[sub][i].x * scale, val[sub][i].y * scale, val[sub][i].z * scale, val[sub][i].w * scale);
+                                m = max_abs_nan(max_abs_nan(m, t[sub][i].x), max_abs_nan(t[sub][i].y, max_abs_nan(t[sub][i].z, t[sub][i].w)));
+                            }
                         }
                     }
                 }
-                if (__any_sync(0xffffffffu, !(fabsf(m) < 1073741824.0f))) {
+                if constexpr (!FIRST) {
+#pragma unroll
+                    for (int cc = 0; cc < CH; ++cc)
+                        if (cc == c) m_run[cc] = max_abs_nan(m_run[cc], m);
+                }
+                if (FIRST || __any_sync(0xffffffffu, !(fabsf(m) < 1073741824.0f))) {
 #pragma unroll
                     for (int i = 0; i < RWC; ++i) {
                         if (off + W * i < FC && c * FC + off + W * i < F) {
@@ -509,15 +569,61 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                                                  max(__float_as_uint(val[sub][i].z) & 0x7fffffffu, __float_as_uint(val[sub][i].w) & 0x7fffffffu)));
                             const int need = static_cast<int>(__reduce_max_sync(0xffffffffu, m8) >> 23) - 126;  // |v| < 2^need
                             if (need > 60) unrepresentable = 1;  // infinities, NaNs, magnitudes beyond 2^60
-                            if (E[i] == kENone) {
+                            if constexpr (FIRST) {
+                                // The row's first scale.  One or two values that stand three bits or more above all
+                                // the others are outliers already (listed, fed as zero), up to four times over: a scale
+                                // set by them would be coarse for everything that follows.
+                                int fit = need, cnt = 0;
+                                if (need <= 60) {
+                                    for (int round = 0; round < 4; ++round) {
+                                        uint32_t top = 0;
+#pragma unroll
+                                        for (int sub = 0; sub < TS; ++sub) {
+                                            const float* v4 = reinterpret_cast<const float*>(&val[sub][i]);
+#pragma unroll
+                                            for (int k = 0; k < 4; ++k) top = max(top, __float_as_uint(v4[k]) & 0x7fffffffu);
+                                        }
+                                        top = __reduce_max_sync(0xffffffffu, top);
+                                        if (top == 0) break;
+                                        fit = static_cast<int>(top >> 23) - 126;
+                                        if (fit <= kELo + 8) break;
+                                        const uint32_t high = static_cast<uint32_t>(fit - 3 + 126) << 23;  // 2^(fit - 3) and up
+                                        int n_high = 0;
+#pragma unroll
+                                        for (int sub = 0; sub < TS; ++sub) {
+                                            const float* v4 = reinterpret_cast<const float*>(&val[sub][i]);
+#pragma unroll
+                                            for (int k = 0; k < 4; ++k) n_high += (__float_as_uint(v4[k]) & 0x7fffffffu) >= high;
+                                        }
+                                        n_high = __reduce_add_sync(0xffffffffu, n_high);
+                                        if (n_high > 2 || cnt + n_high > kOutCap) break;
+#pragma unroll
+                                        for (int sub = 0; sub < TS; ++sub) {
+                                            float* v4 = reinterpret_cast<float*>(&val[sub][i]);
+#pragma unroll
+                                            for (int k = 0; k < 4; ++k) {
+                                                const bool big = (__float_as_uint(v4[k]) & 0x7fffffffu) >= high;
+                                                const unsigned mask = __ballot_sync(0xffffffffu, big);
+                                                if (big) {
+                                                    olist[(static_cast<size_t>(blockIdx.x) * 64 + row) * kOutCap + cnt + __popc(mask & ((1u << lane) - 1u))] =
+                                                        static_cast<int>(j0 + sub * static_cast<int64_t>(gridDim.x) * kTK + k);
+                                                    v4[k] = 0.f;
+                                                }
+                                                cnt += __popc(mask);
+                                            }
+                                        }
+                                        fit = kELo;  // if nothing is left, the finest scale will do
+                                    }
+                                    if (lane == 0 && cnt > 0) n_out[row] = cnt;
+                                }
                                 // one bit of headroom: the finer the step, the tighter the bound on the conversion error
-                                E[i] = clamp_e(need + 1);
+                                E[i] = clamp_e(fit + 1);
                                 if (lane == 0) e_cur[row] = E[i];
                                 const float scale = __int_as_float((30 - E[i] + 127) << 23);
 #pragma unroll
                                 for (int sub = 0; sub < TS; ++sub)
                                     t[sub][i] = make_float4(val[sub][i].x * scale, val[sub][i].y * scale, val[sub][i].z * scale, val[sub][i].w * scale);
-                            } else if (need > E[i]) {
+                            } else if (need > E[i]) {  // (a constexpr-else: steps after the first)
                                 // values of magnitude 2^E or more: how many?
                                 int total = 0;
 #pragma unroll
@@ -596,7 +702,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                     if (fi < FC && c * FC + fi < F) {
                         const int r = c * FC + fi;
                         // a row whose scale changes hands its old exponent to the drain that comes before this step
-                        if (lane == 0) e_stage[o * 64 + r] = old[i] == kENone ? E[i] : old[i];
+                        if (lane == 0) e_stage[o * 64 + r] = FIRST ? E[i] : old[i];
                         // row r of a slice: 128 bytes per row, 16-byte chunk (lane/4) ^ (r%8) within it
                         unsigned char* dst = slot + r * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | lane_word);
                         int small = 0;
@@ -622,10 +728,10 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                     }
                 }
             }
-            if (!ok) break;
+            if (!ok) return;
             if (!have_slot && step >= NO && !mbar_wait_live(&op_empty[o], op_phase ^ 1, dead)) {
                 ok = false;
-                break;
+                return;
             }
             fence_async_smem();
             __syncwarp();
@@ -639,7 +745,12 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                 o = 0;
                 op_phase ^= 1;
             }
+        };
+        if (my_steps > 0) {
+            convert_step(std::true_type{}, 0);
+            tiles_left -= TS;
         }
+        for (int64_t step = 1; step < my_steps && ok; ++step, tiles_left -= TS) convert_step(std::false_type{}, step);
         if (ok) {
             // the slot after the last step: current exponents, nothing to multiply
             if (my_steps >= NO && !mbar_wait_live(&op_empty[o], op_phase ^ 1, dead)) ok = false;

@@ -13,7 +13,9 @@ int pairdist_on_device(const float* v, int f, int64_t d, int64_t ld, double* dis
 size_t pairdist_workspace(int f);
 size_t pairdist_workspace_fp32(int f);
 int pairdist_fp32(const float* v, int f, int64_t d, int64_t ld, double* dist, double* partial, const int* gate, cudaStream_t s);
+int pairdist_f64(const float* v, int f, int64_t d, int64_t ld, double* dist, double* partial, const int* gate, cudaStream_t s);
 int pairdist_path_fp32_only();
+int pairdist_path_fp64_only();
 int pairdist_path_i8_forced();
 int vote_pairdist_i8(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted,
                      double* dist, void* ws, int* flag, int force, cudaStream_t s);  // pairdist_i8.cu
@@ -98,10 +100,10 @@ extern "C" int bz_vote_pairdist(const float* replicas, int r, int f, int64_t d, 
     // Vote + integer distances on the tensor cores wherever that kernel exists (it is the faster single
     // pass on every shape measured).  Two repairs follow, both decided on the device from the kernel's flag
     // words and both returning at once in the ordinary case: the vote alone if the kernel stopped early (its
-    // voted rows are then incomplete), and the binary32 distance kernel if it stopped early or its error
+    // voted rows are then incomplete), and the binary64 distance kernel if it stopped early or its error
     // bound asks for it.
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (d > 0 && r > 1 && !pairdist_path_fp32_only()) {
+    if (d > 0 && r > 1 && !pairdist_path_fp32_only() && !pairdist_path_fp64_only()) {
         int* flag = pairdist_status_words(workspace, f);
         st = vote_pairdist_i8(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, dist, pairdist_i8_part(workspace, f), flag,
                               pairdist_path_i8_forced(), s);
@@ -109,11 +111,13 @@ extern "C" int bz_vote_pairdist(const float* replicas, int r, int f, int64_t d, 
             note_path(BZ_PATH_TENSOR);
             st = vote_if(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, flag + 1, s);
             if (st != BZ_OK) return st;
-            return pairdist_fp32(voted, f, d, ld_voted, dist, static_cast<double*>(workspace), flag, s);
+            return pairdist_f64(voted, f, d, ld_voted, dist, static_cast<double*>(workspace), flag, s);
         }
         if (st != 1) return st;
     }
-    if (d > 0 && r > 1) {
+    // the binary32 single pass: only where the caller asked for binary32 (otherwise the two calls below keep the
+    // tolerance on short rows through the binary64 kernel)
+    if (d > 0 && r > 1 && pairdist_path_fp32_only()) {
         st = vote_pairdist_fused(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, dist,
                                  static_cast<double*>(workspace), s);
         if (st == BZ_OK) {

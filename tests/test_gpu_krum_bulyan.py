@@ -53,6 +53,27 @@ def test_pairdist_close_on_gradients(l, r, q, attack, d):
     assert np.array_equal(bz.pairdist(v.to(DEV)).cpu().numpy(), got)
 
 
+@pytest.mark.parametrize("f,d", [(25, 4), (25, 1000), (49, 5000), (25, 300_000), (49, 200_004)])
+def test_binary64_kernel_matches_the_oracle_to_the_last_digits(f, d, monkeypatch):
+    # differences, squares and sums in double precision: only the order of the additions differs from the oracle's
+    monkeypatch.setenv("BZ_PAIRDIST_PATH", "fp64")
+    g = inputs.true_gradients(f, d, seed=f * d % 1000).numpy()
+    g[1, ::7] *= 1.0e4
+    g[f - 1] = g[0]
+    want = oracle.pairdist(g)
+    got = bz.pairdist(torch.from_numpy(g).to(DEV)).cpu().numpy()
+    assert bz.last_path() == bz.PATH_FP64
+    assert np.array_equal(got, got.T) and (np.diag(got) == 0).all() and got[0, f - 1] == 0
+    nz = want > 0
+    assert (np.abs(got[nz] - want[nz]) <= 1e-12 * want[nz]).all()
+    assert np.array_equal(bz.pairdist(torch.from_numpy(g).to(DEV)).cpu().numpy(), got)
+    # rows too short for the integer kernel take it by default
+    if d < 8192:
+        monkeypatch.delenv("BZ_PAIRDIST_PATH")
+        assert np.array_equal(bz.pairdist(torch.from_numpy(g).to(DEV)).cpu().numpy(), got)
+        assert bz.last_path() == bz.PATH_FP64
+
+
 def test_pairdist_unaligned_rows():
     v = inputs.integer_gradients(25, 1003, seed=2)
     buf = torch.zeros((25, 1100), dtype=torch.float32, device=DEV)
