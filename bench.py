@@ -231,7 +231,7 @@ def multikrum_leg(bz, inputs, torch, dist, world, rank, device, steps, warmup, p
            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                         "algorithmic_bytes_per_step": alg_bytes,
                         "kernels": "pairdist_i8_kernel<49,25,3,25,3,1> (vote + integer MMA distances), mean_rows_kernel"},
-           "status_bits": bz.pairdist_status(ws, f) if world == 1 else None}
+           "status_bits (0 = the integer kernel's distances stood)": bz.pairdist_status(ws, f) if world == 1 else None}
     if world == 1:
         return rec, (rep, voted, out, dmat, res[1])
     del rep
