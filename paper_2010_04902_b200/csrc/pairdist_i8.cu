@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(128)
 //   + 2^-39 (|q_a|^2 + |q_b|^2) for the binary64 sums behind D^ (a few thousand roundings of terms of that size)
 // must stay below kRelTol times the final distance D^ + corr.
 template <int F>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
     pairdist_i8_check_kernel(double* __restrict__ dist, const double* __restrict__ corr, const double* __restrict__ norm2,
                              const int* __restrict__ info, int n_ctas, int force, int* __restrict__ flag) {
     __shared__ double s_n2[F];
@@ -121,14 +121,15 @@ __global__ void __launch_bounds__(256)
     const int tid = threadIdx.x;
     if (tid == 0) s_bad = s_marks = 0;
     __syncthreads();
-    // four threads per row, each over every fourth CTA in order; the four sums are added in a fixed order
-    __shared__ double s_part[4][F];
-    if (tid < 4 * F) {
+    // sixteen threads per row, each over every sixteenth CTA in order; their sums are added in a fixed order
+    constexpr int kParts = 16;
+    __shared__ double s_part[kParts][F];
+    if (tid < kParts * F) {
         const int row = tid % F, part = tid / F;
         double n2 = 0.0;
         int over = 0;
-#pragma unroll 4
-        for (int c = part; c < n_ctas; c += 4) {
+#pragma unroll 5
+        for (int c = part; c < n_ctas; c += kParts) {
             const int* rec = info + c * kInfoStride;
             const double half_step = __longlong_as_double(static_cast<long long>(1023 + rec[kInfoE + row] - 31) << 52);
             n2 += reinterpret_cast<const double*>(rec + kInfoN2)[row] + static_cast<double>(rec[kInfoSmall + row]) * half_step * half_step;
@@ -138,7 +139,12 @@ __global__ void __launch_bounds__(256)
         if (over) atomicOr(&s_marks, kBadValues);
     }
     __syncthreads();
-    if (tid < F) s_n2[tid] = (s_part[0][tid] + s_part[1][tid]) + (s_part[2][tid] + s_part[3][tid]);
+    if (tid < F) {
+        double n2 = 0.0;
+#pragma unroll
+        for (int part = 0; part < kParts; ++part) n2 += s_part[part][tid];
+        s_n2[tid] = n2;
+    }
     for (int c = tid; c < n_ctas; c += blockDim.x)
         if (info[c * kInfoStride + kInfoBad]) atomicOr(&s_marks, info[c * kInfoStride + kInfoBad]);
     __shared__ double s_min_nz[F], s_zero_n2[F];
@@ -182,8 +188,6 @@ __global__ void __launch_bounds__(256)
     }
 }
 
-// rep: R = 1: rows [f][d] with leading dimension ld_file.  R > 1: replicas[r][f][d].
-// Returns 1 if the tensor map cannot express the shape.
 struct Scratch {
     double* tpart;
     int* info;
@@ -229,7 +233,7 @@ int launch_i8(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, floa
     note_launch();
     st = check_launch();
     if (st != BZ_OK) return st;
-    pairdist_i8_check_kernel<F><<<1, 256, 0, s>>>(dist, sc.corr, sc.norm2, sc.info, static_cast<int>(ctas), force, flag);
+    pairdist_i8_check_kernel<F><<<1, 1024, 0, s>>>(dist, sc.corr, sc.norm2, sc.info, static_cast<int>(ctas), force, flag);
     note_launch();
     return check_launch();
 }
