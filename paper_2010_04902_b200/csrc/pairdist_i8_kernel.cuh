@@ -402,6 +402,21 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
         float m_run[CH];
 #pragma unroll
         for (int e = 0; e < CH; ++e) m_run[e] = 0.f;
+        // what stays the same from step to step for each row the warp owns: its exponent (e_cur holds a copy for the
+        // other roles) and this lane's byte offset inside a slice of the operand tile
+        int e_reg[CH * RWC];
+        uint32_t dst_off[CH * RWC];
+#pragma unroll
+        for (int cc = 0; cc < CH; ++cc) {
+            const int off_cc = CH == 1 ? cw : ((cw - cc * FC) % W + W) % W;
+#pragma unroll
+            for (int i = 0; i < RWC; ++i) {
+                const int r = cc * FC + off_cc + W * i;
+                e_reg[cc * RWC + i] = kENone;
+                // row r of a slice: 128 bytes per row, 16-byte chunk (lane/4) ^ (r%8) within it
+                dst_off[cc * RWC + i] = static_cast<uint32_t>(r) * 128u + ((((lane >> 2) ^ (r & 7)) << 4) | lane_word);
+            }
+        }
         // One step.  FIRST: the CTA meets the rows for the first time and fixes their scales; kept apart from the
         // steps that follow so that their code carries none of it.
         auto convert_step = [&](auto first_tag, int64_t step) {
@@ -494,7 +509,12 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                 int old[RWC];
 #pragma unroll
                 for (int i = 0; i < RWC; ++i)
-                    if (off + W * i < FC && c * FC + off + W * i < F) old[i] = FIRST ? static_cast<int>(kENone) : static_cast<int>(e_cur[c * FC + off + W * i]);
+                {
+                    old[i] = kENone;
+#pragma unroll
+                    for (int cc = 0; cc < CH; ++cc)
+                        if (cc == c) old[i] = e_reg[cc * RWC + i];
+                }
                 // Every kLookEvery-th step: did the warp's rows of this box-row leave three bits or more of their
                 // scales unused ever since the last look?  Then they get finer ones (a row's magnitude falls as well
                 // as rises from layer to layer, and a step that stays coarse costs precision for all the values that
@@ -530,6 +550,9 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                                     n2_done[row] += static_cast<double>(so_far) * half_step * half_step;
                                     e_cur[row] = old[i] - finer;
                                 }
+#pragma unroll
+                                for (int cc = 0; cc < CH; ++cc)
+                                    if (cc == c) e_reg[cc * RWC + i] = old[i] - finer;
                                 raise = true;
                             }
                         }
@@ -542,7 +565,10 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
 #pragma unroll
                     for (int i = 0; i < RWC; ++i) {
                         if (off + W * i < FC && c * FC + off + W * i < F) {
-                            E[i] = e_cur[c * FC + off + W * i];
+                            E[i] = kENone;
+#pragma unroll
+                            for (int cc = 0; cc < CH; ++cc)
+                                if (cc == c) E[i] = e_reg[cc * RWC + i];
                             const float scale = __int_as_float((30 - E[i] + 127) << 23);
 #pragma unroll
                             for (int sub = 0; sub < TS; ++sub) {
@@ -619,6 +645,9 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                                 // one bit of headroom: the finer the step, the tighter the bound on the conversion error
                                 E[i] = clamp_e(fit + 1);
                                 if (lane == 0) e_cur[row] = E[i];
+#pragma unroll
+                                for (int cc = 0; cc < CH; ++cc)
+                                    if (cc == c) e_reg[cc * RWC + i] = E[i];
                                 const float scale = __int_as_float((30 - E[i] + 127) << 23);
 #pragma unroll
                                 for (int sub = 0; sub < TS; ++sub)
@@ -678,6 +707,9 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                                     raise = true;
                                     E[i] = clamp_e(need + 1);
                                     if (lane == 0) e_cur[row] = E[i];
+#pragma unroll
+                                    for (int cc = 0; cc < CH; ++cc)
+                                        if (cc == c) e_reg[cc * RWC + i] = E[i];
                                     const float scale = __int_as_float((30 - E[i] + 127) << 23);
 #pragma unroll
                                     for (int sub = 0; sub < TS; ++sub)
@@ -703,8 +735,11 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                         const int r = c * FC + fi;
                         // a row whose scale changes hands its old exponent to the drain that comes before this step
                         if (lane == 0) e_stage[o * 64 + r] = FIRST ? E[i] : old[i];
-                        // row r of a slice: 128 bytes per row, 16-byte chunk (lane/4) ^ (r%8) within it
-                        unsigned char* dst = slot + r * 128 + ((((lane >> 2) ^ (r & 7)) << 4) | lane_word);
+                        uint32_t my_off = 0;
+#pragma unroll
+                        for (int cc = 0; cc < CH; ++cc)
+                            if (cc == c) my_off = dst_off[cc * RWC + i];
+                        unsigned char* dst = slot + my_off;
                         int small = 0;
 #pragma unroll
                         for (int sub = 0; sub < TS; ++sub) {
