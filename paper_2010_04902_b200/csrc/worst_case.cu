@@ -101,7 +101,7 @@ struct WcParams {
 __constant__ uint64_t c_binom[kMaxK + 1][kMaxK + 1];
 
 template <int RP, int T>
-__global__ void __launch_bounds__(kWcBlock)
+__global__ void __launch_bounds__(kWcBlock, 12)
     worst_case_kernel(const __grid_constant__ WcParams prm, WcResult* __restrict__ results) {
     __shared__ uint64_t s_mask[kMaxK];
     __shared__ uint64_t s_begin[kMaxK + 1];

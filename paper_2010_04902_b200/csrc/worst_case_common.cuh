@@ -7,7 +7,7 @@
 namespace bz {
 
 constexpr int kWcBlock = 128;
-constexpr int kWcMaxBlocks = kNumSMs * 8;
+constexpr int kWcMaxBlocks = kNumSMs * 12;
 
 struct Planes {
     uint64_t c0, c1, c2;
