@@ -8,7 +8,7 @@
 //
 // Enumeration: a subset is a prefix of p = q - T workers followed by a tail of T <= 5 workers.  The
 // tail is T nested loops with all state in registers; in the innermost one a subset costs a
-// load, an AND and a popcount.  Prefixes are grouped by their largest worker l: inside a group every prefix has the same
+// load, an AND and a popcount, and the loop above it updates count and mask without a bit-sliced add.  Prefixes are grouped by their largest worker l: inside a group every prefix has the same
 // tail range (l, K), so the threads of a warp run the nested loops with identical trip counts.  A
 // group's prefixes are l plus the (p-1)-subsets of {0..l-1}; threads take chunks of consecutive
 // ones, unrank the first with the combinatorial number system and walk lexicographic successors,
@@ -38,20 +38,27 @@ __device__ __forceinline__ uint64_t member_bits(uint64_t prefix_mem, const TailI
     return mem;
 }
 
-// innermost loop: adding worker x distorts exactly the files that were one holder short, so the
-// count under each x is the count of the enclosing subset plus one popcount
-template <int RP, int DEPTH>
-__device__ __forceinline__ void leaf_loop(const uint64_t* __restrict__ s_mask, const Planes& s, int x_lo, int x_hi,
-                                          uint64_t prefix_mem, const TailIds& ids, Best& best);
-
-template <int RP, int DEPTH>
-__device__ __forceinline__ void leaf_loop(const uint64_t* __restrict__ s_mask, const Planes& s, int x_lo, int x_hi,
+// innermost loop: adding worker x distorts exactly the files that were one holder short (`tip`), so the
+// count under each x is the count of the enclosing subset (`base`) plus one popcount
+template <int DEPTH>
+__device__ __forceinline__ void leaf_loop(const uint64_t* __restrict__ s_mask, int base, uint64_t tip, int x_lo, int x_hi,
                                           uint64_t prefix_mem, const TailIds& ids, Best& best) {
-    const int base = count_at_least<RP>(s);
-    const uint64_t tip = one_short<RP>(s);
     for (int x = x_lo; x < x_hi; ++x) {
         const int cnt = base + __popcll(s_mask[x] & tip);
         if (cnt >= best.cnt) offer(best, cnt, member_bits(prefix_mem, ids, DEPTH, x));
+    }
+}
+
+// The loop above the innermost one needs no bit-sliced add either: with worker y added, the count grows by the
+// one-short files y holds, and the new one-short files are the old ones y does not hold plus the two-short ones
+// it does.
+template <int DEPTH>
+__device__ __forceinline__ void pair_loops(const uint64_t* __restrict__ s_mask, int base, uint64_t tip1, uint64_t tip2, int y_lo,
+                                           int y_hi, int K, uint64_t prefix_mem, TailIds& ids, Best& best) {
+    for (int y = y_lo; y < y_hi; ++y) {
+        ids.w[DEPTH] = y;
+        const uint64_t m = s_mask[y];
+        leaf_loop<DEPTH + 1>(s_mask, base + __popcll(tip1 & m), (tip1 & ~m) | (tip2 & m), y + 1, K, prefix_mem, ids, best);
     }
 }
 
@@ -60,7 +67,9 @@ template <int RP, int LEVEL, int DEPTH>
 __device__ __forceinline__ void tail_loops(const uint64_t* __restrict__ s_mask, const Planes& s, int start, int K,
                                            uint64_t prefix_mem, TailIds& ids, Best& best) {
     if constexpr (LEVEL == 1) {
-        leaf_loop<RP, DEPTH>(s_mask, s, start, K, prefix_mem, ids, best);
+        leaf_loop<DEPTH>(s_mask, count_at_least<RP>(s), one_short<RP>(s), start, K, prefix_mem, ids, best);
+    } else if constexpr (LEVEL == 2) {
+        pair_loops<DEPTH>(s_mask, count_at_least<RP>(s), one_short<RP>(s), two_short<RP>(s), start, K - 1, K, prefix_mem, ids, best);
     } else {
         for (int y = start; y <= K - LEVEL; ++y) {
             ids.w[DEPTH] = y;
@@ -75,7 +84,9 @@ __device__ __forceinline__ void tail_top(const uint64_t* __restrict__ s_mask, co
                                          uint64_t mem, Best& best) {
     TailIds ids;
     if constexpr (LEVEL == 1) {
-        leaf_loop<RP, 0>(s_mask, s, y_lo, y_hi, mem, ids, best);
+        leaf_loop<0>(s_mask, count_at_least<RP>(s), one_short<RP>(s), y_lo, y_hi, mem, ids, best);
+    } else if constexpr (LEVEL == 2) {
+        pair_loops<0>(s_mask, count_at_least<RP>(s), one_short<RP>(s), two_short<RP>(s), y_lo, y_hi, K, mem, ids, best);
     } else {
         for (int y = y_lo; y < y_hi; ++y) {
             ids.w[0] = y;

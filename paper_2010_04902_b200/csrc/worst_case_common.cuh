@@ -49,6 +49,14 @@ template <int RP> __device__ __forceinline__ uint64_t one_short(const Planes& s)
         return s.c0 & s.c1 & ~s.c2;
 }
 
+// files with exactly RP-2 holders: those two more holders would tip over the threshold
+template <int RP> __device__ __forceinline__ uint64_t two_short(const Planes& s) {
+    if constexpr (RP == 1)
+        return 0;
+    else
+        return one_short<RP - 1>(s);
+}
+
 struct Best {
     int cnt;
     uint64_t mem;
