@@ -165,6 +165,17 @@ def test_validation_runs_before_any_launch(lib):
     bad = mask.copy()
     bad[3] = np.uint64(1) << np.uint64(40)  # a file index >= f
     assert L.bz_worst_case(bad.ctypes.data, 15, 25, 3, 2, 0, po, None, None, fake, 1 << 20, None) == bz.ERR_INVALID_ARG
+    # the calls added around the distance stage: status, probe, path
+    st = ctypes.c_int32(0)
+    assert L.bz_pairdist_status(None, 25, ctypes.addressof(st), None) == bz.ERR_INVALID_ARG
+    assert L.bz_pairdist_status(fake, 25, None, None) == bz.ERR_INVALID_ARG
+    assert L.bz_pairdist_status(fake, 0, ctypes.addressof(st), None) == bz.ERR_INVALID_ARG
+    assert L.bz_pairdist_status(fake, 129, ctypes.addressof(st), None) == bz.ERR_UNSUPPORTED
+    assert L.bz_stream_probe(fake, 64, 0, None, None) == bz.ERR_INVALID_ARG
+    assert L.bz_stream_probe(None, 64, 1, fake, None) == bz.ERR_INVALID_ARG
+    assert L.bz_stream_probe(ctypes.c_void_p(264), 64, 0, fake, None) == bz.ERR_INVALID_ARG      # 16-byte alignment
+    assert L.bz_stream_probe(fake, 60, 1, fake, None) == bz.ERR_INVALID_ARG                      # whole 64-bit words
+    assert L.bz_last_path() in range(8)
     assert bz.kernel_launch_count() == n0
 
 
