@@ -383,7 +383,7 @@ def run_ours(args):
 
     # ---- the metric's second aggregator: Multi-Krum (every rank; one all-reduce when N > 1) --------------
     if not args.no_extra and args.coords == 0:
-        sec, keep = multikrum_leg(bz, inputs, torch, dist, world, rank, device, max(5, min(args.steps, 50)), 3, peak)
+        sec, keep = multikrum_leg(bz, inputs, torch, dist, world, rank, device, max(5, min(args.steps, 50)), 10, peak)
         if rank == 0:
             result["secondary"] = sec
             if world == 1 and not args.no_cpu:
