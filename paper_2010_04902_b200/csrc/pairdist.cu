@@ -1,13 +1,14 @@
 // Pairwise squared distances between the f voted gradients - the O(f^2 d) part of the Krum family
-// (Sec. 1.2; cost in Appendix A.1): the binary32 kernels, the dispatch between them and the integer
-// tensor-core kernel (pairdist_i8_kernel.cuh, the default for f = 25 and 49), and the entry point that
-// keeps its scratch in a built-in array.
+// (Sec. 1.2; cost in Appendix A.1): the binary32 and binary64 kernels, the dispatch between them and the
+// integer tensor-core kernel (pairdist_i8_kernel.cuh, the default for f = 25 and 49), and the entry point
+// that keeps its scratch in a built-in array.
 //
-// The kernels here accumulate the difference form sum_j (v_a[j] - v_b[j])^2 in binary32: its accuracy
-// does not depend on a common offset of the rows (gradients share a large per-coordinate mean) nor on
-// the size of an attacker's payload in other rows.  They are bound by the FP32 pipe (f(f-1) add/fma
-// lane-operations per coordinate) and serve every shape the integer kernel does not take, its fall-back
-// when its own error bound or a row's values ask for one, and bz_pairdist_static.
+// The kernels here accumulate the difference form sum_j (v_a[j] - v_b[j])^2: its accuracy does not depend
+// on a common offset of the rows (gradients share a large per-coordinate mean) nor on the size of an
+// attacker's payload in other rows.  The binary32 kernels are bound by the FP32 pipe (f(f-1) add/fma
+// lane-operations per coordinate) and serve the shapes the integer kernel does not take, and
+// bz_pairdist_static.  The binary64 kernel (f = 25 and 49) answers where the integer kernel's error bound
+// or a row's values ask for a recomputation, and for rows too short for that kernel.
 #include <atomic>
 #include <cstdlib>
 #include <cstring>
