@@ -15,7 +15,8 @@
 // every 512 tiles (32-bit headroom), when a row changes its scale and at the end; a drain combines the
 // blocks in binary64 and adds
 //     T[a][b] += 2^(E_a + E_b - 60) * sum_blocks weight * S_i S_j^T [a][b]
-// to the CTA's partial matrix (in shared memory, written out once).  A last kernel forms, per CTA and then over CTAs in a fixed order,
+// to the CTA's partial matrix (in shared memory, written out once).  A last kernel forms, per CTA and
+// then over CTAs in a fixed order,
 //     D[a][b] = (T[a][a] + T[b][b]) - (T[a][b] + T[b][a]).
 // Identical rows give identical integers and therefore exactly equal distances and D = 0.
 //
@@ -23,12 +24,11 @@
 // fixes E_a when it first meets the row: one bit above the power of two that bounds the magnitudes of
 // its first step.  Values whose binary exponent lies within 7 of E_a keep all 24 bits; smaller ones are
 // rounded, by at most half a step, and the converters count them (n_small: a superset, read off the top
-// bytes).  With N_a^2 = sum of
-// n_small * (step/2)^2 over CTAs (and over a row's successive scales) the computed distance obeys
-// |D^ - D| <= 2 (N_a + N_b) sqrt(D^) + (N_a + N_b)^2 (Cauchy-Schwarz): a bound that holds for every
-// input, also for rows whose rounding errors were arranged to line up.  The last kernel compares it with
-// the library's distance tolerance and raises a flag when it does not fit; the caller then runs the
-// binary32 difference-form kernel, which starts by looking at that flag.
+// bytes).  With N_a^2 = sum of n_small * (step/2)^2 over CTAs (and over a row's successive scales) the
+// computed distance obeys |D^ - D| <= 2 (N_a + N_b) sqrt(D^) + (N_a + N_b)^2 (Cauchy-Schwarz): a bound
+// that holds for every input, also for rows whose rounding errors were arranged to line up.  The last
+// kernel compares it with the library's distance tolerance and raises a flag when it does not fit; the
+// caller then runs the binary64 difference-form kernel, which starts by looking at that flag.
 // A later value that does not fit the row's scale (magnitude 2^E_a or more) is an outlier as long as the
 // CTA has met at most kOutCap of them in that row - the rare large values of a heavy-tailed row: it
 // enters the contraction as zero and its coordinate goes on a short list kept per CTA and row; a small
@@ -51,7 +51,7 @@
 // (row r belongs to warp r % W), vote them if there are copies, fix their scales and write the
 // operand tiles (K-major, 128-byte swizzle) of a second ring; one thread issues the MMAs; four warps
 // drain.  Every mbarrier wait is bounded; on expiry the CTA stops, marks its record (the host side then
-// repairs the result with the binary32 kernel) and g_i8_timeouts is raised.  Loads are plain per-CTA loads.
+// repairs the result with the binary64 kernel) and g_i8_timeouts is raised.  Loads are plain per-CTA loads.
 // Every hand-off of shared memory between roles is an mbarrier arrival with release semantics paired with the
 // waiter's acquire: converter -> loader (box read), converter -> MMA thread (operand tiles, exponents, flush
 // request), MMA thread -> drain warps -> MMA thread.
@@ -73,7 +73,7 @@ constexpr int kENone = -1000, kELo = -64, kEHi = 64;
 constexpr int kCtlBytes = 3072;
 // ints per CTA in the record the converters leave: the rows' exponents, their counts of values that may have
 // been rounded, their counts of outliers, then the "bad" mark
-// (kInfoN2: 64 doubles - the squared rounding budget a row used up under earlier, finer scales)
+// (kInfoN2: 64 doubles - the squared rounding budget a row used up under its earlier scales)
 constexpr int kInfoE = 0, kInfoSmall = 64, kInfoOut = 128, kInfoN2 = 192, kInfoBad = 320, kInfoStride = 328;
 constexpr int kLookEvery = 4;        // steps between two looks at whether rows would fit a finer scale
 constexpr int kOutCap = 8;           // listed outliers per CTA and row; a row that has more gets a coarser scale
