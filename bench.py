@@ -226,7 +226,8 @@ def multikrum_leg(bz, inputs, torch, dist, world, rank, device, steps, warmup, p
     rec = {"metric": "aggregated gradient coordinates/sec (vote + Multi-Krum from the replicas)", "value": world * d / (ms * 1e-3),
            "unit": UNIT, "ms_per_step": ms, "ms_best": min(each), "ms_median": statistics.median(each), "steps": steps,
            "workload": "K=21 r=3 l=7 f=49 d=11.2M per GPU, q=5 ALIE, c=5 m=44; bz_vote_multikrum"
-                       + ("" if world == 1 else " per coordinate slab + one all-reduce of the 49x49 fp64 matrix (NCCL)"),
+                       + ("" if world == 1 else " per coordinate slab + one all-reduce of the 49x49 fp64 matrix (%s)"
+                          % os.environ.get("BZ_BENCH_DIST_BACKEND", "nccl")),
            "c_max": cmax, "gpu_launches": int(launches),
            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                         "algorithmic_bytes_per_step": alg_bytes,
@@ -280,11 +281,18 @@ def run_ours(args):
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the aggregation path has no CPU fallback")
+    # one rank per GPU.  (BZ_BENCH_DIST_BACKEND=gloo lets several ranks share the GPUs there are - a functional check of
+    # the multi-rank path on a smaller box, not a measurement: NCCL wants a device per rank.)
+    backend = os.environ.get("BZ_BENCH_DIST_BACKEND", "nccl")
+    local_rank = local_rank if backend == "nccl" else local_rank % torch.cuda.device_count()
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
     if world > 1:
         os.environ.setdefault("NCCL_DEBUG", "INFO")   # NCCL's own account of the transport (NVLS, rings) goes to stderr
-        dist.init_process_group("nccl", device_id=device)
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=device)
+        else:
+            dist.init_process_group(backend)
     if rank == 0:
         bz_build.build()
     if world > 1:
@@ -346,7 +354,8 @@ def run_ours(args):
             "config": {"workload": workload_name(cfg), "coordinates_per_gpu": d, "c_max": cmax,
                        "byzantine_workers": [int(u) for u in byz],
                        "l2": "inputs are %.2f GB per step, far larger than the 126 MB L2; no flush needed" % (4 * r * f * d / 1e9),
-                       "parallelism": "coordinate slabs, no collective" if world > 1 else "single GPU"},
+                       "parallelism": ("coordinate slabs, no collective" + ("" if backend == "nccl" else " (%s backend, ranks sharing GPUs: "
+                                       "functional check only)" % backend)) if world > 1 else "single GPU"},
             "e2e": e2e,
             "gpu_launches": int(launches),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
