@@ -601,7 +601,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                                 // set by them would be coarse for everything that follows.
                                 int fit = need, cnt = 0;
                                 if (need <= 60) {
-                                    for (int round = 0; round < 4; ++round) {
+                                    for (int round = 0; round < 5; ++round) {  // the last round only measures what is left
                                         uint32_t top = 0;
 #pragma unroll
                                         for (int sub = 0; sub < TS; ++sub) {
@@ -610,9 +610,12 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                                             for (int k = 0; k < 4; ++k) top = max(top, __float_as_uint(v4[k]) & 0x7fffffffu);
                                         }
                                         top = __reduce_max_sync(0xffffffffu, top);
-                                        if (top == 0) break;
+                                        if (top == 0) {
+                                            fit = kELo;  // nothing but zeros (left): the finest scale will do
+                                            break;
+                                        }
                                         fit = static_cast<int>(top >> 23) - 126;
-                                        if (fit <= kELo + 8) break;
+                                        if (round == 4 || fit <= kELo + 8) break;
                                         const uint32_t high = static_cast<uint32_t>(fit - 3 + 126) << 23;  // 2^(fit - 3) and up
                                         int n_high = 0;
 #pragma unroll
@@ -638,7 +641,6 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                                                 cnt += __popc(mask);
                                             }
                                         }
-                                        fit = kELo;  // if nothing is left, the finest scale will do
                                     }
                                     if (lane == 0 && cnt > 0) n_out[row] = cnt;
                                 }

@@ -83,6 +83,25 @@ def test_outliers_late_in_a_row():
     _check_close(dist.cpu().numpy(), want)
 
 
+def test_outliers_where_a_cta_first_meets_a_row():
+    # eight isolated values of very different sizes inside the first 256 coordinates (the first step of CTA 0): they
+    # are peeled off two at a time before the row's scale is fixed, so the scale is that of the ordinary values and
+    # nothing of the row is lost; a ninth would set the scale instead (the second case)
+    f, d = 49, 300_000
+    for extra in (0, 1):
+        g = inputs.true_gradients(f, d, seed=31 + extra).numpy()
+        for k, mag in enumerate([3.0e7, -2.0e7, 4.0e5, 3.5e5, -6.0e3, 5.0e3, 90.0, -80.0] + [40.0] * extra):
+            g[12, 3 + 29 * k] = mag
+        g[20, 5] = 1.0e4
+        want = oracle.pairdist(g)
+        ws = bz.alloc_workspace(bz.OP_PAIRDIST, 0, f, d)
+        got = bz.pairdist(torch.from_numpy(g).to(DEV), workspace=ws).cpu().numpy()
+        assert bz.last_path() == bz.PATH_TENSOR
+        _check_close(got, want)
+        if extra == 0:
+            assert bz.pairdist_status(ws, f) == 0
+
+
 def test_a_row_that_outgrows_its_scale():
     # more large values than a list holds (78 inside one tile; and a whole stretch of the row 300 times larger, the
     # way gradients change magnitude from layer to layer): the CTAs that meet them give the row a coarser scale
