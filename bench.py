@@ -517,6 +517,7 @@ def sweep(bz, inputs, torch, device, peak):
     one set per translation orbit beyond)."""
     cells, counts = [], []
     cells.append({"l": 5, "r": 7, "status": "infeasible: r > l (at most l - 1 Latin squares, l parallel classes; Sec. 4.1.1, Eq. 7)"})
+    c_of = {}
     for l, r, q in SWEEP_SHAPES:
         K, f = l * r, l * l
         _, fw, mask = bz.assign_mols(l, r)
@@ -538,8 +539,12 @@ def sweep(bz, inputs, torch, device, peak):
             n_sets += int(n_)
         counts.append({"l": l, "r": r, "K": K, "q": [1, (K - 1) // 2], "c_max": cm, "seconds": time.perf_counter() - t0,
                        "sets_evaluated": n_sets, "first_q_by_orbits": (methods.index("orbits") + 1) if "orbits" in methods else None})
-        cmax_q = cm[q - 1]
-        for d in (1_000_000, 10_000_000, 100_000_000):
+        c_of[(l, r)] = cm[q - 1]
+    # the short cells first: the long ones leave the board at its power cap for a while
+    for d in (1_000_000, 10_000_000, 100_000_000):
+        for l, r, q in SWEEP_SHAPES:
+            f = l * l
+            cmax_q = c_of[(l, r)]
             need = 4 * d * (r * f + f + 3) * 1.03 + (1 << 28)
             free = torch.cuda.mem_get_info()[0]
             cell = {"l": l, "r": r, "f": f, "d": d, "q": q, "c": cmax_q, "m": f - cmax_q}
