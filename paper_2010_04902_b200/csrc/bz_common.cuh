@@ -33,23 +33,17 @@ __device__ __forceinline__ uint32_t key_bits(int key) { return static_cast<uint3
 __device__ __forceinline__ int kmin(int a, int b) { return min(a, b); }
 __device__ __forceinline__ int kmax(int a, int b) { return max(a, b); }
 
-#define BZ_CE(a, b)                         \
-    {                                       \
-        const T lo_ = kmin(k[a], k[b]);     \
-        k[b] = kmax(k[a], k[b]);            \
-        k[a] = lo_;                         \
-    }
 // Integer min/max issue on the ALU pipe (64 lanes per SM and clock) while the multiply-add pipe idles in a
 // comparator network.  max = a + b - min (exact modulo 2^32) as two integer multiply-adds moves one of a
 // comparator's two operations there; the multipliers are read from constant memory so that the compiler
 // cannot fold them into an addition (which would issue on the ALU pipe again).  A loop of comparators alone
-// runs 26 % faster with every other comparator done this way (the networks mark two of three, since the
-// kernels have other ALU work besides); only kernels bound by the ALU pipe ask for it.
+// runs 26 % faster with every other comparator done this way; a network's run<NUM, DEN> does it for NUM of
+// every DEN full comparators, and only kernels bound by the ALU pipe ask for it.
 static __constant__ unsigned int kPipeOne = 1u, kPipeMinusOne = 0xffffffffu;
-#define BZ_CM(a, b)                                                                                               \
+#define BZ_CE(a, b, i)                                                                                            \
     {                                                                                                             \
         const T lo_ = kmin(k[a], k[b]);                                                                           \
-        if constexpr (MIX)                                                                                        \
+        if constexpr (((i) % DEN) < NUM)                                                                          \
             k[b] = static_cast<T>(static_cast<unsigned int>(lo_) * kPipeMinusOne +                                \
                                   (static_cast<unsigned int>(k[a]) * kPipeOne + static_cast<unsigned int>(k[b]))); \
         else                                                                                                      \

@@ -2,9 +2,9 @@
 
 Writes csrc/sort_networks.inc with
   * MedianNet<N>::run  - a network that leaves the element of rank (N-1)/2 on wire (N-1)/2,
-    obtained from Batcher's odd-even merge sort for N inputs by deleting every comparator (or
-    comparator half) the middle output does not depend on;
-  * SortNet<N>::run    - the full odd-even merge sort, for the trimmed mean.
+    obtained from an odd-even merge sort of N inputs by deleting every comparator (or comparator
+    half) the middle output does not depend on;
+  * SortNet<N>::run    - the full merge sort, for the trimmed mean.
 
 The sizes are those of the coordinate-wise median over f = l*l files (l = 3, 5, 7) and of Bulyan's
 selection sets theta = f - 2c for every c with f >= 4c + 3.
@@ -13,6 +13,7 @@ Run `python gen_networks.py` to rewrite the .inc file, `python gen_networks.py -
 that the committed file is current and that every network is correct (0-1 principle: exhaustively
 for N <= 25, on random 0/1 and integer inputs above).
 """
+import functools
 import os
 import random
 import sys
@@ -26,22 +27,71 @@ MEDIAN_SIZES = [9, 25, 49]
 SORT_SIZES = sorted(set([f - 2 * c for f in (25, 49) for c in range(0, (f - 3) // 4 + 1)] + [5, 7, 9]))
 
 
-def batcher(n):
-    """Comparators (lo_wire, hi_wire) of Batcher's odd-even merge sort for any n."""
-    ces = []
-    p = 1
-    while p < n:
-        k = p
-        while k >= 1:
-            j = k % p
-            while j + k < n:
-                for i in range(min(k, n - j - k)):
-                    if (i + j) // (2 * p) == (i + j + k) // (2 * p):
-                        ces.append((i + j, i + j + k))
-                j += 2 * k
-            k //= 2
-        p *= 2
-    return ces
+def odd_even_merge(a, b):
+    """Batcher's odd-even merge of two sorted runs of any lengths.  a, b: the wires holding each run in
+    ascending order.  Returns (comparators, wires of the merged run in ascending order): the elements at
+    even and at odd positions of both runs are merged recursively, then neighbours are exchanged."""
+    if not a:
+        return [], list(b)
+    if not b:
+        return [], list(a)
+    if len(a) == 1 and len(b) == 1:
+        return [(a[0], b[0])], [a[0], b[0]]
+    ces_v, v = odd_even_merge(a[0::2], b[0::2])
+    ces_w, w = odd_even_merge(a[1::2], b[1::2])
+    ces = ces_v + ces_w
+    out = [v[0]]
+    pairs = min(len(w), len(v) - 1)
+    for i in range(pairs):
+        ces.append((w[i], v[i + 1]))
+        out += [w[i], v[i + 1]]
+    out += w[pairs:] + v[pairs + 1:]
+    return ces, out
+
+
+@functools.lru_cache(None)
+def merge_count(m, n):
+    return len(odd_even_merge(list(range(m)), list(range(m, m + n)))[0])
+
+
+@functools.lru_cache(None)
+def best_split(n):
+    """(comparators, size of the first part) of the cheapest merge sort of n wires."""
+    if n <= 1:
+        return 0, 0
+    return min((best_split(a)[0] + best_split(n - a)[0] + merge_count(a, n - a), a) for a in range(1, n // 2 + 1))
+
+
+def merge_sort_wires(wires):
+    n = len(wires)
+    if n <= 1:
+        return [], list(wires)
+    a = best_split(n)[1]
+    ces_a, run_a = merge_sort_wires(wires[:a])
+    ces_b, run_b = merge_sort_wires(wires[a:])
+    ces_m, run = odd_even_merge(run_a, run_b)
+    return ces_a + ces_b + ces_m, run
+
+
+def by_layers(ces):
+    """The same comparators, earliest layer first (a comparator's layer is one more than the later layer of its
+    two wires' previous comparators): independent comparators end up next to each other."""
+    depth, keyed = {}, []
+    for pos, (a, b) in enumerate(ces):
+        layer = 1 + max(depth.get(a, 0), depth.get(b, 0))
+        depth[a] = depth[b] = layer
+        keyed.append((layer, pos, (a, b)))
+    return [ce for _, _, ce in sorted(keyed)]
+
+
+def merge_sort(n):
+    """Comparators (wire of the min, wire of the max) of a merge sort of n wires whose splits minimise the
+    comparator count (Batcher's network when n is a power of two; for other n it saves up to 16 % on padding
+    to the next power).  Wires are renamed so that wire i ends with the element of rank i; a comparator may
+    therefore put its min on the higher-numbered wire."""
+    ces, run = merge_sort_wires(list(range(n)))
+    name = {w: i for i, w in enumerate(run)}
+    return by_layers([(name[a], name[b]) for a, b in ces])
 
 
 def prune(ces, outputs):
@@ -147,23 +197,24 @@ def verify_sort(ces, n):
 def emit():
     lines = [
         "// GENERATED by gen_networks.py - do not edit.  Comparator networks on register arrays:",
-        "// BZ_CE(a,b) orders wires a <= b; BZ_LO / BZ_HI keep only the min on a / the max on b.",
-        "// BZ_CM is a BZ_CE that run<true> computes on the multiply-add pipe (two of three full comparators).",
+        "// BZ_CE(a,b,i) leaves the min on wire a and the max on wire b; BZ_LO / BZ_HI keep only the min on a / the max",
+        "// on b.  i numbers the full comparators: run<NUM, DEN> computes the max of those with i % DEN < NUM on the",
+        "// multiply-add pipe.",
         "",
     ]
     for n in MEDIAN_SIZES:
-        net = prune(batcher(n), [(n - 1) // 2])
+        net = prune(merge_sort(n), [(n - 1) // 2])
         verify_median(net, n)
         ops = sum(int(x) + int(y) for _, _, x, y in net)
         lines.append("// median of %d: %d comparators, %d min/max operations" % (n, len(net), ops))
         lines.append("template <> struct MedianNet<%d> {" % n)
-        lines.append("    template <bool MIX = false, typename T> __device__ __forceinline__ static T run(T (&k)[%d]) {" % n)
+        lines.append("    template <int NUM = 0, int DEN = 1, typename T> __device__ __forceinline__ static T run(T (&k)[%d]) {" % n)
         body = []
         full = 0
         for a, b, na, nb in net:
             if na and nb:
+                body.append("BZ_CE(%d,%d,%d)" % (a, b, full))
                 full += 1
-                body.append(("BZ_CM(%d,%d)" if full % 3 else "BZ_CE(%d,%d)") % (a, b))
             else:
                 body.append(("BZ_LO(%d,%d)" if na else "BZ_HI(%d,%d)") % (a, b))
         for i in range(0, len(body), 8):
@@ -173,12 +224,12 @@ def emit():
         lines.append("};")
         lines.append("")
     for n in SORT_SIZES:
-        ces = batcher(n)
+        ces = merge_sort(n)
         verify_sort(ces, n)
         lines.append("// sort of %d: %d comparators" % (n, len(ces)))
         lines.append("template <> struct SortNet<%d> {" % n)
-        lines.append("    template <bool MIX = false, typename T> __device__ __forceinline__ static void run(T (&k)[%d]) {" % n)
-        body = [("BZ_CM(%d,%d)" if i % 3 else "BZ_CE(%d,%d)") % (a, b) for i, (a, b) in enumerate(ces)]
+        lines.append("    template <int NUM = 0, int DEN = 1, typename T> __device__ __forceinline__ static void run(T (&k)[%d]) {" % n)
+        body = ["BZ_CE(%d,%d,%d)" % (a, b, i) for i, (a, b) in enumerate(ces)]
         for i in range(0, len(body), 8):
             lines.append("        " + " ".join(body[i:i + 8]))
         lines.append("    }")

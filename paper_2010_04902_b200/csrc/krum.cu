@@ -260,35 +260,73 @@ __global__ void __launch_bounds__(256) mean_rows_kernel(const V* __restrict__ v,
     }
 }
 
-// Window of the BETA sorted values closest to the median.  The greedy growth (lower neighbour on
-// ties) is a merge of the two distance sequences: the p-th lower value enters before the q-th upper
-// one iff its distance is not larger, so it belongs to the window iff the (BETA-p)-th upper value
-// does not exist or is at least as far.  The number L of such p fixes the window [MID-L, MID-L+BETA).
-// s[] ascending; returns the mean of the window (binary64 sum, ascending).
+// The window grown one value at a time, as the definition states it: the neighbour (below or above) that is
+// closer to the median in binary32 enters, the lower one on ties.  Used as written by the run-time-theta kernel
+// and, out of line, by the register kernels for columns that hold an infinity or a NaN (a comparison with a NaN
+// distance is false, which takes the upper neighbour).
+__device__ __noinline__ float window_mean_stepwise(const float* s, int theta, int beta) {
+    const int mid = (theta - 1) / 2;
+    const float med = s[mid];
+    int lo = mid, hi = mid;
+    while (hi - lo + 1 < beta) {
+        const bool can_lo = lo > 0, can_hi = hi < theta - 1;
+        bool take_lo = can_lo;
+        if (can_lo && can_hi) take_lo = fabsf(__fsub_rn(s[lo - 1], med)) <= fabsf(__fsub_rn(s[hi + 1], med));
+        if (take_lo) --lo; else ++hi;
+    }
+    double sum = 0.0;
+    for (int t = lo; t <= hi; ++t) sum += static_cast<double>(s[t]);
+    return static_cast<float>(sum / static_cast<double>(beta));
+}
+
+// Window of the BETA sorted values closest to the median, without the steps.  With finite values the two
+// sequences of distances ascend, so growing the window merges them: the p-th lower value enters before the
+// q-th upper one iff its distance is not larger, hence it belongs to the window iff the (BETA-p)-th upper value
+// does not exist or is at least as far.  Of each such pair exactly one is in the window (it holds BETA-1 values
+// besides the median), so the tests themselves are the membership flags and no window bounds are formed.
+// s[] ascending in the total order, which puts every infinity and NaN at an end: those columns take the steps.
+// Returns the mean of the window (binary64 sum, ascending).
 template <int THETA, int BETA> __device__ __forceinline__ float window_mean(const float (&s)[THETA]) {
     constexpr int MID = (THETA - 1) / 2;
+    constexpr float kInf = __builtin_huge_valf();
+    if (!(fabsf(s[0]) < kInf && fabsf(s[THETA - 1]) < kInf)) {
+        float copy[THETA];
+#pragma unroll
+        for (int t = 0; t < THETA; ++t) copy[t] = s[t];
+        return window_mean_stepwise(copy, THETA, BETA);
+    }
     const float med = s[MID];
-    int L = 0;
+    bool in[THETA];
+#pragma unroll
+    for (int t = 0; t < THETA; ++t) in[t] = (t == MID);
 #pragma unroll
     for (int p = 1; p <= MID && p <= BETA - 1; ++p) {
         const int up = MID + (BETA - p);  // index of the (BETA-p)-th upper value
         if (up > THETA - 1) {
-            ++L;
+            in[MID - p] = true;
         } else {
-            const float dl = fabsf(__fsub_rn(s[MID - p], med)), du = fabsf(__fsub_rn(s[up], med));
-            L += (du >= dl);
+            const bool lower = fabsf(__fsub_rn(s[up], med)) >= fabsf(__fsub_rn(s[MID - p], med));
+            in[MID - p] = lower;
+            in[up] = !lower;
         }
     }
-    const int lo = MID - L, hi = lo + BETA - 1;
+    // upper values that no lower value competes with (BETA - u > MID): always in
+#pragma unroll
+    for (int u = 1; u <= BETA - 1 && MID + u <= THETA - 1; ++u)
+        if (BETA - u > MID) in[MID + u] = true;
     double sum = 0.0;
 #pragma unroll
-    for (int t = 0; t < THETA; ++t) {
-        if (t >= MID - (BETA - 1) && t <= MID + (BETA - 1)) {  // the only positions a window can cover
-            if (t >= lo && t <= hi) sum += static_cast<double>(s[t]);
-        }
-    }
+    for (int t = 0; t < THETA; ++t)
+        if (in[t]) sum += static_cast<double>(s[t]);
     return static_cast<float>(sum / static_cast<double>(BETA));
 }
+
+// Share of the sort's comparators whose max goes through the multiply-add pipe (kMaxOnFma of every kMaxOf).
+#ifndef BZ_TM_MAX_ON_FMA
+#define BZ_TM_MAX_ON_FMA 2
+#define BZ_TM_MAX_OF 3
+#endif
+constexpr int kMaxOnFma = BZ_TM_MAX_ON_FMA, kMaxOf = BZ_TM_MAX_OF;
 
 // V coordinates per thread (V = 2, 4: 64- and 128-bit loads, rows aligned accordingly): the address arithmetic
 // and the load instructions are shared by the V coordinates.
@@ -332,7 +370,7 @@ __global__ void __launch_bounds__(128) trimmed_mean_kernel(const float* __restri
         float res[V];
 #pragma unroll
         for (int c = 0; c < V; ++c) {
-            SortNet<THETA>::template run<true>(k[c]);  // bound by the ALU pipe: comparators on two pipes
+            SortNet<THETA>::template run<kMaxOnFma, kMaxOf>(k[c]);  // bound by the ALU pipe: comparators on two pipes
             float s[THETA];
 #pragma unroll
             for (int t = 0; t < THETA; ++t) s[t] = __uint_as_float(key_bits(k[c][t]));
@@ -370,22 +408,9 @@ __global__ void __launch_bounds__(128) trimmed_mean_generic_kernel(const float* 
             }
             k[pos] = x;
         }
-        const int mid = (theta - 1) / 2;
-        const float med = __uint_as_float(key_bits(k[mid]));
-        int lo = mid, hi = mid;
-        while (hi - lo + 1 < beta) {
-            const bool can_lo = lo > 0, can_hi = hi < theta - 1;
-            bool take_lo = can_lo;
-            if (can_lo && can_hi) {
-                const float dl = fabsf(__fsub_rn(__uint_as_float(key_bits(k[lo - 1])), med));
-                const float dh = fabsf(__fsub_rn(__uint_as_float(key_bits(k[hi + 1])), med));
-                take_lo = dl <= dh;
-            }
-            if (take_lo) --lo; else ++hi;
-        }
-        double sum = 0.0;
-        for (int t = lo; t <= hi; ++t) sum += static_cast<double>(__uint_as_float(key_bits(k[t])));
-        out[j] = static_cast<float>(sum / static_cast<double>(beta));
+        float sorted[BZ_MAX_F];
+        for (int t = 0; t < theta; ++t) sorted[t] = __uint_as_float(key_bits(k[t]));
+        out[j] = window_mean_stepwise(sorted, theta, beta);
     }
 }
 

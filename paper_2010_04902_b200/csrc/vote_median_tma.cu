@@ -12,6 +12,11 @@
 // new tiles, drains the loads it has already issued (bounded as well) and returns.
 #include "tma_pipeline.cuh"
 
+#ifndef BZ_VM_MAX_ON_FMA
+#define BZ_VM_MAX_ON_FMA 2
+#define BZ_VM_MAX_OF 3
+#endif
+
 namespace bz {
 
 namespace {
@@ -34,7 +39,8 @@ __global__ void __launch_bounds__(kThreads)
     vote_median_tma_kernel(const __grid_constant__ CUtensorMap map, int64_t d, float* __restrict__ out,
                            const ModelUpdate upd) {
     using S = Shape<R, F, FC>;
-    constexpr bool kMixPipes = R == 1 || (R == 5 && F == 49);  // where the ALU pipe limits the kernel (measured)
+    // where the ALU pipe limits the kernel (measured), two of three comparators compute their max on the other pipe
+    constexpr int kMaxOnFma = (R == 1 || (R == 5 && F == 49)) ? BZ_VM_MAX_ON_FMA : 0, kMaxOf = BZ_VM_MAX_OF;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     float* stages = reinterpret_cast<float*>(smem_raw);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + static_cast<size_t>(STAGES) * S::kStageBytes);
@@ -115,7 +121,7 @@ __global__ void __launch_bounds__(kThreads)
                 if ((tid & 31) == 0) mbar_arrive(&empty[s]);  // this warp is done reading the stage
             }
             if (alive && j < d) {
-                const float med = __uint_as_float(key_bits(MedianNet<F>::template run<kMixPipes>(key)));
+                const float med = __uint_as_float(key_bits(MedianNet<F>::template run<kMaxOnFma, kMaxOf>(key)));
                 if (out != nullptr) out[j] = med;
                 if (has_w) {
                     upd.w[j] = update_lane(w_old, v_old, med, upd.eta, upd.mu, has_v);

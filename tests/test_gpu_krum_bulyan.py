@@ -183,6 +183,28 @@ def test_trimmed_mean_layouts(theta, beta, d, ld, shift, out_shift):
     assert (out_buf[:out_shift] == -7.0).all() and (out_buf[out_shift + d:] == -7.0).all()
 
 
+@pytest.mark.parametrize("theta,beta", [(17, 9), (15, 5), (23, 21), (39, 29), (11, 5)])
+def test_trimmed_mean_with_infinities_and_nans(theta, beta):
+    # Columns holding +-inf or NaN: distances to the median can be NaN, and the window then follows the stepwise
+    # rule (a false comparison takes the upper neighbour).  NaN results compare equal whatever their payload.
+    rng = np.random.default_rng(theta * 7 + beta)
+    f, d = max(theta, 25), 4096
+    v = rng.standard_normal((f, d)).astype(np.float32)
+    specials = np.array([np.inf, -np.inf, np.nan, -np.nan, 3.0e38, -3.0e38], dtype=np.float32)
+    for j in range(0, d, 2):                       # every other column: 1 .. theta special values
+        n = 1 + (j // 2) % theta
+        rows = rng.permutation(f)[:n]
+        v[rows, j] = specials[rng.integers(0, len(specials), n)]
+    v[:, 1::64] = np.inf                            # whole columns of one infinity
+    sel = rng.permutation(f)[:theta].astype(np.int32)
+    want = oracle.trimmed_mean(v, sel, beta)
+    got = bz.trimmed_mean(torch.from_numpy(v).to(DEV), torch.from_numpy(sel).to(DEV), beta).cpu().numpy()
+    assert np.array_equal(np.isnan(got), np.isnan(want))
+    ok = ~np.isnan(want)
+    assert np.array_equal(got[ok].view(np.uint32), want[ok].view(np.uint32))
+    assert (~np.isfinite(v[sel])).any(axis=0).sum() > 1000 and np.isinf(want).sum() > 10   # the stepwise path ran
+
+
 def test_preconditions_reported():
     v = torch.zeros((25, 16), dtype=torch.float32, device=DEV)
     with pytest.raises(bz.BzError) as e:
