@@ -34,7 +34,7 @@ BULYAN = dict(l=5, r=5, q=6, d=25_000_000, attack="constant", seed=0, c=4, heavy
 
 # DRAM bytes per launch of the dominant kernel from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum, scaled to a full launch), or None when no capture of the current kernel exists.
-TRAFFIC_BYTES_PER_LAUNCH = 3_420_054_000  # (600.02 + 10.70) MB at d = 2 M, scaled by 5.6 to d = 11.2 M
+TRAFFIC_BYTES_PER_LAUNCH = 3_422_552_000  # (600.02 + 11.15) MB at d = 2 M, scaled by 5.6 to d = 11.2 M
 
 
 def workload_name(cfg):
