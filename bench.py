@@ -119,6 +119,10 @@ class ClockSampler:
         return {"sm_mhz": (statistics.median([m for _, m, _ in rows]) if rows else None), "sm_max_mhz": self.max_mhz,
                 "reasons": sorted(reasons), "samples": len(rows)}
 
+    def window(self, t0, t1):
+        """Clocks between two time.monotonic() stamps."""
+        return self._summary([r for r in self.samples if t0 <= r[0] <= t1])
+
     def summary(self):
         """Clocks over the marked regions (warm-up + timed steps of the headline), and over the whole run."""
         inside = [s for s in self.samples if any(a <= s[0] <= (b if b is not None else s[0]) for a, b in self.marks)]
@@ -185,7 +189,7 @@ def e2e_leg(bz, torch, dist, world, rep, out, device, steps):
             "d2h_bytes_per_step": d * 4, "steps": n, "matches_device_result": matches}, rep_host
 
 
-def multikrum_leg(bz, inputs, torch, dist, world, rank, device, steps, warmup, peak):
+def multikrum_leg(bz, inputs, torch, dist, world, rank, device, steps, warmup, peak, sampler=None):
     """Multi-Krum from the replicas (vote + distances in one pass, selection, mean) at K = 21, (l, r) = (7, 3),
     f = 49, d = 11.2 M per GPU, q = 5 with the ALIE payload, (c, m) = (5, 44).  With several ranks every rank owns
     a slab of that size and the partial distance matrices are added by one all-reduce."""
@@ -210,11 +214,13 @@ def multikrum_leg(bz, inputs, torch, dist, world, rank, device, steps, warmup, p
         torch.cuda.synchronize()
     n0 = bz.kernel_launch_count()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    t_begin = time.monotonic()
     ev[0].record()
     for i in range(steps):
         res = step()
         ev[i + 1].record()
     torch.cuda.synchronize()
+    t_end = time.monotonic()
     launches = bz.kernel_launch_count() - n0
     ms_total = torch.tensor([ev[0].elapsed_time(ev[steps])], dtype=torch.float64, device=device)
     if world > 1:
@@ -233,6 +239,13 @@ def multikrum_leg(bz, inputs, torch, dist, world, rank, device, steps, warmup, p
                         "algorithmic_bytes_per_step": alg_bytes,
                         "kernels": "pairdist_i8_kernel<49,25,3,25,3,1> (vote + integer MMA distances), mean_rows_kernel"},
            "status_bits (0 = the integer kernel's distances stood)": bz.pairdist_status(ws, f) if world == 1 else None}
+    # this pipeline (tensor cores, conversion and HBM all busy) reaches the board's power limit within tenths of a
+    # second: the later steps run at lower SM clocks than the first ones, and both are reported
+    quarter = max(1, steps // 4)
+    rec["ms_first_quarter"] = sum(each[:quarter]) / quarter
+    rec["ms_last_quarter"] = sum(each[-quarter:]) / quarter
+    if sampler is not None:
+        rec["clocks"] = sampler.window(t_begin, t_end)
     if world == 1:
         return rec, (rep, voted, out, dmat, res[1])
     del rep
@@ -392,7 +405,7 @@ def run_ours(args):
 
     # ---- the metric's second aggregator: Multi-Krum (every rank; one all-reduce when N > 1) --------------
     if not args.no_extra and args.coords == 0:
-        sec, keep = multikrum_leg(bz, inputs, torch, dist, world, rank, device, max(5, min(args.steps, 50)), 10, peak)
+        sec, keep = multikrum_leg(bz, inputs, torch, dist, world, rank, device, max(5, min(args.steps, 50)), 10, peak, sampler)
         if rank == 0:
             result["secondary"] = sec
             if world == 1 and not args.no_cpu:

@@ -109,55 +109,59 @@ __global__ void __launch_bounds__(BZ_MAX_F) bulyan_select_kernel(const double* _
 }
 
 // ------------------------------------------------------------------------------------------------
-// The same selections for f <= 64 with the sorted rows in shared memory, one warp per row.
-// Sorting is by rank counting: the lanes hold the row's distances and each counts how many of them
-// precede its own (by value, then index).  A score is the sum of the first nb ACTIVE entries of the
-// sorted row, added one by one in ascending order - the same sums in the same order as in the kernels above.
+// The same selections for f <= 64 with the sorted rows in shared memory.
+// Sorting is by rank counting: the matrix is staged in shared memory and every thread counts, for a few entries
+// (a, b), how many of row a's distances precede its own (by value, then index).  A score is the sum of the first
+// nb ACTIVE entries of the sorted row, added one by one in ascending order - the same sums in the same order as
+// in the kernels above; one warp per row forms it.
 constexpr int kSelF = 64;
+constexpr int kSelWarps = 32;
 
-__device__ __forceinline__ void sort_rows_shared(const double* __restrict__ dist, int f, double (*sval)[kSelF],
-                                                 unsigned char (*sidx)[kSelF]) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int a = warp; a < f; a += blockDim.x >> 5) {
-        const int b0 = lane, b1 = lane + 32;
-        const double v0 = b0 < f ? dist[a * f + b0] : 0.0, v1 = b1 < f ? dist[a * f + b1] : 0.0;
-        int rank0 = 0, rank1 = 0;
-        for (int b = 0; b < f; ++b) {
-            const double y = __shfl_sync(0xffffffffu, b < 32 ? v0 : v1, b & 31);
-            if (b == a) continue;
-            rank0 += (y < v0) || (y == v0 && b < b0);
-            rank1 += (y < v1) || (y == v1 && b < b1);
+struct SelectShared {
+    double raw[kSelF][kSelF];
+    double sval[kSelF][kSelF];
+    double comp[kSelWarps][kSelF];
+    double score[kSelF];
+    unsigned char sidx[kSelF][kSelF];
+    unsigned char active[kSelF];
+};
+
+__device__ __forceinline__ void sort_rows_shared(const double* __restrict__ dist, int f, SelectShared& sh) {
+    for (int e = threadIdx.x; e < f * f; e += blockDim.x) sh.raw[e / f][e % f] = dist[e];
+    __syncthreads();
+    for (int e = threadIdx.x; e < f * f; e += blockDim.x) {
+        const int a = e / f, b = e % f;
+        if (b == a) continue;
+        const double x = sh.raw[a][b];
+        int rank = 0;
+#pragma unroll 8
+        for (int b2 = 0; b2 < f; ++b2) {
+            const double y = sh.raw[a][b2];
+            rank += (b2 != a) && ((y < x) || (y == x && b2 < b));
         }
-        if (b0 < f && b0 != a) {
-            sval[a][rank0] = v0;
-            sidx[a][rank0] = static_cast<unsigned char>(b0);
-        }
-        if (b1 < f && b1 != a) {
-            sval[a][rank1] = v1;
-            sidx[a][rank1] = static_cast<unsigned char>(b1);
-        }
+        sh.sval[a][rank] = x;
+        sh.sidx[a][rank] = static_cast<unsigned char>(b);
     }
 }
 
 // warp-collective: score of row a among the active rows (the result is valid in lane 0).
 // The lanes compact the first nb active entries into `comp` (positions by prefix counts of the
 // ballots); lane 0 adds them in ascending order.
-constexpr int kSelWarps = 16;
-__device__ __forceinline__ double krum_score_warp(const double (*sval)[kSelF], const unsigned char (*sidx)[kSelF], int f, int a,
-                                                  const unsigned char* active, int nb, double* comp) {
+__device__ __forceinline__ double krum_score_warp(const SelectShared& sh, int f, int a, int nb, double* comp) {
     const int lane = threadIdx.x & 31;
     const int p0 = lane, p1 = lane + 32;
-    const bool act0 = p0 < f - 1 && active[sidx[a][p0]];
-    const bool act1 = p1 < f - 1 && active[sidx[a][p1]];
+    const bool act0 = p0 < f - 1 && sh.active[sh.sidx[a][p0]];
+    const bool act1 = p1 < f - 1 && sh.active[sh.sidx[a][p1]];
     const unsigned m0 = __ballot_sync(0xffffffffu, act0), m1 = __ballot_sync(0xffffffffu, act1);
     const unsigned below = (1u << lane) - 1u;
     const int q0 = __popc(m0 & below), q1 = __popc(m0) + __popc(m1 & below);
-    if (act0 && q0 < nb) comp[q0] = sval[a][p0];
-    if (act1 && q1 < nb) comp[q1] = sval[a][p1];
+    if (act0 && q0 < nb) comp[q0] = sh.sval[a][p0];
+    if (act1 && q1 < nb) comp[q1] = sh.sval[a][p1];
     __syncwarp();
     double s = 0.0;
     if (lane == 0) {
         const int total = min(nb, __popc(m0) + __popc(m1));
+#pragma unroll 4
         for (int k = 0; k < total; ++k) s += comp[k];
     }
     __syncwarp();
@@ -167,24 +171,21 @@ __device__ __forceinline__ double krum_score_warp(const double (*sval)[kSelF], c
 // bulyan == 0: Multi-Krum (first m of the ranking); bulyan != 0: theta = f - 2c picks, one per round
 __global__ void __launch_bounds__(kSelWarps * 32) select_shared_kernel(const double* __restrict__ dist, int f, int c, int m, int bulyan,
                                                              int32_t* __restrict__ selected) {
-    __shared__ double sval[kSelF][kSelF];
-    __shared__ unsigned char sidx[kSelF][kSelF];
-    __shared__ double comp[kSelWarps][kSelF];
-    __shared__ double score[kSelF];
-    __shared__ unsigned char active[kSelF];
+    extern __shared__ __align__(16) unsigned char select_smem[];
+    SelectShared& sh = *reinterpret_cast<SelectShared*>(select_smem);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid < f) active[tid] = 1;
-    sort_rows_shared(dist, f, sval, sidx);
+    if (tid < f) sh.active[tid] = 1;
+    sort_rows_shared(dist, f, sh);
     __syncthreads();
     if (!bulyan) {
         for (int a = warp; a < f; a += kSelWarps) {
-            const double s = krum_score_warp(sval, sidx, f, a, active, f - c - 2, comp[warp]);
-            if (lane == 0) score[a] = s;
+            const double s = krum_score_warp(sh, f, a, f - c - 2, sh.comp[warp]);
+            if (lane == 0) sh.score[a] = s;
         }
         __syncthreads();
         if (tid < f) {
             int rank = 0;
-            for (int b = 0; b < f; ++b) rank += (score[b] < score[tid]) || (score[b] == score[tid] && b < tid);
+            for (int b = 0; b < f; ++b) rank += (sh.score[b] < sh.score[tid]) || (sh.score[b] == sh.score[tid] && b < tid);
             if (rank < m) selected[rank] = tid;
         }
         return;
@@ -196,9 +197,9 @@ __global__ void __launch_bounds__(kSelWarps * 32) select_shared_kernel(const dou
         if (nb < 1) nb = 1;
         if (nb > n - 1) nb = n - 1;
         for (int a = warp; a < f; a += kSelWarps) {
-            if (!active[a]) continue;  // uniform over the warp
-            const double s = (n > 1) ? krum_score_warp(sval, sidx, f, a, active, nb, comp[warp]) : 0.0;
-            if (lane == 0) score[a] = s;
+            if (!sh.active[a]) continue;  // uniform over the warp
+            const double s = (n > 1) ? krum_score_warp(sh, f, a, nb, sh.comp[warp]) : 0.0;
+            if (lane == 0) sh.score[a] = s;
         }
         __syncthreads();
         if (warp == 0) {
@@ -206,8 +207,8 @@ __global__ void __launch_bounds__(kSelWarps * 32) select_shared_kernel(const dou
             double best = 0.0;
             int who = -1;
             for (int a = lane; a < f; a += 32)
-                if (active[a] && (who < 0 || score[a] < best)) {  // a grows: a tie keeps the lower index
-                    best = score[a];
+                if (sh.active[a] && (who < 0 || sh.score[a] < best)) {  // a grows: a tie keeps the lower index
+                    best = sh.score[a];
                     who = a;
                 }
             for (int o = 16; o > 0; o >>= 1) {
@@ -220,11 +221,20 @@ __global__ void __launch_bounds__(kSelWarps * 32) select_shared_kernel(const dou
             }
             if (lane == 0) {
                 selected[t] = who;
-                active[who] = 0;
+                sh.active[who] = 0;
             }
         }
         __syncthreads();
     }
+}
+
+int launch_select_shared(const double* dist, int f, int c, int m, int bulyan, int32_t* selected, cudaStream_t s) {
+    // per device, so set on every call (it is a host-side table entry, not a launch)
+    const cudaError_t attr = cudaFuncSetAttribute(select_shared_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                  static_cast<int>(sizeof(SelectShared)));
+    if (attr != cudaSuccess) return cuda_failed(attr);
+    select_shared_kernel<<<1, kSelWarps * 32, sizeof(SelectShared), s>>>(dist, f, c, m, bulyan, selected);
+    return BZ_OK;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -486,9 +496,10 @@ extern "C" int bz_krum_select(const double* dist, int f, int c, int m, int32_t* 
     if (dist == nullptr || selected == nullptr || f < 1) return BZ_ERR_INVALID_ARG;
     if (f > BZ_MAX_F) return BZ_ERR_UNSUPPORTED;
     if (c < 0 || f < 2 * c + 3 || m < 1 || m > f) return BZ_ERR_PRECONDITION;
-    if (f <= kSelF)
-        select_shared_kernel<<<1, kSelWarps * 32, 0, static_cast<cudaStream_t>(stream)>>>(dist, f, c, m, 0, selected);
-    else
+    if (f <= kSelF) {
+        const int st = launch_select_shared(dist, f, c, m, 0, selected, static_cast<cudaStream_t>(stream));
+        if (st != BZ_OK) return st;
+    } else
         krum_select_kernel<<<1, BZ_MAX_F, 0, static_cast<cudaStream_t>(stream)>>>(dist, f, c, m, selected);
     note_launch();
     return check_launch();
@@ -526,9 +537,10 @@ extern "C" int bz_bulyan_select(const double* dist, int f, int c, int32_t* selec
     if (dist == nullptr || selected == nullptr || f < 1) return BZ_ERR_INVALID_ARG;
     if (f > BZ_MAX_F) return BZ_ERR_UNSUPPORTED;
     if (c < 0 || f < 4 * c + 3) return BZ_ERR_PRECONDITION;
-    if (f <= kSelF)
-        select_shared_kernel<<<1, kSelWarps * 32, 0, static_cast<cudaStream_t>(stream)>>>(dist, f, c, 0, 1, selected);
-    else
+    if (f <= kSelF) {
+        const int st = launch_select_shared(dist, f, c, 0, 1, selected, static_cast<cudaStream_t>(stream));
+        if (st != BZ_OK) return st;
+    } else
         bulyan_select_kernel<<<1, BZ_MAX_F, 0, static_cast<cudaStream_t>(stream)>>>(dist, f, c, selected);
     note_launch();
     return check_launch();

@@ -6,29 +6,43 @@ namespace bz {
 
 namespace {
 
-// After the main kernel: D^ from the CTAs' partial matrices, the exact contribution of the listed outlier
-// coordinates, then the bound on the conversion error and the CTAs' marks (three small kernels).
-// flag[0] = 1 asks for the binary32 kernel: the bound does not fit the tolerance (ignored with force != 0), a
+// After the main kernel, ONE small kernel of F CTAs finishes the job (three launches cost three times the latency of
+// a dependent launch, which at a million coordinates was a fifth of the call):
+//   every CTA: D^ for its share of the pairs from the CTAs' partial matrices; the exact contribution of the
+//              outlier coordinates listed for "its" row; that row's rounding budget N_a^2; the CTAs' marks;
+//   the CTA that finishes last (a ticket counter, no waiting): the bound on the conversion error -> final
+//              distances, flag[0], flag[1].
+// flag[0] = 1 asks for the binary64 kernel: the bound does not fit the tolerance (ignored with force != 0), a
 // row holds values the fixed-point scale cannot carry, an outlier list overflowed, or a CTA stopped early.
 // flag[1] = 1 says the latter: a bounded wait ran out, the partial matrices are incomplete and so are the voted
 // rows of the kernel with the vote in front.
 constexpr double kRelTol = 1e-7;   // the library's tolerance for a squared distance
+constexpr int kFinishThreads = 1024;   // 32 warps: with F CTAs every pair has a warp of its own, and the last CTA covers the matrix in three sweeps
+
+__device__ __forceinline__ double ld_l2(const double* p) { return __ldcg(p); }
 
 // One warp per pair a <= b: lane l takes CTAs l, l+32, ... in order, then the lanes are added in a fixed
 // tree.  Identical rows meet identical numbers in the same order and get identical distances.  The diagonal
-// pairs deliver |q_a|^2 (what the binary64 sums had to carry: the check kernel bounds their rounding with it).
+// pairs deliver |q_a|^2 (what the binary64 sums had to carry: the bound covers their rounding with it).
 template <int F>
-__global__ void __launch_bounds__(256)
-    pairdist_i8_reduce_kernel(const double* __restrict__ tpart, int n_ctas, double* __restrict__ dist, double* __restrict__ norm2) {
-    const int pair = blockIdx.x * (blockDim.x / 32) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-    if (pair >= F * F) return;
-    const int a = pair / F, b = pair % F;
-    if (a > b) return;
-    double s = 0.0;
-    for (int c = lane; c < n_ctas; c += 32) {
-        const double* T = tpart + static_cast<size_t>(c) * F * F;
-        s += a < b ? (T[a * F + a] + T[b * F + b]) - (T[a * F + b] + T[b * F + a]) : T[a * F + a];
+__device__ __forceinline__ void finish_reduce_pair(const double* __restrict__ tpart, int n_ctas, int a, int b, int lane,
+                                                   double* __restrict__ dist, double* __restrict__ norm2) {
+    // at most kNumSMs partial matrices: five per lane, all loads in flight at once, added in the order c = lane, lane + 32, ...
+    constexpr int kPerLane = (kNumSMs + 31) / 32;
+    double t[kPerLane];
+#pragma unroll
+    for (int k = 0; k < kPerLane; ++k) {
+        const int c = lane + 32 * k;
+        t[k] = 0.0;
+        if (c < n_ctas) {
+            const double* T = tpart + static_cast<size_t>(c) * F * F;
+            t[k] = a < b ? (T[a * F + a] + T[b * F + b]) - (T[a * F + b] + T[b * F + a]) : T[a * F + a];
+        }
     }
+    double s = 0.0;
+#pragma unroll
+    for (int k = 0; k < kPerLane; ++k)
+        if (lane + 32 * k < n_ctas) s += t[k];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xffffffffu, s, o);
     if (lane == 0) {
@@ -42,44 +56,45 @@ __global__ void __launch_bounds__(256)
     }
 }
 
-// What the listed outlier coordinates contribute.  CTA a handles row a's lists, thread b the pair (a, b):
+struct FinishShared {
+    int cnt[kNumSMs], off[kNumSMs + 1];
+    int j[kNumSMs * kOutCap];
+    short c[kNumSMs * kOutCap];
+};
+
+// What the listed outlier coordinates contribute.  The CTA handles row a's lists, thread b the pair (a, b):
 //   corr[a][b] = sum over row a's outliers j of (v_a[j] - v_b[j])^2 - (0 - fed_b[j])^2
 // with fed_b[j] what row b fed the contraction at j: its value, or zero if j is on row b's list too (then the
 // pair is handled from the list of the lower row only).  Lists are walked CTA by CTA, entry by entry:
-// a fixed order.  The check kernel adds corr[a][b] + corr[b][a] to D^.
+// a fixed order.  The last CTA adds corr[a][b] + corr[b][a] to D^.  (Block-uniform control flow.)
 template <int F>
-__global__ void __launch_bounds__(128)
-    pairdist_i8_outlier_kernel(const float* __restrict__ v, int64_t ld, const int* __restrict__ info, const int* __restrict__ olist,
-                               int n_ctas, double* __restrict__ corr) {
-    const int a = blockIdx.x, tid = threadIdx.x;
-    __shared__ int s_cnt[kNumSMs], s_off[kNumSMs + 1];
-    __shared__ int s_j[kNumSMs * kOutCap];
-    __shared__ short s_c[kNumSMs * kOutCap];
+__device__ __forceinline__ void finish_outliers(FinishShared& sh, const float* __restrict__ v, int64_t ld, const int* __restrict__ info,
+                                                const int* __restrict__ olist, int n_ctas, int a, double* __restrict__ corr) {
+    const int tid = threadIdx.x;
+    int mine = 0;
     for (int c = tid; c < n_ctas; c += blockDim.x) {
         const int n = info[c * kInfoStride + kInfoOut + a];
-        s_cnt[c] = n > kOutCap ? kOutCap : (n < 0 ? 0 : n);  // an overflowing list sends the caller to the binary32 kernel anyway
+        sh.cnt[c] = n > kOutCap ? kOutCap : (n < 0 ? 0 : n);  // an overflowing list sends the caller to the binary64 kernel anyway
+        mine |= sh.cnt[c];
     }
-    __syncthreads();
-    if (tid == 0) {
-        int run = 0;
-        for (int c = 0; c < n_ctas; ++c) {
-            s_off[c] = run;
-            run += s_cnt[c];
-        }
-        s_off[n_ctas] = run;
-    }
-    __syncthreads();
-    const int total = s_off[n_ctas];
-    if (total == 0) {
+    if (!__syncthreads_or(mine)) {  // nearly always: no CTA listed anything for this row
         if (tid < F) corr[a * F + tid] = 0.0;
         return;
     }
+    // offsets of the CTAs' lists in the compact list: thread c adds the counts before its own
+    for (int c = tid; c <= n_ctas; c += blockDim.x) {
+        int run = 0;
+        for (int k = 0; k < c; ++k) run += sh.cnt[k];
+        sh.off[c] = run;
+    }
+    __syncthreads();
+    const int total = sh.off[n_ctas];
     // row a's entries, CTA by CTA, in list order
     for (int e = tid; e < n_ctas * kOutCap; e += blockDim.x) {
         const int c = e / kOutCap, k = e % kOutCap;
-        if (k < s_cnt[c]) {
-            s_j[s_off[c] + k] = olist[(static_cast<size_t>(c) * 64 + a) * kOutCap + k];
-            s_c[s_off[c] + k] = static_cast<short>(c);
+        if (k < sh.cnt[c]) {
+            sh.j[sh.off[c] + k] = olist[(static_cast<size_t>(c) * 64 + a) * kOutCap + k];
+            sh.c[sh.off[c] + k] = static_cast<short>(c);
         }
     }
     __syncthreads();
@@ -89,8 +104,8 @@ __global__ void __launch_bounds__(128)
     if (b != a) {
 #pragma unroll 4
         for (int e = 0; e < total; ++e) {
-            const int64_t j = s_j[e];
-            const int c = s_c[e];
+            const int64_t j = sh.j[e];
+            const int c = sh.c[e];
             const float va = v[a * ld + j], vb = v[b * ld + j];
             // did row b enter as zero at j as well?  Then j is on its list in the same CTA.
             int n_b = info[c * kInfoStride + kInfoOut + b];
@@ -106,64 +121,102 @@ __global__ void __launch_bounds__(128)
     corr[a * F + b] = sum;
 }
 
-// The bound and the marks -> final distances, flag[0], flag[1].
+// The bound and the marks -> final distances, flag[0], flag[1] (the last CTA).
 //   N_a^2 = sum over CTAs (and a row's successive scales) of n_small * (step / 2)^2, step = 2^(E - 30): every rounded
 //   value moved by at most half a step
 //   |D^ - D~| <= 2 (N_a + N_b) sqrt(D^) + (N_a + N_b)^2, D~ the distance with the outliers as zeros (Cauchy-Schwarz)
 //   + 2^-39 (|q_a|^2 + |q_b|^2) for the binary64 sums behind D^ (a few thousand roundings of terms of that size)
 // must stay below kRelTol times the final distance D^ + corr.
 template <int F>
-__global__ void __launch_bounds__(1024)
-    pairdist_i8_check_kernel(double* __restrict__ dist, const double* __restrict__ corr, const double* __restrict__ norm2,
-                             const int* __restrict__ info, int n_ctas, int force, int* __restrict__ flag) {
-    __shared__ double s_n2[F];
-    __shared__ int s_bad, s_marks;
-    const int tid = threadIdx.x;
-    if (tid == 0) s_bad = s_marks = 0;
-    __syncthreads();
-    // sixteen threads per row, each over every sixteenth CTA in order; their sums are added in a fixed order
+__global__ void __launch_bounds__(kFinishThreads)
+    pairdist_i8_finish_kernel(const double* __restrict__ tpart, const float* __restrict__ v, int64_t ld, int* __restrict__ info,
+                              const int* __restrict__ olist, int n_ctas, double* __restrict__ dist, double* __restrict__ corr,
+                              double* __restrict__ norm2, double* __restrict__ n2_rows, int force, int* __restrict__ flag) {
+    __shared__ FinishShared sh;
     constexpr int kParts = 16;
-    __shared__ double s_part[kParts][F];
-    if (tid < kParts * F) {
-        const int row = tid % F, part = tid / F;
+    __shared__ double s_part[kParts];
+    __shared__ int s_last;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, row = blockIdx.x;
+    // ---- this CTA's share of the pairs a <= b: pair numbers row, row + F, ... (rows of the upper triangle in order)
+    constexpr int kPairs = F * (F + 1) / 2;
+    for (int p = row + F * warp; p < kPairs; p += F * (kFinishThreads / 32)) {
+        int a = 0, rem = p;
+        while (rem >= F - a) {
+            rem -= F - a;
+            ++a;
+        }
+        finish_reduce_pair<F>(tpart, n_ctas, a, a + rem, lane, dist, norm2);
+    }
+    // ---- row `row`: rounding budget (sixteen threads, each over every sixteenth CTA in order; their sums are
+    // added in a fixed order) and the CTAs' marks
+    int marks = 0;
+    if (tid < kParts) {
         double n2 = 0.0;
-        int over = 0;
 #pragma unroll 5
-        for (int c = part; c < n_ctas; c += kParts) {
+        for (int c = tid; c < n_ctas; c += kParts) {
             const int* rec = info + c * kInfoStride;
             const double half_step = __longlong_as_double(static_cast<long long>(1023 + rec[kInfoE + row] - 31) << 52);
             n2 += reinterpret_cast<const double*>(rec + kInfoN2)[row] + static_cast<double>(rec[kInfoSmall + row]) * half_step * half_step;
-            over |= rec[kInfoOut + row] > kOutCap;
+            if (rec[kInfoOut + row] > kOutCap) marks |= kBadValues;
         }
-        s_part[part][row] = n2;
-        if (over) atomicOr(&s_marks, kBadValues);
+        s_part[tid] = n2;
     }
+    if (row == 0)
+        for (int c = tid; c < n_ctas; c += kFinishThreads) marks |= info[c * kInfoStride + kInfoBad];
+    if (marks) atomicOr(&info[kInfoMarks], marks);
+    // ---- row `row`: its outliers (syncs inside: also orders s_part)
+    finish_outliers<F>(sh, v, ld, info, olist, n_ctas, row, corr);
     __syncthreads();
-    if (tid < F) {
+    if (tid == 0) {
         double n2 = 0.0;
 #pragma unroll
-        for (int part = 0; part < kParts; ++part) n2 += s_part[part][tid];
-        s_n2[tid] = n2;
+        for (int part = 0; part < kParts; ++part) n2 += s_part[part];
+        n2_rows[row] = n2;
     }
-    for (int c = tid; c < n_ctas; c += blockDim.x)
-        if (info[c * kInfoStride + kInfoBad]) atomicOr(&s_marks, info[c * kInfoStride + kInfoBad]);
-    __shared__ double s_min_nz[F], s_zero_n2[F];
+    // ---- the last CTA to get here sees what all the others wrote (fence, ticket, fence)
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = atomicAdd(&info[kInfoTicket], 1) == F - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+
+    __shared__ double s_n[F], s_norm2[F], s_min_nz[F], s_zero_n2[F];
+    __shared__ int s_bad;
+    if (tid == 0) s_bad = 0;
     if (tid < F) {
+        s_n[tid] = sqrt(ld_l2(n2_rows + tid));
+        s_norm2[tid] = ld_l2(norm2 + tid);
         s_min_nz[tid] = 1e300;
         s_zero_n2[tid] = 0.0;
     }
     __syncthreads();
     bool bad = false;
-    for (int p = tid; p < F * F; p += blockDim.x) {
+    constexpr int kSweeps = (F * F + kFinishThreads - 1) / kFinishThreads;
+    double dh_[kSweeps], c1_[kSweeps], c2_[kSweeps];
+#pragma unroll
+    for (int k = 0; k < kSweeps; ++k) {  // all loads first: one trip to L2, not three
+        const int p = tid + k * kFinishThreads;
         const int a = p / F, b = p % F;
-        if (a >= b) continue;
-        const double dh = dist[a * F + b];
-        const double df = dh + (corr[a * F + b] + corr[b * F + a]);
-        const double n = sqrt(s_n2[a]) + sqrt(s_n2[b]);
+        dh_[k] = c1_[k] = c2_[k] = 0.0;
+        if (p < F * F && a < b) {
+            dh_[k] = ld_l2(dist + a * F + b);
+            c1_[k] = ld_l2(corr + a * F + b);
+            c2_[k] = ld_l2(corr + b * F + a);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < kSweeps; ++k) {
+        const int p = tid + k * kFinishThreads;
+        const int a = p / F, b = p % F;
+        if (p >= F * F || a >= b) continue;
+        const double dh = dh_[k];
+        const double df = dh + (c1_[k] + c2_[k]);
+        const double n = s_n[a] + s_n[b];
         if (!(dh >= 0.0) || !(df >= 0.0)) {
             bad = true;
         } else {
-            const double err = 2.0 * n * sqrt(dh) + n * n + 1.8189894035458565e-12 * (norm2[a] + norm2[b]);
+            const double err = 2.0 * n * sqrt(dh) + n * n + 1.8189894035458565e-12 * (s_norm2[a] + s_norm2[b]);
             if (df > 0.0) {
                 if (err > kRelTol * df) bad = true;
                 atomicMin(reinterpret_cast<unsigned long long*>(&s_min_nz[a]), static_cast<unsigned long long>(__double_as_longlong(df)));
@@ -183,8 +236,9 @@ __global__ void __launch_bounds__(1024)
     if (tid < F && s_zero_n2[tid] > 0.0 && s_min_nz[tid] < 1e300 && s_zero_n2[tid] > kRelTol * s_min_nz[tid]) atomicOr(&s_bad, 1);
     __syncthreads();
     if (tid == 0) {
-        flag[0] = ((s_bad && !force) || s_marks) ? 1 : 0;
-        flag[1] = (s_marks & kBadStopped) ? 1 : 0;
+        const int all_marks = atomicOr(&info[kInfoMarks], 0);
+        flag[0] = ((s_bad && !force) || all_marks) ? 1 : 0;
+        flag[1] = (all_marks & kBadStopped) ? 1 : 0;
     }
 }
 
@@ -194,6 +248,7 @@ struct Scratch {
     int* olist;
     double* corr;
     double* norm2;
+    double* n2;
 };
 
 // rep: R = 1: rows [f][d] with leading dimension ld_file.  R > 1: replicas[r][f][d].
@@ -222,18 +277,11 @@ int launch_i8(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, floa
     note_launch();
     int st = check_launch();
     if (st != BZ_OK) return st;
-    pairdist_i8_reduce_kernel<F><<<(F * F + 7) / 8, 256, 0, s>>>(sc.tpart, static_cast<int>(ctas), dist, sc.norm2);
-    note_launch();
-    st = check_launch();
-    if (st != BZ_OK) return st;
     // the rows the contraction saw: the given ones, or the winners the kernel has just written
     const float* rows = R > 1 ? voted : rep;
     const int64_t ld_rows = R > 1 ? ld_voted : ld_file;
-    pairdist_i8_outlier_kernel<F><<<F, 128, 0, s>>>(rows, ld_rows, sc.info, sc.olist, static_cast<int>(ctas), sc.corr);
-    note_launch();
-    st = check_launch();
-    if (st != BZ_OK) return st;
-    pairdist_i8_check_kernel<F><<<1, 1024, 0, s>>>(dist, sc.corr, sc.norm2, sc.info, static_cast<int>(ctas), force, flag);
+    pairdist_i8_finish_kernel<F><<<F, kFinishThreads, 0, s>>>(sc.tpart, rows, ld_rows, sc.info, sc.olist, static_cast<int>(ctas), dist,
+                                                            sc.corr, sc.norm2, sc.n2, force, flag);
     note_launch();
     return check_launch();
 }
@@ -242,7 +290,7 @@ size_t tpart_bytes(int f) { return round_up(static_cast<size_t>(kNumSMs) * f * f
 size_t info_bytes() { return round_up(static_cast<size_t>(kNumSMs) * kInfoStride * sizeof(int), 256); }
 size_t olist_bytes() { return round_up(static_cast<size_t>(kNumSMs) * 64 * kOutCap * sizeof(int), 256); }
 size_t corr_bytes(int f) { return round_up(static_cast<size_t>(f) * f * sizeof(double), 256); }
-size_t norm_bytes() { return round_up(64 * sizeof(double), 256); }
+size_t norm_bytes() { return round_up(2 * 64 * sizeof(double), 256); }   // |q_a|^2 and N_a^2 per row
 
 Scratch carve(void* ws, int f) {
     char* p = static_cast<char*>(ws);
@@ -256,6 +304,7 @@ Scratch carve(void* ws, int f) {
     s.corr = reinterpret_cast<double*>(p);
     p += corr_bytes(f);
     s.norm2 = reinterpret_cast<double*>(p);
+    s.n2 = s.norm2 + 64;
     return s;
 }
 

@@ -75,6 +75,8 @@ constexpr int kCtlBytes = 3072;
 // been rounded, their counts of outliers, then the "bad" mark
 // (kInfoN2: 64 doubles - the squared rounding budget a row used up under its earlier scales)
 constexpr int kInfoE = 0, kInfoSmall = 64, kInfoOut = 128, kInfoN2 = 192, kInfoBad = 320, kInfoStride = 328;
+// in CTA 0's record only: the ticket counter and the collected marks of the kernel that finishes the distances
+constexpr int kInfoTicket = 321, kInfoMarks = 322;
 constexpr int kLookEvery = 4;        // steps between two looks at whether rows would fit a finer scale
 constexpr int kOutCap = 8;           // listed outliers per CTA and row; a row that has more gets a coarser scale
 constexpr int kBadValues = 1;        // bits of the mark: a row holds values no fixed-point scale can carry
@@ -201,6 +203,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
         mbar_init(drained, kDrainWarps);
         *dead = 0;
         info[blockIdx.x * kInfoStride + kInfoBad] = 0;
+        if (blockIdx.x == 0) info[kInfoTicket] = info[kInfoMarks] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (tid < 64) {
