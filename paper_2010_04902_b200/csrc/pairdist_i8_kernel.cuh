@@ -15,7 +15,7 @@
 // every 512 tiles (32-bit headroom), when a row changes its scale and at the end; a drain combines the
 // blocks in binary64 and adds
 //     T[a][b] += 2^(E_a + E_b - 60) * sum_blocks weight * S_i S_j^T [a][b]
-// to the CTA's partial matrix (in shared memory, written out once).  A last kernel forms, per CTA and
+// to the CTA's partial matrix (in shared memory, written out once).  A finishing kernel forms, per CTA and
 // then over CTAs in a fixed order,
 //     D[a][b] = (T[a][a] + T[b][b]) - (T[a][b] + T[b][a]).
 // Identical rows give identical integers and therefore exactly equal distances and D = 0.
@@ -26,12 +26,12 @@
 // rounded, by at most half a step, and the converters count them (n_small: a superset, read off the top
 // bytes).  With N_a^2 = sum of n_small * (step/2)^2 over CTAs (and over a row's successive scales) the
 // computed distance obeys |D^ - D| <= 2 (N_a + N_b) sqrt(D^) + (N_a + N_b)^2 (Cauchy-Schwarz): a bound
-// that holds for every input, also for rows whose rounding errors were arranged to line up.  The last
+// that holds for every input, also for rows whose rounding errors were arranged to line up.  The finishing
 // kernel compares it with the library's distance tolerance and raises a flag when it does not fit; the
 // caller then runs the binary64 difference-form kernel, which starts by looking at that flag.
 // A later value that does not fit the row's scale (magnitude 2^E_a or more) is an outlier as long as the
 // CTA has met at most kOutCap of them in that row - the rare large values of a heavy-tailed row: it
-// enters the contraction as zero and its coordinate goes on a short list kept per CTA and row; a small
+// enters the contraction as zero and its coordinate goes on a short list kept per CTA and row; the finishing
 // kernel then adds, in binary64 and in a fixed order, what those coordinates really contribute to every
 // pair.  Past kOutCap the row has outgrown its scale (gradients change magnitude from layer to layer):
 // E_a is set anew from the current step, and the accumulators are read back first, because tensor memory
