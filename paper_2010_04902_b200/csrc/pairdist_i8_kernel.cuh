@@ -146,6 +146,13 @@ __device__ __forceinline__ float max_abs_nan(float a, float b) {
     return m;
 }
 
+// the largest magnitude of a, b and c, one instruction
+__device__ __forceinline__ float max_abs_nan3(float a, float b, float c) {
+    float m;
+    asm("max.NaN.abs.f32 %0, %1, %2, %3;" : "=f"(m) : "f"(a), "f"(b), "f"(c));
+    return m;
+}
+
 // R = 1: distances of the rows of `map` ([f][d]).  R > 1: `map` covers replicas[r][f][d]; row i is the vote
 // (Eq. 3, element by element on bit patterns) over its R copies, which is also written to
 // voted[i*ld_voted + j] (16-byte aligned, ld_voted a multiple of 4).
@@ -427,7 +434,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
             const int n_sub = tiles_left < TS ? tiles_left : TS;
             // this lane's coordinates in the first tile of the step (used by the vote's stores and the outlier lists)
             const int64_t j0 = (blockIdx.x + TS * step * gridDim.x) * kTK + 4 * lane;
-            unsigned char* slot = op + static_cast<uint32_t>(o) * S::kSlotBytes;
+            const uint32_t slot = smem_u32(op) + static_cast<uint32_t>(o) * S::kSlotBytes;
             bool raise = false, have_slot = false;
 #pragma unroll 1
             for (int c = 0; c < CH && ok; ++c) {
@@ -442,7 +449,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                             ok = false;
                             break;
                         }
-                        const uint32_t* src = reinterpret_cast<const uint32_t*>(in) + static_cast<uint32_t>(s) * S::kBoxFloats;
+                        const uint32_t src = smem_u32(in) + static_cast<uint32_t>(s) * S::kBoxBytes + 16 * lane;
                         const int64_t j = j0 + sub * static_cast<int64_t>(gridDim.x) * kTK;
 #pragma unroll
                         for (int i = 0; i < RWC; ++i) {
@@ -450,11 +457,11 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
                             if (fi < FC && c * FC + fi < F) {
                                 uint4 w;
                                 if constexpr (R == 1) {
-                                    w = *reinterpret_cast<const uint4*>(src + fi * kTK + 4 * lane);
+                                    w = lds128(src + fi * (kTK * 4));
                                 } else {
                                     uint4 x[R];
 #pragma unroll
-                                    for (int k = 0; k < R; ++k) x[k] = *reinterpret_cast<const uint4*>(src + (k * FC + fi) * kTK + 4 * lane);
+                                    for (int k = 0; k < R; ++k) x[k] = lds128(src + (k * FC + fi) * (kTK * 4));
                                     uint32_t cp[R];
 #pragma unroll
                                     for (int k = 0; k < R; ++k) cp[k] = x[k].x;
@@ -576,7 +583,7 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
 #pragma unroll
                             for (int sub = 0; sub < TS; ++sub) {
                                 t[sub][i] = make_float4(val[sub][i].x * scale, val[sub][i].y * scale, val[sub][i].z * scale, val[sub][i].w * scale);
-                                m = max_abs_nan(max_abs_nan(m, t[sub][i].x), max_abs_nan(t[sub][i].y, max_abs_nan(t[sub][i].z, t[sub][i].w)));
+                                m = max_abs_nan3(max_abs_nan3(m, t[sub][i].x, t[sub][i].y), t[sub][i].z, t[sub][i].w);
                             }
                         }
                     }
@@ -744,17 +751,17 @@ __global__ void __launch_bounds__(I8Shape<F, W, R, FC, NS, TS>::kThreads, 1)
 #pragma unroll
                         for (int cc = 0; cc < CH; ++cc)
                             if (cc == c) my_off = dst_off[cc * RWC + i];
-                        unsigned char* dst = slot + my_off;
+                        const uint32_t dst = slot + my_off;
                         int small = 0;
 #pragma unroll
                         for (int sub = 0; sub < TS; ++sub) {
                             if (sub < n_sub) {
                                 uint32_t w[4];
                                 slice4(t[sub][i], w);
-                                *reinterpret_cast<uint32_t*>(dst + sub * S::kOpStageBytes + 0 * RP * kTK) = w[3];
-                                *reinterpret_cast<uint32_t*>(dst + sub * S::kOpStageBytes + 1 * RP * kTK) = w[2];
-                                *reinterpret_cast<uint32_t*>(dst + sub * S::kOpStageBytes + 2 * RP * kTK) = w[1];
-                                *reinterpret_cast<uint32_t*>(dst + sub * S::kOpStageBytes + 3 * RP * kTK) = w[0];
+                                sts32(dst + sub * S::kOpStageBytes + 0 * RP * kTK, w[3]);
+                                sts32(dst + sub * S::kOpStageBytes + 1 * RP * kTK, w[2]);
+                                sts32(dst + sub * S::kOpStageBytes + 2 * RP * kTK, w[1]);
+                                sts32(dst + sub * S::kOpStageBytes + 3 * RP * kTK, w[0]);
                                 // A value can only have been rounded if |q| <= 2^23, and then its top byte (of
                                 // q + 0x808080) is 0 or 1: count the bytes of that word whose upper seven bits are
                                 // clear (a zero-byte test; the bytes tested are even, so it has no false positives).

@@ -61,6 +61,14 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, int32_t (&x)[8]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- shared memory by 32-bit address: the offsets of an unrolled loop fold into the instructions ----------
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory"); }
+
 // ---- bounded waits that give up early once another thread of the CTA has ---------------------------
 // Each probe lets the hardware suspend the thread for up to `nap_ns` nanoseconds, so a warp that waits
 // takes no issue slots from the warps that work.  At most `probes` probes.
