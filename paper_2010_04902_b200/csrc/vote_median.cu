@@ -121,7 +121,8 @@ __global__ void __launch_bounds__(256) vote_kernel(const V* __restrict__ rep, in
                                                    const int* __restrict__ gate) {
     if (gate != nullptr && *gate == 0) return;
     constexpr int VEC = Lanes<V>::n;
-    constexpr int U = (12 / R) < 1 ? 1 : (12 / R);  // coordinate groups per thread and trip: ~12 loads in flight
+    // coordinate groups per thread and trip: ~192 bytes of loads in flight whatever the width of a load
+    constexpr int U = (12 * 4 / VEC / R) < 1 ? 1 : (12 * 4 / VEC / R);
     const int i = blockIdx.y;
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
     const V* src = rep + i * ld_file;
