@@ -32,6 +32,19 @@ __device__ __forceinline__ uint32_t key_bits(int key) { return static_cast<uint3
 
 __device__ __forceinline__ int kmin(int a, int b) { return min(a, b); }
 __device__ __forceinline__ int kmax(int a, int b) { return max(a, b); }
+// binary32 comparators for columns of finite values (numeric order = total order up to the sign of zeros, which no
+// result depends on).  A NaN comes out of BOTH sides, so that it reaches the ends of a sorted column, where the
+// caller looks for it.
+__device__ __forceinline__ float kmin(float a, float b) {
+    float m;
+    asm("min.NaN.f32 %0, %1, %2;" : "=f"(m) : "f"(a), "f"(b));
+    return m;
+}
+__device__ __forceinline__ float kmax(float a, float b) {
+    float m;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(m) : "f"(a), "f"(b));
+    return m;
+}
 
 // Integer min/max issue on the ALU pipe (64 lanes per SM and clock) while the multiply-add pipe idles in a
 // comparator network.  max = a + b - min (exact modulo 2^32) as two integer multiply-adds moves one of a

@@ -289,54 +289,73 @@ __device__ __noinline__ float window_mean_stepwise(const float* s, int theta, in
     return static_cast<float>(sum / static_cast<double>(beta));
 }
 
+// sum += x if (du >= dl) == GE, as one compare and one predicated addition (finite values: "not >=" is "<").
+// The test is made where it is used, twice per pair, so that no flag has to live across the other additions:
+// a thread has seven predicate registers, and a flag parked in a general register costs more than the second compare.
+template <bool GE> __device__ __forceinline__ void add_if(double& sum, float x, float du, float dl) {
+    if constexpr (GE)
+        asm("{\n\t.reg .pred p;\n\t.reg .f64 xd;\n\tsetp.ge.f32 p, %2, %3;\n\tcvt.f64.f32 xd, %1;\n\t@p add.rn.f64 %0, %0, xd;\n\t}"
+            : "+d"(sum) : "f"(x), "f"(du), "f"(dl));
+    else
+        asm("{\n\t.reg .pred p;\n\t.reg .f64 xd;\n\tsetp.lt.f32 p, %2, %3;\n\tcvt.f64.f32 xd, %1;\n\t@p add.rn.f64 %0, %0, xd;\n\t}"
+            : "+d"(sum) : "f"(x), "f"(du), "f"(dl));
+}
+
 // Window of the BETA sorted values closest to the median, without the steps.  With finite values the two
 // sequences of distances ascend, so growing the window merges them: the p-th lower value enters before the
 // q-th upper one iff its distance is not larger, hence it belongs to the window iff the (BETA-p)-th upper value
 // does not exist or is at least as far.  Of each such pair exactly one is in the window (it holds BETA-1 values
-// besides the median), so the tests themselves are the membership flags and no window bounds are formed.
-// s[] ascending in the total order, which puts every infinity and NaN at an end: those columns take the steps.
-// Returns the mean of the window (binary64 sum, ascending).
-template <int THETA, int BETA> __device__ __forceinline__ float window_mean(const float (&s)[THETA]) {
+// besides the median), so the tests themselves decide membership and no window bounds are formed.
+// s[] ascending, sorted with the binary32 comparators, which leave every infinity at an end and a NaN at both:
+// for those columns the function returns false (the caller takes the steps, from the column itself).
+// mean: the mean of the window (binary64 sum, ascending).
+template <int THETA, int BETA> __device__ __forceinline__ bool window_mean(const float (&s)[THETA], float& mean) {
     constexpr int MID = (THETA - 1) / 2;
     constexpr float kInf = __builtin_huge_valf();
-    if (!(fabsf(s[0]) < kInf && fabsf(s[THETA - 1]) < kInf)) {
-        float copy[THETA];
-#pragma unroll
-        for (int t = 0; t < THETA; ++t) copy[t] = s[t];
-        return window_mean_stepwise(copy, THETA, BETA);
-    }
+    if (!(fabsf(s[0]) < kInf && fabsf(s[THETA - 1]) < kInf)) return false;
     const float med = s[MID];
-    bool in[THETA];
-#pragma unroll
-    for (int t = 0; t < THETA; ++t) in[t] = (t == MID);
-#pragma unroll
-    for (int p = 1; p <= MID && p <= BETA - 1; ++p) {
-        const int up = MID + (BETA - p);  // index of the (BETA-p)-th upper value
-        if (up > THETA - 1) {
-            in[MID - p] = true;
-        } else {
-            const bool lower = fabsf(__fsub_rn(s[up], med)) >= fabsf(__fsub_rn(s[MID - p], med));
-            in[MID - p] = lower;
-            in[up] = !lower;
-        }
-    }
-    // upper values that no lower value competes with (BETA - u > MID): always in
-#pragma unroll
-    for (int u = 1; u <= BETA - 1 && MID + u <= THETA - 1; ++u)
-        if (BETA - u > MID) in[MID + u] = true;
+    // ascending positions: the lower values (p = distance in rank from the median, descending), the median, the
+    // upper values (u ascending, paired with the lower value p = BETA - u)
     double sum = 0.0;
 #pragma unroll
-    for (int t = 0; t < THETA; ++t)
-        if (in[t]) sum += static_cast<double>(s[t]);
-    return static_cast<float>(sum / static_cast<double>(BETA));
+    for (int p = (MID < BETA - 1 ? MID : BETA - 1); p >= 1; --p) {
+        const int up = MID + (BETA - p);  // index of the (BETA-p)-th upper value
+        if (up > THETA - 1)
+            sum += static_cast<double>(s[MID - p]);
+        else
+            add_if<true>(sum, s[MID - p], fabsf(__fsub_rn(s[up], med)), fabsf(__fsub_rn(s[MID - p], med)));
+    }
+    sum += static_cast<double>(med);
+#pragma unroll
+    for (int u = 1; u <= BETA - 1 && MID + u <= THETA - 1; ++u) {
+        const int p = BETA - u;
+        if (p > MID)  // no lower value competes with it
+            sum += static_cast<double>(s[MID + u]);
+        else
+            add_if<false>(sum, s[MID + u], fabsf(__fsub_rn(s[MID + u], med)), fabsf(__fsub_rn(s[MID - p], med)));
+    }
+    mean = static_cast<float>(sum / static_cast<double>(BETA));
+    return true;
 }
 
-// Share of the sort's comparators whose max goes through the multiply-add pipe (kMaxOnFma of every kMaxOf).
-#ifndef BZ_TM_MAX_ON_FMA
-#define BZ_TM_MAX_ON_FMA 2
-#define BZ_TM_MAX_OF 3
-#endif
-constexpr int kMaxOnFma = BZ_TM_MAX_ON_FMA, kMaxOf = BZ_TM_MAX_OF;
+// One coordinate, out of line: the column is read again, sorted in the total order (insertion sort on order keys in
+// local memory) and its window grown step by step.  For the columns the register kernels hand back: those that
+// hold an infinity or a NaN.
+__device__ __noinline__ float trimmed_column_stepwise(const float* __restrict__ v, const int64_t* row, int64_t j, int theta, int beta) {
+    int k[BZ_MAX_F];
+    for (int t = 0; t < theta; ++t) {
+        const int x = order_key(__float_as_uint(v[row[t] + j]));
+        int pos = t;
+        while (pos > 0 && k[pos - 1] > x) {
+            k[pos] = k[pos - 1];
+            --pos;
+        }
+        k[pos] = x;
+    }
+    float sorted[BZ_MAX_F];
+    for (int t = 0; t < theta; ++t) sorted[t] = __uint_as_float(key_bits(k[t]));
+    return window_mean_stepwise(sorted, theta, beta);
+}
 
 // V coordinates per thread (V = 2, 4: 64- and 128-bit loads, rows aligned accordingly): the address arithmetic
 // and the load instructions are shared by the V coordinates.
@@ -351,40 +370,42 @@ __global__ void __launch_bounds__(128) trimmed_mean_kernel(const float* __restri
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
     for (int64_t g = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; g < groups; g += stride) {
         const int64_t j = g * V;
-        int k[V][THETA];
+        float k[V][THETA];
         const bool whole = j + V <= d;  // the last group may hold fewer coordinates
         if (V == 4 && whole) {
 #pragma unroll
             for (int t = 0; t < THETA; ++t) {
                 const float4 x = __ldcs(reinterpret_cast<const float4*>(v + row[t] + j));
-                k[0][t] = order_key(__float_as_uint(x.x));
-                k[V > 1 ? 1 : 0][t] = order_key(__float_as_uint(x.y));
-                k[V > 2 ? 2 : 0][t] = order_key(__float_as_uint(x.z));
-                k[V > 3 ? 3 : 0][t] = order_key(__float_as_uint(x.w));
+                k[0][t] = x.x;
+                k[V > 1 ? 1 : 0][t] = x.y;
+                k[V > 2 ? 2 : 0][t] = x.z;
+                k[V > 3 ? 3 : 0][t] = x.w;
             }
         } else if (V == 2 && whole) {
 #pragma unroll
             for (int t = 0; t < THETA; ++t) {
                 const float2 x = __ldcs(reinterpret_cast<const float2*>(v + row[t] + j));
-                k[0][t] = order_key(__float_as_uint(x.x));
-                k[V > 1 ? 1 : 0][t] = order_key(__float_as_uint(x.y));
+                k[0][t] = x.x;
+                k[V > 1 ? 1 : 0][t] = x.y;
             }
         } else {
 #pragma unroll
             for (int c = 0; c < V; ++c) {
                 const int64_t jc = j + c < d ? j + c : d - 1;  // past the end: the last coordinate once more
 #pragma unroll
-                for (int t = 0; t < THETA; ++t) k[c][t] = order_key(__float_as_uint(__ldcs(v + row[t] + jc)));
+                for (int t = 0; t < THETA; ++t) k[c][t] = __ldcs(v + row[t] + jc);
             }
         }
         float res[V];
 #pragma unroll
         for (int c = 0; c < V; ++c) {
-            SortNet<THETA>::template run<kMaxOnFma, kMaxOf>(k[c]);  // bound by the ALU pipe: comparators on two pipes
-            float s[THETA];
-#pragma unroll
-            for (int t = 0; t < THETA; ++t) s[t] = __uint_as_float(key_bits(k[c][t]));
-            res[c] = window_mean<THETA, BETA>(s);
+            // Finite columns (all but a handful) sort as numbers: no order keys, half the operations of a comparator on
+            // keys with its max on the other pipe.  The kernel is bound by the ALU pipe and by instruction issue.
+            SortNet<THETA>::run(k[c]);
+            if (!window_mean<THETA, BETA>(k[c], res[c])) {
+                const int64_t jc = j + c < d ? j + c : d - 1;
+                res[c] = trimmed_column_stepwise(v, row, jc, THETA, BETA);
+            }
         }
         if (V == 4 && whole) {
             *reinterpret_cast<float4*>(out + j) = make_float4(res[0], res[V > 1 ? 1 : 0], res[V > 2 ? 2 : 0], res[V > 3 ? 3 : 0]);
