@@ -118,6 +118,24 @@ def test_a_row_that_outgrows_its_scale():
     _check_close(got, want)
 
 
+def test_scale_changes_give_the_same_answer_every_launch():
+    # the same rows as above, 30 launches: a change of scale involves every role of a CTA (converters, the MMA thread's
+    # read-back request, the drain warps), so a hand-off that depended on timing would show as a launch that differs
+    f, d = 49, 400_000
+    g = inputs.true_gradients(f, d, seed=5).numpy()
+    g[17, 222_222:222_300] *= 1.0e3
+    g[:, 300_000:] *= 300.0
+    g[5, 100_000:] *= 1.0e-3
+    want = oracle.pairdist(g)
+    ws = bz.alloc_workspace(bz.OP_PAIRDIST, 0, f, d)
+    v = torch.from_numpy(g).to(DEV)
+    first = bz.pairdist(v, workspace=ws).cpu().numpy()
+    _check_close(first, want)
+    for _ in range(30):
+        again = bz.pairdist(v, workspace=ws).cpu().numpy()
+        assert np.array_equal(again, first) and bz.pairdist_status(ws, f) == 0
+
+
 @pytest.mark.parametrize("seed", range(8))
 def test_randomised_scales_outliers_and_sparse_rows(seed):
     # rows whose magnitude changes from segment to segment (layers), single outliers, rows that start with zeros,
