@@ -414,6 +414,21 @@ def run_ours(args):
         del keep
         torch.cuda.empty_cache()
 
+    # ---- N > 1: the exhaustive worst-case search dealt to the ranks (one gather of the shares' maxima) -------
+    if world > 1 and not args.no_extra and args.coords == 0:
+        from paper_2010_04902_b200 import sharding
+        _, _, mask75 = bz.assign_mols(7, 5)
+        sharding.worst_case(mask75, 49, 5, 9)                      # warm-up (and the binomial table)
+        dist.barrier()
+        t0 = time.perf_counter()
+        c13, set13, n13 = sharding.worst_case(mask75, 49, 5, 13)
+        dist.barrier()
+        dt = time.perf_counter() - t0
+        if rank == 0:
+            result["worst_case_sharded"] = {"K": 35, "f": 49, "r": 5, "q": 13, "subsets": n13, "c_max": c13, "argmax": set13,
+                                            "seconds_wall_all_ranks": dt, "subsets_per_s": n13 / dt,
+                                            "sharding": "subsets dealt to the ranks in fixed-size runs; one all_gather of (c_max, argmax)"}
+
     if rank == 0 and world == 1 and not args.no_extra and args.coords == 0:
         result["config1"] = config1_leg(bz, inputs, torch, device)
         result["unaligned_d"] = unaligned_leg(bz, inputs, torch, device, peak)

@@ -379,6 +379,18 @@ int bz_worst_case(const uint64_t* worker_mask, int K, int f, int r, int q, uint6
                   int32_t* argmax, uint64_t* n_subsets, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * One share of the same search, for several GPUs (or several calls): the q-subsets are dealt to `parts`
+ * shares in fixed-size runs of the enumeration, share `part` (0 <= part < parts) evaluates its own, and the
+ * maximum over all shares - by c_max, then by the lexicographically first argmax - is bz_worst_case's
+ * result (Sec. 5.3.2; nothing else is exchanged).  A share that receives no run reports c_max = -1
+ * (and leaves argmax alone).  n_subsets is C(K, q), the size of the whole search, for every share.
+ * Arguments, limits and errors as bz_worst_case; BZ_ERR_INVALID_ARG for a part outside [0, parts).
+ */
+int bz_worst_case_part(const uint64_t* worker_mask, int K, int f, int r, int q, int part, int parts, uint64_t max_subsets,
+                       int32_t* c_max, int32_t* argmax, uint64_t* n_subsets, void* workspace, size_t workspace_bytes,
+                       void* stream);
+
+/*
  * The same search for the placement bz_assign_mols(l, r) makes (Algorithm 2; Ramanujan Case 2 when
  * r == l), shortened by the design's symmetry: shifting all files by (i, j) -> (i + a, j + b) maps
  * worker (k, s) to (k, s + alpha_k*a + b), so the l*l translations permute the workers inside each

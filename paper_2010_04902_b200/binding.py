@@ -60,6 +60,8 @@ _SIGNATURES = {
     "bz_trimmed_mean": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_vp, _c_int, _c_int, _c_vp, _c_vp]),
     "bz_bulyan": (_c_int, [_c_vp, _c_int, _c_i64, _c_i64, _c_int, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp]),
     "bz_worst_case": (_c_int, [_c_vp, _c_int, _c_int, _c_int, _c_int, _c_u64, _c_vp, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp]),
+    "bz_worst_case_part": (_c_int, [_c_vp, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_u64, _c_vp, _c_vp, _c_vp, _c_vp, _c_sz,
+                                    _c_vp]),
     "bz_vote_pairdist": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_vp, _c_i64, _c_vp, _c_vp, _c_sz, _c_vp]),
     "bz_vote_multikrum": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_int, _c_int, _c_vp, _c_i64, _c_vp, _c_vp,
                                    _c_vp, _c_vp, _c_sz, _c_vp]),
@@ -228,6 +230,22 @@ def worst_case(worker_mask, f: int, r: int, q: int, max_subsets: int = 0, worksp
     st = lib().bz_worst_case(mask.ctypes.data, K, f, r, q, max_subsets, ctypes.addressof(cmax), arg.ctypes.data,
                              ctypes.addressof(n), ws.data_ptr(), ws.numel(), _stream())
     _check(st, "bz_worst_case(K=%d, q=%d)" % (K, q))
+    return int(cmax.value), arg[:q].copy(), int(n.value)
+
+
+def worst_case_part(worker_mask, f: int, r: int, q: int, part: int, parts: int, max_subsets: int = 0,
+                    workspace: torch.Tensor | None = None):
+    """bz_worst_case_part: share `part` of `parts` of the exhaustive search.  Returns (c_max, argmax[q] numpy,
+    n_subsets); c_max is -1 for a share that received nothing."""
+    mask = np.ascontiguousarray(worker_mask, np.uint64)
+    K = int(mask.shape[0])
+    ws = workspace if workspace is not None else alloc_workspace(OP_WORST_CASE, r, f)
+    cmax = ctypes.c_int32(0)
+    n = ctypes.c_uint64(0)
+    arg = np.zeros(max(q, 1), np.int32)
+    st = lib().bz_worst_case_part(mask.ctypes.data, K, f, r, q, part, parts, max_subsets, ctypes.addressof(cmax),
+                                  arg.ctypes.data, ctypes.addressof(n), ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "bz_worst_case_part(K=%d, q=%d, part %d of %d)" % (K, q, part, parts))
     return int(cmax.value), arg[:q].copy(), int(n.value)
 
 

@@ -106,6 +106,7 @@ struct WcParams {
     uint32_t chunk_len[kMaxK];         // prefixes per run
     uint32_t y_width[kMaxK];           // first-tail-worker values per piece
     int K, q, p, n_groups, first_l;   // group g holds the prefixes whose largest worker is first_l + g
+    uint32_t part, parts;             // this launch takes the chunks whose index is part modulo parts
 };
 
 // binom[n][k] for n, k <= 64 (saturating), filled by the host into constant memory
@@ -130,7 +131,9 @@ __global__ void __launch_bounds__(kWcBlock, 12)
     const uint64_t n_chunks = s_begin[prm.n_groups];
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
     int g = 0;
-    for (uint64_t chunk = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; chunk < n_chunks; chunk += stride) {
+    for (uint64_t unit = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;; unit += stride) {
+        const uint64_t chunk = prm.part + prm.parts * unit;
+        if (chunk >= n_chunks) break;
         while (chunk >= s_begin[g + 1]) ++g;  // chunks only move forward
         const int l = prm.first_l + g;        // largest worker of the prefix (p >= 1), or -1 when p == 0
         const int m = p - 1;                  // free prefix elements, from {0..l-1}
@@ -221,10 +224,13 @@ size_t worst_case_workspace_bytes() { return round_up(sizeof(WcResult) * kWcMaxB
 
 using namespace bz;
 
-extern "C" int bz_worst_case(const uint64_t* worker_mask, int K, int f, int r, int q, uint64_t max_subsets,
-                             int32_t* c_max, int32_t* argmax, uint64_t* n_subsets, void* workspace,
-                             size_t workspace_bytes, void* stream) {
+// The search over the chunks whose index is `part` modulo `parts` (the whole search: 0 of 1).  A share without
+// a chunk reports c_max = -1.
+static int worst_case_share(const uint64_t* worker_mask, int K, int f, int r, int q, int part, int parts, uint64_t max_subsets,
+                            int32_t* c_max, int32_t* argmax, uint64_t* n_subsets, void* workspace, size_t workspace_bytes,
+                            void* stream) {
     if (worker_mask == nullptr || c_max == nullptr) return BZ_ERR_INVALID_ARG;
+    if (parts < 1 || part < 0 || part >= parts) return BZ_ERR_INVALID_ARG;
     if (K < 1 || f < 1 || r < 1 || (r % 2) == 0 || q < 0 || q > K) return BZ_ERR_INVALID_ARG;
     if (K > kMaxK || f > 64 || r > 7) return BZ_ERR_UNSUPPORTED;
     if (f < 64)
@@ -239,10 +245,12 @@ extern "C" int bz_worst_case(const uint64_t* worker_mask, int K, int f, int r, i
     if (max_subsets != 0 && total > max_subsets) return BZ_ERR_BUDGET;
     if (n_subsets) *n_subsets = total;
     if (q == 0) {
-        *c_max = 0;
+        *c_max = part == 0 ? 0 : -1;  // the one (empty) set belongs to the first share
         return BZ_OK;
     }
     WcParams prm;
+    prm.part = static_cast<uint32_t>(part);
+    prm.parts = static_cast<uint32_t>(parts);
     for (int u = 0; u < kMaxK; ++u) prm.mask[u] = u < K ? worker_mask[u] : 0;
     const int tail = q < kMaxTail ? q : kMaxTail;
     const int p = q - tail;
@@ -281,7 +289,12 @@ extern "C" int bz_worst_case(const uint64_t* worker_mask, int K, int f, int r, i
         n_chunks += pieces * prm.prefix_chunks[g];
     }
     prm.chunk_begin[prm.n_groups] = n_chunks;
-    uint64_t blocks = (n_chunks + kWcBlock - 1) / kWcBlock;
+    const uint64_t my_chunks = n_chunks > static_cast<uint64_t>(part) ? (n_chunks - part + parts - 1) / parts : 0;
+    if (my_chunks == 0) {
+        *c_max = -1;
+        return BZ_OK;
+    }
+    uint64_t blocks = (my_chunks + kWcBlock - 1) / kWcBlock;
     if (blocks > static_cast<uint64_t>(kWcMaxBlocks)) blocks = kWcMaxBlocks;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     WcResult* dev = static_cast<WcResult*>(workspace);
@@ -296,4 +309,16 @@ extern "C" int bz_worst_case(const uint64_t* worker_mask, int K, int f, int r, i
     st = check_launch();
     if (st != BZ_OK) return st;
     return collect_best(dev, static_cast<int>(blocks), K, q, c_max, argmax, s);
+}
+
+extern "C" int bz_worst_case(const uint64_t* worker_mask, int K, int f, int r, int q, uint64_t max_subsets,
+                             int32_t* c_max, int32_t* argmax, uint64_t* n_subsets, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    return worst_case_share(worker_mask, K, f, r, q, 0, 1, max_subsets, c_max, argmax, n_subsets, workspace, workspace_bytes, stream);
+}
+
+extern "C" int bz_worst_case_part(const uint64_t* worker_mask, int K, int f, int r, int q, int part, int parts,
+                                  uint64_t max_subsets, int32_t* c_max, int32_t* argmax, uint64_t* n_subsets, void* workspace,
+                                  size_t workspace_bytes, void* stream) {
+    return worst_case_share(worker_mask, K, f, r, q, part, parts, max_subsets, c_max, argmax, n_subsets, workspace, workspace_bytes, stream);
 }

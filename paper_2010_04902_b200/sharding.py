@@ -4,6 +4,8 @@ The vote, the median, the means and the trimmed means are independent per coordi
 aggregates its own contiguous slab of coordinates and nothing is exchanged.  The Krum family needs
 one exchange: squared distances are sums over coordinates, so the ranks' partial f x f matrices are
 added with a single all-reduce (at most 128 x 128 doubles) before the - replicated - selection.
+The exhaustive worst-case search shards over its subsets instead: every rank searches its share and
+the ranks' (c_max, argmax) meet in one gather.
 
 ``ops`` is the module that supplies the per-rank operations; it defaults to the CUDA binding.  The
 functions here contain only the partitioning and the exchange.
@@ -89,3 +91,33 @@ def vote_bulyan(replicas_slab: torch.Tensor, c: int, ops=None, group=None):
     sel = ops.bulyan_select(D, c)
     theta = voted.shape[0] - 2 * c
     return ops.trimmed_mean(voted, sel, theta - 2 * c), sel, D, voted
+
+
+def best_of_shares(shares):
+    """The result of the whole search from the shares' (c_max, argmax) pairs: the largest c_max, and among
+    equals the lexicographically first argmax.  Shares that received nothing (c_max < 0) do not count."""
+    best = None
+    for c, arg in shares:
+        if c < 0:
+            continue
+        key = (-int(c), tuple(int(u) for u in arg))
+        if best is None or key < best[0]:
+            best = (key, int(c), [int(u) for u in arg])
+    if best is None:
+        raise ValueError("no share of the search evaluated a subset")
+    return best[1], best[2]
+
+
+def worst_case(worker_mask, f: int, r: int, q: int, max_subsets: int = 0, ops=None, group=None):
+    """Exhaustive c_max^(q) with the subsets dealt to the ranks (bz_worst_case_part), one all-gather of
+    (c_max, argmax).  Returns (c_max, argmax[q] list, n_subsets), the same on every rank and the same as the
+    single-GPU search."""
+    ops = _ops(ops)
+    world = _world(group)
+    rank = dist.get_rank(group) if world > 1 else 0
+    c, arg, n = ops.worst_case_part(worker_mask, f, r, q, rank, world, max_subsets)
+    if world == 1:
+        return best_of_shares([(c, arg)]) + (n,)
+    shares = [None] * world
+    dist.all_gather_object(shares, (int(c), [int(u) for u in arg]), group=group)
+    return best_of_shares(shares) + (n,)

@@ -47,10 +47,12 @@ def _rank(rank, world, port, l, r, q, d, c, ret):
         path_mk = bz.last_path()
         b_out, b_sel, _, _ = sharding.vote_bulyan(slab, min(c, (f - 3) // 4))
         med = sharding.vote_median(slab)
+        _, _, mask = bz.assign_mols(l, r)
+        wc = [sharding.worst_case(mask, f, r, qq) for qq in (2, q)]    # the exhaustive search, dealt to the two ranks
         torch.cuda.synchronize()
         ret[rank] = dict(j=(j0, j1), out=out.cpu().numpy(), sel=sel.cpu().numpy(), D=D.cpu().numpy(),
                          voted=voted.cpu().numpy(), b_out=b_out.cpu().numpy(), b_sel=b_sel.cpu().numpy(),
-                         med=med.cpu().numpy(), timeouts=bz.pipeline_timeouts() - before, path=path_mk)
+                         med=med.cpu().numpy(), timeouts=bz.pipeline_timeouts() - before, path=path_mk, wc=wc)
     finally:
         dist.destroy_process_group()
 
@@ -85,6 +87,10 @@ def test_two_ranks_with_the_cuda_binding(l, r, q, d, c):
         assert p["sel"].tolist() == want_sel.tolist() and p["b_sel"].tolist() == want_bsel.tolist()
         nz = want_D > 0
         assert (np.abs(p["D"][nz] - want_D[nz]) <= 1e-7 * want_D[nz]).all() and (p["D"][~nz] == 0).all()
+    for k, qq in enumerate((2, q)):
+        want_c, want_set, want_n = oracle.worst_case(wf, f, r, qq)
+        for p in parts:
+            assert p["wc"][k] == (want_c, want_set.tolist(), want_n)
     for key, want in (("voted", voted), ("out", want_out), ("b_out", want_b), ("med", want_med)):
         got = np.concatenate([p[key] for p in parts], axis=-1)
         assert np.array_equal(got.view(np.uint32), np.ascontiguousarray(want).view(np.uint32)), key

@@ -101,3 +101,47 @@ def test_symmetric_search_budget_and_arguments():
     with pytest.raises(bz.BzError) as e:
         bz.worst_case_mols(5, 1, 2)
     assert e.value.status == bz.ERR_UNSUPPORTED
+
+
+# ---- the search dealt to several shares (bz_worst_case_part) ----------------------------------------------
+
+@pytest.mark.parametrize("l,r,qs", [(5, 3, [0, 1, 2, 3, 5, 7]), (7, 3, [1, 4, 6]), (5, 5, [3, 6, 9]), (3, 3, [1, 2, 4])])
+def test_shares_combine_to_the_whole_search(l, r, qs):
+    from paper_2010_04902_b200 import sharding
+    wf, _, _ = oracle.assign(l, r)
+    _, _, mask = bz.assign_mols(l, r)
+    f, K = l * l, l * r
+    for q in qs:
+        want, warg, wn = oracle.worst_case(wf, f, r, q)
+        for parts in (1, 2, 3, 8, 1000):
+            shares = []
+            for part in range(parts):
+                c, arg, n = bz.worst_case_part(mask, f, r, q, part, parts)
+                assert n == wn == math.comb(K, q)
+                assert c == -1 or oracle.count_distorted(oracle.assign(l, r)[1], arg) == c   # each share's maximiser is a real set
+                shares.append((c, arg))
+            assert sharding.best_of_shares(shares) == (want, warg.tolist()), (l, r, q, parts)
+            if parts == 1:
+                assert shares[0][0] == bz.worst_case(mask, f, r, q)[0]
+
+
+def test_shares_on_the_row_the_paper_calls_intractable():
+    # (K, f, l, r) = (35, 49, 7, 5), q = 13: 1.48e9 subsets in four shares; the maximum and its first set are those of
+    # the one-call search, and every share's own maximum is at most that
+    from paper_2010_04902_b200 import sharding
+    _, _, mask = bz.assign_mols(7, 5)
+    want, warg, _ = bz.worst_case(mask, 49, 5, 13)
+    shares = [bz.worst_case_part(mask, 49, 5, 13, p, 4)[:2] for p in range(4)]
+    assert all(0 <= c <= want for c, _ in shares)
+    assert sharding.best_of_shares(shares) == (want, warg.tolist())
+
+
+def test_share_arguments():
+    _, _, mask = bz.assign_mols(5, 3)
+    for part, parts in [(-1, 2), (2, 2), (0, 0)]:
+        with pytest.raises(bz.BzError) as e:
+            bz.worst_case_part(mask, 25, 3, 3, part, parts)
+        assert e.value.status == bz.ERR_INVALID_ARG
+    with pytest.raises(bz.BzError) as e:
+        bz.worst_case_part(mask, 25, 3, 7, 0, 2, max_subsets=100)
+    assert e.value.status == bz.ERR_BUDGET

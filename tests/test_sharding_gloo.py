@@ -143,3 +143,81 @@ def test_two_ranks_reproduce_the_single_rank_result(d):
         assert p["mk_sel"].tolist() == want_mk_sel.tolist() and p["bu_sel"].tolist() == want_bu_sel.tolist()
     assert np.array_equal(np.concatenate([p["mk_out"] for p in parts]), want_mk)
     assert np.array_equal(np.concatenate([p["bu_out"] for p in parts]), want_bu)
+
+
+# ---- the exhaustive worst-case search dealt to the ranks ------------------------------------------------
+
+def _brute_force_part(worker_files, f, r, q, part, parts):
+    """A stand-in for bz_worst_case_part with its signature: every q-subset in lexicographic order, subset number n
+    going to share n % parts; returns (c_max, argmax, n_subsets) of the share, c_max = -1 if it is empty."""
+    import itertools
+    K = len(worker_files)
+    need = (r + 1) // 2
+    best, best_set, n = -1, [0] * q, 0
+    for n, S in enumerate(itertools.combinations(range(K), q)):
+        if n % parts != part:
+            continue
+        holders = np.zeros(f, np.int64)
+        for u in S:
+            holders[list(worker_files[u])] += 1
+        c = int((holders >= need).sum())
+        if c > best:
+            best, best_set = c, list(S)
+    return best, np.array(best_set, np.int32), n + 1
+
+
+def test_best_of_shares_rules():
+    assert sharding.best_of_shares([(3, [0, 5, 9]), (4, [1, 2, 3]), (-1, [0, 0, 0])]) == (4, [1, 2, 3])
+    assert sharding.best_of_shares([(4, [1, 2, 4]), (4, [1, 2, 3]), (4, [2, 3, 4])]) == (4, [1, 2, 3])   # first in lexicographic order
+    assert sharding.best_of_shares([(-1, [0]), (0, [7])]) == (0, [7])
+    with pytest.raises(ValueError):
+        sharding.best_of_shares([(-1, [0]), (-1, [0])])
+
+
+def test_shares_of_the_search_combine_to_the_whole():
+    wf, _, _ = oracle.assign(5, 3)
+    for q in (1, 2, 3, 4):
+        want_c, want_set, _ = oracle.worst_case(wf, 25, 3, q)
+        for parts in (1, 2, 3, 7, 40):     # q = 1 has 15 subsets: with 40 shares most are empty
+            shares = [_brute_force_part(wf, 25, 3, q, p, parts)[:2] for p in range(parts)]
+            assert sharding.best_of_shares(shares) == (want_c, [int(u) for u in want_set])
+            if q == 1 and parts == 40:
+                assert sum(c < 0 for c, _ in shares) == 25
+
+
+def _wc_worker(rank, world, port, ret):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        import inspect
+        from paper_2010_04902_b200 import binding
+        wf, _, _ = oracle.assign(5, 3)
+        sig = inspect.signature(binding.worst_case_part)
+
+        def part(mask, f, r, q, p, parts, max_subsets=0):
+            sig.bind(mask, f, r, q, p, parts, max_subsets)      # what the default wiring would hand to the binding
+            assert (p, parts) == (rank, world)
+            return _brute_force_part(wf, f, r, q, p, parts)
+        ops = types.SimpleNamespace(worst_case_part=part)
+        ret[rank] = [sharding.worst_case(None, 25, 3, q, ops=ops) for q in (2, 3, 4)]
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_share_the_worst_case_search():
+    world = 2
+    ctx = mp.get_context("spawn")
+    ret = ctx.Manager().dict()
+    port = _free_port()
+    procs = [ctx.Process(target=_wc_worker, args=(rk, world, port, ret)) for rk in range(world)]
+    for p in procs:
+        p.start()
+    for p in procs:
+        p.join(180)
+        assert p.exitcode == 0
+    wf, _, _ = oracle.assign(5, 3)
+    for k, q in enumerate((2, 3, 4)):
+        want_c, want_set, want_n = oracle.worst_case(wf, 25, 3, q)
+        for rk in range(world):
+            c, arg, n = ret[rk][k]
+            assert (c, arg, n) == (want_c, [int(u) for u in want_set], want_n)
