@@ -215,10 +215,13 @@ int bz_vote_median_host(const float* replicas_host, int r, int f, int64_t d, flo
  *     error ~1e-11.  Two rows closer than binary64 sums of their squared norms can resolve are
  *     reported at distance 0 if the bound on their true distance is below 1e-7 of the smallest
  *     non-zero distance either has; otherwise the binary64 kernel answers.
- *   - Binary64 difference form (same shapes; also rows shorter than 8192): differences, squares and
- *     sums in double precision, the oracle's result to ~1e-15 whatever the data; about 2.5x the
- *     time of the binary32 kernel.  It runs behind the first kernel, reads that kernel's flag and
- *     returns at once unless asked.
+ *   - Binary64 difference form (f = 25 or 49; any d, rows on any 4-byte boundary): differences,
+ *     squares and sums in double precision, the oracle's result to ~1e-15 whatever the data; about
+ *     2.5x the time of the binary32 kernel.  It runs behind the first kernel, reads that kernel's
+ *     flag and returns at once unless asked; and it answers alone for rows shorter than 8192 and
+ *     for rows the first kernel cannot take (not 16-byte aligned, ld not a multiple of 4 - e.g.
+ *     contiguous rows of a length that is not a multiple of 4: pad them and the first kernel runs,
+ *     about twice as fast).
  *   - Binary32 difference form (every other shape, and bz_pairdist_static): differences and squares
  *     in binary32, added in binary32 inside blocks of at most 1024 coordinates (interleaved partial
  *     sums of at most 128 terms) and in binary64 across blocks, in a fixed order.  Its rounding

@@ -28,16 +28,45 @@ namespace {
 // the G groups of a pair are added in binary32 in a fixed order and the result goes into the CTA's
 // binary64 accumulator in shared memory; one fixed-order reduction over CTAs finishes.
 // The result is bit-reproducible from run to run.
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src, int src_bytes) {
+// W bytes per request (16, 8 or 4: what the rows' alignment allows); bytes past src_bytes are filled with zeros
+template <int W> __device__ __forceinline__ void cp_async_w(void* smem_dst, const void* gmem_src, int src_bytes) {
     const unsigned dst = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(gmem_src), "r"(src_bytes));
+    if constexpr (W == 16)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(gmem_src), "r"(src_bytes));
+    else if constexpr (W == 8)
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;\n" ::"r"(dst), "l"(gmem_src), "r"(src_bytes));
+    else
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;\n" ::"r"(dst), "l"(gmem_src), "r"(src_bytes));
+}
+// One tile (kTD coordinates from j0, zeros past d) of F rows into dst[F][kRowStride], NT threads.
+template <int F, int NT, int W>
+__device__ __forceinline__ void stage_rows_w(float* dst, const float* __restrict__ v, int64_t d, int64_t ld, int64_t j0, int tid) {
+    constexpr int E = W / 4, per_row = kTD / E;
+    for (int idx = tid; idx < F * per_row; idx += NT) {
+        const int row = idx / per_row, c = idx - row * per_row;
+        const int64_t j = j0 + E * c;
+        const int64_t left = d - j;
+        const int bytes = left >= E ? W : (left > 0 ? static_cast<int>(left) * 4 : 0);
+        const float* src = bytes ? v + row * ld + j : v;  // zero-byte requests still name a valid address
+        cp_async_w<W>(dst + row * kRowStride + E * c, src, bytes);
+    }
+}
+// width: the bytes per request the rows allow (uniform over the launch)
+template <int F, int NT>
+__device__ __forceinline__ void stage_rows(float* dst, const float* __restrict__ v, int64_t d, int64_t ld, int64_t j0, int tid, int width) {
+    if (width == 16)
+        stage_rows_w<F, NT, 16>(dst, v, d, ld, j0, tid);
+    else if (width == 8)
+        stage_rows_w<F, NT, 8>(dst, v, d, ld, j0, tid);
+    else
+        stage_rows_w<F, NT, 4>(dst, v, d, ld, j0, tid);
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
 
 template <int F, int T, int G>
 __global__ void __launch_bounds__(PairTile<F, T, G>::NT, tiled_ctas_per_sm<F, T, G>())
-    pairdist_tiled_kernel(const float* __restrict__ v, int64_t d, int64_t ld, double* __restrict__ partial,
+    pairdist_tiled_kernel(const float* __restrict__ v, int64_t d, int64_t ld, int width, double* __restrict__ partial,
                           const int* __restrict__ gate) {
     using PT = PairTile<F, T, G>;
     if (gate != nullptr && *gate == 0) return;  // the integer kernel's distances stand
@@ -62,17 +91,7 @@ __global__ void __launch_bounds__(PairTile<F, T, G>::NT, tiled_ctas_per_sm<F, T,
 
     const int64_t n_tiles = (d + kTD - 1) / kTD;
     auto load_tile = [&](int buf, int64_t tile) {
-        const int64_t j0 = tile * kTD;
-        constexpr int per_row = kTD / 4;
-        float* dst = stage0 + buf * F * kRowStride;
-        for (int idx = tid; idx < F * per_row; idx += NT) {
-            const int row = idx / per_row, c4 = idx - row * per_row;
-            const int64_t j = j0 + 4 * c4;
-            const int64_t left = d - j;
-            const int bytes = left >= 4 ? 16 : (left > 0 ? static_cast<int>(left) * 4 : 0);
-            const float* src = bytes ? v + row * ld + j : v;  // zero-byte requests still name a valid address
-            cp_async16(dst + row * kRowStride + 4 * c4, src, bytes);
-        }
+        stage_rows<F, NT>(stage0 + buf * F * kRowStride, v, d, ld, tile * kTD, tid, width);
         cp_async_commit();
     };
 
@@ -133,7 +152,7 @@ template <int F, int T, int G> constexpr size_t f64_smem_bytes() {
 
 template <int F, int T, int G>
 __global__ void __launch_bounds__(PairTile<F, T, G>::NT, 1)
-    pairdist_f64_kernel(const float* __restrict__ v, int64_t d, int64_t ld, double* __restrict__ partial,
+    pairdist_f64_kernel(const float* __restrict__ v, int64_t d, int64_t ld, int width, double* __restrict__ partial,
                         const int* __restrict__ gate) {
     using PT = PairTile<F, T, G>;
     if (gate != nullptr && *gate == 0) return;  // the integer kernel's distances stand
@@ -150,17 +169,7 @@ __global__ void __launch_bounds__(PairTile<F, T, G>::NT, 1)
 
     const int64_t n_tiles = (d + kTD - 1) / kTD;
     auto load_tile = [&](int buf, int64_t tile) {
-        const int64_t j0 = tile * kTD;
-        constexpr int per_row = kTD / 4;
-        float* dst = stage0 + buf * F * kRowStride;
-        for (int idx = tid; idx < F * per_row; idx += NT) {
-            const int row = idx / per_row, c4 = idx - row * per_row;
-            const int64_t j = j0 + 4 * c4;
-            const int64_t left = d - j;
-            const int bytes = left >= 4 ? 16 : (left > 0 ? static_cast<int>(left) * 4 : 0);
-            const float* src = bytes ? v + row * ld + j : v;  // zero-byte requests still name a valid address
-            cp_async16(dst + row * kRowStride + 4 * c4, src, bytes);
-        }
+        stage_rows<F, NT>(stage0 + buf * F * kRowStride, v, d, ld, tile * kTD, tid, width);
         cp_async_commit();
     };
 
@@ -280,6 +289,12 @@ template <int F, int T, int G> constexpr size_t tiled_partial_doubles() {
     return static_cast<size_t>(kNumSMs) * tiled_ctas_per_sm<F, T, G>() * PairTile<F, T, G>::NPB * PairTile<F, T, G>::TT;
 }
 
+// bytes per staging request that every row start allows: 16, 8 or 4
+inline int row_width(const float* v, int64_t ld) {
+    const uintptr_t bits = reinterpret_cast<uintptr_t>(v) | static_cast<uintptr_t>(ld * 4);
+    return bits % 16 == 0 ? 16 : (bits % 8 == 0 ? 8 : 4);
+}
+
 template <int F, int T, int G>
 int launch_pairdist_tiled(const float* v, int64_t d, int64_t ld, double* dist, double* partial, const int* gate, cudaStream_t s) {
     constexpr int NT = PairTile<F, T, G>::NT;
@@ -287,7 +302,7 @@ int launch_pairdist_tiled(const float* v, int64_t d, int64_t ld, double* dist, d
     cudaError_t e = cudaFuncSetAttribute(pairdist_tiled_kernel<F, T, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return cuda_failed(e);
     const int ctas = pairdist_ctas(d, kTD, tiled_ctas_per_sm<F, T, G>());
-    pairdist_tiled_kernel<F, T, G><<<ctas, NT, smem, s>>>(v, d, ld, partial, gate);
+    pairdist_tiled_kernel<F, T, G><<<ctas, NT, smem, s>>>(v, d, ld, row_width(v, ld), partial, gate);
     note_launch();
     int st = check_launch();
     if (st != BZ_OK) return st;
@@ -303,7 +318,7 @@ int launch_pairdist_f64(const float* v, int64_t d, int64_t ld, double* dist, dou
     cudaError_t e = cudaFuncSetAttribute(pairdist_f64_kernel<F, T, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return cuda_failed(e);
     const int ctas = pairdist_ctas(d, kTD, 1);  // never more CTAs than the binary32 kernel's workspace provides for
-    pairdist_f64_kernel<F, T, G><<<ctas, NT, smem, s>>>(v, d, ld, partial, gate);
+    pairdist_f64_kernel<F, T, G><<<ctas, NT, smem, s>>>(v, d, ld, row_width(v, ld), partial, gate);
     note_launch();
     int st = check_launch();
     if (st != BZ_OK) return st;
@@ -362,8 +377,12 @@ int pairdist_clear_status(void* ws, int f, cudaStream_t s) {
 // The binary32 difference-form kernels.  gate != nullptr: they run only if *gate (device) is not 0.
 int pairdist_fp32(const float* v, int f, int64_t d, int64_t ld, double* dist, double* partial, const int* gate, cudaStream_t s);
 
-// The binary64 kernel exists for the shapes of the integer kernel: f = 25 or 49, rows the 128-bit copies accept.
-bool pairdist_f64_has(const float* v, int f, int64_t ld) { return (f == 25 || f == 49) && aligned16(v) && (ld % 4 == 0); }
+// The binary64 kernel exists for the shapes of the integer kernel, f = 25 or 49, rows on any 4-byte boundary.
+bool pairdist_f64_has(const float* v, int f, int64_t ld) {
+    (void)v;
+    (void)ld;
+    return f == 25 || f == 49;
+}
 int pairdist_f64(const float* v, int f, int64_t d, int64_t ld, double* dist, double* partial, const int* gate, cudaStream_t s) {
     if (gate == nullptr) note_path(BZ_PATH_FP64);
     if (f == 25) return launch_pairdist_f64<BZ_PD_25>(v, d, ld, dist, partial, gate, s);
@@ -396,9 +415,8 @@ int pairdist_on_device(const float* v, int f, int64_t d, int64_t ld, double* dis
 
 int pairdist_fp32(const float* v, int f, int64_t d, int64_t ld, double* dist, double* partial, const int* gate, cudaStream_t s) {
     if (gate == nullptr) note_path(BZ_PATH_FP32);
-    const bool vec = aligned16(v) && (ld % 4 == 0);
-    if (vec && f == 25) return launch_pairdist_tiled<BZ_PD_25>(v, d, ld, dist, partial, gate, s);
-    if (vec && f == 49) return launch_pairdist_tiled<BZ_PD_49>(v, d, ld, dist, partial, gate, s);
+    if (f == 25) return launch_pairdist_tiled<BZ_PD_25>(v, d, ld, dist, partial, gate, s);
+    if (f == 49) return launch_pairdist_tiled<BZ_PD_49>(v, d, ld, dist, partial, gate, s);
     const int ctas = pairdist_ctas(d, kGT);
     pairdist_generic_kernel<<<ctas, 256, 0, s>>>(v, f, d, ld, partial);
     note_launch();

@@ -83,6 +83,29 @@ def test_pairdist_unaligned_rows():
     assert np.array_equal(bz.pairdist(buf[:, 4:1007]).cpu().numpy(), oracle.pairdist(v.numpy()))
 
 
+@pytest.mark.parametrize("f", [25, 49])
+@pytest.mark.parametrize("d,shift", [(150_002, 0), (150_001, 0), (150_003, 1), (150_000, 2), (150_000, 3), (1003, 1)])
+@pytest.mark.parametrize("path", ["", "fp32"])
+def test_pairdist_rows_on_8_and_4_byte_boundaries(f, d, shift, path, monkeypatch):
+    # contiguous rows of a length that is not a multiple of 4 (every other row starts 8 or 4 bytes off a 16-byte
+    # boundary) and rows shifted inside a buffer: the tiled kernels stage them with 8- or 4-byte copies.  By default the
+    # binary64 kernel answers (the integer kernel needs 16-byte aligned rows); BZ_PAIRDIST_PATH=fp32 takes the binary32 one.
+    if path:
+        monkeypatch.setenv("BZ_PAIRDIST_PATH", path)
+    g = inputs.true_gradients(f, d, seed=f + d % 100)
+    g[f - 1] = g[2]
+    buf = torch.zeros(f * d + 8, dtype=torch.float32, device=DEV)
+    rows = buf[shift: shift + f * d].view(f, d)
+    rows.copy_(g)
+    want = oracle.pairdist(g.numpy())
+    got = bz.pairdist(rows).cpu().numpy()
+    assert bz.last_path() == (bz.PATH_FP32 if path else bz.PATH_FP64)
+    assert np.array_equal(got, got.T) and (np.diag(got) == 0).all() and got[2, f - 1] == 0
+    nz = want > 0
+    tol = 1e-7 if path else 1e-12
+    assert (np.abs(got[nz] - want[nz]) <= tol * want[nz]).all()
+
+
 def test_krum_hand_cases_on_device():
     v = torch.tensor([[0.0], [1.0], [2.0], [3.0], [10.0]])
     D = bz.pairdist(v.to(DEV))
