@@ -834,7 +834,7 @@ def run_reference(args):
     cores = oracle.num_threads()
     sample = "first %d of %d coordinates of the same workload per step" % (n_sample, cfg["d"])
     print(json.dumps({
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": max(int(os.environ.get("WORLD_SIZE", "1")), int(args.gpus)),
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u32", "data": "synthetic",
         "config": {"workload": workload_name(cfg), "sample": sample},
