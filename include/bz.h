@@ -411,6 +411,14 @@ int bz_worst_case_part(const uint64_t* worker_mask, int K, int f, int r, int q, 
 int bz_worst_case_mols(int l, int r, int q, uint64_t max_subsets, int32_t* c_max, int32_t* argmax,
                        uint64_t* n_orbits, void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * One share of bz_worst_case_mols, as bz_worst_case_part is one of bz_worst_case: share `part` of `parts`
+ * evaluates every parts-th run of the orbit enumeration; the maximum over the shares (by c_max, then by the
+ * lexicographically first argmax) is the one-call result; an empty share reports c_max = -1.
+ */
+int bz_worst_case_mols_part(int l, int r, int q, int part, int parts, uint64_t max_subsets, int32_t* c_max, int32_t* argmax,
+                            uint64_t* n_orbits, void* workspace, size_t workspace_bytes, void* stream);
+
 /* The number of sets bz_worst_case_mols(l, r, q) evaluates.  Host only; needs no GPU. */
 int bz_mols_orbit_count(int l, int r, int q, uint64_t* n_orbits);
 

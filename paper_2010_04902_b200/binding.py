@@ -68,6 +68,7 @@ _SIGNATURES = {
     "bz_vote_bulyan": (_c_int, [_c_vp, _c_int, _c_int, _c_i64, _c_i64, _c_i64, _c_int, _c_vp, _c_i64, _c_vp, _c_vp, _c_vp,
                                 _c_sz, _c_vp]),
     "bz_worst_case_mols": (_c_int, [_c_int, _c_int, _c_int, _c_u64, _c_vp, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp]),
+    "bz_worst_case_mols_part": (_c_int, [_c_int, _c_int, _c_int, _c_int, _c_int, _c_u64, _c_vp, _c_vp, _c_vp, _c_vp, _c_sz, _c_vp]),
     "bz_mols_orbit_count": (_c_int, [_c_int, _c_int, _c_int, _c_vp]),
     "bz_workspace_bytes": (_c_sz, [_c_int, _c_int, _c_int, _c_i64, _c_int, _c_int]),
     "bz_status_string": (ctypes.c_char_p, [_c_int]),
@@ -259,6 +260,20 @@ def worst_case_mols(l: int, r: int, q: int, max_subsets: int = 0, workspace: tor
     st = lib().bz_worst_case_mols(l, r, q, max_subsets, ctypes.addressof(cmax), arg.ctypes.data, ctypes.addressof(n),
                                   ws.data_ptr(), ws.numel(), _stream())
     _check(st, "bz_worst_case_mols(l=%d, r=%d, q=%d)" % (l, r, q))
+    return int(cmax.value), arg[:q].copy(), int(n.value)
+
+
+def worst_case_mols_part(l: int, r: int, q: int, part: int, parts: int, max_subsets: int = 0,
+                         workspace: torch.Tensor | None = None):
+    """bz_worst_case_mols_part: share `part` of `parts` of the orbit search.  Returns (c_max, argmax[q] numpy, n_orbits);
+    c_max is -1 for a share that received nothing."""
+    ws = workspace if workspace is not None else alloc_workspace(OP_WORST_CASE_MOLS, r, l * l)
+    cmax = ctypes.c_int32(0)
+    n = ctypes.c_uint64(0)
+    arg = np.zeros(max(q, 1), np.int32)
+    st = lib().bz_worst_case_mols_part(l, r, q, part, parts, max_subsets, ctypes.addressof(cmax), arg.ctypes.data,
+                                       ctypes.addressof(n), ws.data_ptr(), ws.numel(), _stream())
+    _check(st, "bz_worst_case_mols_part(l=%d, r=%d, q=%d, part %d of %d)" % (l, r, q, part, parts))
     return int(cmax.value), arg[:q].copy(), int(n.value)
 
 

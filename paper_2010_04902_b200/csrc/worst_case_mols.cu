@@ -37,6 +37,7 @@ struct MolsArgs {
     const uint32_t* entries;  // [n_comp][kEntry]
     uint64_t total_heads;
     uint32_t heads_per_chunk;
+    uint32_t part, parts;     // this launch takes the chunks whose index is part modulo parts
     int n_comp, l, r;
 };
 
@@ -62,7 +63,9 @@ __global__ void __launch_bounds__(kWcBlock) worst_case_mols_kernel(const MolsArg
 
     const uint64_t n_chunks = (a.total_heads + a.heads_per_chunk - 1) / a.heads_per_chunk;
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
-    for (uint64_t chunk = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; chunk < n_chunks; chunk += stride) {
+    for (uint64_t unit = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;; unit += stride) {
+        const uint64_t chunk = a.part + a.parts * unit;
+        if (chunk >= n_chunks) break;
         uint64_t head = chunk * a.heads_per_chunk;
         const uint64_t end = head + a.heads_per_chunk < a.total_heads ? head + a.heads_per_chunk : a.total_heads;
         // composition holding this head: the last c with cum[c] <= head
@@ -249,9 +252,11 @@ extern "C" int bz_mols_orbit_count(int l, int r, int q, uint64_t* n_orbits) {
     return BZ_OK;
 }
 
-extern "C" int bz_worst_case_mols(int l, int r, int q, uint64_t max_subsets, int32_t* c_max, int32_t* argmax,
-                                  uint64_t* n_orbits, void* workspace, size_t workspace_bytes, void* stream) {
+// Share `part` of `parts` of the search (the whole search: 0 of 1); a share without a chunk reports c_max = -1.
+static int worst_case_mols_share(int l, int r, int q, int part, int parts, uint64_t max_subsets, int32_t* c_max, int32_t* argmax,
+                                 uint64_t* n_orbits, void* workspace, size_t workspace_bytes, void* stream) {
     if (c_max == nullptr) return BZ_ERR_INVALID_ARG;
+    if (parts < 1 || part < 0 || part >= parts) return BZ_ERR_INVALID_ARG;
     int st = validate_mols(l, r, q);
     if (st != BZ_OK) return st;
     if (r < 3) return BZ_ERR_UNSUPPORTED;
@@ -266,7 +271,7 @@ extern "C" int bz_worst_case_mols(int l, int r, int q, uint64_t max_subsets, int
     if (max_subsets != 0 && C.orbits > max_subsets) return BZ_ERR_BUDGET;
     if (n_orbits) *n_orbits = C.orbits;
     if (q == 0) {
-        *c_max = 0;
+        *c_max = part == 0 ? 0 : -1;  // the one (empty) set belongs to the first share
         return BZ_OK;
     }
     // union of the file masks of each pattern's workers, per class
@@ -316,8 +321,16 @@ extern "C" int bz_worst_case_mols(int l, int r, int q, uint64_t max_subsets, int
     if (per_chunk < 1) per_chunk = 1;
     if (per_chunk > 64) per_chunk = 64;
     a.heads_per_chunk = static_cast<uint32_t>(per_chunk);
+    a.part = static_cast<uint32_t>(part);
+    a.parts = static_cast<uint32_t>(parts);
     const uint64_t n_chunks = (a.total_heads + per_chunk - 1) / per_chunk;
-    uint64_t blocks = (n_chunks + kWcBlock - 1) / kWcBlock;
+    const uint64_t my_chunks = n_chunks > static_cast<uint64_t>(part) ? (n_chunks - part + parts - 1) / parts : 0;
+    if (my_chunks == 0) {
+        cudaStreamSynchronize(s);  // the host vectors of the copies above go out of scope
+        *c_max = -1;
+        return BZ_OK;
+    }
+    uint64_t blocks = (my_chunks + kWcBlock - 1) / kWcBlock;
     if (blocks > static_cast<uint64_t>(kWcMaxBlocks)) blocks = kWcMaxBlocks;
     const int grid = static_cast<int>(blocks);
     switch ((r + 1) / 2) {
@@ -332,4 +345,14 @@ extern "C" int bz_worst_case_mols(int l, int r, int q, uint64_t max_subsets, int
         return st;
     }
     return collect_best(dev_results, grid, K, q, c_max, argmax, s);  // waits for the stream: the vectors may go
+}
+
+extern "C" int bz_worst_case_mols(int l, int r, int q, uint64_t max_subsets, int32_t* c_max, int32_t* argmax,
+                                  uint64_t* n_orbits, void* workspace, size_t workspace_bytes, void* stream) {
+    return worst_case_mols_share(l, r, q, 0, 1, max_subsets, c_max, argmax, n_orbits, workspace, workspace_bytes, stream);
+}
+
+extern "C" int bz_worst_case_mols_part(int l, int r, int q, int part, int parts, uint64_t max_subsets, int32_t* c_max,
+                                       int32_t* argmax, uint64_t* n_orbits, void* workspace, size_t workspace_bytes, void* stream) {
+    return worst_case_mols_share(l, r, q, part, parts, max_subsets, c_max, argmax, n_orbits, workspace, workspace_bytes, stream);
 }

@@ -121,3 +121,17 @@ def worst_case(worker_mask, f: int, r: int, q: int, max_subsets: int = 0, ops=No
     shares = [None] * world
     dist.all_gather_object(shares, (int(c), [int(u) for u in arg]), group=group)
     return best_of_shares(shares) + (n,)
+
+
+def worst_case_mols(l: int, r: int, q: int, max_subsets: int = 0, ops=None, group=None):
+    """The same for the orbit search of the MOLS placement (bz_worst_case_mols_part).  Returns (c_max, argmax[q]
+    list, n_orbits)."""
+    ops = _ops(ops)
+    world = _world(group)
+    rank = dist.get_rank(group) if world > 1 else 0
+    c, arg, n = ops.worst_case_mols_part(l, r, q, rank, world, max_subsets)
+    if world == 1:
+        return best_of_shares([(c, arg)]) + (n,)
+    shares = [None] * world
+    dist.all_gather_object(shares, (int(c), [int(u) for u in arg]), group=group)
+    return best_of_shares(shares) + (n,)

@@ -145,3 +145,20 @@ def test_share_arguments():
     with pytest.raises(bz.BzError) as e:
         bz.worst_case_part(mask, 25, 3, 7, 0, 2, max_subsets=100)
     assert e.value.status == bz.ERR_BUDGET
+
+
+@pytest.mark.parametrize("l,r,qs", [(5, 3, [0, 1, 3, 7]), (7, 3, [2, 6, 10]), (5, 5, [4, 9, 12]), (7, 5, [5, 13]), (7, 7, [7, 12])])
+def test_orbit_search_shares_combine_to_the_whole(l, r, qs):
+    from paper_2010_04902_b200 import sharding
+    for q in qs:
+        want, warg, wn = bz.worst_case_mols(l, r, q)
+        for parts in (1, 2, 5, 64):
+            shares = []
+            for part in range(parts):
+                c, arg, n = bz.worst_case_mols_part(l, r, q, part, parts)
+                assert n == wn
+                shares.append((c, arg))
+            assert sharding.best_of_shares(shares) == (want, warg.tolist()), (l, r, q, parts)
+    with pytest.raises(bz.BzError) as e:
+        bz.worst_case_mols_part(l, r, 1, 3, 3)
+    assert e.value.status == bz.ERR_INVALID_ARG
