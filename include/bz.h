@@ -99,6 +99,11 @@ int bz_assign_ramanujan(int m, int s, int32_t* worker_files, int32_t* file_worke
  * the paper describes; r odd rules out two-way ties (Sec. 2).
  *   replicas  device, [r][f][d] with ld_file, ld_replica;  voted  device, [f][d] with ld_voted.
  *   voted must not overlap replicas.
+ * Two kernels: one on 128-/64-/32-bit register loads (any layout), and - for (r, f) in {3,5}x{25,49} and
+ * (7,49), replicas 16-byte aligned with ld_file, ld_replica multiples of 4 - the fused kernel's staged
+ * loads with the winners stored directly (any voted layout).  The second is the default from r = 5 up,
+ * where it is the faster one; BZ_VOTE_PATH=staged / =registers (environment, read at every call) forces
+ * one of them.  Its bounded waits are counted by bz_pipeline_timeouts like the fused kernel's.
  */
 int bz_vote(const float* replicas, int r, int f, int64_t d, int64_t ld_file, int64_t ld_replica, float* voted,
             int64_t ld_voted, void* stream);

@@ -13,6 +13,8 @@
 namespace bz {
 
 // vote_median_tma.cu: BZ_OK / error, or 1 when the staged path does not apply
+int vote_tma(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted,
+             cudaStream_t s);
 int vote_median_tma(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* out,
                     const ModelUpdate& upd, cudaStream_t s);
 
@@ -29,6 +31,17 @@ bool staged_path_enabled() {
         return !(v != nullptr && std::strcmp(v, "registers") == 0);
     }();
     return on;
+}
+
+// The vote alone through the fused kernel's bulk-copy ring: the loads do not care how the rows sit relative to
+// 128-byte lines, but the winners leave as 32-bit stores.  Measured against the register kernel (d = 11.2 M, f = 49):
+// r = 3 0.83 against 0.98 of the copy rate, r = 5 0.97 against 0.96, r = 7 0.88 against 0.78 - so it is the default
+// from five copies up.  BZ_VOTE_PATH=staged / =registers forces one or the other (read at every call).
+bool vote_staged_enabled(int r) {
+    const char* v = std::getenv("BZ_VOTE_PATH");
+    if (v != nullptr && std::strcmp(v, "staged") == 0) return true;
+    if (v != nullptr && std::strcmp(v, "registers") == 0) return false;
+    return r >= 5;
 }
 
 template <typename V> struct Lanes;
@@ -449,6 +462,13 @@ extern "C" int bz_vote(const float* replicas, int r, int f, int64_t d, int64_t l
     if ((voted == nullptr && d > 0) || ld_voted < d) return BZ_ERR_INVALID_ARG;
     if (d == 0) return BZ_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (r > 1 && vote_staged_enabled(r)) {
+        st = vote_tma(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, s);
+        if (st != 1) {
+            if (st == BZ_OK) note_path(BZ_PATH_STAGED);
+            return st;
+        }
+    }
     int vec = 1;
     if (aligned16(replicas) && aligned16(voted) && (ld_file % 4 == 0) && (ld_voted % 4 == 0) && (r == 1 || ld_replica % 4 == 0))
         vec = 4;

@@ -34,9 +34,11 @@ template <int R, int F, int FC> struct Shape {
 
 // Dynamic shared memory: [STAGES][R][FC][kTileD] floats (each stage 128-byte aligned), then the
 // full/empty barriers.
-template <int R, int F, int FC, int STAGES>
+// VOTE_ONLY: the winners themselves go to out[file * ld_out + j] (bz_vote through the same ring: the loads no
+// longer depend on how the rows sit relative to 128-byte lines); otherwise out[j] is their median.
+template <int R, int F, int FC, int STAGES, bool VOTE_ONLY = false>
 __global__ void __launch_bounds__(kThreads)
-    vote_median_tma_kernel(const __grid_constant__ CUtensorMap map, int64_t d, float* __restrict__ out,
+    vote_median_tma_kernel(const __grid_constant__ CUtensorMap map, int64_t d, float* __restrict__ out, int64_t ld_out,
                            const ModelUpdate upd) {
     using S = Shape<R, F, FC>;
     // where the ALU pipe limits the kernel (measured), two of three comparators compute their max on the other pipe
@@ -87,7 +89,7 @@ __global__ void __launch_bounds__(kThreads)
         }
     } else {
         // ---------------------------------------------------------------- consumers: one coordinate each
-        int key[F];
+        int key[VOTE_ONLY ? 1 : F];
         const bool has_w = upd.w != nullptr, has_v = upd.v != nullptr;
         int64_t item = 0;
         bool alive = true;
@@ -114,18 +116,24 @@ __global__ void __launch_bounds__(kThreads)
                         uint32_t copies[R];
 #pragma unroll
                         for (int k = 0; k < R; ++k) copies[k] = base[(k * FC + fi) * kTileD];
-                        key[chunk * FC + fi] = order_key(vote_bits<R>(copies));
+                        if constexpr (VOTE_ONLY) {
+                            if (j < d) out[(chunk * FC + fi) * ld_out + j] = __uint_as_float(vote_bits<R>(copies));
+                        } else {
+                            key[chunk * FC + fi] = order_key(vote_bits<R>(copies));
+                        }
                     }
                 }
                 __syncwarp();
                 if ((tid & 31) == 0) mbar_arrive(&empty[s]);  // this warp is done reading the stage
             }
-            if (alive && j < d) {
-                const float med = __uint_as_float(key_bits(MedianNet<F>::template run<kMaxOnFma, kMaxOf>(key)));
-                if (out != nullptr) out[j] = med;
-                if (has_w) {
-                    upd.w[j] = update_lane(w_old, v_old, med, upd.eta, upd.mu, has_v);
-                    if (has_v) upd.v[j] = v_old;
+            if constexpr (!VOTE_ONLY) {
+                if (alive && j < d) {
+                    const float med = __uint_as_float(key_bits(MedianNet<F>::template run<kMaxOnFma, kMaxOf>(key)));
+                    if (out != nullptr) out[j] = med;
+                    if (has_w) {
+                        upd.w[j] = update_lane(w_old, v_old, med, upd.eta, upd.mu, has_v);
+                        if (has_v) upd.v[j] = v_old;
+                    }
                 }
             }
         }
@@ -135,8 +143,8 @@ __global__ void __launch_bounds__(kThreads)
 
 // ---- host side ----------------------------------------------------------------------------------
 
-template <int R, int F, int FC, int STAGES>
-int launch_tma(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, float* out, const ModelUpdate& upd,
+template <int R, int F, int FC, int STAGES, bool VOTE_ONLY = false>
+int launch_tma(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, float* out, int64_t ld_out, const ModelUpdate& upd,
                cudaStream_t s) {
     using S = Shape<R, F, FC>;
     EncodeTiledFn enc = encode_tiled();
@@ -151,14 +159,14 @@ int launch_tma(const float* rep, int64_t d, int64_t ld_file, int64_t ld_rep, flo
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (cr != CUDA_SUCCESS) return 1;  // shape the descriptor cannot express: use the register path
     constexpr int smem = STAGES * S::kStageBytes + 2 * STAGES * 8;
-    auto kern = vote_median_tma_kernel<R, F, FC, STAGES>;
+    auto kern = vote_median_tma_kernel<R, F, FC, STAGES, VOTE_ONLY>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return cuda_failed(e);
     constexpr int fit = (227 * 1024) / (smem + 1024);  // CTAs whose rings fit in one SM (1 KB reserved each)
     constexpr int ctas_per_sm = fit >= 4 ? 4 : (fit >= 1 ? fit : 1);
     int64_t grid = (d + kTileD - 1) / kTileD;
     if (grid > kNumSMs * ctas_per_sm) grid = kNumSMs * ctas_per_sm;
-    kern<<<static_cast<int>(grid), kThreads, smem, s>>>(map, d, out, upd);
+    kern<<<static_cast<int>(grid), kThreads, smem, s>>>(map, d, out, ld_out, upd);
     note_launch();
     return check_launch();
 }
@@ -173,7 +181,7 @@ int vote_median_tma(const float* rep, int r, int f, int64_t d, int64_t ld_file, 
     if (!aligned16(rep) || (ld_file % 4) != 0 || (r > 1 && (ld_rep % 4) != 0) || d >= (int64_t(1) << 31)) return 1;
     if (d < 4 * kTileD) return 1;  // tiny inputs: not worth a descriptor
 #define BZ_TMA_CASE(R_, F_, FC_, ST_) \
-    if (r == R_ && f == F_) return launch_tma<R_, F_, FC_, ST_>(rep, d, ld_file, ld_rep, out, upd, s);
+    if (r == R_ && f == F_) return launch_tma<R_, F_, FC_, ST_>(rep, d, ld_file, ld_rep, out, 0, upd, s);
     BZ_TMA_CASE(3, 25, 25, 3)
     BZ_TMA_CASE(3, 49, 25, 3)
     BZ_TMA_CASE(5, 25, 13, 2)
@@ -182,6 +190,23 @@ int vote_median_tma(const float* rep, int r, int f, int64_t d, int64_t ld_file, 
     BZ_TMA_CASE(1, 25, 25, 4)
     BZ_TMA_CASE(1, 49, 49, 2)
 #undef BZ_TMA_CASE
+    return 1;
+}
+
+// bz_vote through the ring.  Returns BZ_OK / an error, or 1 when this path does not apply (same requirements as
+// above, and ld_voted a multiple of 4 is not needed: the winners are stored with 32-bit stores, one line per warp).
+int vote_tma(const float* rep, int r, int f, int64_t d, int64_t ld_file, int64_t ld_rep, float* voted, int64_t ld_voted,
+             cudaStream_t s) {
+    if (!aligned16(rep) || (ld_file % 4) != 0 || (ld_rep % 4) != 0 || d >= (int64_t(1) << 31) || d < 4 * kTileD) return 1;
+    const ModelUpdate none{nullptr, nullptr, 0.f, 0.f};
+#define BZ_TMA_VOTE(R_, F_, FC_, ST_) \
+    if (r == R_ && f == F_) return launch_tma<R_, F_, FC_, ST_, true>(rep, d, ld_file, ld_rep, voted, ld_voted, none, s);
+    BZ_TMA_VOTE(3, 25, 25, 3)
+    BZ_TMA_VOTE(3, 49, 25, 3)
+    BZ_TMA_VOTE(5, 25, 13, 2)
+    BZ_TMA_VOTE(5, 49, 13, 2)
+    BZ_TMA_VOTE(7, 49, 10, 2)
+#undef BZ_TMA_VOTE
     return 1;
 }
 

@@ -159,6 +159,37 @@ def test_edge_values_through_the_staged_kernels(r, f, kind):
     _check_staged(rep, buf[:, :, 4:4 + d])
 
 
+@pytest.mark.parametrize("kind", ["ties", "special", "independent"])
+@pytest.mark.parametrize("r,f", [(3, 25), (3, 49), (5, 25), (5, 49), (7, 49)])
+def test_vote_alone_through_the_staged_kernel(r, f, kind, monkeypatch):
+    # bz_vote through the fused kernel's ring (the default from five copies up; forced here for three): the winners,
+    # bit for bit, on aligned sizes, a ragged last tile, padded replica rows and an output with its own leading dimension
+    monkeypatch.setenv("BZ_VOTE_PATH", "staged")
+    rng = np.random.default_rng(77 * r + f + len(kind))
+    for d in (512, 4484, 148 * 128 + 36):
+        rep = _staged_inputs(kind, r, f, d, rng)
+        got = bz.vote(torch.from_numpy(rep).to(DEV))
+        assert bz.last_path() == bz.PATH_STAGED
+        assert np.array_equal(_bits(got), _bits(oracle.vote(rep)))
+    d, ld = 3076, 3100
+    rep = _staged_inputs(kind, r, f, d, rng)
+    buf = torch.full((r, f, ld), float("nan"), dtype=torch.float32, device=DEV)
+    buf[:, :, 4:4 + d] = torch.from_numpy(rep).to(DEV)
+    out_buf = torch.full((f, d + 7), -7.0, dtype=torch.float32, device=DEV)
+    out = out_buf[:, 3:3 + d]                       # rows 12 bytes off, leading dimension d + 7: 32-bit stores do not mind
+    bz.vote(buf[:, :, 4:4 + d], out)
+    assert bz.last_path() == bz.PATH_STAGED
+    assert np.array_equal(_bits(out), _bits(oracle.vote(rep)))
+    assert (out_buf[:, :3] == -7.0).all() and (out_buf[:, 3 + d:] == -7.0).all()
+    # the register kernel on request, and by default for three copies
+    monkeypatch.setenv("BZ_VOTE_PATH", "registers")
+    got = bz.vote(torch.from_numpy(rep).to(DEV))
+    assert bz.last_path() == bz.PATH_REGISTERS and np.array_equal(_bits(got), _bits(oracle.vote(rep)))
+    monkeypatch.delenv("BZ_VOTE_PATH")
+    bz.vote(torch.from_numpy(rep).to(DEV))
+    assert bz.last_path() == (bz.PATH_STAGED if r >= 5 else bz.PATH_REGISTERS)
+
+
 @pytest.mark.parametrize("f", [25, 49])
 def test_median_of_given_rows_on_the_staged_kernel(f):
     # Gaussian rows with a block of rounded values (many equal keys), at a size with many tiles per CTA
