@@ -34,14 +34,13 @@ bool staged_path_enabled() {
 }
 
 // The vote alone through the fused kernel's bulk-copy ring: the loads do not care how the rows sit relative to
-// 128-byte lines, but the winners leave as 32-bit stores.  Measured against the register kernel (d = 11.2 M, f = 49):
-// r = 3 0.83 against 0.98 of the copy rate, r = 5 0.97 against 0.96, r = 7 0.88 against 0.78 - so it is the default
-// from five copies up.  BZ_VOTE_PATH=staged / =registers forces one or the other (read at every call).
-bool vote_staged_enabled(int r) {
+// 128-byte lines, and the winners leave as 128-bit stores from the stage (32-bit ones where the output is not
+// 16-byte aligned).  Measured against the register kernel at d = 11.2 M: r = 3, f = 49 1.05 against 0.98 of the copy
+// rate (rows off 128-byte lines: 1.00 against 0.86), r = 5 0.99 against 0.96, r = 7 0.89 against 0.78 - so it is the
+// default wherever it applies.  BZ_VOTE_PATH=registers / =staged forces one or the other (read at every call).
+bool vote_staged_enabled() {
     const char* v = std::getenv("BZ_VOTE_PATH");
-    if (v != nullptr && std::strcmp(v, "staged") == 0) return true;
-    if (v != nullptr && std::strcmp(v, "registers") == 0) return false;
-    return r >= 5;
+    return !(v != nullptr && std::strcmp(v, "registers") == 0);
 }
 
 template <typename V> struct Lanes;
@@ -462,7 +461,11 @@ extern "C" int bz_vote(const float* replicas, int r, int f, int64_t d, int64_t l
     if ((voted == nullptr && d > 0) || ld_voted < d) return BZ_ERR_INVALID_ARG;
     if (d == 0) return BZ_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (r > 1 && vote_staged_enabled(r)) {
+    // (small inputs stay on the register kernel unless asked: below ~100 MB of replicas the call is bound by its
+    // launch, and the staged kernel adds a descriptor and a ring to that - 27 -> 46 us at d = 100 000)
+    const bool asked = std::getenv("BZ_VOTE_PATH") != nullptr;
+    const bool large = static_cast<double>(r) * f * static_cast<double>(d) * 4.0 >= 128.0 * 1024 * 1024;
+    if (r > 1 && vote_staged_enabled() && (large || asked)) {
         st = vote_tma(replicas, r, f, d, ld_file, ld_replica, voted, ld_voted, s);
         if (st != 1) {
             if (st == BZ_OK) note_path(BZ_PATH_STAGED);

@@ -90,6 +90,8 @@ __global__ void __launch_bounds__(kThreads)
     } else {
         // ---------------------------------------------------------------- consumers: one coordinate each
         int key[VOTE_ONLY ? 1 : F];
+        // vote only: 128-bit stores where the output allows them (16-byte aligned rows, whole groups of four)
+        const bool wide_out = VOTE_ONLY && ((reinterpret_cast<uintptr_t>(out) | static_cast<uintptr_t>(ld_out * 4)) & 15) == 0 && (d & 3) == 0;
         const bool has_w = upd.w != nullptr, has_v = upd.v != nullptr;
         int64_t item = 0;
         bool alive = true;
@@ -117,13 +119,36 @@ __global__ void __launch_bounds__(kThreads)
 #pragma unroll
                         for (int k = 0; k < R; ++k) copies[k] = base[(k * FC + fi) * kTileD];
                         if constexpr (VOTE_ONLY) {
-                            if (j < d) out[(chunk * FC + fi) * ld_out + j] = __uint_as_float(vote_bits<R>(copies));
+                            // the winner takes copy 0's place in the stage (only this thread reads that column)
+                            if (wide_out)
+                                const_cast<uint32_t*>(base)[fi * kTileD] = vote_bits<R>(copies);
+                            else if (j < d)
+                                out[(chunk * FC + fi) * ld_out + j] = __uint_as_float(vote_bits<R>(copies));
                         } else {
                             key[chunk * FC + fi] = order_key(vote_bits<R>(copies));
                         }
                     }
                 }
                 __syncwarp();
+                if constexpr (VOTE_ONLY) {
+                    if (wide_out) {
+                        // the warp's 32 columns of the FC winner rows leave as 128-bit stores: lane -> (row, four columns)
+                        const int warp = tid >> 5, lane = tid & 31;
+                        const int64_t j4 = (blockIdx.x + t * gridDim.x) * kTileD + warp * 32;
+                        const float* rows = stages + static_cast<size_t>(s) * S::kStageFloats + warp * 32;
+                        for (int idx = lane; idx < FC * 8; idx += 32) {
+                            const int row = idx >> 3, c4 = (idx & 7) * 4;
+                            if (chunk * FC + row < F && j4 + c4 < d) {   // d is a multiple of 4 on this path
+                                const float4 w = *reinterpret_cast<const float4*>(rows + row * kTileD + c4);
+                                __stcs(reinterpret_cast<float4*>(out + (chunk * FC + row) * ld_out + j4 + c4), w);
+                            }
+                        }
+                        // this thread wrote the stage through the generic proxy; the bulk copy that refills it
+                        // writes through the asynchronous one
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                    }
+                }
                 if ((tid & 31) == 0) mbar_arrive(&empty[s]);  // this warp is done reading the stage
             }
             if constexpr (!VOTE_ONLY) {

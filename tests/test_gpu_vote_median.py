@@ -162,7 +162,7 @@ def test_edge_values_through_the_staged_kernels(r, f, kind):
 @pytest.mark.parametrize("kind", ["ties", "special", "independent"])
 @pytest.mark.parametrize("r,f", [(3, 25), (3, 49), (5, 25), (5, 49), (7, 49)])
 def test_vote_alone_through_the_staged_kernel(r, f, kind, monkeypatch):
-    # bz_vote through the fused kernel's ring (the default from five copies up; forced here for three): the winners,
+    # bz_vote through the fused kernel's ring (the default where it applies): the winners,
     # bit for bit, on aligned sizes, a ragged last tile, padded replica rows and an output with its own leading dimension
     monkeypatch.setenv("BZ_VOTE_PATH", "staged")
     rng = np.random.default_rng(77 * r + f + len(kind))
@@ -181,13 +181,21 @@ def test_vote_alone_through_the_staged_kernel(r, f, kind, monkeypatch):
     assert bz.last_path() == bz.PATH_STAGED
     assert np.array_equal(_bits(out), _bits(oracle.vote(rep)))
     assert (out_buf[:, :3] == -7.0).all() and (out_buf[:, 3 + d:] == -7.0).all()
-    # the register kernel on request, and by default for three copies
+    # the register kernel on request
     monkeypatch.setenv("BZ_VOTE_PATH", "registers")
     got = bz.vote(torch.from_numpy(rep).to(DEV))
     assert bz.last_path() == bz.PATH_REGISTERS and np.array_equal(_bits(got), _bits(oracle.vote(rep)))
+    # by default: the register kernel for an input this small, the staged one from ~100 MB of replicas up
     monkeypatch.delenv("BZ_VOTE_PATH")
     bz.vote(torch.from_numpy(rep).to(DEV))
-    assert bz.last_path() == (bz.PATH_STAGED if r >= 5 else bz.PATH_REGISTERS)
+    assert bz.last_path() == bz.PATH_REGISTERS
+    if kind == "ties":
+        d_big = (128 * 1024 * 1024) // (4 * r * f) // 128 * 128 + 128
+        big = torch.from_numpy(rng.integers(0, 3, size=(r, f, d_big)).astype(np.float32))
+        got = bz.vote(big.to(DEV))
+        assert bz.last_path() == bz.PATH_STAGED
+        sample = np.concatenate([np.arange(0, 300), np.arange(d_big - 300, d_big), rng.integers(0, d_big, 5000)])
+        assert np.array_equal(_bits(got[:, sample]), _bits(oracle.vote(big[:, :, sample].numpy())))
 
 
 @pytest.mark.parametrize("f", [25, 49])
